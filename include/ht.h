@@ -1,0 +1,174 @@
+/*
+ * ht.h -- C ABI of the B200 tree-verify library for Hidden Transfer decoding
+ * (arXiv 2404.12022).  One decoding round verifies a flattened draft tree and the
+ * pseudo positions produced by the hidden-transfer projection in a single forward; this
+ * library holds the four data-parallel operations of that forward that are specific to
+ * the method.  Everything else of the transformer layer (norms, Q/K/V/O and MLP GEMMs,
+ * rotary embedding, lm-head) is the caller's.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers unless a comment says "host".  The caller owns every
+ *     buffer, workspace included; the library allocates no device memory and keeps no
+ *     state between calls.
+ *   - Work is enqueued on the caller's stream (`stream` is a cudaStream_t passed as
+ *     void*; NULL = the default stream) and the call returns without synchronising.
+ *   - The return value is a host-checkable status (HT_OK or HT_ERR_*).  When it is not
+ *     HT_OK nothing was launched and ht_last_error_string() describes why.
+ *   - Errors only the device can see (an illegal parent array, a cache length that does
+ *     not fit, a malformed accepted path) are written to `status` -- one int32 per
+ *     sequence, HT_STATUS_* -- and that sequence's work is skipped.  Device code never
+ *     traps or asserts.  Every call that takes `status` writes all B entries.
+ *   - Tensors are dense row-major with the last index fastest; every base pointer must
+ *     be 16-byte aligned.
+ *
+ * Shapes: B sequences; N query rows per sequence = T draft-tree nodes followed by P
+ * pseudo positions; Hq query heads sharing Hkv KV heads (Hq % Hkv == 0); head size D;
+ * `cap` rows of cache capacity per (sequence, KV head); vocabulary V; hidden size d;
+ * k transfer steps.
+ */
+#ifndef HT_H_
+#define HT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { HT_F32 = 0, HT_F16 = 1, HT_BF16 = 2 } ht_dtype;
+
+enum {
+    HT_OK = 0,
+    HT_ERR_INVALID_ARG = 1, /* null / misaligned pointer, non-positive or inconsistent size */
+    HT_ERR_UNSUPPORTED = 2, /* a legal request this build has no kernel for */
+    HT_ERR_BAD_TREE = 3,    /* reserved for host-side tree checks */
+    HT_ERR_WORKSPACE = 4,   /* workspace smaller than ht_tree_attention_workspace() */
+    HT_ERR_CUDA = 5,        /* the CUDA runtime reported an error at launch */
+    HT_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (reported via status) */
+};
+
+enum {
+    HT_STATUS_OK = 0,
+    HT_STATUS_BAD_TREE = 1,      /* some parent[r] is outside [-1, r) */
+    HT_STATUS_BAD_LEN = 2,       /* kv_len[b] < 0 or kv_len[b] + N > cap */
+    HT_STATUS_BAD_PATH = 3,      /* accepted path not increasing / out of range */
+    HT_STATUS_PATH_TOO_LONG = 4, /* the accepted path has more than max_path nodes */
+    HT_STATUS_TIMEOUT = 6
+};
+
+/* ht_attn_desc.flags */
+#define HT_ATTN_FORCE_SIMT 1u /* use the fp32-ALU kernel even where a tensor-core kernel applies */
+
+typedef struct {
+    int32_t B, N, Hq, Hkv, D, cap;
+    int32_t dtype;        /* ht_dtype of q, caches and out */
+    float scale;          /* softmax scale; <= 0 selects 1/sqrt(D) */
+    int64_t kv_stride_b;  /* elements between sequences in each cache; 0 = Hkv*cap*D */
+    int64_t kv_stride_h;  /* elements between KV heads; 0 = cap*D.  Rows are D apart. */
+    int32_t num_splits;   /* KV splits per (sequence, head); 0 = library chooses */
+    uint32_t flags;
+} ht_attn_desc;
+
+typedef struct {
+    int32_t layers, B, Hkv, cap, D;
+    int32_t dtype;        /* ht_dtype (only its width matters) */
+    int32_t N;            /* tree rows behind each context: accepted indices lie in [0, N) */
+    int64_t stride_layer; /* elements; 0 = B*Hkv*cap*D */
+    int64_t stride_b;     /* elements; 0 = Hkv*cap*D */
+    int64_t stride_h;     /* elements; 0 = cap*D */
+} ht_cache_desc;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int ht_version(void);
+
+/* Host string describing the most recent non-HT_OK return on the calling thread. */
+const char *ht_last_error_string(void);
+
+/*
+ * Hidden-transfer projection -- Section "Hidden Transfer" and the displayed equation of
+ * Section "Training stage":  h~ = W^i_{t_i} . h  with W^i in R^{d x d}, 1 <= i <= k, a
+ * plain linear map (no bias, no activation).
+ *   h_src [B, d]      hidden state of the source token of each sequence
+ *   W     [k, d, d]   W[i][r][c]: output feature r, input feature c (W acts on a column)
+ *   out   [B, k, d]   out[b][i][r] = sum_c W[i][r][c] * h_src[b][c]
+ * fp32 accumulation, result rounded once to `dtype`.  d must be a multiple of 4 (fp32)
+ * or 8 (fp16 / bf16).  B*k*d == 0 is a no-op.
+ */
+int ht_transfer(const void *h_src, const void *W, void *out, int B, int k, int d, int dtype,
+                void *stream);
+
+/*
+ * Tree attention -- Section "Tree attention": the draft tree is flattened into a
+ * sequence and "a token only attends to its ancestors" (and the context); pseudo
+ * positions follow Section "Training stage" (a pseudo state sees the context, earlier
+ * pseudo states and itself) and are given as ordinary rows of `parent`.
+ *   q        [B, N, Hq, D]
+ *   k_cache, v_cache  [B, Hkv, cap, D] (strides in desc); sequence b holds kv_len[b]
+ *            context rows; the K/V of query row r must already sit at row kv_len[b] + r
+ *   kv_len   [B] int32
+ *   parent   [B, N] int32, parent[b][r] in [-1, r); -1 attaches r to the context
+ *   out      [B, N, Hq, D]:  out[b,r,h] = softmax(scale * q[b,r,h] . K^T) V over cache rows
+ *            [0, kv_len[b]) of KV head h / (Hq/Hkv) and rows kv_len[b] + c for c = r and
+ *            every ancestor c of r.  fp32 (fp16 / bf16 inputs: tensor-core products with
+ *            fp32 accumulation) softmax and accumulation, rounded once to `dtype`.
+ *   workspace, workspace_bytes  scratch of at least ht_tree_attention_workspace(desc)
+ *            bytes, 16-byte aligned; contents need no initialisation and are undefined
+ *            afterwards.  Calls that run concurrently need distinct workspaces.
+ *   status   [B] int32 out: HT_STATUS_BAD_TREE / HT_STATUS_BAD_LEN sequences are skipped
+ *            (their rows of `out` are left untouched).
+ * Cache rows at or beyond kv_len[b] + N are never used for a result, whatever they hold.
+ * Supported: D in {64, 128}; N <= 1024.  B == 0 or N == 0 is a no-op.
+ */
+size_t ht_tree_attention_workspace(const ht_attn_desc *desc /* host */);
+int ht_tree_attention(const ht_attn_desc *desc /* host */, const void *q, const void *k_cache,
+                      const void *v_cache, const int32_t *kv_len, const int32_t *parent, void *out,
+                      void *workspace, size_t workspace_bytes, int32_t *status, void *stream);
+
+/*
+ * Greedy verification -- Fig. 2 caption ("find the last accepted token position"),
+ * Section "Inference stage", Section "Setup" (greedy sampling; output identical to
+ * auto-regressive decoding).
+ *   logits    [B, N, V] of `dtype`
+ *   tokens    [B, T] int32 draft token of each tree node (T <= N)
+ *   parent    [B, N] int32 (rows < T are consulted)
+ *   root_pred [B] int32 or NULL: the token greedy decoding emits after the context (the
+ *             argmax carried over from the previous round).  Top-level nodes (parent -1)
+ *             are checked against it; with NULL they are taken as known-correct.
+ *   pred      [B, N] int32 out, required: argmax_v logits[b,r,v]; the lowest index wins
+ *             ties, NaN never wins, a row of NaNs gives 0
+ *   accept_len  [B] out: number of nodes on the longest root path all of whose nodes c
+ *             satisfy tokens[c] == pred[parent[c]] (top level: == root_pred); ties between
+ *             paths of equal length go to the smallest terminal node index
+ *   accept_path [B, max_path] out: that path, root first, padded with -1
+ *   next_token  [B] out: pred at the path's last node; root_pred[b] (or -1 without
+ *             root_pred) when nothing is accepted
+ *   status    [B] out: HT_STATUS_BAD_TREE, HT_STATUS_PATH_TOO_LONG (accept_len 0, next -1)
+ */
+int ht_verify_greedy(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
+                     const int32_t *root_pred, int B, int N, int T, int V, int max_path,
+                     int32_t *pred, int32_t *accept_len, int32_t *accept_path,
+                     int32_t *next_token, int32_t *status, void *stream);
+
+/*
+ * KV compaction -- implied by verifying under a KV cache (Fig. 1 caption; Section
+ * "Inference stage"): after acceptance only the accepted path's K/V may follow the
+ * context.  For every layer, sequence b, KV head and j < accept_len[b], cache row
+ * kv_len[b] + j receives what row kv_len[b] + accept_path[b][j] held before the call (K and
+ * V alike); new_kv_len[b] = kv_len[b] + accept_len[b].  In place and safe when source and
+ * destination rows overlap.  Rows below kv_len[b] are untouched; rows at or beyond
+ * new_kv_len[b] are unspecified afterwards.
+ *   k_cache, v_cache  [layers, B, Hkv, cap, D] (strides in desc)
+ *   accept_path [B, max_path], strictly increasing, accept_path[b][j] in [j, N)
+ *   status [B] out: HT_STATUS_BAD_LEN / HT_STATUS_BAD_PATH sequences are left unchanged and
+ *            new_kv_len[b] = kv_len[b].
+ * max_path <= 64.  D * element size must be a multiple of 16 bytes.
+ */
+int ht_kv_compact(void *k_cache, void *v_cache, const ht_cache_desc *desc /* host */,
+                  const int32_t *kv_len, const int32_t *accept_len, const int32_t *accept_path,
+                  int max_path, int32_t *new_kv_len, int32_t *status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HT_H_ */

@@ -1,0 +1,139 @@
+// C ABI of the tree-verify library: argument checks and dispatch.  Declarations and the
+// meaning of every argument are in include/ht.h.
+#include <stdarg.h>
+#include <stdio.h>
+
+#include "ht_common.cuh"
+
+namespace ht {
+
+static thread_local char g_err[512] = "no error";
+
+int fail(int code, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int check_launch(const char *what) {
+    const cudaError_t e = cudaPeekAtLastError();
+    if (e != cudaSuccess) {
+        cudaGetLastError();  // clear the non-sticky launch error so later calls are judged on their own
+        return fail(HT_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+    }
+    return HT_OK;
+}
+
+static int check_attn_desc(const ht_attn_desc *d) {
+    if (!d) return fail(HT_ERR_INVALID_ARG, "desc is NULL");
+    if (d->B < 0 || d->N < 0) return fail(HT_ERR_INVALID_ARG, "negative B or N");
+    if (d->Hq <= 0 || d->Hkv <= 0 || d->Hq % d->Hkv != 0)
+        return fail(HT_ERR_INVALID_ARG, "Hq = %d must be a positive multiple of Hkv = %d", d->Hq, d->Hkv);
+    if (!valid_dtype(d->dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", d->dtype);
+    if (d->D != 64 && d->D != 128) return fail(HT_ERR_UNSUPPORTED, "head size %d (64 and 128 are built)", d->D);
+    if (d->cap <= 0) return fail(HT_ERR_INVALID_ARG, "cap must be positive");
+    if (d->N > d->cap) return fail(HT_ERR_INVALID_ARG, "N = %d rows cannot fit in cap = %d", d->N, d->cap);
+    if (d->num_splits < 0 || d->num_splits > 1024) return fail(HT_ERR_INVALID_ARG, "num_splits out of range");
+    const long long sh = d->kv_stride_h ? d->kv_stride_h : (long long)d->cap * d->D;
+    const long long sb = d->kv_stride_b ? d->kv_stride_b : (long long)d->Hkv * d->cap * d->D;
+    if (sh < (long long)d->cap * d->D || sb < sh * d->Hkv)
+        return fail(HT_ERR_INVALID_ARG, "cache strides overlap");
+    if ((sh * elem_bytes(d->dtype)) % 16 || (sb * elem_bytes(d->dtype)) % 16)
+        return fail(HT_ERR_INVALID_ARG, "cache strides must be multiples of 16 bytes");
+    return HT_OK;
+}
+
+}  // namespace ht
+
+using namespace ht;
+
+extern "C" {
+
+int ht_version(void) { return 100; }
+
+const char *ht_last_error_string(void) { return g_err; }
+
+int ht_transfer(const void *h_src, const void *W, void *out, int B, int k, int d, int dtype,
+                void *stream) {
+    if (B < 0 || k < 0 || d < 0) return fail(HT_ERR_INVALID_ARG, "negative size");
+    if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if ((long long)B * k * d == 0) return HT_OK;
+    if (!h_src || !W || !out) return fail(HT_ERR_INVALID_ARG, "NULL pointer");
+    if (!aligned16(h_src) || !aligned16(W) || !aligned16(out))
+        return fail(HT_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    const int ve = 16 / elem_bytes(dtype);
+    if (d % ve) return fail(HT_ERR_UNSUPPORTED, "d = %d must be a multiple of %d for this dtype", d, ve);
+    if ((long long)k * d > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "k*d too large");
+    return launch_transfer(h_src, W, out, B, k, d, dtype, static_cast<cudaStream_t>(stream));
+}
+
+size_t ht_tree_attention_workspace(const ht_attn_desc *desc) {
+    if (check_attn_desc(desc) != HT_OK) return 0;
+    if (desc->B == 0 || desc->N == 0) return 0;
+    size_t need = attn_simt_workspace(*desc, nullptr);
+    return (need + 255) / 256 * 256;
+}
+
+int ht_tree_attention(const ht_attn_desc *desc, const void *q, const void *k_cache, const void *v_cache,
+                      const int32_t *kv_len, const int32_t *parent, void *out, void *workspace,
+                      size_t workspace_bytes, int32_t *status, void *stream) {
+    int rc = check_attn_desc(desc);
+    if (rc != HT_OK) return rc;
+    if (desc->B == 0 || desc->N == 0) return HT_OK;
+    if (!q || !k_cache || !v_cache || !kv_len || !parent || !out || !status)
+        return fail(HT_ERR_INVALID_ARG, "NULL pointer");
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out) ||
+        (workspace && !aligned16(workspace)))
+        return fail(HT_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    const size_t need = ht_tree_attention_workspace(desc);
+    if (need > 0 && (!workspace || workspace_bytes < need))
+        return fail(HT_ERR_WORKSPACE, "workspace holds %zu bytes, %zu needed", workspace ? workspace_bytes : 0, need);
+    return launch_attn_simt(*desc, q, k_cache, v_cache, kv_len, parent, out, workspace, workspace_bytes,
+                            status, static_cast<cudaStream_t>(stream));
+}
+
+int ht_verify_greedy(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
+                     const int32_t *root_pred, int B, int N, int T, int V, int max_path, int32_t *pred,
+                     int32_t *accept_len, int32_t *accept_path, int32_t *next_token, int32_t *status,
+                     void *stream) {
+    if (B < 0 || N < 0 || T < 0 || T > N) return fail(HT_ERR_INVALID_ARG, "need 0 <= T <= N and B >= 0");
+    if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if (B == 0) return HT_OK;
+    if (N == 0 || V <= 0) return fail(HT_ERR_INVALID_ARG, "N and V must be positive");
+    if (max_path <= 0) return fail(HT_ERR_INVALID_ARG, "max_path must be positive");
+    if (!logits || !parent || !pred || !accept_len || !accept_path || !next_token || !status || (T > 0 && !tokens))
+        return fail(HT_ERR_INVALID_ARG, "NULL pointer");
+    if (!aligned16(logits)) return fail(HT_ERR_INVALID_ARG, "logits must be 16-byte aligned");
+    if ((long long)B * N > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "B*N too large");
+    return launch_verify(logits, dtype, tokens, parent, root_pred, B, N, T, V, max_path, pred, accept_len,
+                         accept_path, next_token, status, static_cast<cudaStream_t>(stream));
+}
+
+int ht_kv_compact(void *k_cache, void *v_cache, const ht_cache_desc *desc, const int32_t *kv_len,
+                  const int32_t *accept_len, const int32_t *accept_path, int max_path,
+                  int32_t *new_kv_len, int32_t *status, void *stream) {
+    if (!desc) return fail(HT_ERR_INVALID_ARG, "desc is NULL");
+    if (desc->layers <= 0 || desc->B < 0 || desc->Hkv <= 0 || desc->cap <= 0 || desc->D <= 0 || desc->N < 0)
+        return fail(HT_ERR_INVALID_ARG, "bad cache sizes");
+    if (!valid_dtype(desc->dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", desc->dtype);
+    if (max_path <= 0 || max_path > 64) return fail(HT_ERR_INVALID_ARG, "max_path must be in 1..64");
+    if (desc->B == 0) return HT_OK;
+    const int row_bytes = desc->D * elem_bytes(desc->dtype);
+    if (row_bytes % 16) return fail(HT_ERR_UNSUPPORTED, "a cache row must be a multiple of 16 bytes");
+    if ((long long)max_path * (row_bytes / 16) > 4096)
+        return fail(HT_ERR_UNSUPPORTED, "max_path * row size too large for one block");
+    if (!kv_len || !accept_len || !accept_path || !new_kv_len || !status || !k_cache || !v_cache)
+        return fail(HT_ERR_INVALID_ARG, "NULL pointer");
+    if (!aligned16(k_cache) || !aligned16(v_cache)) return fail(HT_ERR_INVALID_ARG, "caches must be 16-byte aligned");
+    const long long e = elem_bytes(desc->dtype);
+    if ((desc->stride_layer * e) % 16 || (desc->stride_b * e) % 16 || (desc->stride_h * e) % 16)
+        return fail(HT_ERR_INVALID_ARG, "cache strides must be multiples of 16 bytes");
+    if (2ll * desc->layers * desc->B * desc->Hkv > 0x7fffffffLL)
+        return fail(HT_ERR_UNSUPPORTED, "too many (layer, sequence, head) units");
+    return launch_compact(k_cache, v_cache, *desc, kv_len, accept_len, accept_path, max_path, new_kv_len, status,
+                          static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

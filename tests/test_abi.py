@@ -1,0 +1,77 @@
+"""The C-ABI library loads, exports what include/ht.h declares, and rejects bad arguments on
+the host before anything is launched (no GPU needed for any of this)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2404_12022_b200 import build, binding
+    build.build()
+    return binding.load()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "ht.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ht_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    from paper_2404_12022_b200 import binding
+    names = _declared()
+    assert set(names) == set(binding.EXPORTS)
+    for n in names:
+        assert getattr(lib, n) is not None
+    assert lib.ht_version() >= 100
+
+
+def test_host_side_rejections(lib):
+    from paper_2404_12022_b200 import binding as hb
+    buf = (ctypes.c_char * 4096)()
+    base = ctypes.addressof(buf)
+    p = (base + 255) // 256 * 256          # a 16-byte aligned host address: never dereferenced here
+    assert lib.ht_transfer(None, p, p, 1, 1, 8, hb.HT_BF16, None) == hb.HT_ERR_INVALID_ARG
+    assert b"NULL" in lib.ht_last_error_string()
+    assert lib.ht_transfer(p + 2, p, p, 1, 1, 8, hb.HT_BF16, None) == hb.HT_ERR_INVALID_ARG
+    assert lib.ht_transfer(p, p, p, 1, 1, 12, hb.HT_BF16, None) == hb.HT_ERR_UNSUPPORTED
+    assert lib.ht_transfer(p, p, p, 1, 1, 8, 7, None) == hb.HT_ERR_INVALID_ARG
+    assert lib.ht_transfer(p, p, p, 0, 3, 8, hb.HT_F32, None) == hb.HT_OK      # empty batch: no-op
+
+    d = hb.AttnDesc(1, 4, 6, 4, 128, 64, hb.HT_F16, 0.0, 0, 0, 0, 0)           # Hq % Hkv != 0
+    assert lib.ht_tree_attention(ctypes.byref(d), p, p, p, p, p, p, None, 0, p, None) == hb.HT_ERR_INVALID_ARG
+    d = hb.AttnDesc(1, 4, 4, 4, 96, 64, hb.HT_F16, 0.0, 0, 0, 0, 0)            # head size not built
+    assert lib.ht_tree_attention(ctypes.byref(d), p, p, p, p, p, p, None, 0, p, None) == hb.HT_ERR_UNSUPPORTED
+    d = hb.AttnDesc(1, 100, 4, 4, 128, 64, hb.HT_F16, 0.0, 0, 0, 0, 0)         # N > cap
+    assert lib.ht_tree_attention(ctypes.byref(d), p, p, p, p, p, p, None, 0, p, None) == hb.HT_ERR_INVALID_ARG
+    d = hb.AttnDesc(4, 91, 32, 32, 128, 4224, hb.HT_BF16, 0.0, 0, 0, 4, 0)     # needs a workspace
+    need = lib.ht_tree_attention_workspace(ctypes.byref(d))
+    assert need > 0 and need % 256 == 0
+    assert lib.ht_tree_attention(ctypes.byref(d), p, p, p, p, p, p, p, need - 16, p, None) == hb.HT_ERR_WORKSPACE
+    assert lib.ht_tree_attention(ctypes.byref(d), p, p, p, p, p, p, None, 0, p, None) == hb.HT_ERR_WORKSPACE
+    d = hb.AttnDesc(0, 91, 32, 32, 128, 4224, hb.HT_BF16, 0.0, 0, 0, 0, 0)     # empty batch
+    assert lib.ht_tree_attention(ctypes.byref(d), None, None, None, None, None, None, None, 0, None, None) == hb.HT_OK
+
+    assert lib.ht_verify_greedy(p, hb.HT_F16, p, p, None, 1, 4, 5, 100, 8, p, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG
+    assert lib.ht_verify_greedy(p, hb.HT_F16, p, p, None, 1, 4, 3, 100, 8, None, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG
+    assert lib.ht_verify_greedy(p, hb.HT_F16, p, p, None, 1, 4, 3, 100, 0, p, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG
+
+    c = hb.CacheDesc(2, 1, 4, 64, 128, hb.HT_BF16, 8, 0, 0, 0)
+    assert lib.ht_kv_compact(p, p, ctypes.byref(c), p, p, p, 65, p, p, None) == hb.HT_ERR_INVALID_ARG
+    assert lib.ht_kv_compact(None, p, ctypes.byref(c), p, p, p, 8, p, p, None) == hb.HT_ERR_INVALID_ARG
+    c = hb.CacheDesc(2, 1, 4, 64, 3, hb.HT_BF16, 8, 0, 0, 0)                   # 6-byte rows
+    assert lib.ht_kv_compact(p, p, ctypes.byref(c), p, p, p, 8, p, p, None) == hb.HT_ERR_UNSUPPORTED
+
+
+def test_binding_refuses_cpu_tensors_and_has_no_fallback():
+    import torch
+    from paper_2404_12022_b200 import binding as hb
+    with pytest.raises(ValueError):
+        hb.transfer(torch.zeros(1, 8), torch.zeros(1, 8, 8))
+    src = open(os.path.join(ROOT, "paper_2404_12022_b200", "binding.py")).read()
+    assert "oracle" not in src.replace("no fallback", "")

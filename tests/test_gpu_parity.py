@@ -1,0 +1,438 @@
+"""Parity of the CUDA library (through the C ABI) with the CPU oracle, element by element,
+on the same seeded inputs.  Tolerances:
+  fp32            |g - o| <= 1e-5
+  fp16 / bf16     |g - o| <= 2e-3 + 1e-2 |o|   (inputs rounded to the dtype, fp32 accumulation,
+                  one final rounding of an O(1) output: half an ulp of bf16 at 1.0 is 3.9e-3,
+                  so a pure absolute 2e-3 cannot hold where |o| approaches 1)
+  integers, bytes bit-exact
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2404_12022_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+DT = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
+
+
+@pytest.fixture(scope="module")
+def hb():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2404_12022_b200 import binding
+    binding.load()
+    return binding
+
+
+def f32np(t):
+    return t.detach().float().cpu().numpy()
+
+
+def assert_close(got, ref, dtype, what=""):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert np.isfinite(got).all(), what + ": non-finite output"
+    err = np.abs(got - ref)
+    if dtype == torch.float32:
+        assert err.max() <= 1e-5, "%s: max abs err %.3e" % (what, err.max())
+    else:
+        bound = 2e-3 + 1e-2 * np.abs(ref)
+        worst = (err - bound).max()
+        assert worst <= 0, "%s: max abs err %.3e (over bound by %.3e)" % (what, err.max(), worst)
+
+
+def rand_tree(rng, N, kind):
+    par = np.full(N, -1, np.int32)
+    for r in range(1, N):
+        if kind == "chain":
+            par[r] = r - 1
+        elif kind == "roots":
+            par[r] = -1
+        else:
+            par[r] = rng.integers(-1, r)
+    return par
+
+
+def make_attn_case(seed, dtype, B, N, Hq, Hkv, D, lens, cap, tree="random", garbage=True):
+    rng = np.random.default_rng(seed)
+    dt = DT[dtype]
+    q = wl.normal_tensor(seed, 1, (B, N, Hq, D), "cuda", 1.0, dt)
+    k = wl.normal_tensor(seed, 2, (B, Hkv, cap, D), "cuda", 1.0, dt)
+    v = wl.normal_tensor(seed, 3, (B, Hkv, cap, D), "cuda", 1.0, dt)
+    parent = np.stack([rand_tree(rng, N, tree) for _ in range(B)])
+    kv_len = np.array(lens, np.int32)
+    if garbage:   # rows past the tree must never influence a result, whatever they hold
+        for b in range(B):
+            k[b, :, lens[b] + N:] = float("nan")
+            v[b, :, lens[b] + N:] = float("inf")
+    return q, k, v, torch.from_numpy(kv_len).cuda(), torch.from_numpy(parent).cuda()
+
+
+def oracle_attn(oracle, q, k, v, kv_len, parent, scale=None):
+    kk, vv = f32np(k), f32np(v)
+    kk[~np.isfinite(kk)] = 0.0       # the oracle never reads those rows; keep its inputs finite anyway
+    vv[~np.isfinite(vv)] = 0.0
+    return oracle.tree_attention(f32np(q), kk, vv, kv_len.cpu().numpy(), parent.cpu().numpy(), scale)
+
+
+SMALL_CASES = [
+    # B, N, Hq, Hkv, D, lens, cap, tree
+    (1, 1, 2, 2, 64, [0], 8, "roots"),             # empty context, single row: out = v
+    (1, 1, 4, 1, 128, [1], 130, "roots"),
+    (2, 7, 4, 2, 64, [5, 70], 96, "random"),       # ragged lengths, tail tile
+    (1, 18, 4, 4, 64, [128], 160, "random"),
+    (3, 23, 8, 2, 128, [0, 33, 257], 300, "random"),
+    (1, 40, 8, 8, 128, [300], 417, "chain"),
+    (1, 33, 8, 1, 128, [100], 256, "roots"),
+    (2, 91, 8, 8, 128, [1024, 1000], 1152, "random"),
+    (1, 259, 8, 1, 128, [130], 512, "random"),     # more than 256 rows, 9 bitmask words
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("case", SMALL_CASES, ids=lambda c: "B%dN%dHq%dHkv%dD%d" % c[:5])
+def test_attention_small_cases(hb, oracle, dtype, case):
+    B, N, Hq, Hkv, D, lens, cap, tree = case
+    q, k, v, kv_len, parent = make_attn_case(11, dtype, B, N, Hq, Hkv, D, lens, cap, tree)
+    out, status = hb.tree_attention(q, k, v, kv_len, parent)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0] * B
+    ref = oracle_attn(oracle, q, k, v, kv_len, parent)
+    assert_close(f32np(out), ref, DT[dtype], "attention")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("splits", [1, 2, 3, 8, 17])
+def test_attention_split_count_invariance(hb, oracle, dtype, splits):
+    q, k, v, kv_len, parent = make_attn_case(12, dtype, 2, 37, 4, 2, 128, [513, 64], 640)
+    out, status = hb.tree_attention(q, k, v, kv_len, parent, num_splits=splits)
+    ref = oracle_attn(oracle, q, k, v, kv_len, parent)
+    assert_close(f32np(out), ref, DT[dtype], "splits=%d" % splits)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_attention_forced_simt_path(hb, oracle, dtype):
+    q, k, v, kv_len, parent = make_attn_case(13, dtype, 1, 50, 8, 2, 128, [700], 768)
+    out, _ = hb.tree_attention(q, k, v, kv_len, parent, flags=hb.HT_ATTN_FORCE_SIMT)
+    assert_close(f32np(out), oracle_attn(oracle, q, k, v, kv_len, parent), DT[dtype], "simt")
+
+
+def test_attention_custom_scale_and_strided_layer_view(hb, oracle):
+    """A layer of a [layers, B, Hkv, cap, D] cache is passed as a view; scale is a parameter."""
+    dt = torch.float16
+    layers, B, N, Hq, Hkv, D, cap = 3, 2, 20, 4, 2, 128, 200
+    kc = wl.normal_tensor(5, 1, (layers, B, Hkv, cap, D), "cuda", 1.0, dt)
+    vc = wl.normal_tensor(5, 2, (layers, B, Hkv, cap, D), "cuda", 1.0, dt)
+    q = wl.normal_tensor(5, 3, (B, N, Hq, D), "cuda", 1.0, dt)
+    rng = np.random.default_rng(5)
+    parent = torch.from_numpy(np.stack([rand_tree(rng, N, "random") for _ in range(B)])).cuda()
+    kv_len = torch.tensor([150, 17], dtype=torch.int32, device="cuda")
+    # heads interleaved differently: take a strided head view too
+    out, status = hb.tree_attention(q, kc[1], vc[1], kv_len, parent, scale=0.05)
+    ref = oracle.tree_attention(f32np(q), f32np(kc[1]), f32np(vc[1]), kv_len.cpu().numpy(),
+                                parent.cpu().numpy(), 0.05)
+    assert_close(f32np(out), ref, dt, "strided")
+
+
+def test_attention_flags_bad_sequences_and_leaves_their_rows_alone(hb, oracle):
+    q, k, v, kv_len, parent = make_attn_case(14, "f32", 3, 9, 4, 2, 64, [10, 20, 30], 64, garbage=False)
+    parent[1, 4] = 4                      # not an earlier row
+    kv_len[2] = 60                        # 60 + 9 > cap
+    out = torch.full_like(q, 7.0)
+    out, status = hb.tree_attention(q, k, v, kv_len, parent, out=out)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [hb.HT_STATUS_OK, hb.HT_STATUS_BAD_TREE, hb.HT_STATUS_BAD_LEN]
+    assert (out[1:] == 7.0).all()
+    good_parent = parent.clone()
+    good_parent[1, 4] = -1
+    kv_len[2] = 30
+    ref = oracle_attn(oracle, q, k, v, kv_len, good_parent)
+    assert_close(f32np(out[0]), ref[0], torch.float32, "good sequence")
+
+
+def _sample_units(rng, B, Hkv, n):
+    units = set()
+    units.add((0, 0))
+    while len(units) < min(n, B * Hkv):
+        units.add((int(rng.integers(B)), int(rng.integers(Hkv))))
+    return sorted(units)
+
+
+def check_sampled_units(hb, oracle, q, k, v, kv_len, parent, out, n_units, dtype, seed=0):
+    """Full-size parity: all rows and query heads of a seeded sample of (sequence, KV head)
+    units, each reduced to a B=1, Hkv=1 problem for the oracle."""
+    B, N, Hq, D = q.shape
+    Hkv = k.shape[1]
+    g = Hq // Hkv
+    rng = np.random.default_rng(seed)
+    rows = 0
+    for b, hk in _sample_units(rng, B, Hkv, n_units):
+        L = int(kv_len[b])
+        qs = f32np(q[b:b + 1, :, hk * g:(hk + 1) * g])
+        ks = f32np(k[b:b + 1, hk:hk + 1, :L + N])
+        vs = f32np(v[b:b + 1, hk:hk + 1, :L + N])
+        ref = oracle.tree_attention(qs, ks, vs, np.array([L], np.int32), parent[b:b + 1].cpu().numpy())
+        got = f32np(out[b:b + 1, :, hk * g:(hk + 1) * g])
+        assert_close(got, ref, dtype, "unit b=%d hk=%d" % (b, hk))
+        rows += N * g
+    return rows
+
+
+def test_config_c1_all_operations(hb, oracle):
+    for want in (2, 3):
+        w = wl.config_c1(want)
+        inp = wl.make_inputs(w, "cuda")
+        out, status = hb.tree_attention(inp.q[0], inp.k_cache[0], inp.v_cache[0], inp.kv_len, inp.parent)
+        ref = oracle.tree_attention(f32np(inp.q[0]), f32np(inp.k_cache[0]), f32np(inp.v_cache[0]),
+                                    inp.kv_len.cpu().numpy(), inp.parent.cpu().numpy())
+        assert_close(f32np(out), ref, torch.float32, "c1 attention")
+        pseudo = hb.transfer(inp.h_src, inp.W)
+        assert_close(f32np(pseudo), oracle.transfer(f32np(inp.h_src), f32np(inp.W)), torch.float32, "c1 transfer")
+        _verify_and_compact(hb, oracle, inp, want)
+
+
+def _verify_and_compact(hb, oracle, inp, want_first=None):
+    w = inp.w
+    pred, alen, apath, nxt, status = hb.verify_greedy(inp.logits, inp.tokens, inp.parent, inp.root_pred, w.max_path)
+    o_pred, o_alen, o_apath, o_nxt, o_status = oracle.verify_greedy(
+        f32np(inp.logits), inp.tokens.cpu().numpy(), inp.parent.cpu().numpy(),
+        None if inp.root_pred is None else inp.root_pred.cpu().numpy(), w.max_path)
+    assert np.array_equal(pred.cpu().numpy(), o_pred)
+    assert np.array_equal(alen.cpu().numpy(), o_alen)
+    assert np.array_equal(apath.cpu().numpy(), o_apath)
+    assert np.array_equal(nxt.cpu().numpy(), o_nxt)
+    assert np.array_equal(status.cpu().numpy(), o_status)
+    assert o_alen.tolist() == inp.want_len
+    if want_first is not None:
+        assert o_alen[0] == want_first
+    # compaction, bit-exact on the raw storage
+    view = torch.int32 if inp.k_cache.dtype == torch.float32 else torch.int16
+    k_before = inp.k_cache.view(view).cpu().numpy()
+    v_before = inp.v_cache.view(view).cpu().numpy()
+    new_len, cstatus = hb.kv_compact(inp.k_cache, inp.v_cache, w.N, inp.kv_len, alen, apath)
+    k_ref, v_ref, len_ref, st_ref = oracle.kv_compact(k_before, v_before, w.N, inp.kv_len.cpu().numpy(),
+                                                      o_alen, o_apath)
+    assert np.array_equal(new_len.cpu().numpy(), len_ref)
+    assert np.array_equal(cstatus.cpu().numpy(), st_ref)
+    k_after = inp.k_cache.view(view).cpu().numpy()
+    v_after = inp.v_cache.view(view).cpu().numpy()
+    for b in range(w.B):
+        n = int(len_ref[b])
+        assert np.array_equal(k_after[:, b, :, :n], k_ref[:, b, :, :n])
+        assert np.array_equal(v_after[:, b, :, :n], v_ref[:, b, :, :n])
+
+
+def test_config_c2_all_operations(hb, oracle):
+    w = wl.config_c2()
+    inp = wl.make_inputs(w, "cuda")
+    out, status = hb.tree_attention(inp.q[0], inp.k_cache[0], inp.v_cache[0], inp.kv_len, inp.parent)
+    assert status.cpu().tolist() == [0]
+    ref = oracle.tree_attention(f32np(inp.q[0]), f32np(inp.k_cache[0]), f32np(inp.v_cache[0]),
+                                inp.kv_len.cpu().numpy(), inp.parent.cpu().numpy())
+    assert_close(f32np(out), ref, torch.float16, "c2 attention")
+    pseudo = hb.transfer(inp.h_src, inp.W)
+    assert_close(f32np(pseudo), oracle.transfer(f32np(inp.h_src), f32np(inp.W)), torch.float16, "c2 transfer")
+    _verify_and_compact(hb, oracle, inp)
+
+
+@pytest.mark.parametrize("want", [0, 1, 2, 3, 4])
+def test_config_c2_every_accepted_length(hb, oracle, want):
+    w = dataclasses.replace(wl.config_c2(), want_len=[want], kv_len=[64], d=64)
+    inp = wl.make_inputs(w, "cuda")
+    _verify_and_compact(hb, oracle, inp, want)
+
+
+def test_config_c3_full_size_layers_sampled(hb, oracle):
+    """Config 3 at full size (B=4, 32 heads, KV 4096, bf16): one layer before the transfer
+    (88 rows) and one after it (91 rows), checked on sampled (sequence, head) units; then the
+    step's transfer, verification and compaction over the materialised layers."""
+    w = wl.config_c3()
+    inp = wl.make_inputs(w, "cuda", layers=[3, 20])
+    total_rows = 0
+    for i, layer in enumerate((3, 20)):
+        rows = w.rows_at_layer(layer)
+        parent = inp.parent_tree if rows == w.T else inp.parent
+        out, status = hb.tree_attention(inp.q[i], inp.k_cache[i], inp.v_cache[i], inp.kv_len, parent)
+        assert status.cpu().tolist() == [0] * w.B
+        total_rows += check_sampled_units(hb, oracle, inp.q[i], inp.k_cache[i], inp.v_cache[i],
+                                          inp.kv_len.cpu().numpy(), parent, out, 24, torch.bfloat16, seed=layer)
+    assert total_rows >= 4096
+    pseudo = hb.transfer(inp.h_src, inp.W)
+    assert_close(f32np(pseudo), oracle.transfer(f32np(inp.h_src), f32np(inp.W)), torch.bfloat16, "c3 transfer")
+    _verify_and_compact(hb, oracle, inp)
+
+
+def test_config_c4_ragged_full_size_sampled(hb, oracle):
+    w = wl.config_c4()
+    inp = wl.make_inputs(w, "cuda")
+    out, status = hb.tree_attention(inp.q[0], inp.k_cache[0], inp.v_cache[0], inp.kv_len, inp.parent)
+    assert status.cpu().tolist() == [0] * w.B
+    rows = check_sampled_units(hb, oracle, inp.q[0], inp.k_cache[0], inp.v_cache[0],
+                               inp.kv_len.cpu().numpy(), inp.parent, out, 64, torch.bfloat16)
+    assert rows >= 4096
+    pseudo = hb.transfer(inp.h_src, inp.W)
+    assert_close(f32np(pseudo), oracle.transfer(f32np(inp.h_src), f32np(inp.W)), torch.bfloat16, "c4 transfer")
+    _verify_and_compact(hb, oracle, inp)
+    assert sorted(set(inp.want_len)) == sorted(set(inp.want_len) & {0, 1, 2, 3, 4})
+
+
+@pytest.mark.parametrize("point", [(512, 16, 1), (2048, 64, 4), (8192, 128, 1), (512, 256, 16), (32768, 16, 4)],
+                         ids=lambda p: "kv%d_t%d_b%d" % p)
+def test_config_c5_gqa_points_sampled(hb, oracle, point):
+    w = wl.config_c5(*point)
+    inp = wl.make_inputs(w, "cuda", with_transfer=False)
+    out, status = hb.tree_attention(inp.q[0], inp.k_cache[0], inp.v_cache[0], inp.kv_len, inp.parent)
+    assert status.cpu().tolist() == [0] * w.B
+    n_units = 2 if point[0] * w.N > 2_000_000 else 6
+    check_sampled_units(hb, oracle, inp.q[0], inp.k_cache[0], inp.v_cache[0], inp.kv_len.cpu().numpy(),
+                        inp.parent, out, n_units, torch.bfloat16)
+    _verify_and_compact(hb, oracle, inp)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("shape", [(1, 1, 32), (2, 3, 256), (5, 2, 520), (16, 3, 1024), (9, 1, 4096)],
+                         ids=lambda s: "B%dk%dd%d" % s)
+def test_transfer_shapes(hb, oracle, dtype, shape):
+    B, k, d = shape
+    dt = DT[dtype]
+    h = wl.normal_tensor(21, 1, (B, d), "cuda", 1.0, dt)
+    W = wl.normal_tensor(21, 2, (k, d, d), "cuda", 1.0 / np.sqrt(d), dt)
+    out = hb.transfer(h, W)
+    assert_close(f32np(out), oracle.transfer(f32np(h), f32np(W)), dt, "transfer")
+
+
+def test_transfer_identity_is_exact(hb):
+    d = 512
+    h = wl.normal_tensor(22, 1, (3, d), "cuda", 1.0, torch.bfloat16)
+    W = torch.eye(d, dtype=torch.bfloat16, device="cuda")[None].contiguous()
+    assert torch.equal(hb.transfer(h, W)[:, 0], h)
+
+
+def test_transfer_c5_shape(hb, oracle):
+    B, k, d = 16, 3, 8192
+    h = wl.normal_tensor(23, 1, (B, d), "cuda", 1.0, torch.bfloat16)
+    W = wl.normal_tensor(23, 2, (k, d, d), "cuda", 0.02, torch.bfloat16)
+    out = hb.transfer(h, W)
+    assert_close(f32np(out), oracle.transfer(f32np(h), f32np(W)), torch.bfloat16, "transfer c5")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("V", [50, 1000, 32000, 32003])
+def test_row_argmax_with_ties_and_nans(hb, oracle, dtype, V):
+    dt = DT[dtype]
+    B, N, T = 2, 6, 4
+    rng = np.random.default_rng(V)
+    x = np.round(rng.standard_normal((B, N, V)) * 2) / 2          # coarse values: ties at the maximum
+    x[0, 0, :] = np.nan
+    x[0, 1, 0] = np.nan
+    x[0, 2, :] = -np.inf
+    x[1, 0, V - 1] = np.inf
+    x[1, 1, V // 2:] = x[1, 1].max() + 1                          # a long run of equal maxima
+    logits = torch.from_numpy(x).to(dt).cuda()
+    parent = torch.from_numpy(np.stack([rand_tree(rng, N, "random") for _ in range(B)])).cuda()
+    tokens = torch.from_numpy(rng.integers(0, V, (B, T)).astype(np.int32)).cuda()
+    pred, alen, apath, nxt, status = hb.verify_greedy(logits, tokens, parent, None, 8)
+    ref = oracle.row_argmax(f32np(logits))
+    assert np.array_equal(pred.cpu().numpy(), ref)
+    assert ref[0, 0] == 0 and ref[0, 2] == 0 and ref[1, 0] == V - 1 and ref[1, 1] == V // 2
+
+
+def test_acceptance_random_trees_small_alphabet(hb, oracle):
+    """Many sequences, random trees, 3-symbol alphabet: duplicates among siblings, ties between
+    equally long paths, forests, with and without root_pred."""
+    rng = np.random.default_rng(3)
+    B, T, P, V = 300, 30, 3, 16
+    N = T + P
+    parent = np.stack([rand_tree(rng, N, "random") for _ in range(B)])
+    tokens = rng.integers(0, 3, (B, T)).astype(np.int32)
+    logits = np.zeros((B, N, V), np.float32)
+    hot = rng.integers(0, 3, (B, N))
+    np.put_along_axis(logits, hot[..., None], 1.0, axis=2)
+    root_pred = rng.integers(0, 3, B).astype(np.int32)
+    for rp in (None, root_pred):
+        got = hb.verify_greedy(torch.from_numpy(logits).cuda(), torch.from_numpy(tokens).cuda(),
+                               torch.from_numpy(parent).cuda(),
+                               None if rp is None else torch.from_numpy(rp).cuda(), 16)
+        ref = oracle.verify_greedy(logits, tokens, parent, rp, 16)
+        for g, r in zip(got, ref):
+            assert np.array_equal(g.cpu().numpy(), r)
+    assert len(set(ref[1].tolist())) >= 4          # several different accepted lengths occurred
+
+
+def test_acceptance_statuses(hb, oracle):
+    N = T = 6
+    parent = np.array([[-1, 0, 1, 2, 3, 4], [-1, 0, 5, 1, 2, 3]], np.int32)     # second tree is illegal
+    tokens = np.array([[1, 2, 3, 4, 5, 6]] * 2, np.int32)
+    logits = np.zeros((2, N, 8), np.float32)
+    for r in range(N):
+        logits[:, r, min(r + 2, 7)] = 1.0
+    args = (torch.from_numpy(logits).cuda(), torch.from_numpy(tokens).cuda(), torch.from_numpy(parent).cuda(),
+            torch.tensor([1, 1], dtype=torch.int32, device="cuda"))
+    got = hb.verify_greedy(*args, 4)                                                # chain of 6 > max_path 4
+    ref = oracle.verify_greedy(logits, tokens, parent, np.array([1, 1], np.int32), 4)
+    for g, r in zip(got, ref):
+        assert np.array_equal(g.cpu().numpy(), r)
+    assert got[4].cpu().tolist() == [hb.HT_STATUS_PATH_TOO_LONG, hb.HT_STATUS_BAD_TREE]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_compaction_paths_aliasing_strides_and_errors(hb, oracle, dtype):
+    dt = DT[dtype]
+    layers, B, Hkv, cap, D, N = 3, 5, 2, 40, 64, 12
+    big_k = wl.normal_tensor(31, 1, (layers, B, Hkv + 1, cap, D), "cuda", 1.0, dt)
+    big_v = wl.normal_tensor(31, 2, (layers, B, Hkv + 1, cap, D), "cuda", 1.0, dt)
+    k = big_k[:, :, :Hkv]                       # strided over heads
+    v = big_v[:, :, :Hkv]
+    kv_len = np.array([7, 0, 20, 28, 3], np.int32)
+    alen = np.array([3, 4, 0, 2, 2], np.int32)
+    apath = np.array([[0, 2, 5, -1, -1], [0, 1, 2, 3, -1], [-1] * 5, [1, 11, -1, -1, -1], [4, 3, -1, -1, -1]], np.int32)
+    view = torch.int32 if dt == torch.float32 else torch.int16
+    k_before = k.contiguous().view(view).cpu().numpy()
+    v_before = v.contiguous().view(view).cpu().numpy()
+    untouched = big_k[:, :, Hkv].clone()
+    new_len, status = hb.kv_compact(k, v, N, torch.from_numpy(kv_len).cuda(), torch.from_numpy(alen).cuda(),
+                                    torch.from_numpy(apath).cuda())
+    k_ref, v_ref, len_ref, st_ref = oracle.kv_compact(k_before, v_before, N, kv_len, alen, apath)
+    assert np.array_equal(new_len.cpu().numpy(), len_ref) and np.array_equal(status.cpu().numpy(), st_ref)
+    assert st_ref.tolist() == [0, 0, 0, 0, oracle.BAD_PATH]
+    assert np.array_equal(k.contiguous().view(view).cpu().numpy(), k_ref)
+    assert np.array_equal(v.contiguous().view(view).cpu().numpy(), v_ref)
+    assert torch.equal(big_k[:, :, Hkv], untouched)
+
+
+def test_toy_lossless_loop_on_the_gpu(hb):
+    """Draft-and-verify rounds through the library reproduce plain greedy decoding (fp32)."""
+    from toy_lm import run_lossless_loop
+
+    class GpuOps:
+        def attention(self, q, k_cache, v_cache, kv_len, parent):
+            out, status = hb.tree_attention(torch.from_numpy(q).cuda(), torch.from_numpy(np.ascontiguousarray(k_cache)).cuda(),
+                                            torch.from_numpy(np.ascontiguousarray(v_cache)).cuda(),
+                                            torch.from_numpy(np.ascontiguousarray(kv_len)).cuda(),
+                                            torch.from_numpy(parent).cuda())
+            assert status.cpu().tolist() == [0] * q.shape[0]
+            return out.cpu().numpy()
+
+        def transfer(self, h, W):
+            return hb.transfer(torch.from_numpy(h).cuda(), torch.from_numpy(W).cuda()).cpu().numpy()
+
+        def verify(self, logits, tokens, parent, root_pred, max_path):
+            res = hb.verify_greedy(torch.from_numpy(logits).cuda(), torch.from_numpy(tokens).cuda(),
+                                   torch.from_numpy(parent).cuda(),
+                                   None if root_pred is None else torch.from_numpy(root_pred).cuda(), max_path)
+            return tuple(r.cpu().numpy() for r in res)
+
+        def compact(self, k_cache, v_cache, N, kv_len, alen, apath):
+            k = torch.from_numpy(k_cache).cuda()
+            v = torch.from_numpy(v_cache).cuda()
+            new_len, status = hb.kv_compact(k, v, N, torch.from_numpy(np.ascontiguousarray(kv_len)).cuda(),
+                                            torch.from_numpy(alen).cuda(), torch.from_numpy(apath).cuda())
+            assert status.cpu().tolist() == [0] * k.shape[1]
+            return k.cpu().numpy(), v.cpu().numpy(), new_len.cpu().numpy()
+
+    for with_root in (True, False):
+        assert run_lossless_loop(GpuOps(), with_root, seed=3, n_new=24, atol_cache=5e-4, D=64) < 24

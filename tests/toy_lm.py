@@ -137,11 +137,11 @@ def single_token_parent(P):
     return np.array([[-1] + list(range(P))], np.int32)
 
 
-def run_lossless_loop(ops, with_root, seed=0, n_new=24, atol_cache=1e-5):
+def run_lossless_loop(ops, with_root, seed=0, n_new=24, atol_cache=1e-5, D=8):
     """Tree-verify rounds against plain greedy decoding for two sequences with different
     prompt lengths.  Returns the number of rounds used (fewer than n_new means drafts were
     accepted)."""
-    lm = ToyLM(seed)
+    lm = ToyLM(seed, D=D)
     rng = np.random.default_rng(seed + 100)
     prompts = [list(rng.integers(0, lm.V, 5)), list(rng.integers(0, lm.V, 9))]
     B = len(prompts)
