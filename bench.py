@@ -1,0 +1,402 @@
+"""Benchmark of the tree-verify step (one JSON line on stdout).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c2|c4] [--impl reference]
+
+A step is one pass of the whole hot path over one batch of synthetic input: per layer a
+tree-attention call, the hidden-transfer projection at the transfer layer, greedy
+verification of the logits and KV compaction over all layers.  Default workload: config 3
+(LLaMA-7B-shaped full step: 32 layers, batch 4, KV length 4096, 88-node trees plus 3
+pseudo positions, bf16), the largest single-GPU configuration that is a whole step.
+
+The path does not shard (one GPU, no collectives): with --gpus N each rank runs an
+independent replica ("replicas only") and the value is the sum over ranks divided by the
+slowest rank's time.
+
+--impl reference times the CPU oracle (plain fp64 C) on the host cores on a bounded sample
+of the same workload; it is a deliberately slow baseline, not a target.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "tree_verify_step_hbm_gbs"
+UNIT = "GB/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4"])
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling small cases)")
+    ap.add_argument("--kv", type=int, default=0, help="override the KV length of c3 (profiling small cases)")
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--simt", action="store_true", help="force the fp32-ALU attention kernel")
+    ap.add_argument("--no-extras", action="store_true", help="skip e2e, cpu baseline and per-kernel timing")
+    return ap.parse_args()
+
+
+def make_workload(args):
+    from paper_2404_12022_b200 import workloads as wl
+    if args.workload == "c2":
+        return wl.config_c2()
+    if args.workload == "c4":
+        return wl.config_c4()
+    kw = {}
+    if args.layers:
+        kw["layers"] = args.layers
+    if args.kv:
+        kw["kv"] = args.kv
+    return wl.config_c3(**kw)
+
+
+def workload_config(w, n_gpus):
+    return {"workload": w.name, "layers": w.layers, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv,
+            "head_dim": w.D, "kv_len": (w.kv_len[0] if len(set(w.kv_len)) == 1 else "ragged %d..%d" % (min(w.kv_len), max(w.kv_len))),
+            "tree_nodes": w.T, "pseudo_rows": w.P, "hidden": w.d, "transfer_steps": w.k, "vocab": w.V,
+            "parallelism": "replicas x%d" % n_gpus if n_gpus > 1 else "single GPU",
+            "l2_policy": "inputs larger than L2 (KV cache of a step >> 126 MB)"}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle sample (reference arm and cpu_baseline leg)
+# ------------------------------------------------------------------------------------------
+
+class OracleSample:
+    """A bounded sample of the step for the CPU oracle: attention on a few (sequence, KV head)
+    units of one post-transfer layer, the transfer projection, verification of all logits and
+    compaction of one layer.  Inputs are the workload's own values, regenerated on the host."""
+
+    def __init__(self, w, n_units=16):
+        import dataclasses
+        import numpy as np
+        from oracle import ht_oracle
+        from paper_2404_12022_b200 import workloads as wl
+        self.np, self.oracle, self.w = np, ht_oracle, w
+        ht_oracle.build()
+        layer = w.layers - 1
+        inp = wl.make_inputs(w, "cpu", layers=[layer])
+        self.inp = inp
+        f = lambda t: t.float().numpy()
+        rng = np.random.default_rng(0)
+        units = sorted({(int(rng.integers(w.B)), int(rng.integers(w.Hkv))) for _ in range(4 * n_units)})[:n_units]
+        g = w.Hq // w.Hkv
+        self.units = []
+        for b, hk in units:
+            L = w.kv_len[b]
+            self.units.append((f(inp.q[0][b:b + 1, :, hk * g:(hk + 1) * g]), f(inp.k_cache[0, b:b + 1, hk:hk + 1, :L + w.N]),
+                               f(inp.v_cache[0, b:b + 1, hk:hk + 1, :L + w.N]), np.array([L], np.int32),
+                               inp.parent[b:b + 1].numpy()))
+        self.h, self.W = f(inp.h_src), f(inp.W)
+        self.logits = f(inp.logits)
+        self.tokens, self.parent = inp.tokens.numpy(), inp.parent.numpy()
+        self.root_pred = None if inp.root_pred is None else inp.root_pred.numpy()
+        self.kview = inp.k_cache.view(torch_int_view(inp.k_cache)).numpy()
+        self.vview = inp.v_cache.view(torch_int_view(inp.v_cache)).numpy()
+        e = w.elem_bytes()
+        attn_bytes = sum(2 * (int(u[3][0]) + w.N) * w.D * e + 2 * w.N * g * w.D * e for u in self.units)
+        self.bytes = (attn_bytes + w.k * w.d * w.d * e + w.B * w.N * w.V * e +
+                      4 * sum(inp.want_len) * w.Hkv * w.D * e)
+        self.describe = ("attention on %d of %d (sequence, KV head) units of one layer, the transfer projection, "
+                         "verification of all logits, compaction of one layer" % (len(self.units), w.B * w.Hkv))
+
+    def run(self):
+        o = self.oracle
+        for q, k, v, L, par in self.units:
+            o.tree_attention(q, k, v, L, par)
+        o.transfer(self.h, self.W)
+        pred, alen, apath, nxt, st = o.verify_greedy(self.logits, self.tokens, self.parent, self.root_pred,
+                                                     self.w.max_path)
+        o.kv_compact(self.kview, self.vview, self.w.N, self.np.array(self.w.kv_len, self.np.int32), alen, apath)
+
+
+def torch_int_view(t):
+    import torch
+    return torch.int32 if t.dtype == torch.float32 else torch.int16
+
+
+def time_oracle(sample, steps, warmup, budget_s=None):
+    for _ in range(warmup):
+        sample.run()
+    t0 = time.perf_counter()
+    done = 0
+    for _ in range(steps):
+        sample.run()
+        done += 1
+        if budget_s is not None and time.perf_counter() - t0 > budget_s:
+            break
+    dt = (time.perf_counter() - t0) / done
+    return dt, done
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import ht_oracle
+    w = make_workload(args)
+    sample = OracleSample(w)
+    dt, done = time_oracle(sample, args.steps, args.warmup)
+    value = sample.bytes / dt / 1e9
+    cores = ht_oracle.num_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": done, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w, 1),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample.describe},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+# Native arm
+# ------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        import torch
+        self.proc = None
+        try:
+            uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", uuid, "--query-gpu=" + self.QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in out.strip().splitlines():
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def run_native(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2404_12022_b200 import binding as hb
+    from paper_2404_12022_b200 import workloads as wl
+    from paper_2404_12022_b200.step import VerifyStep
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    w = make_workload(args)
+    inp = wl.make_inputs(w, "cuda")
+    step = VerifyStep(inp, num_splits=args.splits, flags=hb.HT_ATTN_FORCE_SIMT if args.simt else 0)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step.run(stream)
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step.run(stream)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    step_bytes = step.step_bytes()
+    value = world * step_bytes / (ms_step * 1e-3) / 1e9
+
+    # correctness of what was just timed: status words and the seeded accepted lengths
+    assert int(step.attn_status.abs().sum()) == 0 and int(step.verify_status.abs().sum()) == 0
+    assert step.accept_len.cpu().tolist() == inp.want_len, "accepted lengths differ from the seeded ones"
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": w.dtype, "data": "synthetic", "config": workload_config(w, world),
+            "step_us": ms_step * 1e3, "step_bytes": step_bytes, "clocks": clocks}
+    # launches of this library's kernels per step: attention (+ combine when split), transfer
+    # (one per batch slice of 8), argmax + acceptance, compaction
+    attn_launches = sum(1 for _ in range(step.layers))
+    line["gpu_launches"] = args.steps * (attn_launches * kernels_per_attention(step) + ((w.B + 7) // 8) + 2 + 1)
+
+    if rank == 0 and not args.no_extras:
+        line["roofline"], line["kernels"] = per_kernel_pass(args, step, stream, torch)
+        line["e2e"] = e2e_pass(args, step, inp, torch, world)
+        sample = OracleSample(w)
+        dt, done = time_oracle(sample, 1000, 0, budget_s=12.0)
+        from oracle import ht_oracle
+        line["cpu_baseline"] = {"value": sample.bytes / dt / 1e9, "unit": UNIT, "cores": ht_oracle.num_threads(),
+                                "kind": "oracle", "sample": sample.describe + " (%d passes, %.2f s each)" % (done, dt)}
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
+def kernels_per_attention(step):
+    return 2 if step.ws_bytes > 0 else 1
+
+
+def per_kernel_pass(args, step, stream, torch):
+    """Same steps again with CUDA events around every library call, on the launching stream."""
+    n = min(args.steps, 10)
+    names = ["attention", "transfer", "verify", "compact"]
+    ev = {k: [] for k in names}
+
+    def pair():
+        return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    for _ in range(n):
+        for i in range(step.layers):
+            if i == step.transfer_at:
+                a, b = pair(); a.record(); step.transfer(stream); b.record(); ev["transfer"].append((a, b))
+            a, b = pair(); a.record(); step.attention(i, stream); b.record(); ev["attention"].append((a, b, i))
+        if step.transfer_at >= step.layers:
+            a, b = pair(); a.record(); step.transfer(stream); b.record(); ev["transfer"].append((a, b))
+        a, b = pair(); a.record(); step.verify(stream); b.record(); ev["verify"].append((a, b))
+        a, b = pair(); a.record(); step.compact(stream); b.record(); ev["compact"].append((a, b))
+    torch.cuda.synchronize()
+    tot = {k: sum(x[0].elapsed_time(x[1]) for x in v) for k, v in ev.items()}
+    all_ms = sum(tot.values())
+    attn_ms = tot["attention"] / len(ev["attention"])
+    attn_bytes = sum(step.attention_bytes(x[2]) for x in ev["attention"]) / len(ev["attention"])
+    attn_flops = sum(step.attention_flops(x[2]) for x in ev["attention"]) / len(ev["attention"])
+    peak, how = measured_peaks()
+    achieved = attn_bytes / (attn_ms * 1e-3) / 1e9
+    roofline = {"kernel": "ht_tree_attention", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "frac_of_nominal_8tbs": achieved / 8000.0, "peak_source": how,
+                "traffic": None, "bytes_per_launch": attn_bytes, "us_per_launch": attn_ms * 1e3,
+                "tflops": attn_flops / (attn_ms * 1e-3) / 1e12}
+    bytes_of = {"transfer": step.transfer_bytes(), "verify": step.verify_bytes(), "compact": step.compact_bytes()}
+    kernels = {"attention": {"us": attn_ms * 1e3, "share": tot["attention"] / all_ms, "gbs": achieved}}
+    for k in ("transfer", "verify", "compact"):
+        us = tot[k] / len(ev[k]) * 1e3
+        kernels[k] = {"us": us, "share": tot[k] / all_ms, "gbs": bytes_of[k] / (us * 1e-6) / 1e9}
+    return roofline, kernels
+
+
+def e2e_pass(args, step, inp, torch, world):
+    """The same step with its per-step inputs arriving from pinned host memory and its results
+    read back: q of every layer, the new K/V rows of the tree, logits, tree structure and the
+    source hidden state go host -> device; attention outputs, pseudo hidden states and the
+    acceptance results come back.  The KV cache and the transfer weights are resident state."""
+    w = step.w
+    n = min(args.steps, 5)
+    dev = inp.k_cache.device
+    pin = lambda t: t.cpu().pin_memory()
+    host_q = [pin(q) for q in inp.q]
+    L = torch.tensor(w.kv_len, device=dev)
+    idx = (L[:, None] + torch.arange(w.N, device=dev)[None]).long()          # [B, N] cache rows of the tree
+    gather = lambda c: torch.stack([c[:, b][:, :, idx[b]] for b in range(w.B)], 1)   # [layers, B, Hkv, N, D]
+    host_k, host_v = pin(gather(inp.k_cache)), pin(gather(inp.v_cache))
+    host_small = [pin(t) for t in (inp.logits, inp.parent, inp.parent_tree, inp.tokens, inp.h_src, inp.kv_len)]
+    host_rp = pin(inp.root_pred) if inp.root_pred is not None else None
+    dev_k, dev_v = torch.empty_like(host_k, device=dev), torch.empty_like(host_v, device=dev)
+    small_targets = [inp.logits, inp.parent, inp.parent_tree, inp.tokens, inp.h_src, inp.kv_len]
+    host_out = [torch.empty_like(o, device="cpu").pin_memory() for o in step.outs]
+    host_res = [torch.empty_like(t, device="cpu").pin_memory() for t in
+                (step.pseudo, step.pred, step.accept_len, step.accept_path, step.next_token, step.new_kv_len)]
+    res_src = [step.pseudo, step.pred, step.accept_len, step.accept_path, step.next_token, step.new_kv_len]
+    h2d = sum(t.numel() * t.element_size() for t in host_q + [host_k, host_v] + host_small + ([host_rp] if host_rp is not None else []))
+    d2h = sum(t.numel() * t.element_size() for t in host_out + host_res)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def one():
+        for q, hq in zip(inp.q, host_q):
+            q.copy_(hq, non_blocking=True)
+        dev_k.copy_(host_k, non_blocking=True)
+        dev_v.copy_(host_v, non_blocking=True)
+        for b in range(w.B):                                   # new K/V rows into the cache tail
+            inp.k_cache[:, b, :, w.kv_len[b]:w.kv_len[b] + w.N] = dev_k[:, b]
+            inp.v_cache[:, b, :, w.kv_len[b]:w.kv_len[b] + w.N] = dev_v[:, b]
+        for t, h in zip(small_targets, host_small):
+            t.copy_(h, non_blocking=True)
+        if host_rp is not None:
+            inp.root_pred.copy_(host_rp, non_blocking=True)
+        step.run(stream)
+        for o, h in zip(step.outs, host_out):
+            h.copy_(o, non_blocking=True)
+        for s, h in zip(res_src, host_res):
+            h.copy_(s, non_blocking=True)
+        torch.cuda.synchronize()
+
+    one()
+    one()
+    t0 = time.perf_counter()
+    for _ in range(n):
+        one()
+    dt = (time.perf_counter() - t0) / n
+    return {"value": world * step.step_bytes() / dt / 1e9, "unit": UNIT, "ms_per_step": dt * 1e3,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "note": "KV cache and transfer weights resident; per-step inputs from pinned host memory"}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_native(args)
+
+
+if __name__ == "__main__":
+    main()
