@@ -168,6 +168,31 @@ int ht_kv_compact(void *k_cache, void *v_cache, const ht_cache_desc *desc /* hos
                   const int32_t *kv_len, const int32_t *accept_len, const int32_t *accept_path,
                   int max_path, int32_t *new_kv_len, int32_t *status, void *stream);
 
+/*
+ * Tree attention without a caller-provided workspace.  (The paper has no counterpart: this
+ * entry point exists for integration, not for the method.)
+ *
+ * Same operation, arguments and results as ht_tree_attention, computed by the split-KV
+ * fp32-ALU kernel, for callers that cannot give the library scratch memory because they
+ * cannot allocate any: code running where cudaMalloc must not be called, plugin
+ * interfaces that pass only inputs and outputs, processes whose device memory is fully
+ * committed.  The split partials live in a fixed array of HT_STATIC_SCRATCH_BYTES inside
+ * the library image; every GPU context that loads the library holds that array until it
+ * exits, used or not.  The call allocates and frees nothing.
+ *   - A problem whose partials exceed the array is refused with HT_ERR_WORKSPACE and a
+ *     message giving both sizes; desc->num_splits = 1 never needs scratch.
+ *   - The first call on each device looks up the array's device address (with the caller's
+ *     current device, which must be the one the pointers and the stream belong to).  Make
+ *     that first call outside any stream capture.
+ *   - All calls share the array and it keeps the previous call's contents.  Nothing in it
+ *     needs clearing, but calls that overlap on the GPU (two streams, two host threads)
+ *     race on it: serialise them.
+ */
+#define HT_STATIC_SCRATCH_BYTES (16u << 20)
+int ht_tree_attention_static(const ht_attn_desc *desc /* host */, const void *q, const void *k_cache,
+                             const void *v_cache, const int32_t *kv_len, const int32_t *parent,
+                             void *out, int32_t *status, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,8 @@ HT_STATUS_OK, HT_STATUS_BAD_TREE, HT_STATUS_BAD_LEN, HT_STATUS_BAD_PATH, HT_STAT
 HT_ATTN_FORCE_SIMT = 1
 
 EXPORTS = ("ht_version", "ht_last_error_string", "ht_transfer", "ht_tree_attention_workspace",
-           "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact")
+           "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact", "ht_tree_attention_static")
+HT_STATIC_SCRATCH_BYTES = 16 << 20
 
 _DTYPES = {torch.float32: HT_F32, torch.float16: HT_F16, torch.bfloat16: HT_BF16}
 
@@ -70,6 +71,8 @@ def load() -> ctypes.CDLL:
         lib.ht_tree_attention_workspace.argtypes = [ctypes.POINTER(AttnDesc)]
         lib.ht_tree_attention.restype = i32
         lib.ht_tree_attention.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        lib.ht_tree_attention_static.restype = i32
+        lib.ht_tree_attention_static.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.ht_verify_greedy.restype = i32
         lib.ht_verify_greedy.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         lib.ht_kv_compact.restype = i32
@@ -157,6 +160,25 @@ def tree_attention(q, k_cache, v_cache, kv_len, parent, out=None, workspace=None
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(load().ht_tree_attention(ctypes.byref(desc), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(kv_len),
                                     _ptr(parent), _ptr(out), _ptr(workspace), ws_bytes, _ptr(status), _stream()))
+    return out, status
+
+
+def tree_attention_static(q, k_cache, v_cache, kv_len, parent, out=None, status=None, scale: float = 0.0,
+                          num_splits: int = 0):
+    """Tree attention for callers that cannot allocate scratch: same results as
+    ``tree_attention``, with the split partials in the library's built-in array (at most
+    ``HT_STATIC_SCRATCH_BYTES``; larger problems raise).  Calls must not overlap on the GPU.
+    ``out`` and ``status`` may be passed in so that the call itself allocates nothing."""
+    _need(q, name="q")
+    _need(kv_len, torch.int32, "kv_len")
+    _need(parent, torch.int32, "parent")
+    desc = make_attn_desc(q, k_cache, scale, num_splits, 0)
+    if out is None:
+        out = torch.empty_like(q)
+    if status is None:
+        status = torch.empty(desc.B, dtype=torch.int32, device=q.device)
+    _check(load().ht_tree_attention_static(ctypes.byref(desc), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(kv_len),
+                                           _ptr(parent), _ptr(out), _ptr(status), _stream()))
     return out, status
 
 

@@ -26,7 +26,7 @@ int check_launch(const char *what) {
     return HT_OK;
 }
 
-static int check_attn_desc(const ht_attn_desc *d) {
+int check_attn_desc(const ht_attn_desc *d) {
     if (!d) return fail(HT_ERR_INVALID_ARG, "desc is NULL");
     if (d->B < 0 || d->N < 0) return fail(HT_ERR_INVALID_ARG, "negative B or N");
     if (d->Hq <= 0 || d->Hkv <= 0 || d->Hq % d->Hkv != 0)

@@ -12,6 +12,9 @@ namespace ht {
 // Records a message for ht_last_error_string() and returns `code`.
 int fail(int code, const char *fmt, ...);
 
+// Host-side checks of an attention descriptor (sizes, dtype, strides).
+int check_attn_desc(const ht_attn_desc *d);
+
 // Checks the launch status of the kernel just enqueued.
 int check_launch(const char *what);
 
