@@ -73,6 +73,7 @@ size_t ht_tree_attention_workspace(const ht_attn_desc *desc) {
     if (check_attn_desc(desc) != HT_OK) return 0;
     if (desc->B == 0 || desc->N == 0) return 0;
     size_t need = attn_simt_workspace(*desc, nullptr);
+    if (attn_tc_applicable(*desc)) need = attn_tc_workspace(*desc) > need ? attn_tc_workspace(*desc) : need;
     return (need + 255) / 256 * 256;
 }
 
@@ -90,6 +91,9 @@ int ht_tree_attention(const ht_attn_desc *desc, const void *q, const void *k_cac
     const size_t need = ht_tree_attention_workspace(desc);
     if (need > 0 && (!workspace || workspace_bytes < need))
         return fail(HT_ERR_WORKSPACE, "workspace holds %zu bytes, %zu needed", workspace ? workspace_bytes : 0, need);
+    if (attn_tc_applicable(*desc))
+        return launch_attn_tc(*desc, q, k_cache, v_cache, kv_len, parent, out, workspace, workspace_bytes, status,
+                              static_cast<cudaStream_t>(stream));
     return launch_attn_simt(*desc, q, k_cache, v_cache, kv_len, parent, out, workspace, workspace_bytes,
                             status, static_cast<cudaStream_t>(stream));
 }

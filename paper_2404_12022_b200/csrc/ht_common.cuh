@@ -74,6 +74,10 @@ size_t attn_simt_workspace(const ht_attn_desc &d, int *splits_out);
 int launch_attn_simt(const ht_attn_desc &d, const void *q, const void *kc, const void *vc,
                      const int32_t *kv_len, const int32_t *parent, void *out, void *ws, size_t ws_bytes,
                      int32_t *status, cudaStream_t s);
+bool attn_tc_applicable(const ht_attn_desc &d);
+size_t attn_tc_workspace(const ht_attn_desc &d);
+int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const void *vc, const int32_t *kv_len,
+                   const int32_t *parent, void *out, void *ws, size_t ws_bytes, int32_t *status, cudaStream_t s);
 int launch_verify(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
                   const int32_t *root_pred, int B, int N, int T, int V, int max_path, int32_t *pred,
                   int32_t *accept_len, int32_t *accept_path, int32_t *next_token, int32_t *status,
