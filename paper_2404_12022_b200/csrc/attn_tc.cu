@@ -168,6 +168,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t *r) {
           "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
           "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ float ex2(float x) {             // 2^x, -inf -> 0
@@ -408,7 +416,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const int node = sg.rt * p.rows_per_tile_nodes + row / p.g;
             if (s == 0) {
                 const bool real = node < p.N;
-                for (int w = 0; w < words; ++w) sm.anc[w][row] = real ? 0u : 0xFFFFFFFFu;
+                for (int w = 0; w < words; ++w) sm.anc[w][row] = 0u;   // padding rows see the context only; their results are dropped
                 if (real)
                     for (int c = node; c >= 0; c = sm.parent[c]) sm.anc[c >> 5][row] |= 1u << (c & 31);
             }
@@ -422,24 +430,45 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int kt = sg.kt0 + i;
                 mbar_wait(&sm.s_full[s], (jj >> 1) & 1, abort_flag);
                 tc_fence_after();
-                float x[kTile];
                 const uint32_t s_addr = tmem + lane_base + s * 128;
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) tmem_ld32(s_addr + c4 * 32, x + c4 * 32);
-                tmem_ld_wait();
                 const int tile_lo = kt * kTile;
-                if (tile_lo + kTile > L) {             // reaches into the tree rows / the tail
+                const bool boundary = tile_lo + kTile > L;   // reaches into the tree rows / the tail
+                // Visibility of this tile's 128 keys for this row, one bit per key: context keys are
+                // visible, tree key c iff bit c of the row's ancestor words, the tail never.
+                uint32_t vis[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+                if (boundary) {
 #pragma unroll
-                    for (int c = 0; c < kTile; ++c) {
-                        const int cc = tile_lo + c - L;
-                        bool vis = cc < 0;
-                        if (cc >= 0 && cc < p.N) vis = (sm.anc[cc >> 5][row] >> (cc & 31)) & 1u;
-                        x[c] = vis ? x[c] : -INFINITY;
+                    for (int w = 0; w < 4; ++w) {
+                        const int cc0 = tile_lo + 32 * w - L;           // tree index of the word's first key
+                        if (cc0 > -32) {
+                            const int wi = cc0 >> 5, sh = cc0 & 31;     // arithmetic shift: -1 for cc0 in (-32, 0)
+                            const uint32_t lo = wi < 0 ? 0xFFFFFFFFu : (wi < words ? sm.anc[wi][row] : 0u);
+                            const uint32_t hi = wi + 1 < words ? sm.anc[wi + 1][row] : 0u;
+                            vis[w] = __funnelshift_r(lo, hi, sh);
+                        }
                     }
                 }
-                float mx = x[0];
+                // --- pass 1: row maximum over the visible keys, 32 scores at a time ---
+                float xa[32], xb[32];
+                float mx = -INFINITY;
+                tmem_ld32(s_addr, xa);
 #pragma unroll
-                for (int c = 1; c < kTile; ++c) mx = fmaxf(mx, x[c]);
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    float *cur = (c4 & 1) ? xb : xa, *nxt = (c4 & 1) ? xa : xb;
+                    tmem_ld_wait();
+                    tmem_ld32(s_addr + ((c4 + 1) & 3) * 32, nxt);   // after the last chunk: chunk 0 again, for pass 2
+                    if (boundary) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) cur[c] = ((vis[c4] >> c) & 1u) ? cur[c] : -INFINITY;
+                    }
+                    float m0 = fmaxf(cur[0], cur[1]), m1 = fmaxf(cur[2], cur[3]);
+#pragma unroll
+                    for (int c = 4; c < 32; c += 4) {
+                        m0 = fmaxf(m0, fmaxf(cur[c], cur[c + 1]));
+                        m1 = fmaxf(m1, fmaxf(cur[c + 2], cur[c + 3]));
+                    }
+                    mx = fmaxf(mx, fmaxf(m0, m1));
+                }
                 mx *= p.scale_log2;                    // scale > 0: max commutes with scaling
                 // --- running maximum, raised lazily ---
                 const float m_new = fmaxf(m_ref, mx);
@@ -450,14 +479,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     // (the tensor pipe runs in issue order), so its accumulator may be rescaled here.
                     const float f = grow ? exp2f(m_ref - m_new) : 1.f;
                     const uint32_t o_addr = tmem + lane_base + 256 + s * 128;
+                    tmem_ld_wait();                    // the prefetched chunk lands in xa before xb is reused
 #pragma unroll
                     for (int c4 = 0; c4 < 4; ++c4) {
-                        float o[32];
                         uint32_t r[32];
-                        tmem_ld32(o_addr + c4 * 32, o);
+                        tmem_ld32(o_addr + c4 * 32, xb);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(o[c] * f);
+                        for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(xb[c] * f);
                         tmem_st32(o_addr + c4 * 32, r);
                     }
                     tmem_st_wait();
@@ -465,21 +494,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     if (grow) m_ref = m_new;
                 }
                 const float base = (m_ref == -INFINITY) ? 0.f : m_ref;
-                // --- exponentials, row sum, P to TMEM as packed 16-bit pairs ---
-                float acc = 0.f;
+                // --- pass 2: exponentials, row sum, P to TMEM as packed 16-bit pairs.  P chunk c4 lands
+                // in columns [16 c4, 16 c4 + 16), which hold scores already consumed. ---
+                float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
-                for (int c4 = 0; c4 < 2; ++c4) {
-                    uint32_t r[32];
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    float *cur = (c4 & 1) ? xb : xa, *nxt = (c4 & 1) ? xa : xb;
+                    tmem_ld_wait();
+                    if (c4 < 3) tmem_ld32(s_addr + (c4 + 1) * 32, nxt);
+                    uint32_t r[16];
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float p0 = ex2(fmaf(x[c4 * 64 + 2 * c], p.scale_log2, -base));
-                        const float p1 = ex2(fmaf(x[c4 * 64 + 2 * c + 1], p.scale_log2, -base));
-                        acc += p0 + p1;
+                    for (int c = 0; c < 16; ++c) {
+                        float p0 = ex2(fmaf(cur[2 * c], p.scale_log2, -base));
+                        float p1 = ex2(fmaf(cur[2 * c + 1], p.scale_log2, -base));
+                        if (boundary) {
+                            p0 = ((vis[c4] >> (2 * c)) & 1u) ? p0 : 0.f;
+                            p1 = ((vis[c4] >> (2 * c + 1)) & 1u) ? p1 : 0.f;
+                        }
+                        acc0 += p0;
+                        acc1 += p1;
                         r[c] = pack2<kBf16>(p0, p1);
                     }
-                    tmem_st32(s_addr + c4 * 32, r);
+                    tmem_st16(s_addr + c4 * 16, r);
                 }
-                l_sum += acc;
+                l_sum += acc0 + acc1;
                 tmem_st_wait();
                 // --- last tile of the unit: rows of V past the tree are not data; make them zero ---
                 if (kt == sg.nkt - 1) {
