@@ -29,8 +29,9 @@
 //                        that reach past the context length are masked.
 //   work split         : all (sequence, KV head, row tile) units are laid end to end as
 //                        a list of 128-key tiles; CTA i takes tiles [i*per, (i+1)*per).  A
-//                        unit that is cut writes (m, l, O) partials to the workspace and a
-//                        second small kernel merges them -- nobody waits on another CTA.
+//                        unit that is cut writes (m, l, O) partials to the workspace and
+//                        takes a ticket; the CTA that delivers the last part of a unit
+//                        merges all parts -- nobody waits on another CTA.
 //
 // Every wait on an mbarrier is bounded; when one runs out the CTA raises an abort flag,
 // reports HT_STATUS_TIMEOUT, runs to the end of its control flow without further waiting,
@@ -51,7 +52,7 @@ constexpr int kSlabBytes = kEntryBytes / 2;   // [128 rows][64 elements] = 16 Ki
 constexpr int kThreads = 320;
 constexpr int kMaxB = 256;
 constexpr int kMaxWords = 16;              // ancestor words per row -> N <= 512
-constexpr int kPartStride = 132;           // floats per partial row: O[128], m, l, pad
+constexpr int kSlotFloats = kRows * kD + 2 * kRows;   // one partial result: O as [32 feature groups][128 rows][4], m[128], l[128]
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;  // log2 domain
 
@@ -59,12 +60,25 @@ struct Params {
     const int32_t *kv_len, *parent;
     int32_t *status;
     void *out;
-    float *part;
+    float *part;           // partial results of cut units: [grid][2][kSlotFloats]
+    unsigned int *tickets; // one arrival counter per unit, zero on entry
     int B, N, Hq, Hkv, g, cap, n_rt, rows_per_tile_nodes;   // rows_per_tile_nodes = 128 / g
     float scale_log2;
     int is_bf16;
     int grid;
+#ifdef HT_TC_TRACE
+    long long *trace;
+#endif
 };
+
+// Optional timeline of one CTA (clock64 stamps per role / tile / event) for tuning builds.
+#ifdef HT_TC_TRACE
+#define HT_TR(role, j, ev) do { if (p.trace && blockIdx.x == HT_TC_TRACE && (threadIdx.x & 31) == 0 && ((role) < 2 || (threadIdx.x & 127) == 0) && (j) < 40) p.trace[((role) * 40 + (j)) * 4 + (ev)] = clock64(); } while (0)
+#define HT_TR_CTA(ev) do { if (p.trace && (threadIdx.x & 31) == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); p.trace[1000 + blockIdx.x * 4 + (ev)] = (long long)gt; } } while (0)
+#else
+#define HT_TR(role, j, ev) do { } while (0)
+#define HT_TR_CTA(ev) do { } while (0)
+#endif
 
 struct __align__(1024) Smem {
     unsigned char q[kEntryBytes];
@@ -78,7 +92,8 @@ struct __align__(1024) Smem {
     unsigned long long kv_full[kStages], kv_empty[kStages], q_full, q_empty, s_full[2], p_ready[2], o_done[2], mma_drain;
     uint32_t tmem_base;
     int abort;
-    int bad;
+    int merge_here[2];
+    int direct;
 };
 
 // ---------------------------------------------------------------------------------------
@@ -184,6 +199,37 @@ __device__ __forceinline__ float ex2(float x) {             // 2^x, -inf -> 0
     return y;
 }
 
+
+__device__ __forceinline__ unsigned int ld_relaxed_gpu(const unsigned int *ptr) {
+    unsigned int v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// Two fp32 values in one 64-bit register, for the paired fp32 instructions.
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+    unsigned long long d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
 __device__ __forceinline__ void softmax_groups_sync() {   // the 256 softmax threads
     asm volatile("bar.sync 1, 256;" ::: "memory");
 }
@@ -225,10 +271,34 @@ __device__ __forceinline__ Segment locate(const int32_t *pre, const int32_t *nkt
 
 __device__ __forceinline__ int tiles_per_cta(int total, int grid) { return (total + grid - 1) / grid; }
 
+// Tiles per CTA.  An even share cuts nearly every unit in two, and every cut costs a partial
+// result in the workspace and a merge at the end.  While the cache is streamed at memory speed a
+// few idle SMs cost less than that, so when all sequences are equally long and some whole
+// multiple or whole fraction of a unit lies within 20 % above the even share, ranges of that
+// length are used and cuts fall on unit boundaries (or, for fractions, near them).
+__device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nkt, int B) {
+    const int even = tiles_per_cta(total, grid);
+    int n = 0;
+    for (int b = 0; b < B; ++b) {
+        if (nkt[b] == 0) continue;
+        if (n != 0 && nkt[b] != n) return even;
+        n = nkt[b];
+    }
+    if (n == 0 || even == 0) return even;
+    int cand;
+    if (n >= even) {
+        const int k = n / even;                       // largest count of parts whose length is >= even
+        cand = (n + k - 1) / k;
+    } else {
+        cand = (even + n - 1) / n * n;                // whole units
+    }
+    return (cand * 5 <= even * 6) ? cand : even;
+}
+
 // Validates every sequence and fills len / nkt / pre.  Called by all threads of a block.
 template <int NT>
 __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, int32_t *s_nkt, int32_t *s_pre,
-                                               int *s_bad_scratch, bool write_status) {
+                                               bool write_status) {
     for (int b = threadIdx.x; b < p.B; b += NT) s_nkt[b] = 0;       // 0 = legal so far
     __syncthreads();
     for (int i = threadIdx.x; i < p.B * p.N; i += NT) {
@@ -256,7 +326,6 @@ __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, 
         s_pre[p.B] = acc;
     }
     __syncthreads();
-    (void)s_bad_scratch;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -273,6 +342,56 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     }
 }
 
+// A unit that was cut between CTAs: which one, and which CTAs hold its parts.
+struct CutUnit {
+    int valid, unit, b, hk, rt, t0, c_lo, c_hi;
+};
+
+// Merge of the parts of a cut unit by the 256 softmax threads of the CTA that delivered the
+// last part.  Threads r and r + 128 own query row r, 64 features each; a warp reads 32
+// consecutive rows of one feature group at a time (contiguous in the part's layout), and the
+// loads of a part are independent of one another so that one round trip to L2 fetches it.
+template <bool kBf16>
+__device__ __noinline__ void merge_parts(const Params &p, const CutUnit &cu, int per, int tid256) {
+    const int row = tid256 & 127, half = tid256 >> 7;
+    const int node = cu.rt * p.rows_per_tile_nodes + row / p.g;
+    if (node >= p.N) return;
+    const int head = cu.hk * p.g + row % p.g;
+    float M = -INFINITY, l = 0.f;
+    float acc[64];
+#pragma unroll
+    for (int x = 0; x < 64; ++x) acc[x] = 0.f;
+#pragma unroll 1
+    for (int c = cu.c_lo; c <= cu.c_hi; ++c) {
+        const int slot = 2 * c + ((max(cu.t0, c * per) == c * per) ? 0 : 1);
+        const float *pslot = p.part + (size_t)slot * kSlotFloats;
+        const float m = __ldcg(pslot + kRows * kD + row), lp = __ldcg(pslot + kRows * kD + kRows + row);
+        float4 v[16];
+#pragma unroll
+        for (int x = 0; x < 16; ++x) v[x] = __ldcg(reinterpret_cast<const float4 *>(pslot) + (half * 16 + x) * kRows + row);
+        const float Mn = fmaxf(M, m);
+        const float fa = (M == -INFINITY) ? 0.f : exp2f(M - Mn);
+        const float fb = (m == -INFINITY) ? 0.f : exp2f(m - Mn);
+        l = l * fa + lp * fb;
+#pragma unroll
+        for (int x = 0; x < 16; ++x) {
+            acc[4 * x] = acc[4 * x] * fa + v[x].x * fb;
+            acc[4 * x + 1] = acc[4 * x + 1] * fa + v[x].y * fb;
+            acc[4 * x + 2] = acc[4 * x + 2] * fa + v[x].z * fb;
+            acc[4 * x + 3] = acc[4 * x + 3] * fa + v[x].w * fb;
+        }
+        M = Mn;
+    }
+    const float inv = 1.f / l;
+    unsigned char *dst = static_cast<unsigned char *>(p.out) +
+                         ((((size_t)cu.b * p.N + node) * p.Hq + head) * kD + half * 64) * 2;
+#pragma unroll
+    for (int x = 0; x < 8; ++x)
+        *reinterpret_cast<uint4 *>(dst + x * 16) =
+            make_uint4(pack2<kBf16>(acc[8 * x] * inv, acc[8 * x + 1] * inv), pack2<kBf16>(acc[8 * x + 2] * inv, acc[8 * x + 3] * inv),
+                       pack2<kBf16>(acc[8 * x + 4] * inv, acc[8 * x + 5] * inv), pack2<kBf16>(acc[8 * x + 6] * inv, acc[8 * x + 7] * inv));
+}
+
 template <bool kBf16>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -281,6 +400,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &sm.abort;
+    if (threadIdx.x == 0) HT_TR_CTA(0);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&sm.kv_full[i], 1); mbar_init(&sm.kv_empty[i], 1); }
@@ -295,14 +415,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, &sm.bad, blockIdx.x == 0);
+    plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
 
     const int total = sm.pre[p.B];
-    const int per = tiles_per_cta(total, p.grid);
+    const int per = choose_per(total, p.grid, sm.nkt, p.B);
     const int t_begin = min((int)blockIdx.x * per, total);
     const int t_end = min(t_begin + per, total);
 
@@ -310,6 +430,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // ------------------------------- TMA producer -------------------------------
         if (lane == 0) {
             int b_hint = 0, ring_i = 0, seg_i = 0;
+            HT_TR_CTA(1);
             for (int t = t_begin; t < t_end && !*abort_flag;) {
                 const Segment s = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
                 if (seg_i > 0 && !mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag)) break;
@@ -321,6 +442,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     const int kt = s.kt0 + (i >> 1);
                     const int slot = ring_i % kStages, use = ring_i / kStages;
                     if (use > 0 && !mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag)) break;
+                    HT_TR(0, ring_i >> 1, ring_i & 1);
                     const CUtensorMap *tm = (i & 1) ? &tm_v : &tm_k;
                     mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
                     tma_load_4d(sm.ring[slot], tm, &sm.kv_full[slot], 0, kt * kTile, s.hk, s.b);
@@ -347,6 +469,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             auto issue_pv = [&](int jj, int first) {
                 const int s = jj & 1;
                 mbar_wait(&sm.p_ready[s], (jj >> 1) & 1, abort_flag);
+                HT_TR(1, jj, 2);
                 const int e = 2 * jj + 1, slot = e % kStages;
                 mbar_wait(&sm.kv_full[slot], (e / kStages) & 1, abort_flag);
                 tc_fence_after();
@@ -372,6 +495,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     const int e = 2 * j, slot = e % kStages;
                     mbar_wait(&sm.kv_full[slot], (e / kStages) & 1, abort_flag);
                     tc_fence_after();
+                    HT_TR(1, j, 0);
                     if (!*abort_flag) {
                         const uint32_t k_addr = smem_u32(sm.ring[slot]);
 #pragma unroll
@@ -404,72 +528,111 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int row = threadIdx.x & 127;             // query row within the tile = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const int tid256 = threadIdx.x;                // 0..255 among the softmax threads
-        int b_hint = 0, J = 0, cta_seg = 0;
+        const int words = (p.N + 31) >> 5;
+        const unsigned long long scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+        int b_hint = 0, J = 0;
+        float xa_e[32], xb_e[32];
+        CutUnit cut[2];
+        unsigned int ticket[2] = {0u, 0u};
+        cut[0].valid = cut[1].valid = 0;
+        int anc_b = -1, anc_rt = -1;           // sequence / row tile the ancestor words were built for
         for (int t = t_begin; t < t_end;) {
             const Segment sg = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
             const int L = sm.len[sg.b];
-            const int words = (p.N + 31) >> 5;
-            // --- ancestor masks of this tile's rows ---
-            softmax_groups_sync();                     // previous segment no longer reads parent / anc
-            for (int c = tid256; c < p.N; c += 256) sm.parent[c] = p.parent[(size_t)sg.b * p.N + c];
-            softmax_groups_sync();
+            // --- ancestor masks of this tile's rows (kept while sequence and row tile stay the same) ---
             const int node = sg.rt * p.rows_per_tile_nodes + row / p.g;
-            if (s == 0) {
-                const bool real = node < p.N;
-                for (int w = 0; w < words; ++w) sm.anc[w][row] = 0u;   // padding rows see the context only; their results are dropped
-                if (real)
-                    for (int c = node; c >= 0; c = sm.parent[c]) sm.anc[c >> 5][row] |= 1u << (c & 31);
+            const bool real = node < p.N;
+            if (sg.b != anc_b || sg.rt != anc_rt) {
+                softmax_groups_sync();                 // previous segment no longer reads parent / anc
+                for (int c = tid256; c < p.N; c += 256) sm.parent[c] = p.parent[(size_t)sg.b * p.N + c];
+                softmax_groups_sync();
+                if (s == 0) {
+                    for (int w = 0; w < words; ++w) sm.anc[w][row] = 0u;   // padding rows see the context only; their results are dropped
+                    if (real)
+                        for (int c = node; c >= 0; c = sm.parent[c]) sm.anc[c >> 5][row] |= 1u << (c & 31);
+                }
+                softmax_groups_sync();
+                anc_b = sg.b;
+                anc_rt = sg.rt;
             }
-            softmax_groups_sync();
+
+            // A segment that is only part of its unit: which CTAs hold the other parts.  How many of
+            // them have been delivered is asked anew at every tile and looked at in the epilogue, so
+            // that the answer never has to be waited for.
+            const bool complete = sg.kt0 == 0 && sg.len == sg.nkt;
+            const int cut_k = (t == t_begin) ? 0 : 1;
+            unsigned int delivered = 0, delivered_old = 0;   // newest answer, and the one before it
+            if (!complete) {
+                CutUnit &cu = cut[cut_k];
+                cu.unit = (sg.b * p.Hkv + sg.hk) * p.n_rt + sg.rt;
+                cu.b = sg.b; cu.hk = sg.hk; cu.rt = sg.rt;
+                cu.t0 = sm.pre[sg.b] + (sg.hk * p.n_rt + sg.rt) * sg.nkt;
+                cu.c_lo = cu.t0 / per;
+                cu.c_hi = (cu.t0 + sg.nkt - 1) / per;
+            }
 
             float m_ref = -INFINITY, l_sum = 0.f;
             int n_mine = 0, last_jj = 0;
+#pragma unroll 1
             for (int i = 0; i < sg.len; ++i) {
                 const int jj = J + i;
                 if ((jj & 1) != s) continue;
                 const int kt = sg.kt0 + i;
+                if (!complete && tid256 == 0) {
+                    delivered_old = delivered;
+                    delivered = ld_relaxed_gpu(&p.tickets[cut[cut_k].unit]);
+                }
+                HT_TR(2 + s, jj, 0);
                 mbar_wait(&sm.s_full[s], (jj >> 1) & 1, abort_flag);
                 tc_fence_after();
+                HT_TR(2 + s, jj, 1);
                 const uint32_t s_addr = tmem + lane_base + s * 128;
                 const int tile_lo = kt * kTile;
-                const bool boundary = tile_lo + kTile > L;   // reaches into the tree rows / the tail
-                // Visibility of this tile's 128 keys for this row, one bit per key: context keys are
-                // visible, tree key c iff bit c of the row's ancestor words, the tail never.
-                uint32_t vis[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
-                if (boundary) {
-#pragma unroll
+                float *const xa = xa_e, *const xb = xb_e;
+                if (tile_lo + kTile > L) {
+                    // The tile reaches into the tree rows / the tail: overwrite the scores of keys this
+                    // row must not see with -inf, in place, so that the two passes below need no mask.
+                    // Context keys are visible, tree key c iff bit c of the row's ancestor words, the
+                    // tail never (whatever those cache rows hold, NaN included).
+#pragma unroll 1
                     for (int w = 0; w < 4; ++w) {
                         const int cc0 = tile_lo + 32 * w - L;           // tree index of the word's first key
-                        if (cc0 > -32) {
-                            const int wi = cc0 >> 5, sh = cc0 & 31;     // arithmetic shift: -1 for cc0 in (-32, 0)
-                            const uint32_t lo = wi < 0 ? 0xFFFFFFFFu : (wi < words ? sm.anc[wi][row] : 0u);
-                            const uint32_t hi = wi + 1 < words ? sm.anc[wi + 1][row] : 0u;
-                            vis[w] = __funnelshift_r(lo, hi, sh);
-                        }
+                        if (cc0 <= -32) continue;
+                        const int wi = cc0 >> 5, sh = cc0 & 31;         // arithmetic shift: -1 for cc0 in (-32, 0)
+                        const uint32_t lo = wi < 0 ? 0xFFFFFFFFu : (wi < words ? sm.anc[wi][row] : 0u);
+                        const uint32_t hi = (wi + 1 >= 0 && wi + 1 < words) ? sm.anc[wi + 1][row] : 0u;
+                        const uint32_t vis = __funnelshift_r(lo, hi, sh);
+                        tmem_ld32(s_addr + w * 32, xa);
+                        tmem_ld_wait();
+                        uint32_t r[32];
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) r[c] = ((vis >> c) & 1u) ? __float_as_uint(xa[c]) : 0xFF800000u;
+                        tmem_st32(s_addr + w * 32, r);
                     }
+                    tmem_st_wait();
                 }
-                // --- pass 1: row maximum over the visible keys, 32 scores at a time ---
-                float xa[32], xb[32];
-                float mx = -INFINITY;
+                // --- pass 1: row maximum, 32 scores at a time, the next chunk in flight meanwhile ---
+                float mx0 = -INFINITY, mx1 = -INFINITY;
                 tmem_ld32(s_addr, xa);
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    float *cur = (c4 & 1) ? xb : xa, *nxt = (c4 & 1) ? xa : xb;
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {
                     tmem_ld_wait();
-                    tmem_ld32(s_addr + ((c4 + 1) & 3) * 32, nxt);   // after the last chunk: chunk 0 again, for pass 2
-                    if (boundary) {
+                    tmem_ld32(s_addr + (2 * h + 1) * 32, xb);
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) cur[c] = ((vis[c4] >> c) & 1u) ? cur[c] : -INFINITY;
+                    for (int c = 0; c < 32; c += 4) {
+                        mx0 = max3(mx0, xa[c], xa[c + 1]);
+                        mx1 = max3(mx1, xa[c + 2], xa[c + 3]);
                     }
-                    float m0 = fmaxf(cur[0], cur[1]), m1 = fmaxf(cur[2], cur[3]);
+                    tmem_ld_wait();
+                    tmem_ld32(s_addr + ((2 * h + 2) & 3) * 32, xa);   // after the last chunk: chunk 0 again, for pass 2
 #pragma unroll
-                    for (int c = 4; c < 32; c += 4) {
-                        m0 = fmaxf(m0, fmaxf(cur[c], cur[c + 1]));
-                        m1 = fmaxf(m1, fmaxf(cur[c + 2], cur[c + 3]));
+                    for (int c = 0; c < 32; c += 4) {
+                        mx0 = max3(mx0, xb[c], xb[c + 1]);
+                        mx1 = max3(mx1, xb[c + 2], xb[c + 3]);
                     }
-                    mx = fmaxf(mx, fmaxf(m0, m1));
                 }
-                mx *= p.scale_log2;                    // scale > 0: max commutes with scaling
+                const float mx = fmaxf(mx0, mx1) * p.scale_log2;   // scale > 0: max commutes with scaling
+                HT_TR(2 + s, jj, 2);
                 // --- running maximum, raised lazily ---
                 const float m_new = fmaxf(m_ref, mx);
                 const bool grow = (m_ref != -INFINITY) && (m_new > m_ref + kRescaleThreshold);
@@ -479,8 +642,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     // (the tensor pipe runs in issue order), so its accumulator may be rescaled here.
                     const float f = grow ? exp2f(m_ref - m_new) : 1.f;
                     const uint32_t o_addr = tmem + lane_base + 256 + s * 128;
-                    tmem_ld_wait();                    // the prefetched chunk lands in xa before xb is reused
-#pragma unroll
+                    tmem_ld_wait();                    // the prefetched chunk has landed in xa before xb is reused
+#pragma unroll 1
                     for (int c4 = 0; c4 < 4; ++c4) {
                         uint32_t r[32];
                         tmem_ld32(o_addr + c4 * 32, xb);
@@ -494,30 +657,43 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     if (grow) m_ref = m_new;
                 }
                 const float base = (m_ref == -INFINITY) ? 0.f : m_ref;
-                // --- pass 2: exponentials, row sum, P to TMEM as packed 16-bit pairs.  P chunk c4 lands
-                // in columns [16 c4, 16 c4 + 16), which hold scores already consumed. ---
-                float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    float *cur = (c4 & 1) ? xb : xa, *nxt = (c4 & 1) ? xa : xb;
-                    tmem_ld_wait();
-                    if (c4 < 3) tmem_ld32(s_addr + (c4 + 1) * 32, nxt);
+                // --- pass 2: exponentials, row sum, P to TMEM as packed 16-bit pairs.  P chunk c lands
+                // in columns [16 c, 16 c + 16), which hold scores already consumed. ---
+                const unsigned long long nbase2 = pack_f32x2(-base, -base);
+                unsigned long long acc2 = pack_f32x2(0.f, 0.f);
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {
                     uint32_t r[16];
+                    tmem_ld_wait();
+                    tmem_ld32(s_addr + (2 * h + 1) * 32, xb);
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
-                        float p0 = ex2(fmaf(cur[2 * c], p.scale_log2, -base));
-                        float p1 = ex2(fmaf(cur[2 * c + 1], p.scale_log2, -base));
-                        if (boundary) {
-                            p0 = ((vis[c4] >> (2 * c)) & 1u) ? p0 : 0.f;
-                            p1 = ((vis[c4] >> (2 * c + 1)) & 1u) ? p1 : 0.f;
-                        }
-                        acc0 += p0;
-                        acc1 += p1;
+                        float p0, p1;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(xa[2 * c], xa[2 * c + 1]), scale2, nbase2), p0, p1);
+                        p0 = ex2(p0);
+                        p1 = ex2(p1);
+                        acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
                         r[c] = pack2<kBf16>(p0, p1);
                     }
-                    tmem_st16(s_addr + c4 * 16, r);
+                    tmem_st16(s_addr + (2 * h) * 16, r);
+                    tmem_ld_wait();
+                    if (h == 0) tmem_ld32(s_addr + 2 * 32, xa);
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        float p0, p1;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(xb[2 * c], xb[2 * c + 1]), scale2, nbase2), p0, p1);
+                        p0 = ex2(p0);
+                        p1 = ex2(p1);
+                        acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
+                        r[c] = pack2<kBf16>(p0, p1);
+                    }
+                    tmem_st16(s_addr + (2 * h + 1) * 16, r);
                 }
-                l_sum += acc0 + acc1;
+                {
+                    float a0, a1;
+                    unpack_f32x2(acc2, a0, a1);
+                    l_sum += a0 + a1;
+                }
                 tmem_st_wait();
                 // --- last tile of the unit: rows of V past the tree are not data; make them zero ---
                 if (kt == sg.nkt - 1) {
@@ -534,6 +710,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     }
                 }
                 tc_fence_before();
+                HT_TR(2 + s, jj, 3);
                 mbar_arrive(&sm.p_ready[s]);
                 ++n_mine;
                 last_jj = jj;
@@ -543,13 +720,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 mbar_wait(&sm.o_done[s], (last_jj >> 1) & 1, abort_flag);
                 tc_fence_after();
             }
+            HT_TR(4, J, 0);
             sm.ml[s][row][0] = m_ref;
             sm.ml[s][row][1] = l_sum;
+            // With one other part and that part already in the workspace, this CTA finishes the unit
+            // from its registers; otherwise it leaves its own part there.
+            if (tid256 == 0) sm.direct = !complete && cut[cut_k].c_hi - cut[cut_k].c_lo == 1 && delivered_old == 1u;
             tc_fence_before();
             softmax_groups_sync();
             tc_fence_after();
             const float m0 = sm.ml[0][row][0], l0 = sm.ml[0][row][1];
             const float m1 = sm.ml[1][row][0], l1 = sm.ml[1][row][1];
+            const bool direct = sm.direct;
             const float M = fmaxf(m0, m1);
             const float f0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - M);
             const float f1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - M);
@@ -557,54 +739,104 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             // which streams own tiles of this segment (uniform over the CTA)
             const bool has0 = sg.len >= 2 || (J & 1) == 0;
             const bool has1 = sg.len >= 2 || (J & 1) == 1;
-            const bool complete = sg.kt0 == 0 && sg.len == sg.nkt;
             const int head = sg.hk * p.g + row % p.g;
-            const bool real = node < p.N;
-            const int slot_idx = 2 * (int)blockIdx.x + ((t == t_begin) ? 0 : 1);
-            float *prow = p.part + ((size_t)slot_idx * kRows + row) * kPartStride;
-#pragma unroll
+            float *pslot = p.part + (size_t)(2 * (int)blockIdx.x + cut_k) * kSlotFloats;
+            const float *oslot = pslot;                // the other part, when finishing the unit here
+            float g0, g1, gb = 0.f;
+            if (direct) {
+                const CutUnit &cu = cut[cut_k];
+                const int oc = (cu.c_lo == (int)blockIdx.x) ? cu.c_hi : cu.c_lo;
+                oslot = p.part + (size_t)(2 * oc + ((max(cu.t0, oc * per) == oc * per) ? 0 : 1)) * kSlotFloats;
+                __threadfence();
+                const float m_o = __ldcg(oslot + kRows * kD + row), l_o = __ldcg(oslot + kRows * kD + kRows + row);
+                const float Mn = fmaxf(M, m_o);
+                const float fa = (M == -INFINITY) ? 0.f : exp2f(M - Mn);
+                const float fb = (m_o == -INFINITY) ? 0.f : exp2f(m_o - Mn);
+                const float inv = 1.f / (l_tot * fa + l_o * fb);
+                g0 = f0 * fa * inv;
+                g1 = f1 * fa * inv;
+                gb = fb * inv;
+            } else {
+                const float inv = complete ? 1.f / l_tot : 1.f;
+                g0 = f0 * inv;
+                g1 = f1 * inv;
+            }
+            const bool final = complete || direct;
+#pragma unroll 1
             for (int c2 = 0; c2 < 2; ++c2) {
                 const int col0 = s * 64 + c2 * 32;
-                float o[32], o1[32];
-                if (has0) tmem_ld32(tmem + lane_base + 256 + col0, o);
-                if (has1) tmem_ld32(tmem + lane_base + 384 + col0, o1);
+                tmem_ld32(tmem + lane_base + 256 + col0, xa_e);
+                tmem_ld32(tmem + lane_base + 384 + col0, xb_e);
                 tmem_ld_wait();
+                // an accumulator no tile of this segment wrote holds stale numbers (possibly NaN)
 #pragma unroll
-                for (int c = 0; c < 32; ++c) o[c] = (has0 ? f0 * o[c] : 0.f) + (has1 ? f1 * o1[c] : 0.f);
-                if (complete) {
-                    if (real) {
-                        const float inv = 1.f / l_tot;
-                        uint32_t w[16];
+                for (int c = 0; c < 32; ++c) xa_e[c] = (has0 ? g0 * xa_e[c] : 0.f) + (has1 ? g1 * xb_e[c] : 0.f);
+                if (!real) continue;
+                if (direct) {
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) w[c] = pack2<kBf16>(o[2 * c] * inv, o[2 * c + 1] * inv);
-                        unsigned char *dst = static_cast<unsigned char *>(p.out) +
-                                             ((((size_t)sg.b * p.N + node) * p.Hq + head) * kD + col0) * 2;
-#pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            *reinterpret_cast<uint4 *>(dst + c * 16) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+                    for (int c = 0; c < 8; ++c) {
+                        const float4 v = __ldcg(reinterpret_cast<const float4 *>(oslot) + (col0 / 4 + c) * kRows + row);
+                        xa_e[4 * c] = fmaf(gb, v.x, xa_e[4 * c]);
+                        xa_e[4 * c + 1] = fmaf(gb, v.y, xa_e[4 * c + 1]);
+                        xa_e[4 * c + 2] = fmaf(gb, v.z, xa_e[4 * c + 2]);
+                        xa_e[4 * c + 3] = fmaf(gb, v.w, xa_e[4 * c + 3]);
                     }
+                }
+                if (final) {
+                    uint32_t w[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) w[c] = pack2<kBf16>(xa_e[2 * c], xa_e[2 * c + 1]);
+                    unsigned char *dst = static_cast<unsigned char *>(p.out) +
+                                         ((((size_t)sg.b * p.N + node) * p.Hq + head) * kD + col0) * 2;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        *reinterpret_cast<uint4 *>(dst + c * 16) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
                 } else {
 #pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        *reinterpret_cast<float4 *>(prow + col0 + 4 * c) = make_float4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                    for (int c = 0; c < 8; ++c)      // 32 consecutive rows of one feature group: 512 contiguous bytes per warp
+                        reinterpret_cast<float4 *>(pslot)[(col0 / 4 + c) * kRows + row] = make_float4(xa_e[4 * c], xa_e[4 * c + 1], xa_e[4 * c + 2], xa_e[4 * c + 3]);
                 }
             }
-            if (!complete && s == 0) {
-                prow[128] = M;
-                prow[129] = l_tot;
+            if (!final && s == 0 && real) {
+                pslot[kRows * kD + row] = M;
+                pslot[kRows * kD + kRows + row] = l_tot;
             }
             tc_fence_before();
             softmax_groups_sync();                     // both accumulators are free for the next segment
+            if (!final) {
+                // This CTA's part is in the workspace: take the unit's ticket.  One thread orders the
+                // CTA's stores (the barrier above collected them) and draws; the answer is looked at
+                // after the CTA's last segment.
+                cut[cut_k].valid = 1;
+                if (tid256 == 0) {
+                    __threadfence();
+                    ticket[cut_k] = atomicAdd(&p.tickets[cut[cut_k].unit], 1u);
+                }
+            }
+            HT_TR(4, J, 1);
             J += sg.len;
             t += sg.len;
-            ++cta_seg;
         }
-        (void)cta_seg;
+        if (tid256 == 0) HT_TR_CTA(2);
+        // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
+        if (cut[0].valid || cut[1].valid) {
+            if (tid256 == 0)
+                for (int k = 0; k < 2; ++k)
+                    sm.merge_here[k] = cut[k].valid && ticket[k] == (unsigned)(cut[k].c_hi - cut[k].c_lo);
+            softmax_groups_sync();
+            for (int k = 0; k < 2; ++k)
+                if (sm.merge_here[k]) {
+                    __threadfence();
+                    merge_parts<kBf16>(p, cut[k], per, tid256);
+                }
+        }
+        HT_TR(4, 39, 0);
     }
 
     // ------------------------------- teardown -------------------------------
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) HT_TR_CTA(3);
     if (sm.abort && threadIdx.x == 0) {
         for (int b = 0; b < p.B; ++b)
             if (sm.nkt[b] > 0) p.status[b] = HT_STATUS_TIMEOUT;
@@ -612,64 +844,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (warp == 8) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
-    }
-}
-
-// ---------------------------------------------------------------------------------------
-// Merge of the partials of units that were cut between CTAs.  One block per unit.
-// ---------------------------------------------------------------------------------------
-template <bool kBf16>
-__global__ void __launch_bounds__(128)
-attn_tc_merge_kernel(const Params p) {
-    __shared__ int32_t s_len[kMaxB], s_nkt[kMaxB], s_pre[kMaxB + 1];
-    __shared__ int s_bad;
-    plan_sequences<128>(p, s_len, s_nkt, s_pre, &s_bad, false);
-    const int units_per_seq = p.Hkv * p.n_rt;
-    const int b = blockIdx.x / units_per_seq;
-    const int unit = blockIdx.x - b * units_per_seq;
-    const int nkt = s_nkt[b];
-    if (nkt == 0) return;
-    const int total = s_pre[p.B];
-    const int per = tiles_per_cta(total, p.grid);
-    const int t0 = s_pre[b] + unit * nkt, t1 = t0 + nkt;
-    const int c_lo = t0 / per, c_hi = (t1 - 1) / per;
-    if (c_lo == c_hi) return;                          // the unit was computed whole by one CTA
-    const int hk = unit / p.n_rt, rt = unit - hk * p.n_rt;
-    const int row = threadIdx.x;
-    const int node = rt * p.rows_per_tile_nodes + row / p.g;
-    if (node >= p.N) return;
-    const int head = hk * p.g + row % p.g;
-    float M = -INFINITY;
-    for (int c = c_lo; c <= c_hi; ++c) {
-        const int slot = 2 * c + ((max(t0, c * per) == c * per) ? 0 : 1);
-        M = fmaxf(M, p.part[((size_t)slot * kRows + row) * kPartStride + 128]);
-    }
-    float l = 0.f;
-    float o[kD];
-#pragma unroll
-    for (int x = 0; x < kD; ++x) o[x] = 0.f;
-    for (int c = c_lo; c <= c_hi; ++c) {
-        const int slot = 2 * c + ((max(t0, c * per) == c * per) ? 0 : 1);
-        const float *prow = p.part + ((size_t)slot * kRows + row) * kPartStride;
-        const float m = prow[128];
-        if (m == -INFINITY) continue;
-        const float f = exp2f(m - M);
-        l += f * prow[129];
-#pragma unroll
-        for (int x = 0; x < kD; x += 4) {
-            const float4 v = *reinterpret_cast<const float4 *>(prow + x);
-            o[x] = fmaf(f, v.x, o[x]); o[x + 1] = fmaf(f, v.y, o[x + 1]);
-            o[x + 2] = fmaf(f, v.z, o[x + 2]); o[x + 3] = fmaf(f, v.w, o[x + 3]);
-        }
-    }
-    const float inv = 1.f / l;
-    unsigned char *dst = static_cast<unsigned char *>(p.out) + (((size_t)b * p.N + node) * p.Hq + head) * kD * 2;
-#pragma unroll
-    for (int x = 0; x < kD; x += 8) {
-        uint32_t w[4];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) w[c] = pack2<kBf16>(o[x + 2 * c] * inv, o[x + 2 * c + 1] * inv);
-        *reinterpret_cast<uint4 *>(dst + x * 2) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 
@@ -717,9 +891,30 @@ bool attn_tc_applicable(const ht_attn_desc &d) {
     return true;
 }
 
+static size_t ticket_bytes(const ht_attn_desc &d) {
+    const int g = d.Hq / d.Hkv;
+    const size_t units = (size_t)d.B * d.Hkv * ((d.N * g + tc::kRows - 1) / tc::kRows);
+    return (units * sizeof(unsigned int) + 255) / 256 * 256;
+}
+
+// Arrival counters of the units, then two partial-result slots per CTA.
 size_t attn_tc_workspace(const ht_attn_desc &d) {
-    (void)d;
-    return (size_t)2 * sm_count() * tc::kRows * tc::kPartStride * sizeof(float);
+    return ticket_bytes(d) + (size_t)2 * sm_count() * tc::kSlotFloats * sizeof(float);
+}
+
+// The kernels' dynamic shared memory limit is raised once per device.
+static cudaError_t ensure_smem_attr(size_t smem) {
+    static bool done[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(tc::attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(tc::attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) done[dev] = true;
+    return cudaSuccess;
 }
 
 static int make_map(CUtensorMap *map, const void *base, int dtype, const cuuint64_t dims[4], const cuuint64_t strides_b[3],
@@ -733,6 +928,11 @@ static int make_map(CUtensorMap *map, const void *base, int dtype, const cuuint6
     if (r != CUDA_SUCCESS) return fail(HT_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", (int)r);
     return HT_OK;
 }
+
+#ifdef HT_TC_TRACE
+static long long *g_trace = nullptr;
+extern "C" void ht_set_trace(void *ptr) { g_trace = static_cast<long long *>(ptr); }
+#endif
 
 int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const void *vc, const int32_t *kv_len,
                    const int32_t *parent, void *out, void *ws, size_t ws_bytes, int32_t *status, cudaStream_t s) {
@@ -759,7 +959,8 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
         if (rc != HT_OK) return rc;
     }
     tc::Params p;
-    p.kv_len = kv_len; p.parent = parent; p.status = status; p.out = out; p.part = static_cast<float *>(ws);
+    p.kv_len = kv_len; p.parent = parent; p.status = status; p.out = out; p.tickets = static_cast<unsigned int *>(ws);
+    p.part = reinterpret_cast<float *>(static_cast<unsigned char *>(ws) + ticket_bytes(d));
     p.B = d.B; p.N = d.N; p.Hq = d.Hq; p.Hkv = d.Hkv; p.g = g; p.cap = d.cap;
     p.rows_per_tile_nodes = tc::kRows / g;
     p.n_rt = (d.N * g + tc::kRows - 1) / tc::kRows;
@@ -767,24 +968,19 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     p.scale_log2 = scale * 1.4426950408889634f;
     p.is_bf16 = d.dtype == HT_BF16;
     p.grid = sm_count();
+#ifdef HT_TC_TRACE
+    p.trace = g_trace;
+#endif
     const size_t smem = sizeof(tc::Smem) + 1024;
     const long long units = (long long)d.B * d.Hkv * p.n_rt;
     if (units > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "too many (sequence, head, row tile) units");
-    cudaError_t e;
-    if (d.dtype == HT_BF16) {
-        e = cudaFuncSetAttribute(tc::attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        tc::attn_tc_kernel<true><<<p.grid, tc::kThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
-    } else {
-        e = cudaFuncSetAttribute(tc::attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        tc::attn_tc_kernel<false><<<p.grid, tc::kThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
-    }
-    int rc = check_launch("ht_tree_attention (tcgen05)");
-    if (rc != HT_OK) return rc;
-    if (d.dtype == HT_BF16) tc::attn_tc_merge_kernel<true><<<(unsigned)units, 128, 0, s>>>(p);
-    else tc::attn_tc_merge_kernel<false><<<(unsigned)units, 128, 0, s>>>(p);
-    return check_launch("ht_tree_attention (tcgen05 merge)");
+    cudaError_t e = ensure_smem_attr(smem);
+    if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    e = cudaMemsetAsync(p.tickets, 0, (size_t)units * sizeof(unsigned int), s);
+    if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    if (d.dtype == HT_BF16) tc::attn_tc_kernel<true><<<p.grid, tc::kThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
+    else tc::attn_tc_kernel<false><<<p.grid, tc::kThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
+    return check_launch("ht_tree_attention (tcgen05)");
 }
 
 }  // namespace ht
