@@ -6,78 +6,101 @@
 // ridge for the batch sizes of decoding, so tensor cores are not used here and the
 // design goal is 16-byte coalesced loads with enough of them in flight.
 //
-// One warp owns R consecutive rows of the flattened [k*d, d] weight; its lanes stride
-// over the input features in 16-byte vectors, keep R x BT fp32 accumulators and reduce
-// them with shuffles at the end.  The R rows share each loaded h vector, which cuts the
-// L1 traffic for h by R.
+// Every warp of a grid that just fills the GPU owns an equal, contiguous share of the k*d rows of
+// the flattened [k*d, d] weight and walks it R rows at a time.  Its lanes stride over the input
+// features in 16-byte vectors; U such steps (R x U independent 16-byte loads per lane) are issued
+// before the first is used, which keeps over 100 KB of weight in flight per SM -- what a stream
+// needs to run at memory speed.  R x BT fp32 accumulators per lane, reduced with shuffles at
+// the end of a row group.  The R rows share each loaded h vector (h is small and cache resident).
 #include "ht_common.cuh"
 
 namespace ht {
 
-template <typename T, int R, int BT>
-__global__ void __launch_bounds__(128)
+constexpr int kTransferBlocksPerSm = 4;
+
+template <typename T, int R, int BT, int U>
+__global__ void __launch_bounds__(128, kTransferBlocksPerSm)
 transfer_kernel(const T *__restrict__ h, const T *__restrict__ W, T *__restrict__ out,
-                int B, int rows_total, int d, int b0) {
+                int rows_total, int d, int b0, int nb) {
     constexpr int VE = Vec16<T>::n;
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    constexpr int BC = BT < 4 ? BT : 4;              // batch columns handled per pass over the loaded weights
     const int lane = threadIdx.x & 31;
-    const int row0 = warp * R;
-    if (row0 >= rows_total) return;
+    const long long warp = (long long)blockIdx.x * 4 + (threadIdx.x >> 5), n_warps = (long long)gridDim.x * 4;
+    const int r_begin = (int)(warp * rows_total / n_warps), r_end = (int)((warp + 1) * rows_total / n_warps);
 
-    float acc[R][BT];
+    for (int row0 = r_begin; row0 < r_end; row0 += R) {
+        float acc[R][BT];
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+        for (int r = 0; r < R; ++r)
 #pragma unroll
-        for (int b = 0; b < BT; ++b) acc[r][b] = 0.f;
+            for (int b = 0; b < BT; ++b) acc[r][b] = 0.f;
 
-    const int nb = min(BT, B - b0);
-    for (int c = lane * VE; c < d; c += 32 * VE) {
-        uint4 wraw[R];
+        for (int c0 = lane * VE; c0 < d; c0 += 32 * VE * U) {
+            uint4 wraw[U][R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const int row = min(row0 + r, rows_total - 1);
-            wraw[r] = ld_nc16(W + (size_t)row * d + c);
-        }
-        float hv[BT][VE];
+            for (int u = 0; u < U; ++u) {
+                const int c = c0 + u * 32 * VE;
 #pragma unroll
-        for (int b = 0; b < BT; ++b) {
-            if (b < nb) {
-                const uint4 raw = *reinterpret_cast<const uint4 *>(h + (size_t)(b0 + b) * d + c);
-                unpack16<T>(raw, hv[b]);
-            } else {
+                for (int r = 0; r < R; ++r) {
+                    const int row = min(row0 + r, r_end - 1);      // a short last group repeats its last row
+                    wraw[u][r] = c < d ? ld_nc16(W + (size_t)row * d + c) : make_uint4(0, 0, 0, 0);
+                }
+            }
 #pragma unroll
-                for (int e = 0; e < VE; ++e) hv[b][e] = 0.f;
+            for (int u = 0; u < U; ++u) {
+                const int c = min(c0 + u * 32 * VE, d - VE);       // past the end the weights above are zero
+                float wf[R][VE];
+#pragma unroll
+                for (int r = 0; r < R; ++r) unpack16<T>(wraw[u][r], wf[r]);
+#pragma unroll
+                for (int bb = 0; bb < BT; bb += BC) {
+                    float hv[BC][VE];
+#pragma unroll
+                    for (int b = 0; b < BC; ++b) {
+                        const int bi = min(bb + b, nb - 1);        // unused batch columns repeat the last one
+                        unpack16<T>(*reinterpret_cast<const uint4 *>(h + (size_t)(b0 + bi) * d + c), hv[b]);
+                    }
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int b = 0; b < BC; ++b)
+#pragma unroll
+                            for (int e = 0; e < VE; ++e) acc[r][bb + b] = fmaf(wf[r][e], hv[b][e], acc[r][bb + b]);
+                }
             }
         }
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            float wf[VE];
-            unpack16<T>(wraw[r], wf);
+        for (int r = 0; r < R; ++r)
 #pragma unroll
-            for (int b = 0; b < BT; ++b)
+            for (int b = 0; b < BT; ++b) {
+                float v = acc[r][b];
 #pragma unroll
-                for (int e = 0; e < VE; ++e) acc[r][b] = fmaf(wf[e], hv[b][e], acc[r][b]);
-        }
+                for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+                if (lane == 0 && b < nb && row0 + r < r_end)
+                    out[(size_t)(b0 + b) * rows_total + row0 + r] = from_float<T>(v);
+            }
     }
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int b = 0; b < BT; ++b) {
-            float v = acc[r][b];
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-            if (lane == 0 && b < nb && row0 + r < rows_total)
-                out[(size_t)(b0 + b) * rows_total + row0 + r] = from_float<T>(v);
-        }
 }
 
-template <typename T, int R, int BT>
-static int launch_one(const void *h, const void *W, void *out, int B, int rows_total, int d, int b0,
+static int transfer_grid(int rows_total, int R) {
+    static int sms[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+    if (!sms[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        sms[dev] = n;
+    }
+    const int full = sms[dev] * kTransferBlocksPerSm;              // every CTA resident at once
+    const int need = (rows_total + 4 * R - 1) / (4 * R);           // at least one row group per warp
+    return need < full ? need : full;
+}
+
+template <typename T, int R, int BT, int U>
+static int launch_one(const void *h, const void *W, void *out, int rows_total, int d, int b0, int nb,
                       cudaStream_t s) {
-    const int warps = (rows_total + R - 1) / R;
-    const int blocks = (warps + 3) / 4;
-    transfer_kernel<T, R, BT><<<blocks, 128, 0, s>>>(static_cast<const T *>(h), static_cast<const T *>(W),
-                                                     static_cast<T *>(out), B, rows_total, d, b0);
+    transfer_kernel<T, R, BT, U><<<transfer_grid(rows_total, R), 128, 0, s>>>(
+        static_cast<const T *>(h), static_cast<const T *>(W), static_cast<T *>(out), rows_total, d, b0, nb);
     return check_launch("ht_transfer");
 }
 
@@ -85,13 +108,14 @@ template <typename T>
 static int launch_typed(const void *h, const void *W, void *out, int B, int k, int d, cudaStream_t s) {
     const int rows_total = k * d;
     // out is [B, k*d]: batch b writes at out + b*rows_total, so batch slices are independent.
-    for (int b0 = 0; b0 < B; b0 += 8) {
-        const int nb = min(8, B - b0);
+    for (int b0 = 0; b0 < B; b0 += 16) {
+        const int nb = min(16, B - b0);
         int rc;
-        if (nb == 1) rc = launch_one<T, 4, 1>(h, W, out, B, rows_total, d, b0, s);
-        else if (nb == 2) rc = launch_one<T, 4, 2>(h, W, out, B, rows_total, d, b0, s);
-        else if (nb <= 4) rc = launch_one<T, 4, 4>(h, W, out, B, rows_total, d, b0, s);
-        else rc = launch_one<T, 2, 8>(h, W, out, B, rows_total, d, b0, s);
+        if (nb == 1) rc = launch_one<T, 4, 1, 4>(h, W, out, rows_total, d, b0, nb, s);
+        else if (nb == 2) rc = launch_one<T, 4, 2, 4>(h, W, out, rows_total, d, b0, nb, s);
+        else if (nb <= 4) rc = launch_one<T, 4, 4, 4>(h, W, out, rows_total, d, b0, nb, s);
+        else if (nb <= 8) rc = launch_one<T, 2, 8, 4>(h, W, out, rows_total, d, b0, nb, s);
+        else rc = launch_one<T, 2, 16, 4>(h, W, out, rows_total, d, b0, nb, s);
         if (rc != HT_OK) return rc;
     }
     return HT_OK;

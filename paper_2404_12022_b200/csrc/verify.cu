@@ -29,14 +29,25 @@ row_argmax_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pre
     const bool vec_ok = ((size_t)V * sizeof(T)) % 16 == 0;
     if (vec_ok) {
         const int nvec = V / VE;
-        for (int j = threadIdx.x; j < nvec; j += blockDim.x) {
-            float f[VE];
-            unpack16<T>(ld_nc16(row + (size_t)j * VE), f);
+        constexpr int U = 8;                       // independent 16-byte loads in flight per thread
+        for (int j0 = threadIdx.x; j0 < nvec; j0 += U * blockDim.x) {
+            uint4 raw[U];
 #pragma unroll
-            for (int e = 0; e < VE; ++e) {
-                // NaN compares false both ways and is skipped; -inf at a lower index than
-                // the current -inf candidate is taken through the equality branch.
-                if (f[e] > best.v || (f[e] == best.v && j * VE + e < best.i)) best = Best{f[e], j * VE + e};
+            for (int u = 0; u < U; ++u) {
+                const int j = j0 + u * blockDim.x;
+                raw[u] = ld_nc16(row + (size_t)min(j, nvec - 1) * VE);   // past the end: the last vector again
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int j = min(j0 + u * (int)blockDim.x, nvec - 1);
+                float f[VE];
+                unpack16<T>(raw[u], f);
+#pragma unroll
+                for (int e = 0; e < VE; ++e) {
+                    // NaN compares false both ways and is skipped; -inf at a lower index than
+                    // the current -inf candidate is taken through the equality branch.
+                    if (f[e] > best.v || (f[e] == best.v && j * VE + e < best.i)) best = Best{f[e], j * VE + e};
+                }
             }
         }
     } else {
