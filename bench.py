@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--simt", action="store_true", help="force the fp32-ALU attention kernel")
     ap.add_argument("--no-extras", action="store_true", help="skip e2e, cpu baseline and per-kernel timing")
+    ap.add_argument("--sweep", default="", help="instead of the step benchmark, time ht_tree_attention alone on a set of "
+                    "workloads and print one JSON line per point: 'configs' (c2, c2 at KV 2048, a c3 layer, c4) or "
+                    "'c5' (the 48 grouped-query points) or 'c5-quick' (12 of them)")
     return ap.parse_args()
 
 
@@ -209,6 +212,25 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+# DRAM traffic per launch of the attention kernel on a c3 layer, from the ncu capture summarised in
+# profiles/attn_tc_kernel_c3_layer.md (dram__bytes_read.sum + dram__bytes_write.sum).  It is only
+# reported while the kernel source is the one that was profiled.
+NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.6e6,
+               "source": "paper_2404_12022_b200/csrc/attn_tc.cu",
+               "sha256": "1b044cd0f375668c8fa40579add77eb8132f52e19b7c7b8e2851f4c239b195f8"}
+
+
+def ncu_traffic(w):
+    import hashlib
+    try:
+        digest = hashlib.sha256(open(os.path.join(ROOT, NCU_TRAFFIC["source"]), "rb").read()).hexdigest()
+    except OSError:
+        return None
+    if digest != NCU_TRAFFIC["sha256"] or w.name != NCU_TRAFFIC["workload"] or w.kv_len[0] != 4096 or w.B != 4:
+        return None
+    return NCU_TRAFFIC["bytes_per_launch"]
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -324,7 +346,7 @@ def per_kernel_pass(args, step, stream, torch):
     achieved = attn_bytes / (attn_ms * 1e-3) / 1e9
     roofline = {"kernel": "ht_tree_attention", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_nominal_8tbs": achieved / 8000.0, "peak_source": how,
-                "traffic": None, "bytes_per_launch": attn_bytes, "us_per_launch": attn_ms * 1e3,
+                "traffic": ncu_traffic(step.w), "bytes_per_launch": attn_bytes, "us_per_launch": attn_ms * 1e3,
                 "tflops": attn_flops / (attn_ms * 1e-3) / 1e12}
     bytes_of = {"transfer": step.transfer_bytes(), "verify": step.verify_bytes(), "compact": step.compact_bytes()}
     kernels = {"attention": {"us": attn_ms * 1e3, "share": tot["attention"] / all_ms, "gbs": achieved}}
@@ -390,8 +412,79 @@ def e2e_pass(args, step, inp, torch, world):
             "note": "KV cache and transfer weights resident; per-step inputs from pinned host memory"}
 
 
+# ------------------------------------------------------------------------------------------
+# Attention-only sweep over the other workloads (not the bench line; feeds the results tables)
+# ------------------------------------------------------------------------------------------
+
+def sweep_points(which):
+    from paper_2404_12022_b200 import workloads as wl
+    import dataclasses
+    if which == "configs":
+        c2 = wl.config_c2()
+        return [c2, dataclasses.replace(c2, name="c2_at_kv2048", kv_len=[2048]), wl.config_c3(layers=1), wl.config_c4()]
+    pts = wl.c5_points()
+    if which == "c5-quick":
+        pts = [p for p in pts if p[2] == 4 and p[1] in (16, 64, 256)]
+    return [wl.config_c5(*p) for p in pts]
+
+
+def run_sweep(args):
+    """CUDA-event time of ht_tree_attention per call, replayed from a CUDA graph of `reps` calls
+    that rotate over enough copies of the cache to exceed twice the L2 (cold-L2 protocol)."""
+    import torch
+    from paper_2404_12022_b200 import binding as hb
+    from paper_2404_12022_b200 import workloads as wl
+    torch.cuda.set_device(0)
+    peak, how = measured_peaks()
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    for w in sweep_points(args.sweep):
+        inp = wl.make_inputs(w, "cuda", with_logits=False, with_transfer=False, layers=[w.layers - 1])
+        q, kv_len, parent = inp.q[0], inp.kv_len, inp.parent
+        e = w.elem_bytes()
+        cache_bytes = 2 * inp.k_cache[0].numel() * e
+        nbuf = int(min(64, max(2, -(-2 * l2 // cache_bytes))))
+        ks = [inp.k_cache[0]] + [wl.normal_tensor(w.seed, 10 + i, tuple(inp.k_cache[0].shape), "cuda", 1.0, w.torch_dtype())
+                                 for i in range(nbuf - 1)]
+        vs = [inp.v_cache[0]] + [wl.normal_tensor(w.seed, 100 + i, tuple(inp.k_cache[0].shape), "cuda", 1.0, w.torch_dtype())
+                                 for i in range(nbuf - 1)]
+        out = torch.empty_like(q)
+        st = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+        desc = hb.make_attn_desc(q, ks[0])
+        ws = torch.empty(max(hb.tree_attention_workspace(desc), 16), dtype=torch.uint8, device="cuda")
+        reps = max(nbuf, 16)
+        call = lambda i: hb.tree_attention(q, ks[i % nbuf], vs[i % nbuf], kv_len, parent, out=out, workspace=ws, status=st)
+        for i in range(3):
+            call(i)
+        torch.cuda.synchronize()
+        graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side), torch.cuda.graph(graph, stream=side):
+            for i in range(reps):
+                call(i)
+        torch.cuda.synchronize()
+        graph.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        times = []
+        for _ in range(5):
+            e0.record(); graph.replay(); e1.record(); torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1) / reps * 1e3)
+        us = statistics.median(times)
+        rows = q.shape[1]
+        byts = sum(2 * w.Hkv * (L + rows) * w.D * e for L in w.kv_len) + 2 * w.B * rows * w.Hq * w.D * e + 4 * w.B * rows
+        flops = sum(4 * rows * w.Hq * (L + rows) * w.D for L in w.kv_len)
+        assert int(st.abs().sum()) == 0
+        print(json.dumps({"workload": w.name, "batch": w.B, "kv_len": w.kv_len[0] if len(set(w.kv_len)) == 1 else "ragged",
+                          "rows": rows, "q_heads": w.Hq, "kv_heads": w.Hkv, "dtype": w.dtype, "us": round(us, 2),
+                          "hbm_gbs": round(byts / us / 1e3, 1), "frac_of_measured_hbm": round(byts / us / 1e3 / peak, 3),
+                          "frac_of_8tbs": round(byts / us / 1e3 / 8000.0, 3), "tflops": round(flops / us / 1e6, 1),
+                          "flop_per_byte": round(flops / byts, 1), "cold_l2_copies": nbuf}), flush=True)
+        del ks, vs, inp, ws, graph
+
+
 def main():
     args = parse_args()
+    if args.sweep:
+        return run_sweep(args)
     if args.impl == "reference":
         run_reference(args)
     else:
