@@ -1,0 +1,363 @@
+// Building blocks shared by the tensor-core tree-attention kernels: PTX wrappers (mbarrier, TMA,
+// tcgen05), the work plan every role evaluates identically, and the merge of cut units.
+#pragma once
+#include <cuda.h>
+
+#include "ht_common.cuh"
+
+namespace ht {
+namespace tc {
+
+constexpr int kTile = 128;                 // keys per tile
+constexpr int kRows = 128;                 // query rows per tile (UMMA M)
+constexpr int kD = 128;
+constexpr int kStages = 5;                 // ring entries (each one K or one V tile)
+constexpr int kEntryBytes = kTile * kD * 2;
+constexpr int kSlabBytes = kEntryBytes / 2;   // [128 rows][64 elements] = 16 KiB
+constexpr int kThreads = 320;
+constexpr int kMaxB = 256;
+constexpr int kMaxWords = 16;              // ancestor words per row -> N <= 512
+constexpr int kSlotFloats = kRows * kD + 2 * kRows;   // one partial result: O as [32 feature groups][128 rows][4], m[128], l[128]
+constexpr uint32_t kTmemCols = 512;
+constexpr float kRescaleThreshold = 8.0f;  // log2 domain
+
+struct Params {
+    const int32_t *kv_len, *parent;
+    int32_t *status;
+    void *out;
+    float *part;           // partial results of cut units: [grid][2][kSlotFloats]
+    unsigned int *tickets; // one arrival counter per unit, zero on entry
+    int B, N, Hq, Hkv, g, cap, n_rt, rows_per_tile_nodes;   // n_rt: units per (sequence, KV head); rows_per_tile_nodes = 128 / g
+    int n_row_tiles;       // 128-row tiles of the N*g query rows (= n_rt, or 2 n_rt - 1 / 2 n_rt when units are tile pairs)
+    float scale_log2;
+    int is_bf16;
+    int grid;
+#ifdef HT_TC_TRACE
+    long long *trace;
+#endif
+};
+
+// Optional timeline of one CTA (clock64 stamps per role / tile / event) for tuning builds.
+#ifdef HT_TC_TRACE
+#define HT_TR(role, j, ev) do { if (p.trace && blockIdx.x == HT_TC_TRACE && (threadIdx.x & 31) == 0 && ((role) < 2 || (threadIdx.x & 127) == 0) && (j) < 40) p.trace[((role) * 40 + (j)) * 4 + (ev)] = clock64(); } while (0)
+#define HT_TR_CTA(ev) do { if (p.trace && (threadIdx.x & 31) == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); p.trace[1000 + blockIdx.x * 4 + (ev)] = (long long)gt; } } while (0)
+#else
+#define HT_TR(role, j, ev) do { } while (0)
+#define HT_TR_CTA(ev) do { } while (0)
+#endif
+
+struct __align__(1024) Smem {
+    unsigned char q[kEntryBytes];
+    unsigned char ring[kStages][kEntryBytes];
+    uint32_t anc[kMaxWords][kRows];
+    int32_t parent[kMaxWords * 32];
+    float ml[2][kRows][2];
+    int32_t len[kMaxB];
+    int32_t nkt[kMaxB];
+    int32_t pre[kMaxB + 1];
+    unsigned long long kv_full[kStages], kv_empty[kStages], q_full, q_empty, s_full[2], p_ready[2], o_done[2], mma_drain;
+    uint32_t tmem_base;
+    int abort;
+    int merge_here[2];
+    int direct;
+};
+
+// ---------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(void *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(void *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait for the completion of the phase with the given parity.  Returns false (and
+// raises the CTA's abort flag) when about a second passes without it.
+__device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, volatile int *abort_flag,
+                                          bool honor_abort = true) {
+    if (honor_abort && *abort_flag) return false;
+    const uint32_t addr = smem_u32(bar);
+    long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((it & 63u) == 63u) {
+            if (honor_abort && *abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 2000000000ll) { *abort_flag = 1; return false; }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, void *bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(void *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// 32 consecutive TMEM columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t *r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
+          "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {             // 2^x, -inf -> 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+
+__device__ __forceinline__ unsigned int ld_relaxed_gpu(const unsigned int *ptr) {
+    unsigned int v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// Two fp32 values in one 64-bit register, for the paired fp32 instructions.
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+    unsigned long long d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+__device__ __forceinline__ void softmax_groups_sync() {   // the 256 softmax threads
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  Offsets are in 16-byte units.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo16, uint32_t sbo16) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)lbo16 << 16) | ((uint64_t)sbo16 << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor of kind::f16: fp32 accumulate, M = 128, N = n (a multiple of 16).
+__device__ __forceinline__ uint32_t instr_desc(int is_bf16, int b_mn_major, uint32_t n = 128u) {
+    const uint32_t fmt = is_bf16 ? 1u : 0u;
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)b_mn_major << 16) | ((n >> 3) << 17) |
+           ((128u >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------------------
+// Work partition, evaluated identically by every role and by the merge kernel.
+// ---------------------------------------------------------------------------------------
+struct Segment {
+    int b, hk, rt, kt0, len, nkt;
+};
+
+__device__ __forceinline__ Segment locate(const int32_t *pre, const int32_t *nkt, int B, int n_rt, int t, int t_end, int &b_hint) {
+    int b = b_hint;
+    while (b < B - 1 && t >= pre[b + 1]) ++b;
+    b_hint = b;
+    Segment s;
+    s.b = b;
+    s.nkt = nkt[b];
+    const int local = t - pre[b];
+    const int unit = local / s.nkt;
+    s.kt0 = local - unit * s.nkt;
+    s.hk = unit / n_rt;
+    s.rt = unit - s.hk * n_rt;
+    s.len = min(s.nkt - s.kt0, t_end - t);
+    return s;
+}
+
+__device__ __forceinline__ int tiles_per_cta(int total, int grid) { return (total + grid - 1) / grid; }
+
+// Tiles per CTA.  An even share cuts nearly every unit in two, and every cut costs a partial
+// result in the workspace and a merge at the end.  While the cache is streamed at memory speed a
+// few idle SMs cost less than that, so when all sequences are equally long and some whole
+// multiple or whole fraction of a unit lies within 20 % above the even share, ranges of that
+// length are used and cuts fall on unit boundaries (or, for fractions, near them).
+__device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nkt, int B) {
+    const int even = tiles_per_cta(total, grid);
+    int n = 0;
+    for (int b = 0; b < B; ++b) {
+        if (nkt[b] == 0) continue;
+        if (n != 0 && nkt[b] != n) return even;
+        n = nkt[b];
+    }
+    if (n == 0 || even == 0) return even;
+    int cand;
+    if (n >= even) {
+        const int k = n / even;                       // largest count of parts whose length is >= even
+        cand = (n + k - 1) / k;
+    } else {
+        cand = (even + n - 1) / n * n;                // whole units
+    }
+    return (cand * 5 <= even * 6) ? cand : even;
+}
+
+// Validates every sequence and fills len / nkt / pre.  Called by all threads of a block.
+template <int NT>
+__device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, int32_t *s_nkt, int32_t *s_pre,
+                                               bool write_status) {
+    for (int b = threadIdx.x; b < p.B; b += NT) s_nkt[b] = 0;       // 0 = legal so far
+    __syncthreads();
+    for (int i = threadIdx.x; i < p.B * p.N; i += NT) {
+        const int b = i / p.N, c = i - b * p.N;
+        const int par = p.parent[i];
+        if (par < -1 || par >= c) s_nkt[b] = -1;                     // benign race: all writers store -1
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < p.B; b += NT) {
+        const int L = p.kv_len[b];
+        int code = HT_STATUS_OK;
+        if (s_nkt[b] < 0) code = HT_STATUS_BAD_TREE;
+        if (L < 0 || (long long)L + p.N > p.cap) code = HT_STATUS_BAD_LEN;
+        s_len[b] = L;
+        s_nkt[b] = code == HT_STATUS_OK ? (L + p.N + kTile - 1) / kTile : 0;
+        if (write_status) p.status[b] = code;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int b = 0; b < p.B; ++b) {
+            s_pre[b] = acc;
+            acc += s_nkt[b] * p.Hkv * p.n_rt;
+        }
+        s_pre[p.B] = acc;
+    }
+    __syncthreads();
+}
+
+// ---------------------------------------------------------------------------------------
+// Main kernel
+// ---------------------------------------------------------------------------------------
+template <bool kBf16>
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    if (kBf16) {
+        __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t *>(&v);
+    } else {
+        __half2 v = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<uint32_t *>(&v);
+    }
+}
+
+// A unit that was cut between CTAs: which one, and which CTAs hold its parts.
+struct CutUnit {
+    int valid, unit, b, hk, rt, t0, c_lo, c_hi;
+};
+
+// Merge of the parts of a cut unit by the 256 softmax threads of the CTA that delivered the
+// last part.  Threads r and r + 128 own query row r, 64 features each; a warp reads 32
+// consecutive rows of one feature group at a time (contiguous in the part's layout), and the
+// loads of a part are independent of one another so that one round trip to L2 fetches it.
+// `row_tile` is the 128-row tile the part holds; a workspace slot has `subs` parts, this is `sub`.
+template <bool kBf16>
+__device__ __noinline__ void merge_parts(const Params &p, const CutUnit &cu, int per, int tid256, int row_tile, int sub, int subs) {
+    const int row = tid256 & 127, half = tid256 >> 7;
+    const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
+    if (node >= p.N) return;
+    const int head = cu.hk * p.g + row % p.g;
+    float M = -INFINITY, l = 0.f;
+    float acc[64];
+#pragma unroll
+    for (int x = 0; x < 64; ++x) acc[x] = 0.f;
+#pragma unroll 1
+    for (int c = cu.c_lo; c <= cu.c_hi; ++c) {
+        const int slot = 2 * c + ((max(cu.t0, c * per) == c * per) ? 0 : 1);
+        const float *pslot = p.part + ((size_t)slot * subs + sub) * kSlotFloats;
+        const float m = __ldcg(pslot + kRows * kD + row), lp = __ldcg(pslot + kRows * kD + kRows + row);
+        float4 v[16];
+#pragma unroll
+        for (int x = 0; x < 16; ++x) v[x] = __ldcg(reinterpret_cast<const float4 *>(pslot) + (half * 16 + x) * kRows + row);
+        const float Mn = fmaxf(M, m);
+        const float fa = (M == -INFINITY) ? 0.f : exp2f(M - Mn);
+        const float fb = (m == -INFINITY) ? 0.f : exp2f(m - Mn);
+        l = l * fa + lp * fb;
+#pragma unroll
+        for (int x = 0; x < 16; ++x) {
+            acc[4 * x] = acc[4 * x] * fa + v[x].x * fb;
+            acc[4 * x + 1] = acc[4 * x + 1] * fa + v[x].y * fb;
+            acc[4 * x + 2] = acc[4 * x + 2] * fa + v[x].z * fb;
+            acc[4 * x + 3] = acc[4 * x + 3] * fa + v[x].w * fb;
+        }
+        M = Mn;
+    }
+    const float inv = 1.f / l;
+    unsigned char *dst = static_cast<unsigned char *>(p.out) +
+                         ((((size_t)cu.b * p.N + node) * p.Hq + head) * kD + half * 64) * 2;
+#pragma unroll
+    for (int x = 0; x < 8; ++x)
+        *reinterpret_cast<uint4 *>(dst + x * 16) =
+            make_uint4(pack2<kBf16>(acc[8 * x] * inv, acc[8 * x + 1] * inv), pack2<kBf16>(acc[8 * x + 2] * inv, acc[8 * x + 3] * inv),
+                       pack2<kBf16>(acc[8 * x + 4] * inv, acc[8 * x + 5] * inv), pack2<kBf16>(acc[8 * x + 6] * inv, acc[8 * x + 7] * inv));
+}
+
+}  // namespace tc
+}  // namespace ht

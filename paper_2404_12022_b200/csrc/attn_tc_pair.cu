@@ -1,0 +1,521 @@
+// Tree attention on the 5th-generation tensor cores, variant for more than 128 query rows per
+// KV head (grouped-query attention: N * Hq/Hkv rows; Section "Tree attention").
+//
+// With several 128-row tiles per KV head, streaming the cache once per tile would fetch and
+// stage every K/V tile several times.  Here a CTA works on TWO row tiles at once: each K/V tile
+// is fetched into shared memory once and multiplied with both Q tiles.  The roles are those of
+// the one-tile kernel (warp 8: TMA producer, warps 9 and 10: tcgen05.mma issue for stream 0 / 1,
+// warps 0-3 / 4-7: one softmax group per row tile, thread i owns row i of its tile), with these
+// differences:
+//   - stream s = row tile 2*pair + s; every stream sees every K/V tile, keeps its own running
+//     max, sum and TMEM accumulator, and there is nothing to merge between streams.
+//   - the unit of softmax / MMA work is half a K/V tile (64 keys).  Each stream has two 64-column
+//     score buffers in TMEM, so Q K^T of the next half is computed while the softmax of the
+//     current one runs, and P V follows as soon as P is written.  TMEM: 4 x 64 (S/P) + 2 x 128 (O).
+//   - shared memory: two Q tiles and a ring of four 32 KiB K / V tiles.
+//   - a unit (sequence, KV head, tile pair) whose second tile does not exist runs with stream 1 idle.
+// Work split, cut units, tickets and merges are those of the one-tile kernel; a workspace slot
+// holds one part per stream.  Every wait is bounded.
+#include "attn_tc.cuh"
+
+namespace ht {
+namespace tc {
+
+constexpr int kPStages = 4;
+constexpr int kPThreads = kThreads + 32;      // + the second MMA-issuing warp
+constexpr int kHalf = 64;                     // keys per softmax / MMA step
+
+struct __align__(1024) PSmem {
+    unsigned char q[2][kEntryBytes];
+    unsigned char ring[kPStages][kEntryBytes];
+    uint32_t anc[2][kMaxWords][kRows];
+    int32_t parent[kMaxWords * 32];
+    int32_t len[kMaxB];
+    int32_t nkt[kMaxB];
+    int32_t pre[kMaxB + 1];
+    unsigned long long kv_full[kPStages], kv_empty[kPStages], q_full, q_empty, s_full[2][2], p_ready[2][2], o_done[2][2], mma_drain;
+    uint32_t tmem_base;
+    int abort;
+    int merge_here[2];
+    int direct;
+};
+
+template <bool kBf16>
+__global__ void __launch_bounds__(kPThreads, 1)
+attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                    const __grid_constant__ CUtensorMap tm_v, const Params p) {
+    extern __shared__ unsigned char smem_raw[];
+    PSmem &sm = *reinterpret_cast<PSmem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *abort_flag = &sm.abort;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kPStages; ++i) { mbar_init(&sm.kv_full[i], 1); mbar_init(&sm.kv_empty[i], 2); }
+        mbar_init(&sm.q_full, 1);
+        mbar_init(&sm.q_empty, 2);          // one arrival per issuing thread
+        mbar_init(&sm.mma_drain, 2);
+        for (int s = 0; s < 2; ++s)
+            for (int h = 0; h < 2; ++h) {
+                mbar_init(&sm.s_full[s][h], 1);
+                mbar_init(&sm.p_ready[s][h], 128);
+                mbar_init(&sm.o_done[s][h], 1);
+            }
+        sm.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 8) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+
+    const int total = sm.pre[p.B];
+    const int per = choose_per(total, p.grid, sm.nkt, p.B);
+    const int t_begin = min((int)blockIdx.x * per, total);
+    const int t_end = min(t_begin + per, total);
+
+    if (warp == 8) {
+        // ------------------------------- TMA producer -------------------------------
+        if (lane == 0) {
+            int b_hint = 0, ring_i = 0, seg_i = 0;
+            for (int t = t_begin; t < t_end && !*abort_flag;) {
+                const Segment s = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
+                const bool two = 2 * s.rt + 1 < p.n_row_tiles;
+                if (seg_i > 0 && !mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag)) break;
+                mbar_expect_tx(&sm.q_full, two ? 2 * kEntryBytes : kEntryBytes);
+                for (int x = 0; x < (two ? 2 : 1); ++x) {
+                    const int node0 = (2 * s.rt + x) * p.rows_per_tile_nodes;
+                    tma_load_4d(sm.q[x], &tm_q, &sm.q_full, 0, s.hk * p.g, node0, s.b);
+                    tma_load_4d(sm.q[x] + kSlabBytes, &tm_q, &sm.q_full, 64, s.hk * p.g, node0, s.b);
+                }
+                ++seg_i;
+                for (int i = 0; i < 2 * s.len; ++i) {
+                    const int kt = s.kt0 + (i >> 1);
+                    const int slot = ring_i % kPStages, use = ring_i / kPStages;
+                    if (use > 0 && !mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag)) break;
+                    HT_TR(0, ring_i >> 1, ring_i & 1);
+                    const CUtensorMap *tm = (i & 1) ? &tm_v : &tm_k;
+                    mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
+                    tma_load_4d(sm.ring[slot], tm, &sm.kv_full[slot], 0, kt * kTile, s.hk, s.b);
+                    tma_load_4d(sm.ring[slot] + kSlabBytes, tm, &sm.kv_full[slot], 64, kt * kTile, s.hk, s.b);
+                    ++ring_i;
+                }
+                t += s.len;
+            }
+            if (*abort_flag) {
+                // Every copy this thread issued must have landed before the CTA exits.
+                for (int e = max(0, ring_i - kPStages); e < ring_i; ++e)
+                    mbar_wait(&sm.kv_full[e % kPStages], (e / kPStages) & 1, abort_flag, false);
+                if (seg_i > 0) mbar_wait(&sm.q_full, (seg_i - 1) & 1, abort_flag, false);
+            }
+        }
+    } else if (warp >= 9) {
+        // ------------------------------- MMA issuers -------------------------------
+        // One issuing thread per stream (warp 9: stream 0, warp 10: stream 1), so that neither stream
+        // ever waits for the other's softmax.  Per half tile H (64 keys): Q K^T into score buffer H & 1,
+        // then P V of half H - 1; a score buffer is rewritten only after the P V that read it has been
+        // issued.  A tcgen05.commit covers the issuing thread's own operations, so the K / V slots and the
+        // Q buffers are released by one arrival from each of the two threads; in a unit without a second
+        // tile the thread of stream 1 issues nothing and only keeps step with the ring.
+        if (lane == 0) {
+            const int s = warp - 9;
+            const uint32_t idesc_qk = instr_desc(kBf16, 0, kHalf), idesc_pv = instr_desc(kBf16, 1, 128);
+            const uint32_t q_addr = smem_u32(sm.q[s]);
+            int b_hint = 0, j = 0, seg_i = 0;
+            uint32_t uses[2] = {0, 0};                      // completed uses of p_ready[s][h]
+            bool pend = false, pend_first = false;          // the half tile whose P V is still to be issued
+            int pend_j = 0, pend_h = 0;
+            auto issue_pv = [&]() {
+                const int e = 2 * pend_j + 1, slot = e % kPStages;
+                mbar_wait(&sm.kv_full[slot], (e / kPStages) & 1, abort_flag);
+                mbar_wait(&sm.p_ready[s][pend_h], uses[pend_h] & 1, abort_flag);
+                ++uses[pend_h];
+                if (s == 0) HT_TR(1, pend_j, 2 + pend_h);
+                tc_fence_after();
+                if (!*abort_flag) {
+                    const uint32_t v_addr = smem_u32(sm.ring[slot]) + pend_h * (kHalf * 128);
+#pragma unroll
+                    for (int kk = 0; kk < kHalf / 16; ++kk) {
+                        // V as B operand, MN-major: 64 features contiguous per key (one swizzled 128-byte
+                        // line), the second 64-feature slab one slab further (LBO), groups of 8 keys
+                        // 1 KiB apart (SBO); 16 keys per instruction = 2 KiB.
+                        const uint64_t b_desc = smem_desc(v_addr + kk * 2048, kSlabBytes >> 4, 1024 >> 4);
+                        mma_ts(tmem + 256 + s * 128, tmem + s * 128 + pend_h * kHalf + kk * 8, b_desc, idesc_pv,
+                               (kk > 0 || !pend_first) ? 1u : 0u);
+                    }
+                }
+                tc_commit(&sm.o_done[s][pend_h]);
+                if (pend_h == 1) tc_commit(&sm.kv_empty[slot]);
+                pend = false;
+            };
+            for (int t = t_begin; t < t_end;) {
+                const Segment sg = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
+                const bool act = s == 0 || 2 * sg.rt + 1 < p.n_row_tiles;
+                mbar_wait(&sm.q_full, seg_i & 1, abort_flag);
+                for (int i = 0; i < sg.len; ++i) {
+                    const int e = 2 * j, slot = e % kPStages;
+                    mbar_wait(&sm.kv_full[slot], (e / kPStages) & 1, abort_flag);
+                    tc_fence_after();
+                    if (!act) {
+                        // keep step with the ring: hand both slots of this tile back once they are loaded
+                        if (pend) issue_pv();
+                        tc_commit(&sm.kv_empty[slot]);
+                        if (i == sg.len - 1) tc_commit(&sm.q_empty);
+                        const int ev = e + 1, vslot = ev % kPStages;
+                        mbar_wait(&sm.kv_full[vslot], (ev / kPStages) & 1, abort_flag);
+                        tc_commit(&sm.kv_empty[vslot]);
+                        ++j;
+                        continue;
+                    }
+                    for (int h = 0; h < 2; ++h) {
+                        if (s == 0) HT_TR(1, j, h);
+                        if (!*abort_flag) {
+                            const uint32_t k_addr = smem_u32(sm.ring[slot]) + h * (kHalf * 128);
+#pragma unroll
+                            for (int kk = 0; kk < kD / 16; ++kk) {
+                                // K-major operands: 16 features = 32 bytes inside the 128-byte swizzled
+                                // line; the second 64-feature slab lies one slab further.
+                                const uint32_t off = (kk >> 2) * kSlabBytes + (kk & 3) * 32;
+                                mma_ss(tmem + s * 128 + h * kHalf, smem_desc(q_addr + off, 1, 1024 >> 4),
+                                       smem_desc(k_addr + off, 1, 1024 >> 4), idesc_qk, kk > 0 ? 1u : 0u);
+                            }
+                        }
+                        tc_commit(&sm.s_full[s][h]);
+                        if (h == 1) {
+                            tc_commit(&sm.kv_empty[slot]);
+                            if (i == sg.len - 1) tc_commit(&sm.q_empty);
+                        }
+                        if (pend) issue_pv();
+                        pend = true;
+                        pend_first = (i == 0 && h == 0);
+                        pend_j = j;
+                        pend_h = h;
+                    }
+                    ++j;
+                }
+                t += sg.len;
+                ++seg_i;
+            }
+            if (pend) issue_pv();
+            // No tensor-core operation of this CTA may be in flight when its TMEM is freed.
+            tc_commit(&sm.mma_drain);
+            mbar_wait(&sm.mma_drain, 0, abort_flag, false);
+        }
+    } else {
+        // ------------------------------- softmax groups -------------------------------
+        const int s = warp >> 2;                       // stream of this group = which tile of the pair
+        const int row = threadIdx.x & 127;             // query row within the tile = TMEM lane
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const int tid256 = threadIdx.x;                // 0..255 among the softmax threads
+        const int words = (p.N + 31) >> 5;
+        const unsigned long long scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+        const uint32_t o_addr = tmem + lane_base + 256 + s * 128;
+        int b_hint = 0, J = 0;
+        float xa[32], xb[32];
+        CutUnit cut[2];
+        unsigned int ticket[2] = {0u, 0u};
+        cut[0].valid = cut[1].valid = 0;
+        int anc_b = -1, anc_rt = -1;                   // sequence / tile pair the ancestor words were built for
+        uint32_t uses_s[2] = {0, 0}, uses_o[2] = {0, 0};   // uses of s_full[s][h] / o_done[s][h] so far
+        for (int t = t_begin; t < t_end;) {
+            const Segment sg = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
+            const int L = sm.len[sg.b];
+            const int row_tile = 2 * sg.rt + s;
+            const bool active = row_tile < p.n_row_tiles;
+            const bool two = 2 * sg.rt + 1 < p.n_row_tiles;
+            const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
+            const bool real = active && node < p.N;
+            if (sg.b != anc_b || sg.rt != anc_rt) {
+                softmax_groups_sync();                 // previous segment no longer reads parent / anc
+                for (int c = tid256; c < p.N; c += 256) sm.parent[c] = p.parent[(size_t)sg.b * p.N + c];
+                softmax_groups_sync();
+                for (int w = 0; w < words; ++w) sm.anc[s][w][row] = 0u;   // padding rows see the context only; their results are dropped
+                if (real)
+                    for (int c = node; c >= 0; c = sm.parent[c]) sm.anc[s][c >> 5][row] |= 1u << (c & 31);
+                softmax_groups_sync();
+                anc_b = sg.b;
+                anc_rt = sg.rt;
+            }
+            // A segment that is only part of its unit: see the one-tile kernel.
+            const bool complete = sg.kt0 == 0 && sg.len == sg.nkt;
+            const int cut_k = (t == t_begin) ? 0 : 1;
+            unsigned int delivered = 0, delivered_old = 0;
+            if (!complete) {
+                CutUnit &cu = cut[cut_k];
+                cu.unit = (sg.b * p.Hkv + sg.hk) * p.n_rt + sg.rt;
+                cu.b = sg.b; cu.hk = sg.hk; cu.rt = sg.rt;
+                cu.t0 = sm.pre[sg.b] + (sg.hk * p.n_rt + sg.rt) * sg.nkt;
+                cu.c_lo = cu.t0 / per;
+                cu.c_hi = (cu.t0 + sg.nkt - 1) / per;
+            }
+
+            float m_ref = -INFINITY, l_sum = 0.f;
+            int last_h = -1;                            // score buffer of this stream's latest P V in this segment
+            if (active) {
+#pragma unroll 1
+                for (int ih = 0; ih < 2 * sg.len; ++ih) {
+                    const int i = ih >> 1, h = ih & 1;
+                    const int kt = sg.kt0 + i;
+                    if (!complete && tid256 == 0 && h == 0) {
+                        delivered_old = delivered;
+                        delivered = ld_relaxed_gpu(&p.tickets[cut[cut_k].unit]);
+                    }
+                    if (h == 0) HT_TR(2 + s, J + i, 0);
+                    mbar_wait(&sm.s_full[s][h], uses_s[h] & 1, abort_flag);
+                    ++uses_s[h];
+                    HT_TR(2 + s, J + i, 1 + h);
+                    tc_fence_after();
+                    const uint32_t s_addr = tmem + lane_base + s * 128 + h * kHalf;
+                    const int key_lo = kt * kTile + h * kHalf;
+                    if (key_lo + kHalf > L) {
+                        // Reaches into the tree rows / the tail: scores of keys this row must not see
+                        // become -inf in place (context visible, tree key c iff ancestor bit c, tail never).
+#pragma unroll 1
+                        for (int w = 0; w < 2; ++w) {
+                            const int cc0 = key_lo + 32 * w - L;
+                            if (cc0 <= -32) continue;
+                            const int wi = cc0 >> 5, sh = cc0 & 31;
+                            const uint32_t lo = wi < 0 ? 0xFFFFFFFFu : (wi < words ? sm.anc[s][wi][row] : 0u);
+                            const uint32_t hi = (wi + 1 >= 0 && wi + 1 < words) ? sm.anc[s][wi + 1][row] : 0u;
+                            const uint32_t vis = __funnelshift_r(lo, hi, sh);
+                            tmem_ld32(s_addr + w * 32, xa);
+                            tmem_ld_wait();
+                            uint32_t r[32];
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) r[c] = ((vis >> c) & 1u) ? __float_as_uint(xa[c]) : 0xFF800000u;
+                            tmem_st32(s_addr + w * 32, r);
+                        }
+                        tmem_st_wait();
+                    }
+                    // --- pass 1: row maximum over the 64 scores (they stay in registers for pass 2) ---
+                    float mx0 = -INFINITY, mx1 = -INFINITY;
+                    tmem_ld32(s_addr, xa);
+                    tmem_ld32(s_addr + 32, xb);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4) {
+                        mx0 = max3(mx0, xa[c], xa[c + 1]);
+                        mx1 = max3(mx1, xa[c + 2], xa[c + 3]);
+                    }
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4) {
+                        mx0 = max3(mx0, xb[c], xb[c + 1]);
+                        mx1 = max3(mx1, xb[c + 2], xb[c + 3]);
+                    }
+                    const float mx = fmaxf(mx0, mx1) * p.scale_log2;
+                    // --- running maximum, raised lazily ---
+                    const float m_new = fmaxf(m_ref, mx);
+                    const bool grow = (m_ref != -INFINITY) && (m_new > m_ref + kRescaleThreshold);
+                    if (m_ref == -INFINITY) m_ref = m_new;
+                    if (__any_sync(0xffffffffu, grow)) {
+                        // The accumulator may be rescaled once this stream's latest P V has completed
+                        // (the next one is not issued before this thread reports P ready).
+                        if (last_h >= 0) {
+                            mbar_wait(&sm.o_done[s][last_h], (uses_o[last_h] - 1) & 1, abort_flag);
+                            tc_fence_after();
+                        }
+                        const float f = grow ? exp2f(m_ref - m_new) : 1.f;
+#pragma unroll 1
+                        for (int c4 = 0; c4 < 4; ++c4) {
+                            float o[32];
+                            uint32_t r[32];
+                            tmem_ld32(o_addr + c4 * 32, o);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(o[c] * f);
+                            tmem_st32(o_addr + c4 * 32, r);
+                        }
+                        tmem_st_wait();
+                        l_sum *= f;
+                        if (grow) m_ref = m_new;
+                    }
+                    const float base = (m_ref == -INFINITY) ? 0.f : m_ref;
+                    // --- pass 2: exponentials, row sum, P as packed 16-bit pairs over the consumed scores ---
+                    const unsigned long long nbase2 = pack_f32x2(-base, -base);
+                    unsigned long long acc2 = pack_f32x2(0.f, 0.f);
+                    {
+                        uint32_t r[16];
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            float p0, p1;
+                            unpack_f32x2(fma_f32x2(pack_f32x2(xa[2 * c], xa[2 * c + 1]), scale2, nbase2), p0, p1);
+                            p0 = ex2(p0);
+                            p1 = ex2(p1);
+                            acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
+                            r[c] = pack2<kBf16>(p0, p1);
+                        }
+                        tmem_st16(s_addr, r);
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            float p0, p1;
+                            unpack_f32x2(fma_f32x2(pack_f32x2(xb[2 * c], xb[2 * c + 1]), scale2, nbase2), p0, p1);
+                            p0 = ex2(p0);
+                            p1 = ex2(p1);
+                            acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
+                            r[c] = pack2<kBf16>(p0, p1);
+                        }
+                        tmem_st16(s_addr + 16, r);
+                    }
+                    {
+                        float a0, a1;
+                        unpack_f32x2(acc2, a0, a1);
+                        l_sum += a0 + a1;
+                    }
+                    tmem_st_wait();
+                    // --- last tile of the unit: rows of V past the tree are not data; make them zero (both
+                    // streams write the same zeros, each before it lets its own P V go) ---
+                    if (kt == sg.nkt - 1 && h == 0) {
+                        const int valid = L + p.N - kt * kTile;
+                        if (valid < kTile) {
+                            const int e = 2 * (J + i) + 1, slot = e % kPStages;
+                            mbar_wait(&sm.kv_full[slot], (e / kPStages) & 1, abort_flag);
+                            const int vecs = (kTile - valid) * 8;               // 16-byte vectors per slab
+                            for (int v = row; v < vecs; v += 128) {
+                                *reinterpret_cast<uint4 *>(sm.ring[slot] + valid * 128 + v * 16) = make_uint4(0, 0, 0, 0);
+                                *reinterpret_cast<uint4 *>(sm.ring[slot] + kSlabBytes + valid * 128 + v * 16) = make_uint4(0, 0, 0, 0);
+                            }
+                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        }
+                    }
+                    tc_fence_before();
+                    if (h == 1) HT_TR(2 + s, J + i, 3);
+                    mbar_arrive(&sm.p_ready[s][h]);
+                    ++uses_o[h];                        // the P V of this half will arrive on o_done[s][h]
+                    last_h = h;
+                }
+                // the segment's last P V of this stream
+                mbar_wait(&sm.o_done[s][last_h], (uses_o[last_h] - 1) & 1, abort_flag);
+                tc_fence_after();
+            }
+            // --- segment epilogue: write the result, finish a cut unit, or leave a part ---
+            if (tid256 == 0) sm.direct = !complete && cut[cut_k].c_hi - cut[cut_k].c_lo == 1 && delivered_old == 1u;
+            tc_fence_before();
+            softmax_groups_sync();
+            tc_fence_after();
+            const bool direct = sm.direct;
+            const bool final = complete || direct;
+            if (active) {
+                const int head = sg.hk * p.g + row % p.g;
+                float *pslot = p.part + ((size_t)(2 * (int)blockIdx.x + cut_k) * 2 + s) * kSlotFloats;
+                const float *oslot = pslot;            // the other part, when finishing the unit here
+                float g0, gb = 0.f;
+                if (direct) {
+                    const CutUnit &cu = cut[cut_k];
+                    const int oc = (cu.c_lo == (int)blockIdx.x) ? cu.c_hi : cu.c_lo;
+                    oslot = p.part + ((size_t)(2 * oc + ((max(cu.t0, oc * per) == oc * per) ? 0 : 1)) * 2 + s) * kSlotFloats;
+                    __threadfence();
+                    const float m_o = __ldcg(oslot + kRows * kD + row), l_o = __ldcg(oslot + kRows * kD + kRows + row);
+                    const float Mn = fmaxf(m_ref, m_o);
+                    const float fa = (m_ref == -INFINITY) ? 0.f : exp2f(m_ref - Mn);
+                    const float fb = (m_o == -INFINITY) ? 0.f : exp2f(m_o - Mn);
+                    const float inv = 1.f / (l_sum * fa + l_o * fb);
+                    g0 = fa * inv;
+                    gb = fb * inv;
+                } else {
+                    g0 = complete ? 1.f / l_sum : 1.f;
+                }
+#pragma unroll 1
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    const int col0 = c4 * 32;
+                    tmem_ld32(o_addr + col0, xa);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) xa[c] *= g0;
+                    if (!real) continue;
+                    if (direct) {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const float4 v = __ldcg(reinterpret_cast<const float4 *>(oslot) + (col0 / 4 + c) * kRows + row);
+                            xa[4 * c] = fmaf(gb, v.x, xa[4 * c]);
+                            xa[4 * c + 1] = fmaf(gb, v.y, xa[4 * c + 1]);
+                            xa[4 * c + 2] = fmaf(gb, v.z, xa[4 * c + 2]);
+                            xa[4 * c + 3] = fmaf(gb, v.w, xa[4 * c + 3]);
+                        }
+                    }
+                    if (final) {
+                        uint32_t w[16];
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) w[c] = pack2<kBf16>(xa[2 * c], xa[2 * c + 1]);
+                        unsigned char *dst = static_cast<unsigned char *>(p.out) +
+                                             ((((size_t)sg.b * p.N + node) * p.Hq + head) * kD + col0) * 2;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            *reinterpret_cast<uint4 *>(dst + c * 16) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)
+                            reinterpret_cast<float4 *>(pslot)[(col0 / 4 + c) * kRows + row] = make_float4(xa[4 * c], xa[4 * c + 1], xa[4 * c + 2], xa[4 * c + 3]);
+                    }
+                }
+                if (!final && real) {
+                    pslot[kRows * kD + row] = m_ref;
+                    pslot[kRows * kD + kRows + row] = l_sum;
+                }
+            }
+            tc_fence_before();
+            softmax_groups_sync();                     // the accumulators are free for the next segment
+            if (!final) {
+                cut[cut_k].valid = two ? 3 : 1;         // which streams left a part
+                if (tid256 == 0) {
+                    __threadfence();
+                    ticket[cut_k] = atomicAdd(&p.tickets[cut[cut_k].unit], 1u);
+                }
+            }
+            J += sg.len;
+            t += sg.len;
+        }
+        // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
+        if (cut[0].valid || cut[1].valid) {
+            if (tid256 == 0)
+                for (int k = 0; k < 2; ++k)
+                    sm.merge_here[k] = cut[k].valid && ticket[k] == (unsigned)(cut[k].c_hi - cut[k].c_lo);
+            softmax_groups_sync();
+            for (int k = 0; k < 2; ++k)
+                if (sm.merge_here[k]) {
+                    __threadfence();
+                    for (int x = 0; x < 2; ++x)
+                        if (cut[k].valid & (1 << x)) merge_parts<kBf16>(p, cut[k], per, tid256, 2 * cut[k].rt + x, x, 2);
+                }
+        }
+    }
+
+    // ------------------------------- teardown -------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (sm.abort && threadIdx.x == 0) {
+        for (int b = 0; b < p.B; ++b)
+            if (sm.nkt[b] > 0) p.status[b] = HT_STATUS_TIMEOUT;
+    }
+    if (warp == 8) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+}  // namespace tc
+
+// Raises the kernels' dynamic shared memory limit (once per device) and launches.
+int launch_attn_tc_pair_kernel(const CUtensorMap &tm_q, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const tc::Params &p,
+                               bool bf16, cudaStream_t s) {
+    static bool done[64];
+    const size_t smem = sizeof(tc::PSmem) + 1024;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    if (!(dev >= 0 && dev < 64 && done[dev])) {
+        e = cudaFuncSetAttribute(tc::attn_tc_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tc::attn_tc_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+        if (dev >= 0 && dev < 64) done[dev] = true;
+    }
+    if (bf16) tc::attn_tc_pair_kernel<true><<<p.grid, tc::kPThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
+    else tc::attn_tc_pair_kernel<false><<<p.grid, tc::kPThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
+    return check_launch("ht_tree_attention (tcgen05, tile pairs)");
+}
+
+}  // namespace ht
