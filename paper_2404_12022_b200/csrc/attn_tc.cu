@@ -191,6 +191,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             // --- ancestor masks of this tile's rows (kept while sequence and row tile stay the same) ---
             const int node = sg.rt * p.rows_per_tile_nodes + row / p.g;
             const bool real = node < p.N;
+            // a warp none of whose 32 rows is a query row keeps step with the barriers but computes nothing
+            const bool warp_real = sg.rt * p.rows_per_tile_nodes + (row & ~31) / p.g < p.N;
             if (sg.b != anc_b || sg.rt != anc_rt) {
                 softmax_groups_sync();                 // previous segment no longer reads parent / anc
                 for (int c = tid256; c < p.N; c += 256) sm.parent[c] = p.parent[(size_t)sg.b * p.N + c];
@@ -238,6 +240,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const uint32_t s_addr = tmem + lane_base + s * 128;
                 const int tile_lo = kt * kTile;
                 float *const xa = xa_e, *const xb = xb_e;
+                if (warp_real) {
                 if (tile_lo + kTile > L) {
                     // The tile reaches into the tree rows / the tail: overwrite the scores of keys this
                     // row must not see with -inf, in place, so that the two passes below need no mask.
@@ -344,6 +347,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     l_sum += a0 + a1;
                 }
                 tmem_st_wait();
+                }
                 // --- last tile of the unit: rows of V past the tree are not data; make them zero ---
                 if (kt == sg.nkt - 1) {
                     const int valid = L + p.N - tile_lo;
@@ -412,7 +416,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
             const bool final = complete || direct;
 #pragma unroll 1
-            for (int c2 = 0; c2 < 2; ++c2) {
+            for (int c2 = 0; c2 < (warp_real ? 2 : 0); ++c2) {
                 const int col0 = s * 64 + c2 * 32;
                 tmem_ld32(tmem + lane_base + 256 + col0, xa_e);
                 tmem_ld32(tmem + lane_base + 384 + col0, xb_e);

@@ -229,6 +229,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const bool two = 2 * sg.rt + 1 < p.n_row_tiles;
             const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
             const bool real = active && node < p.N;
+            // a warp none of whose 32 rows is a query row keeps step with the barriers but computes nothing
+            const bool warp_real = active && row_tile * p.rows_per_tile_nodes + (row & ~31) / p.g < p.N;
             if (sg.b != anc_b || sg.rt != anc_rt) {
                 softmax_groups_sync();                 // previous segment no longer reads parent / anc
                 for (int c = tid256; c < p.N; c += 256) sm.parent[c] = p.parent[(size_t)sg.b * p.N + c];
@@ -271,6 +273,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tc_fence_after();
                     const uint32_t s_addr = tmem + lane_base + s * 128 + h * kHalf;
                     const int key_lo = kt * kTile + h * kHalf;
+                    if (warp_real) {
                     if (key_lo + kHalf > L) {
                         // Reaches into the tree rows / the tail: scores of keys this row must not see
                         // become -inf in place (context visible, tree key c iff ancestor bit c, tail never).
@@ -366,6 +369,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         l_sum += a0 + a1;
                     }
                     tmem_st_wait();
+                    }
                     // --- last tile of the unit: rows of V past the tree are not data; make them zero (both
                     // streams write the same zeros, each before it lets its own P V go) ---
                     if (kt == sg.nkt - 1 && h == 0) {
@@ -419,7 +423,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     g0 = complete ? 1.f / l_sum : 1.f;
                 }
 #pragma unroll 1
-                for (int c4 = 0; c4 < 4; ++c4) {
+                for (int c4 = 0; c4 < (warp_real ? 4 : 0); ++c4) {
                     const int col0 = c4 * 32;
                     tmem_ld32(o_addr + col0, xa);
                     tmem_ld_wait();
