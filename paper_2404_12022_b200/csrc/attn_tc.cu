@@ -41,6 +41,72 @@
 namespace ht {
 namespace tc {
 
+// Reduction of a unit's parts inside a thread-block cluster, by the 256 softmax threads of each CTA.
+// On entry this CTA's part (m, l, O in the layout of a workspace slot) lies at the start of its K / V
+// ring, which nothing else uses any more.  Every CTA owns 128 / k of the 128 output features: once all
+// peers have said that their rings are idle, each CTA copies, for every peer, that peer's feature
+// slice of its part (and m, l) into the peer's ring through distributed shared memory; after a
+// second round of arrivals each CTA merges the k slices it holds and writes its features of the
+// result.  No global memory, no atomics; both waits are bounded.
+constexpr int kXchgRecvOffset = (kSlotFloats * 4 + 1023) / 1024 * 1024;   // bytes from the ring's start
+
+template <bool kBf16>
+__device__ __noinline__ void cluster_exchange(const Params &p, Smem &sm, int rank, int b, int hk, bool valid,
+                                              int tid256, volatile int *abort_flag) {
+    const int k = p.cluster_k;
+    const int cg_per_slice = 32 / k;                    // 4-feature groups per CTA's slice
+    unsigned char *ring = &sm.ring[0][0];
+    const float4 *own4 = reinterpret_cast<const float4 *>(ring);
+    const float *own_ml = reinterpret_cast<const float *>(ring) + kRows * kD;
+    float4 *recv4 = reinterpret_cast<float4 *>(ring + kXchgRecvOffset);          // [sender][group in slice][row]
+    float *recv_ml = reinterpret_cast<float *>(ring + kXchgRecvOffset) + kRows * kD;   // [sender][m | l][row]
+    softmax_groups_sync();                              // this CTA's part is complete
+    if (tid256 == 0)
+        for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&sm.xb[0]), (uint32_t)c));
+    mbar_wait_cluster(&sm.xb[0], 0, abort_flag);        // every peer's ring is idle
+    if (!*abort_flag) {
+        for (int idx = tid256; idx < 32 * kRows; idx += 256) {
+            const int cg = idx >> 7, r = idx & 127, c = cg / cg_per_slice, x = cg - c * cg_per_slice;
+            st_peer_f4(map_to_peer(smem_u32(recv4 + (rank * cg_per_slice + x) * kRows + r), (uint32_t)c), own4[idx]);
+        }
+        const float ml = own_ml[tid256];                // 128 m then 128 l
+        for (int c = 0; c < k; ++c) st_peer_f1(map_to_peer(smem_u32(recv_ml + rank * 2 * kRows + tid256), (uint32_t)c), ml);
+    }
+    asm volatile("fence.acq_rel.cluster;" ::: "memory");
+    softmax_groups_sync();
+    if (tid256 == 0)
+        for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&sm.xb[1]), (uint32_t)c));
+    mbar_wait_cluster(&sm.xb[1], 0, abort_flag);        // every part has arrived here
+    const int row = tid256 & 127, half = tid256 >> 7;
+    const int node = row / p.g;
+    if (!valid || node >= p.N || *abort_flag) return;
+    float M = -INFINITY;
+    for (int c = 0; c < k; ++c) M = fmaxf(M, recv_ml[c * 2 * kRows + row]);
+    float l = 0.f;
+    for (int c = 0; c < k; ++c) {
+        const float m = recv_ml[c * 2 * kRows + row];
+        if (m != -INFINITY) l = fmaf(exp2f(m - M), recv_ml[c * 2 * kRows + kRows + row], l);
+    }
+    const float inv = 1.f / l;
+    const int head = hk * p.g + row % p.g;
+    const int x_per_half = cg_per_slice / 2 > 0 ? cg_per_slice / 2 : 1;
+    for (int xi = 0; xi < x_per_half; ++xi) {
+        const int x = half * x_per_half + xi;
+        if (x >= cg_per_slice) break;
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = 0; c < k; ++c) {
+            const float m = recv_ml[c * 2 * kRows + row];
+            if (m == -INFINITY) continue;
+            const float f = exp2f(m - M);
+            const float4 v = recv4[(c * cg_per_slice + x) * kRows + row];
+            o.x = fmaf(f, v.x, o.x); o.y = fmaf(f, v.y, o.y); o.z = fmaf(f, v.z, o.z); o.w = fmaf(f, v.w, o.w);
+        }
+        unsigned char *dst = static_cast<unsigned char *>(p.out) +
+                             ((((size_t)b * p.N + node) * p.Hq + head) * kD + (rank * cg_per_slice + x) * 4) * 2;
+        *reinterpret_cast<uint2 *>(dst) = make_uint2(pack2<kBf16>(o.x * inv, o.y * inv), pack2<kBf16>(o.z * inv, o.w * inv));
+    }
+}
+
 template <bool kBf16>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -56,6 +122,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         mbar_init(&sm.q_full, 1);
         mbar_init(&sm.q_empty, 1);
         mbar_init(&sm.mma_drain, 1);
+        for (int i = 0; i < 2; ++i) mbar_init(&sm.xb[i], p.cluster_k > 1 ? p.cluster_k : 1);
         for (int i = 0; i < 2; ++i) { mbar_init(&sm.s_full[i], 1); mbar_init(&sm.p_ready[i], 128); mbar_init(&sm.o_done[i], 1); }
         sm.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -72,8 +139,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
     const int total = sm.pre[p.B];
     const int per = choose_per(total, p.grid, sm.nkt, p.B);
-    const int t_begin = min((int)blockIdx.x * per, total);
-    const int t_end = min(t_begin + per, total);
+    int t_begin = min((int)blockIdx.x * per, total);
+    int t_end = min(t_begin + per, total);
+    const bool clustered = p.cluster_k > 1;
+    uint32_t c_rank = 0;
+    if (clustered) {
+        // One cluster per (sequence, KV head); the cluster's CTAs take equal shares of its tiles.  The
+        // peers' barriers must exist before anyone arrives on them.
+        cluster_sync_all();
+        c_rank = cluster_ctarank();
+        const int unit = (int)blockIdx.x / p.cluster_k, b = unit / p.Hkv, hk = unit - b * p.Hkv;
+        const int nk = sm.nkt[b], share = (nk + p.cluster_k - 1) / p.cluster_k;
+        const int t0 = sm.pre[b] + hk * nk;
+        t_begin = t0 + min((int)c_rank * share, nk);
+        t_end = t0 + min(((int)c_rank + 1) * share, nk);
+    }
 
     if (warp == 8) {
         // ------------------------------- TMA producer -------------------------------
@@ -229,7 +309,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int jj = J + i;
                 if ((jj & 1) != s) continue;
                 const int kt = sg.kt0 + i;
-                if (!complete && tid256 == 0) {
+                if (!complete && !clustered && tid256 == 0) {
                     delivered_old = delivered;
                     delivered = ld_relaxed_gpu(&p.tickets[cut[cut_k].unit]);
                 }
@@ -378,7 +458,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             sm.ml[s][row][1] = l_sum;
             // With one other part and that part already in the workspace, this CTA finishes the unit
             // from its registers; otherwise it leaves its own part there.
-            if (tid256 == 0) sm.direct = !complete && cut[cut_k].c_hi - cut[cut_k].c_lo == 1 && delivered_old == 1u;
+            if (tid256 == 0) sm.direct = !clustered && !complete && cut[cut_k].c_hi - cut[cut_k].c_lo == 1 && delivered_old == 1u;
             tc_fence_before();
             softmax_groups_sync();
             tc_fence_after();
@@ -393,7 +473,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const bool has0 = sg.len >= 2 || (J & 1) == 0;
             const bool has1 = sg.len >= 2 || (J & 1) == 1;
             const int head = sg.hk * p.g + row % p.g;
-            float *pslot = p.part + (size_t)(2 * (int)blockIdx.x + cut_k) * kSlotFloats;
+            // a part goes to the workspace -- or, in a cluster, to this CTA's own (by now idle) K / V ring
+            float *pslot = clustered ? reinterpret_cast<float *>(&sm.ring[0][0]) : p.part + (size_t)(2 * (int)blockIdx.x + cut_k) * kSlotFloats;
             const float *oslot = pslot;                // the other part, when finishing the unit here
             float g0, g1, gb = 0.f;
             if (direct) {
@@ -410,11 +491,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 g1 = f1 * fa * inv;
                 gb = fb * inv;
             } else {
-                const float inv = complete ? 1.f / l_tot : 1.f;
+                const float inv = (complete && !clustered) ? 1.f / l_tot : 1.f;
                 g0 = f0 * inv;
                 g1 = f1 * inv;
             }
-            const bool final = complete || direct;
+            const bool final = (complete && !clustered) || direct;
 #pragma unroll 1
             for (int c2 = 0; c2 < (warp_real ? 2 : 0); ++c2) {
                 const int col0 = s * 64 + c2 * 32;
@@ -456,7 +537,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
             tc_fence_before();
             softmax_groups_sync();                     // both accumulators are free for the next segment
-            if (!final) {
+            if (!final && !clustered) {
                 // This CTA's part is in the workspace: take the unit's ticket.  One thread orders the
                 // CTA's stores (the barrier above collected them) and draws; the answer is looked at
                 // after the CTA's last segment.
@@ -471,6 +552,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             t += sg.len;
         }
         if (tid256 == 0) HT_TR_CTA(2);
+        if (clustered) {
+            const bool had_tiles = t_end > t_begin;
+            if (!had_tiles && s == 0) {                // an empty share still delivers a part: nothing seen
+                float *pslot = reinterpret_cast<float *>(&sm.ring[0][0]);
+                pslot[kRows * kD + row] = -INFINITY;
+                pslot[kRows * kD + kRows + row] = 0.f;
+            }
+            const int unit = (int)blockIdx.x / p.cluster_k, b = unit / p.Hkv;
+            cluster_exchange<kBf16>(p, sm, (int)c_rank, b, unit - b * p.Hkv, sm.nkt[b] > 0, tid256, abort_flag);
+        }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
         if (cut[0].valid || cut[1].valid) {
             if (tid256 == 0)
@@ -489,6 +580,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // ------------------------------- teardown -------------------------------
     tc_fence_before();
     __syncthreads();
+    if (clustered) cluster_sync_all();       // no CTA leaves while a peer may still write into its shared memory
     if (threadIdx.x == 0) HT_TR_CTA(3);
     if (sm.abort && threadIdx.x == 0) {
         for (int b = 0; b < p.B; ++b)
@@ -549,6 +641,17 @@ bool attn_tc_applicable(const ht_attn_desc &d) {
 static int row_tiles(const ht_attn_desc &d) { return (d.N * (d.Hq / d.Hkv) + tc::kRows - 1) / tc::kRows; }
 static bool pair_mode(const ht_attn_desc &d) { return row_tiles(d) >= 2; }
 static int units_per_head(const ht_attn_desc &d) { return pair_mode(d) ? (row_tiles(d) + 1) / 2 : 1; }
+
+// Cluster size for the one-tile kernel when the (sequence, KV head) units are so few that a CTA
+// per unit would leave most SMs idle: the largest of 8, 4, 2 whose clusters fit the GPU at once.
+static int cluster_size(const ht_attn_desc &d) {
+    if (pair_mode(d)) return 0;
+    const long long units = (long long)d.B * d.Hkv;
+    const int sms = sm_count();
+    for (int k = 8; k >= 2; k /= 2)
+        if (units * k <= sms) return k;
+    return 0;
+}
 
 static size_t ticket_bytes(const ht_attn_desc &d) {
     const size_t units = (size_t)d.B * d.Hkv * units_per_head(d);
@@ -631,17 +734,45 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     p.scale_log2 = scale * 1.4426950408889634f;
     p.is_bf16 = d.dtype == HT_BF16;
     p.grid = sm_count();
+    p.cluster_k = 0;
 #ifdef HT_TC_TRACE
     p.trace = g_trace;
 #endif
     const size_t smem = sizeof(tc::Smem) + 1024;
     const long long units = (long long)d.B * d.Hkv * p.n_rt;
     if (units > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "too many (sequence, head, row tile) units");
-    cudaError_t e = cudaMemsetAsync(p.tickets, 0, (size_t)units * sizeof(unsigned int), s);
+    const int k = cluster_size(d);
+    cudaError_t e = cudaSuccess;
+    if (k <= 1) e = cudaMemsetAsync(p.tickets, 0, (size_t)units * sizeof(unsigned int), s);   // clusters use no tickets
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
     if (pair_mode(d)) return launch_attn_tc_pair_kernel(tm_q, tm_k, tm_v, p, d.dtype == HT_BF16, s);
     e = ensure_smem_attr(smem);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    // Few (sequence, KV head) units: one cluster of 8, 4 or 2 CTAs per unit, parts reduced through
+    // distributed shared memory; otherwise one persistent CTA per SM.
+    if (k > 1) {
+        p.cluster_k = k;
+        p.grid = (int)units * k;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)p.grid);
+        cfg.blockDim = dim3(tc::kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)k;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = d.dtype == HT_BF16 ? cudaLaunchKernelEx(&cfg, tc::attn_tc_kernel<true>, tm_q, tm_k, tm_v, p)
+                               : cudaLaunchKernelEx(&cfg, tc::attn_tc_kernel<false>, tm_q, tm_k, tm_v, p);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(HT_ERR_CUDA, "ht_tree_attention (tcgen05, clusters of %d): %s", k, cudaGetErrorString(e));
+        }
+        return HT_OK;
+    }
     if (d.dtype == HT_BF16) tc::attn_tc_kernel<true><<<p.grid, tc::kThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
     else tc::attn_tc_kernel<false><<<p.grid, tc::kThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
     return check_launch("ht_tree_attention (tcgen05)");

@@ -32,6 +32,7 @@ struct Params {
     float scale_log2;
     int is_bf16;
     int grid;
+    int cluster_k;         // > 1: launched as clusters of this many CTAs, one cluster per (sequence, KV head)
 #ifdef HT_TC_TRACE
     long long *trace;
 #endif
@@ -56,6 +57,7 @@ struct __align__(1024) Smem {
     int32_t nkt[kMaxB];
     int32_t pre[kMaxB + 1];
     unsigned long long kv_full[kStages], kv_empty[kStages], q_full, q_empty, s_full[2], p_ready[2], o_done[2], mma_drain;
+    unsigned long long xb[2];          // cluster exchange: peers ready to receive / all parts delivered
     uint32_t tmem_base;
     int abort;
     int merge_here[2];
@@ -170,6 +172,49 @@ __device__ __forceinline__ unsigned int ld_relaxed_gpu(const unsigned int *ptr) 
     unsigned int v;
     asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
     return v;
+}
+
+// ---- thread-block cluster: rank, peer shared memory, barriers in a peer's shared memory ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_peer(uint32_t local_smem_addr, uint32_t rank) {
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_smem_addr), "r"(rank));
+    return ra;
+}
+__device__ __forceinline__ void st_peer_f4(uint32_t peer_addr, float4 v) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(peer_addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_peer_f1(uint32_t peer_addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_peer(uint32_t peer_bar_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(peer_bar_addr) : "memory");
+}
+// Bounded wait on a barrier of this CTA that peers arrive on.
+__device__ __forceinline__ bool mbar_wait_cluster(void *bar, uint32_t parity, volatile int *abort_flag) {
+    if (*abort_flag) return false;
+    const uint32_t addr = smem_u32(bar);
+    long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 2000000000ll) { *abort_flag = 1; return false; }
+        }
+    }
+}
+__device__ __forceinline__ void cluster_sync_all() {   // every thread of every CTA of the cluster
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;

@@ -138,6 +138,67 @@ def test_attention_custom_scale_and_strided_layer_view(hb, oracle):
     assert_close(f32np(out), ref, dt, "strided")
 
 
+# Shapes that select each work split of the tensor-core kernels (16-bit, head size 128):
+# few (sequence, KV head) units -> clusters of 8 / 4 / 2 CTAs reducing through distributed shared
+# memory (with empty shares when a unit has fewer tiles than the cluster has CTAs); many units ->
+# persistent CTAs with whole units, or with units cut between CTAs (ticket merge / direct merge);
+# more than 128 rows per KV head -> tile pairs, with and without a second tile, cut and uncut.
+SPLIT_CASES = [
+    # B, N, Hq, Hkv, lens, tree
+    (1, 5, 2, 2, [0], "chain"),                       # clusters of 8, one tile, seven empty shares
+    (1, 91, 32, 32, [2048], "random"),                # clusters of 4, 17 tiles over 4 CTAs
+    (2, 20, 32, 32, [700, 129], "random"),            # clusters of 2, ragged
+    (3, 64, 8, 4, [1500, 3, 800], "random"),          # clusters of 8, ragged, a nearly empty sequence
+    (5, 37, 32, 32, [900, 640, 33, 1200, 512], "random"),   # 160 units: persistent, ragged, cut units
+    (4, 30, 40, 40, [1024] * 4, "random"),            # 160 units of 9 tiles: persistent, equal lengths
+    (2, 19, 64, 8, [3000, 2500], "random"),           # 152 rows: a pair whose second tile is small; cut units
+    (9, 40, 16, 2, [200, 300, 100, 150, 260, 90, 310, 128, 5], "random"),   # 320 rows: pair + single tile
+    (1, 300, 8, 1, [1000], "random"),                 # 2400 rows: 19 tiles, 10 units
+]
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("case", SPLIT_CASES, ids=lambda c: "B%dN%dHq%dHkv%d" % c[:4])
+def test_attention_every_work_split(hb, oracle, dtype, case):
+    B, N, Hq, Hkv, lens, tree = case
+    cap = max(lens) + N + 5
+    q, k, v, kv_len, parent = make_attn_case(15, dtype, B, N, Hq, Hkv, 128, lens, cap, tree)
+    out, status = hb.tree_attention(q, k, v, kv_len, parent)
+    assert status.cpu().tolist() == [0] * B
+    n_units = 8 if B * Hkv > 16 else B * Hkv
+    check_sampled_units(hb, oracle, q, k, v, kv_len.cpu().numpy(), parent, out, n_units, DT[dtype], seed=B, p_rounding=True)
+    # A second call agrees to the last place or the one next to it: which CTA merges a cut unit, and
+    # from registers or from the workspace, depends on arrival order, and so does the rounding order.
+    out2, _ = hb.tree_attention(q, k, v, kv_len, parent)
+    a, b2 = out.float(), out2.float()
+    ulp = 2.0 ** -7 if dtype == "bf16" else 2.0 ** -10
+    assert bool(((a - b2).abs() <= ulp * a.abs() + 1e-6).all())
+
+
+@pytest.mark.parametrize("shape", [(3, 9, 4, 2), (3, 40, 32, 8), (40, 9, 8, 4)], ids=lambda s: "B%dN%dHq%dHkv%d" % s)
+def test_attention_tensor_core_paths_skip_bad_sequences(hb, oracle, shape):
+    """Status words and untouched rows on the 16-bit kernels (clusters, tile pairs, persistent)."""
+    B, N, Hq, Hkv = shape
+    lens = [10 + 7 * b for b in range(B)]
+    cap = max(lens) + N + 3
+    q, k, v, kv_len, parent = make_attn_case(16, "bf16", B, N, Hq, Hkv, 128, lens, cap, garbage=False)
+    parent[1, N - 1] = N - 1              # not an earlier row
+    kv_len[2] = cap - N + 1               # does not fit
+    out = torch.full_like(q, 7.0)
+    out, status = hb.tree_attention(q, k, v, kv_len, parent, out=out)
+    torch.cuda.synchronize()
+    want = [hb.HT_STATUS_OK] * B
+    want[1], want[2] = hb.HT_STATUS_BAD_TREE, hb.HT_STATUS_BAD_LEN
+    assert status.cpu().tolist() == want
+    assert (out[1:3] == 7.0).all()
+    good_parent = parent.clone()
+    good_parent[1, N - 1] = -1
+    kv_len[2] = lens[2]
+    ref = oracle_attn(oracle, q, k, v, kv_len, good_parent)
+    for b in [0] + list(range(3, min(B, 6))):
+        assert_close(f32np(out[b]), ref[b], torch.bfloat16, "good sequence %d" % b)
+
+
 def test_attention_flags_bad_sequences_and_leaves_their_rows_alone(hb, oracle):
     q, k, v, kv_len, parent = make_attn_case(14, "f32", 3, 9, 4, 2, 64, [10, 20, 30], 64, garbage=False)
     parent[1, 4] = 4                      # not an earlier row
@@ -162,7 +223,23 @@ def _sample_units(rng, B, Hkv, n):
     return sorted(units)
 
 
-def check_sampled_units(hb, oracle, q, k, v, kv_len, parent, out, n_units, dtype, seed=0):
+def assert_close_with_p_rounding(got, ref, ref_abs_v, dtype, what=""):
+    """The 16-bit bound plus the one term the arithmetic adds when few keys carry a row's weight:
+    the tensor-core product takes the softmax weights rounded to the input type (relative error
+    2^-9 for bf16, 2^-11 for fp16), which moves an output by at most that fraction of
+    sum_i w_i |v_i| -- the attention output of |V|, which the oracle supplies.  With thousands of
+    diffuse weights the term is invisible; with three visible keys and cancelling values it is not."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert np.isfinite(got).all(), what + ": non-finite output"
+    eps_p = 2.0 ** -9 if dtype == torch.bfloat16 else 2.0 ** -11
+    bound = 2e-3 + 1e-2 * np.abs(ref) + eps_p * np.asarray(ref_abs_v, dtype=np.float64)
+    err = np.abs(got - ref)
+    worst = (err - bound).max()
+    assert worst <= 0, "%s: max abs err %.3e (over bound by %.3e)" % (what, err.max(), worst)
+
+
+def check_sampled_units(hb, oracle, q, k, v, kv_len, parent, out, n_units, dtype, seed=0, p_rounding=False):
     """Full-size parity: all rows and query heads of a seeded sample of (sequence, KV head)
     units, each reduced to a B=1, Hkv=1 problem for the oracle."""
     B, N, Hq, D = q.shape
@@ -177,7 +254,11 @@ def check_sampled_units(hb, oracle, q, k, v, kv_len, parent, out, n_units, dtype
         vs = f32np(v[b:b + 1, hk:hk + 1, :L + N])
         ref = oracle.tree_attention(qs, ks, vs, np.array([L], np.int32), parent[b:b + 1].cpu().numpy())
         got = f32np(out[b:b + 1, :, hk * g:(hk + 1) * g])
-        assert_close(got, ref, dtype, "unit b=%d hk=%d" % (b, hk))
+        if p_rounding:
+            ref_abs_v = oracle.tree_attention(qs, ks, np.abs(vs), np.array([L], np.int32), parent[b:b + 1].cpu().numpy())
+            assert_close_with_p_rounding(got, ref, ref_abs_v, dtype, "unit b=%d hk=%d" % (b, hk))
+        else:
+            assert_close(got, ref, dtype, "unit b=%d hk=%d" % (b, hk))
         rows += N * g
     return rows
 
