@@ -60,23 +60,32 @@ __device__ __noinline__ void cluster_exchange(const Params &p, Smem &sm, int ran
     const float *own_ml = reinterpret_cast<const float *>(ring) + kRows * kD;
     float4 *recv4 = reinterpret_cast<float4 *>(ring + kXchgRecvOffset);          // [sender][group in slice][row]
     float *recv_ml = reinterpret_cast<float *>(ring + kXchgRecvOffset) + kRows * kD;   // [sender][m | l][row]
+    HT_TR(4, 30, 0);
     softmax_groups_sync();                              // this CTA's part is complete
     if (tid256 == 0)
         for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&sm.xb[0]), (uint32_t)c));
     mbar_wait_cluster(&sm.xb[0], 0, abort_flag);        // every peer's ring is idle
+    HT_TR(4, 31, 0);
     if (!*abort_flag) {
-        for (int idx = tid256; idx < 32 * kRows; idx += 256) {
-            const int cg = idx >> 7, r = idx & 127, c = cg / cg_per_slice, x = cg - c * cg_per_slice;
-            st_peer_f4(map_to_peer(smem_u32(recv4 + (rank * cg_per_slice + x) * kRows + r), (uint32_t)c), own4[idx]);
+        // thread t moves rows t & 127 of feature groups (t >> 7) + 2 j; k is a power of two
+        const int sh = 5 - __ffs(k) + 1;                // log2(cg_per_slice)
+        const uint32_t recv_base = smem_u32(recv4 + rank * cg_per_slice * kRows + (tid256 & 127));
+#pragma unroll 4
+        for (int j = 0; j < 16; ++j) {
+            const int cg = (tid256 >> 7) + 2 * j, c = cg >> sh, x = cg & (cg_per_slice - 1);
+            st_peer_f4(map_to_peer(recv_base + x * kRows * 16, (uint32_t)c), own4[cg * kRows + (tid256 & 127)]);
         }
         const float ml = own_ml[tid256];                // 128 m then 128 l
         for (int c = 0; c < k; ++c) st_peer_f1(map_to_peer(smem_u32(recv_ml + rank * 2 * kRows + tid256), (uint32_t)c), ml);
     }
+    HT_TR(4, 32, 0);
     asm volatile("fence.acq_rel.cluster;" ::: "memory");
     softmax_groups_sync();
+    HT_TR(4, 33, 0);
     if (tid256 == 0)
         for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&sm.xb[1]), (uint32_t)c));
     mbar_wait_cluster(&sm.xb[1], 0, abort_flag);        // every part has arrived here
+    HT_TR(4, 34, 0);
     const int row = tid256 & 127, half = tid256 >> 7;
     const int node = row / p.g;
     if (!valid || node >= p.N || *abort_flag) return;
@@ -126,6 +135,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         for (int i = 0; i < 2; ++i) { mbar_init(&sm.s_full[i], 1); mbar_init(&sm.p_ready[i], 128); mbar_init(&sm.o_done[i], 1); }
         sm.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (threadIdx.x == 32) {                 // descriptors on their way while the CTA sets itself up
+        prefetch_tensormap(&tm_q);
+        prefetch_tensormap(&tm_k);
+        prefetch_tensormap(&tm_v);
     }
     if (warp == 8) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");

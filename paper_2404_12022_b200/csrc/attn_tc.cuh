@@ -106,6 +106,10 @@ __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, v
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(void *bar) {
@@ -310,6 +314,10 @@ __device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nk
 template <int NT>
 __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, int32_t *s_nkt, int32_t *s_pre,
                                                bool write_status) {
+    // The lengths are asked for first and used last, so that their round trip to memory overlaps
+    // the scan of the parent arrays (B <= kMaxB <= NT: one sequence per thread).
+    const int my_b = threadIdx.x;
+    const int my_L = my_b < p.B ? p.kv_len[my_b] : 0;
     for (int b = threadIdx.x; b < p.B; b += NT) s_nkt[b] = 0;       // 0 = legal so far
     __syncthreads();
     for (int i = threadIdx.x; i < p.B * p.N; i += NT) {
@@ -318,8 +326,8 @@ __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, 
         if (par < -1 || par >= c) s_nkt[b] = -1;                     // benign race: all writers store -1
     }
     __syncthreads();
-    for (int b = threadIdx.x; b < p.B; b += NT) {
-        const int L = p.kv_len[b];
+    if (my_b < p.B) {
+        const int b = my_b, L = my_L;
         int code = HT_STATUS_OK;
         if (s_nkt[b] < 0) code = HT_STATUS_BAD_TREE;
         if (L < 0 || (long long)L + p.N > p.cap) code = HT_STATUS_BAD_LEN;
