@@ -36,7 +36,7 @@ UNIT = "GB/s"
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4"])
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
@@ -44,10 +44,13 @@ def parse_args():
     ap.add_argument("--kv", type=int, default=0, help="override the KV length of c3 (profiling small cases)")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--simt", action="store_true", help="force the fp32-ALU attention kernel")
+    ap.add_argument("--eager", action="store_true", help="enqueue every library call from the host instead of replaying a CUDA graph of the step")
     ap.add_argument("--no-extras", action="store_true", help="skip e2e, cpu baseline and per-kernel timing")
     ap.add_argument("--sweep", default="", help="instead of the step benchmark, time ht_tree_attention alone on a set of "
                     "workloads and print one JSON line per point: 'configs' (c2, c2 at KV 2048, a c3 layer, c4) or "
                     "'c5' (the 48 grouped-query points) or 'c5-quick' (12 of them)")
+    ap.add_argument("--only", default="", help="with --sweep: keep the workloads whose name contains this text")
+    ap.add_argument("--sweep-reps", type=int, default=0, help="with --sweep: calls per graph (profiling small cases)")
     return ap.parse_args()
 
 
@@ -179,7 +182,7 @@ class ClockSampler:
         try:
             uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
             self.proc = subprocess.Popen(["nvidia-smi", "-i", uuid, "--query-gpu=" + self.QUERY,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -215,15 +218,15 @@ class ClockSampler:
 # DRAM traffic per launch of the attention kernel on a c3 layer, from the ncu capture summarised in
 # profiles/attn_tc_kernel_c3_layer.md (dram__bytes_read.sum + dram__bytes_write.sum).  It is only
 # reported while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.6e6,
-               "source": "paper_2404_12022_b200/csrc/attn_tc.cu",
-               "sha256": "1b044cd0f375668c8fa40579add77eb8132f52e19b7c7b8e2851f4c239b195f8"}
+NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.8e6,
+               "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh"],
+               "sha256": "d76973c628f86da03769293b941ef571a75d3782f42af551f63984b184db5c73"}
 
 
 def ncu_traffic(w):
     import hashlib
     try:
-        digest = hashlib.sha256(open(os.path.join(ROOT, NCU_TRAFFIC["source"]), "rb").read()).hexdigest()
+        digest = hashlib.sha256(b"".join(open(os.path.join(ROOT, f), "rb").read() for f in NCU_TRAFFIC["source"])).hexdigest()
     except OSError:
         return None
     if digest != NCU_TRAFFIC["sha256"] or w.name != NCU_TRAFFIC["workload"] or w.kv_len[0] != 4096 or w.B != 4:
@@ -266,14 +269,19 @@ def run_native(args):
             dist.barrier()
             torch.cuda.synchronize()
 
+    step.run(stream)                      # eager once: per-device set-up inside the library
+    torch.cuda.synchronize()
+    if not args.eager:
+        step.capture()                    # the step as one CUDA graph: same kernels, no host work between them
+    run_step = (lambda: step.run(stream)) if args.eager else step.replay
     for _ in range(max(args.warmup, 3)):
-        step.run(stream)
+        run_step()
     barrier()
     sampler = ClockSampler(local) if rank == 0 else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
-        step.run(stream)
+        run_step()
     e1.record()
     barrier()
     ms_total = e0.elapsed_time(e1)
@@ -293,7 +301,8 @@ def run_native(args):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": w.dtype, "data": "synthetic", "config": workload_config(w, world),
-            "step_us": ms_step * 1e3, "step_bytes": step_bytes, "clocks": clocks}
+            "step_us": ms_step * 1e3, "step_bytes": step_bytes, "clocks": clocks,
+            "launch": "eager C-ABI calls" if args.eager else "CUDA graph of the step's C-ABI calls"}
     # launches of this library's kernels per step: attention (+ combine when split), transfer
     # (one per batch slice of 8), argmax + acceptance, compaction
     attn_launches = sum(1 for _ in range(step.layers))
@@ -437,7 +446,7 @@ def run_sweep(args):
     torch.cuda.set_device(0)
     peak, how = measured_peaks()
     l2 = torch.cuda.get_device_properties(0).L2_cache_size
-    for w in sweep_points(args.sweep):
+    for w in [x for x in sweep_points(args.sweep) if args.only in x.name]:
         inp = wl.make_inputs(w, "cuda", with_logits=False, with_transfer=False, layers=[w.layers - 1])
         q, kv_len, parent = inp.q[0], inp.kv_len, inp.parent
         e = w.elem_bytes()
@@ -451,7 +460,7 @@ def run_sweep(args):
         st = torch.zeros(w.B, dtype=torch.int32, device="cuda")
         desc = hb.make_attn_desc(q, ks[0])
         ws = torch.empty(max(hb.tree_attention_workspace(desc), 16), dtype=torch.uint8, device="cuda")
-        reps = max(nbuf, 16)
+        reps = args.sweep_reps or max(nbuf, 16)
         call = lambda i: hb.tree_attention(q, ks[i % nbuf], vs[i % nbuf], kv_len, parent, out=out, workspace=ws, status=st)
         for i in range(3):
             call(i)

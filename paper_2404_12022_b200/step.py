@@ -54,6 +54,7 @@ class VerifyStep:
         self.dtype_code = hb._DTYPES[kc.dtype]
         self.transfer_at = min(w.transfer_after_layer, self.layers)
         self.launches_per_step = 0
+        self.graph = None
 
     def attention(self, i: int, stream: int) -> None:
         inp = self.inp
@@ -99,6 +100,20 @@ class VerifyStep:
             self.transfer(s)
         self.verify(s)
         self.compact(s)
+
+    def capture(self) -> None:
+        """Record one whole step into a CUDA graph (after at least one eager ``run``, which does the
+        library's once-per-device set-up).  ``replay`` then enqueues the step with a single launch:
+        the same kernels on the same buffers, without per-call host work between them."""
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side), torch.cuda.graph(self.graph, stream=side):
+            self.run(side.cuda_stream)
+        torch.cuda.current_stream().wait_stream(side)
+
+    def replay(self) -> None:
+        self.graph.replay()
 
     # ---- algorithmic bytes (what each kernel must move at least once) ----
     def attention_bytes(self, i: int) -> int:
