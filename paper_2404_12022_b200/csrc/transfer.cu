@@ -12,6 +12,15 @@
 // before the first is used, which keeps over 100 KB of weight in flight per SM -- what a stream
 // needs to run at memory speed.  R x BT fp32 accumulators per lane, reduced with shuffles at
 // the end of a row group.  The R rows share each loaded h vector (h is small and cache resident).
+//
+// 16-bit inputs take a second kernel: unpacking bf16 / fp16 and multiplying on the fp32 ALUs costs
+// about 15 issue slots per weight element, which caps the stream near 3 TB/s.  The warp-level
+// tensor-core instruction (m16n8k16, fp32 accumulate) consumes the 16-bit words as loaded.  The
+// order of the contraction index is free as long as both operands agree, so each lane loads
+// plain 16-byte vectors (8 consecutive features of one weight row, the same 8 features of one
+// batch row) and the pairs of those vectors are dealt to the instruction's k slots in place:
+// no shuffles, no shared memory.  (tcgen05 would stage both operands through shared memory for
+// an M = 128 tile; with 4 to 16 batch columns this skinny product gains nothing from it.)
 #include "ht_common.cuh"
 
 namespace ht {
@@ -121,12 +130,106 @@ static int launch_typed(const void *h, const void *W, void *out, int B, int k, i
     return HT_OK;
 }
 
+
+// ---------------------------------------------------------------------------------------
+// 16-bit inputs: m16n8k16 tensor-core products on the words as loaded
+// ---------------------------------------------------------------------------------------
+template <typename T> struct MmaOp;
+template <> struct MmaOp<__half> {
+    static __device__ __forceinline__ void run(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    }
+};
+template <> struct MmaOp<__nv_bfloat16> {
+    static __device__ __forceinline__ void run(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    }
+};
+
+// A warp owns an equal, contiguous share of the groups of 16 weight rows.  Lane (g, t) = (lane / 4,
+// lane % 4) loads features [f + 8 t, f + 8 t + 8) of rows g and g + 8 of the group and of batch row
+// g of each 8-column batch tile; words 0 / 1 of those vectors fill k slots (2t, 2t+1) / (2t+8, 2t+9)
+// of one instruction, words 2 / 3 those of a second one.  U steps of 32 features are loaded before
+// the first is used.  The accumulator fragment holds rows g, g + 8 and batch columns 2t, 2t + 1.
+template <typename T, int NB, int U>
+__global__ void __launch_bounds__(128, kTransferBlocksPerSm)
+transfer_mma_kernel(const T *__restrict__ h, const T *__restrict__ W, T *__restrict__ out,
+                    int rows_total, int d, int b0, int nb) {
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const long long warp = (long long)blockIdx.x * 4 + (threadIdx.x >> 5), n_warps = (long long)gridDim.x * 4;
+    const int groups = (rows_total + 15) / 16;
+    const int g_begin = (int)(warp * groups / n_warps), g_end = (int)((warp + 1) * groups / n_warps);
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+
+    for (int grp = g_begin; grp < g_end; ++grp) {
+        const int r0 = grp * 16;
+        const T *wa_row = W + (size_t)min(r0 + g, rows_total - 1) * d;        // rows past the end repeat the last one
+        const T *wb_row = W + (size_t)min(r0 + g + 8, rows_total - 1) * d;
+        float acc[NB][4];
+#pragma unroll
+        for (int n = 0; n < NB; ++n)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[n][i] = 0.f;
+
+        for (int fb = 0; fb < d; fb += 32 * U) {             // warp-uniform trip count: the products are warp-wide
+            uint4 wa[U], wb[U], hb[U][NB];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int f = fb + u * 32 + t * 8;
+                const bool in = f < d;                                           // d is a multiple of 8
+                wa[u] = in ? ld_nc16(wa_row + f) : zero;
+                wb[u] = in ? ld_nc16(wb_row + f) : zero;
+#pragma unroll
+                for (int n = 0; n < NB; ++n) {
+                    const int b = n * 8 + g;
+                    hb[u][n] = (in && b < nb) ? *reinterpret_cast<const uint4 *>(h + (size_t)(b0 + b) * d + f) : zero;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int n = 0; n < NB; ++n) {
+                    MmaOp<T>::run(acc[n], wa[u].x, wb[u].x, wa[u].y, wb[u].y, hb[u][n].x, hb[u][n].y);
+                    MmaOp<T>::run(acc[n], wa[u].z, wb[u].z, wa[u].w, wb[u].w, hb[u][n].z, hb[u][n].w);
+                }
+        }
+#pragma unroll
+        for (int n = 0; n < NB; ++n)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = r0 + g + (i >> 1) * 8, b = n * 8 + 2 * t + (i & 1);
+                if (row < rows_total && b < nb) out[(size_t)(b0 + b) * rows_total + row] = from_float<T>(acc[n][i]);
+            }
+    }
+}
+
+template <typename T, int NB, int U>
+static int launch_mma(const void *h, const void *W, void *out, int rows_total, int d, int b0, int nb, cudaStream_t s) {
+    transfer_mma_kernel<T, NB, U><<<transfer_grid(rows_total, 16), 128, 0, s>>>(
+        static_cast<const T *>(h), static_cast<const T *>(W), static_cast<T *>(out), rows_total, d, b0, nb);
+    return check_launch("ht_transfer");
+}
+
+template <typename T>
+static int launch_typed16(const void *h, const void *W, void *out, int B, int k, int d, cudaStream_t s) {
+    const int rows_total = k * d;
+    for (int b0 = 0; b0 < B; b0 += 16) {
+        const int nb = min(16, B - b0);
+        const int rc = nb <= 8 ? launch_mma<T, 1, 8>(h, W, out, rows_total, d, b0, nb, s)
+                               : launch_mma<T, 2, 4>(h, W, out, rows_total, d, b0, nb, s);
+        if (rc != HT_OK) return rc;
+    }
+    return HT_OK;
+}
+
 int launch_transfer(const void *h, const void *W, void *out, int B, int k, int d, int dtype,
                     cudaStream_t s) {
     switch (dtype) {
         case HT_F32: return launch_typed<float>(h, W, out, B, k, d, s);
-        case HT_F16: return launch_typed<__half>(h, W, out, B, k, d, s);
-        default: return launch_typed<__nv_bfloat16>(h, W, out, B, k, d, s);
+        case HT_F16: return launch_typed16<__half>(h, W, out, B, k, d, s);
+        default: return launch_typed16<__nv_bfloat16>(h, W, out, B, k, d, s);
     }
 }
 
