@@ -169,6 +169,35 @@ int ht_kv_compact(void *k_cache, void *v_cache, const ht_cache_desc *desc /* hos
                   int max_path, int32_t *new_kv_len, int32_t *status, void *stream);
 
 /*
+ * Draft tree for the next round -- Section "Inference stage" (the candidate sequences are made
+ * "into a tree structure by merging their common ancestors" and the tree is flattened) and Section
+ * "Tree attention" ("a pre-defined tree structure and parser"; tokens keep their positional indices).
+ * The candidates are the most likely tokens of the pseudo positions' distributions (Section "Hidden
+ * Transfer": the lm-head decodes the pseudo hidden states).  The pre-defined structure is a template
+ * shared by all sequences: node n at level i takes the tmpl_rank[n]-th most likely token (0 = the
+ * most likely) of pseudo position i, so merging common ancestors costs nothing at run time.
+ *   logits      [B, rows, V] of `dtype`; pseudo position i (1..P) of sequence b is row first_row + i - 1
+ *   tmpl_parent [T] int32, tmpl_parent[n] in [-1, n)
+ *   tmpl_rank   [T] int32, in [0, K) for nodes of level >= 1
+ *   root_token  [B] int32 or NULL.  Given: nodes with parent -1 are the known next token (level 0,
+ *               e.g. next_token of ht_verify_greedy) and their children are level 1.  NULL: nodes
+ *               with parent -1 are level 1 themselves (a forest of first drafts).
+ *   base_pos    [B] int32: position id of the top-level nodes (e.g. new_kv_len of ht_kv_compact)
+ *   topk        [B, P, K] out: the K most likely tokens per pseudo position -- larger value first,
+ *               lower index first among equal values, NaN below everything
+ *   tokens      [B, T] out: draft token of every template node
+ *   pos         [B, T] out: base_pos[b] + depth of the node (top-level nodes: depth 0)
+ *   status      [B] out: HT_STATUS_BAD_TREE when the template is malformed (a parent that is not an
+ *               earlier node, a level beyond P, a rank outside [0, K)); tokens and pos are then -1.
+ * 1 <= K <= 16, K <= V, T >= 1.  B == 0 is a no-op.  The parent array of the next round's
+ * ht_tree_attention is tmpl_parent followed by the pseudo rows.
+ */
+int ht_draft_tree(const void *logits, int dtype, int B, int rows, int V, int first_row, int P, int K,
+                  const int32_t *tmpl_parent, const int32_t *tmpl_rank, int T, const int32_t *root_token,
+                  const int32_t *base_pos, int32_t *topk, int32_t *tokens, int32_t *pos, int32_t *status,
+                  void *stream);
+
+/*
  * Tree attention without a caller-provided workspace.  (The paper has no counterpart: this
  * entry point exists for integration, not for the method.)
  *

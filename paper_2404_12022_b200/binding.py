@@ -23,7 +23,7 @@ HT_STATUS_OK, HT_STATUS_BAD_TREE, HT_STATUS_BAD_LEN, HT_STATUS_BAD_PATH, HT_STAT
 HT_ATTN_FORCE_SIMT = 1
 
 EXPORTS = ("ht_version", "ht_last_error_string", "ht_transfer", "ht_tree_attention_workspace",
-           "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact", "ht_tree_attention_static")
+           "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact", "ht_draft_tree", "ht_tree_attention_static")
 HT_STATIC_SCRATCH_BYTES = 16 << 20
 
 _DTYPES = {torch.float32: HT_F32, torch.float16: HT_F16, torch.bfloat16: HT_BF16}
@@ -77,6 +77,8 @@ def load() -> ctypes.CDLL:
         lib.ht_verify_greedy.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         lib.ht_kv_compact.restype = i32
         lib.ht_kv_compact.argtypes = [vp, vp, ctypes.POINTER(CacheDesc), vp, vp, vp, i32, vp, vp, vp]
+        lib.ht_draft_tree.restype = i32
+        lib.ht_draft_tree.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
         _lib = lib
     return _lib
 
@@ -231,3 +233,26 @@ def kv_compact(k_cache, v_cache, n_rows: int, kv_len, accept_len, accept_path, n
                                 _ptr(accept_len), _ptr(accept_path), max_path, _ptr(new_kv_len),
                                 _ptr(status), _stream()))
     return new_kv_len, status
+
+
+def draft_tree(logits, first_row: int, P: int, K: int, tmpl_parent, tmpl_rank, root_token, base_pos):
+    """logits [B, rows, V]; pseudo position i (1..P) is row first_row + i - 1; tmpl_parent, tmpl_rank
+    [T] int32; root_token [B] int32 or None; base_pos [B] int32.
+    Returns (topk [B, P, K], tokens [B, T], pos [B, T], status [B])."""
+    _need(logits, name="logits")
+    _need(tmpl_parent, torch.int32, "tmpl_parent")
+    _need(tmpl_rank, torch.int32, "tmpl_rank")
+    _need(base_pos, torch.int32, "base_pos")
+    if root_token is not None:
+        _need(root_token, torch.int32, "root_token")
+    B, rows, V = logits.shape
+    T = tmpl_parent.shape[0]
+    dev = logits.device
+    topk = torch.empty((B, P, K), dtype=torch.int32, device=dev)
+    tokens = torch.empty((B, T), dtype=torch.int32, device=dev)
+    pos = torch.empty((B, T), dtype=torch.int32, device=dev)
+    status = torch.empty(B, dtype=torch.int32, device=dev)
+    _check(load().ht_draft_tree(_ptr(logits), _DTYPES[logits.dtype], B, rows, V, first_row, P, K, _ptr(tmpl_parent),
+                                _ptr(tmpl_rank), T, _ptr(root_token), _ptr(base_pos), _ptr(topk), _ptr(tokens),
+                                _ptr(pos), _ptr(status), _stream()))
+    return topk, tokens, pos, status

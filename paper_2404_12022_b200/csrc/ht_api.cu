@@ -140,4 +140,22 @@ int ht_kv_compact(void *k_cache, void *v_cache, const ht_cache_desc *desc, const
                           static_cast<cudaStream_t>(stream));
 }
 
+int ht_draft_tree(const void *logits, int dtype, int B, int rows, int V, int first_row, int P, int K,
+                  const int32_t *tmpl_parent, const int32_t *tmpl_rank, int T, const int32_t *root_token,
+                  const int32_t *base_pos, int32_t *topk, int32_t *tokens, int32_t *pos, int32_t *status,
+                  void *stream) {
+    if (B < 0 || rows < 0 || P < 0 || first_row < 0) return fail(HT_ERR_INVALID_ARG, "negative size");
+    if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if (B == 0) return HT_OK;
+    if (T <= 0 || V <= 0) return fail(HT_ERR_INVALID_ARG, "T and V must be positive");
+    if (K < 1 || K > 16 || K > V) return fail(HT_ERR_INVALID_ARG, "K = %d must lie in [1, min(16, V)]", K);
+    if ((long long)first_row + P > rows) return fail(HT_ERR_INVALID_ARG, "pseudo rows [%d, %d) exceed the %d rows", first_row, first_row + P, rows);
+    if (!tmpl_parent || !tmpl_rank || !base_pos || !tokens || !pos || !status || (P > 0 && (!logits || !topk)))
+        return fail(HT_ERR_INVALID_ARG, "NULL pointer");
+    if (P > 0 && !aligned16(logits)) return fail(HT_ERR_INVALID_ARG, "logits must be 16-byte aligned");
+    if ((long long)B * (P > 0 ? P : 1) > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "B*P too large");
+    return launch_draft(logits, dtype, B, rows, V, first_row, P, K, tmpl_parent, tmpl_rank, T, root_token, base_pos,
+                        topk, tokens, pos, status, static_cast<cudaStream_t>(stream));
+}
+
 }  // extern "C"

@@ -67,6 +67,13 @@ def test_host_side_rejections(lib):
     c = hb.CacheDesc(2, 1, 4, 64, 3, hb.HT_BF16, 8, 0, 0, 0)                   # 6-byte rows
     assert lib.ht_kv_compact(p, p, ctypes.byref(c), p, p, p, 8, p, p, None) == hb.HT_ERR_UNSUPPORTED
 
+    # ht_draft_tree(logits, dtype, B, rows, V, first_row, P, K, tmpl_parent, tmpl_rank, T, root, base, topk, tokens, pos, status, stream)
+    assert lib.ht_draft_tree(p, hb.HT_F16, 1, 10, 100, 7, 3, 17, p, p, 5, None, p, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG   # K > 16
+    assert lib.ht_draft_tree(p, hb.HT_F16, 1, 10, 100, 8, 3, 4, p, p, 5, None, p, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG    # rows 8..10 of 10
+    assert lib.ht_draft_tree(p, hb.HT_F16, 1, 10, 3, 7, 3, 4, p, p, 5, None, p, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG      # K > V
+    assert lib.ht_draft_tree(p, hb.HT_F16, 1, 10, 100, 7, 3, 4, p, None, 5, None, p, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG
+    assert lib.ht_draft_tree(None, hb.HT_F16, 0, 10, 100, 7, 3, 4, None, None, 5, None, None, None, None, None, None, None) == hb.HT_OK
+
 
 def test_binding_refuses_cpu_tensors_and_has_no_fallback():
     import torch

@@ -517,3 +517,87 @@ def test_toy_lossless_loop_on_the_gpu(hb):
 
     for with_root in (True, False):
         assert run_lossless_loop(GpuOps(), with_root, seed=3, n_new=24, atol_cache=5e-4, D=64) < 24
+
+
+# ------------------------------------------------------------------------------------------
+# Draft tree for the next round (top tokens of the pseudo positions in a pre-defined tree)
+# ------------------------------------------------------------------------------------------
+
+def _template(rng, T, P, K, has_root):
+    parent, rank, depth = [], [], []
+    for n in range(T):
+        while True:
+            par = int(rng.integers(-1, n)) if n else -1
+            d = 0 if par < 0 else depth[par] + 1
+            if d + (0 if has_root else 1) <= P:
+                break
+        parent.append(par)
+        depth.append(d)
+        rank.append(int(rng.integers(0, K)))
+    return np.array(parent, np.int32), np.array(rank, np.int32)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("shape", [(1, 50, 3, 4, 15, True), (3, 1000, 2, 8, 40, False), (4, 32000, 3, 10, 88, False),
+                                   (2, 32003, 4, 16, 64, True)], ids=lambda s: "B%dV%dP%dK%dT%d%s" % (s[:5] + ("root" if s[5] else "",)))
+def test_draft_tree_matches_the_oracle_bit_for_bit(hb, dtype, shape):
+    from oracle import draft_oracle as do
+    B, V, P, K, T, has_root = shape
+    dt = DT[dtype]
+    rng = np.random.default_rng(V + K)
+    rows, first_row = T + P, T
+    x = np.round(rng.standard_normal((B, rows, V)) * 4) / 4               # coarse values: ties within the top K
+    x[0, first_row, 1] = np.nan
+    x[0, first_row, V // 3] = np.inf
+    x[B - 1, first_row + P - 1, :] = -np.inf
+    x[B - 1, first_row + P - 1, 5] = np.nan
+    logits = torch.from_numpy(x).to(dt).cuda()
+    parent, rank = _template(rng, T, P, K, has_root)
+    root = rng.integers(0, V, B).astype(np.int32) if has_root else None
+    base = rng.integers(0, 5000, B).astype(np.int32)
+    got = hb.draft_tree(logits, first_row, P, K, torch.from_numpy(parent).cuda(), torch.from_numpy(rank).cuda(),
+                        None if root is None else torch.from_numpy(root).cuda(), torch.from_numpy(base).cuda())
+    ref = do.draft_tree(f32np(logits), first_row, P, K, parent.tolist(), rank.tolist(), root, base)
+    for g, r, what in zip(got, ref, ("topk", "tokens", "pos", "status")):
+        assert np.array_equal(g.cpu().numpy(), r), what
+    assert ref[3].tolist() == [0] * B
+
+
+def test_draft_tree_flags_bad_templates(hb):
+    from oracle import draft_oracle as do
+    logits = wl.normal_tensor(41, 1, (2, 6, 500), "cuda", 1.0, torch.bfloat16)
+    base = torch.tensor([10, 20], dtype=torch.int32, device="cuda")
+    for parent, rank in (([-1, 1, 0], [0, 0, 0]), ([-1, 0, 1, 2], [0, 0, 0, 0]), ([-1, 0, 0], [0, 4, 0])):
+        got = hb.draft_tree(logits, 3, 2, 4, torch.tensor(parent, dtype=torch.int32, device="cuda"),
+                            torch.tensor(rank, dtype=torch.int32, device="cuda"), None, base)
+        ref = do.draft_tree(f32np(logits), 3, 2, 4, parent, rank, None, base.cpu().numpy())
+        for g, r in zip(got, ref):
+            assert np.array_equal(g.cpu().numpy(), r)
+        assert got[3].cpu().tolist() == [hb.HT_STATUS_BAD_TREE] * 2
+
+
+def test_draft_tree_closes_the_round_on_the_device(hb):
+    """verify -> compact -> draft: the next round's tree hangs off the verified next token at the
+    compacted length, without a host round trip in between (config 2 shapes)."""
+    from oracle import draft_oracle as do
+    w = wl.config_c2()
+    inp = wl.make_inputs(w, "cuda")
+    pred, alen, apath, nxt, vst = hb.verify_greedy(inp.logits, inp.tokens, inp.parent, inp.root_pred, w.max_path)
+    new_len, cst = hb.kv_compact(inp.k_cache, inp.v_cache, w.N, inp.kv_len, alen, apath)
+    parent = np.concatenate([[-1], inp.parent_tree.cpu().numpy()[0] + 1]).astype(np.int32)    # a root above the (4,3,2,2) forest
+    parent[1:][inp.parent_tree.cpu().numpy()[0] < 0] = 0
+    depth = do.template_depths(parent.tolist())
+    rng = np.random.default_rng(3)
+    rank = np.array([0] + [int(rng.integers(0, 4)) for _ in range(w.T)], np.int32)
+    assert max(depth) == 4                                    # four levels below the root need four pseudo rows: use P = 3 and cut
+    keep = np.array([d <= w.P for d in depth])
+    remap = np.cumsum(keep) - 1
+    parent = np.array([-1 if parent[n] < 0 else remap[parent[n]] for n in range(len(parent)) if keep[n]], np.int32)
+    rank = rank[keep]
+    got = hb.draft_tree(inp.logits, w.T, w.P, 4, torch.from_numpy(parent).cuda(), torch.from_numpy(rank).cuda(), nxt, new_len)
+    torch.cuda.synchronize()
+    ref = do.draft_tree(f32np(inp.logits), w.T, w.P, 4, parent.tolist(), rank.tolist(), nxt.cpu().numpy(), new_len.cpu().numpy())
+    for g, r in zip(got, ref):
+        assert np.array_equal(g.cpu().numpy(), r)
+    assert got[1][0, 0].item() == nxt[0].item() and got[2][0, 0].item() == new_len[0].item()
+
