@@ -36,7 +36,7 @@ UNIT = "GB/s"
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4"])
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
@@ -303,10 +303,10 @@ def run_native(args):
             "vs_baseline": None, "dtype": w.dtype, "data": "synthetic", "config": workload_config(w, world),
             "step_us": ms_step * 1e3, "step_bytes": step_bytes, "clocks": clocks,
             "launch": "eager C-ABI calls" if args.eager else "CUDA graph of the step's C-ABI calls"}
-    # launches of this library's kernels per step: attention (+ combine when split), transfer
-    # (one per batch slice of 8), argmax + acceptance, compaction
+    # launches of this library's kernels per step: one per attention call, transfer (one per batch
+    # slice of 16), verification (argmax and acceptance in one), compaction
     attn_launches = sum(1 for _ in range(step.layers))
-    line["gpu_launches"] = args.steps * (attn_launches * kernels_per_attention(step) + ((w.B + 7) // 8) + 2 + 1)
+    line["gpu_launches"] = args.steps * (attn_launches * kernels_per_attention(step) + ((w.B + 15) // 16) + 1 + 1)
 
     if rank == 0 and not args.no_extras:
         line["roofline"], line["kernels"] = per_kernel_pass(args, step, stream, torch)

@@ -2,8 +2,10 @@
 // row argmax of the logits, then the longest root path of the draft tree whose tokens
 // are the ones greedy decoding would emit.
 //
-// Kernel 1 streams the logits once (HBM-bound scan, 16-byte loads, shuffle reductions);
-// kernel 2 is a few hundred integer operations per sequence.
+// One launch: a block per logits row streams it once (16-byte loads, eight in flight per thread,
+// shuffle reductions) and stores the row's argmax; the block that finishes a sequence's last row
+// (a ticket per sequence, drawn on the accept_len word, which a memset clears ahead of the launch)
+// runs the path search for that sequence -- a few hundred integer operations.  Nobody waits.
 #include <limits.h>
 
 #include "ht_common.cuh"
@@ -20,9 +22,86 @@ __device__ __forceinline__ Best better(Best a, Best b) {
     return (b.v > a.v || (b.v == a.v && b.i < a.i)) ? b : a;
 }
 
+// Path search of one sequence by one block.  Every thread walks the root path of its nodes (parent[c] < c
+// makes the walk finite), checks the match rule on the way and proposes (depth, node);
+// the block keeps the deepest valid node, lowest index on ties.
+__device__ __forceinline__ void accept_sequence(const int b, const int32_t *__restrict__ tokens, const int32_t *__restrict__ parent,
+              const int32_t *__restrict__ root_pred, const int32_t *pred, int N, int T,
+              int max_path, int32_t *accept_len, int32_t *__restrict__ accept_path,
+              int32_t *__restrict__ next_token, int32_t *__restrict__ status) {
+    const int32_t *par = parent + (size_t)b * N;
+    const int32_t *tok = tokens + (size_t)b * T;
+    const int32_t *prd = pred + (size_t)b * N;
+    int32_t *path = accept_path + (size_t)b * max_path;
+    __shared__ int s_bad;
+    __shared__ unsigned long long s_key[8];
+    if (threadIdx.x == 0) s_bad = 0;
+    __syncthreads();
+    for (int c = threadIdx.x; c < N; c += blockDim.x)
+        if (par[c] < -1 || par[c] >= c) s_bad = 1;
+    for (int j = threadIdx.x; j < max_path; j += blockDim.x) path[j] = -1;
+    __syncthreads();
+    if (s_bad) {
+        if (threadIdx.x == 0) {
+            status[b] = HT_STATUS_BAD_TREE;
+            accept_len[b] = 0;
+            next_token[b] = -1;
+        }
+        return;
+    }
+    const bool has_root = root_pred != nullptr;
+    const int rp = has_root ? root_pred[b] : -1;
+    // key = depth << 32 | (0xFFFFFFFF - node): max picks the deepest, then the lowest node
+    unsigned long long key = 0;
+    for (int n = threadIdx.x; n < T; n += blockDim.x) {
+        int depth = 0;
+        bool ok = true;
+        for (int c = n; c >= 0; c = par[c]) {
+            const int p = par[c];
+            const bool m = p < 0 ? (!has_root || tok[c] == rp) : (tok[c] == __ldcg(prd + p));
+            ok = ok && m;
+            ++depth;
+        }
+        if (ok) {
+            const unsigned long long k2 = ((unsigned long long)depth << 32) | (0xFFFFFFFFu - (unsigned)n);
+            key = k2 > key ? k2 : key;
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, key, off);
+        key = o > key ? o : key;
+    }
+    if ((threadIdx.x & 31) == 0) s_key[threadIdx.x >> 5] = key;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) key = s_key[w] > key ? s_key[w] : key;
+        const int len = (int)(key >> 32);
+        const int node = (int)(0xFFFFFFFFu - (unsigned)(key & 0xFFFFFFFFu));
+        if (len > max_path) {
+            status[b] = HT_STATUS_PATH_TOO_LONG;
+            accept_len[b] = 0;
+            next_token[b] = -1;
+        } else {
+            status[b] = HT_STATUS_OK;
+            accept_len[b] = len;
+            if (len == 0) {
+                next_token[b] = has_root ? rp : -1;
+            } else {
+                int j = len - 1;
+                for (int c = node; c >= 0; c = par[c]) path[j--] = c;
+                next_token[b] = __ldcg(prd + node);
+            }
+        }
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256)
-row_argmax_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pred) {
+verify_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pred, const int32_t *__restrict__ tokens,
+              const int32_t *__restrict__ parent, const int32_t *__restrict__ root_pred, int N, int Tn, int max_path,
+              int32_t *__restrict__ accept_len, int32_t *__restrict__ accept_path, int32_t *__restrict__ next_token,
+              int32_t *__restrict__ status) {
     constexpr int VE = Vec16<T>::n;
     const T *row = logits + (size_t)blockIdx.x * V;
     Best best{-INFINITY, INT_MAX};
@@ -74,82 +153,17 @@ row_argmax_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pre
         }
         if (lane == 0) pred[blockIdx.x] = best.i == INT_MAX ? 0 : best.i;
     }
-}
-
-// One block per sequence.  Every thread walks the root path of its nodes (parent[c] < c
-// makes the walk finite), checks the match rule on the way and proposes (depth, node);
-// the block keeps the deepest valid node, lowest index on ties.
-__global__ void __launch_bounds__(128)
-accept_kernel(const int32_t *__restrict__ tokens, const int32_t *__restrict__ parent,
-              const int32_t *__restrict__ root_pred, const int32_t *__restrict__ pred, int N, int T,
-              int max_path, int32_t *__restrict__ accept_len, int32_t *__restrict__ accept_path,
-              int32_t *__restrict__ next_token, int32_t *__restrict__ status) {
-    const int b = blockIdx.x;
-    const int32_t *par = parent + (size_t)b * N;
-    const int32_t *tok = tokens + (size_t)b * T;
-    const int32_t *prd = pred + (size_t)b * N;
-    int32_t *path = accept_path + (size_t)b * max_path;
-    __shared__ int s_bad;
-    __shared__ unsigned long long s_key[4];
-    if (threadIdx.x == 0) s_bad = 0;
-    __syncthreads();
-    for (int c = threadIdx.x; c < N; c += blockDim.x)
-        if (par[c] < -1 || par[c] >= c) s_bad = 1;
-    for (int j = threadIdx.x; j < max_path; j += blockDim.x) path[j] = -1;
-    __syncthreads();
-    if (s_bad) {
-        if (threadIdx.x == 0) {
-            status[b] = HT_STATUS_BAD_TREE;
-            accept_len[b] = 0;
-            next_token[b] = -1;
-        }
-        return;
-    }
-    const bool has_root = root_pred != nullptr;
-    const int rp = has_root ? root_pred[b] : -1;
-    // key = depth << 32 | (0xFFFFFFFF - node): max picks the deepest, then the lowest node
-    unsigned long long key = 0;
-    for (int n = threadIdx.x; n < T; n += blockDim.x) {
-        int depth = 0;
-        bool ok = true;
-        for (int c = n; c >= 0; c = par[c]) {
-            const int p = par[c];
-            const bool m = p < 0 ? (!has_root || tok[c] == rp) : (tok[c] == prd[p]);
-            ok = ok && m;
-            ++depth;
-        }
-        if (ok) {
-            const unsigned long long k2 = ((unsigned long long)depth << 32) | (0xFFFFFFFFu - (unsigned)n);
-            key = k2 > key ? k2 : key;
-        }
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const unsigned long long o = __shfl_xor_sync(0xffffffffu, key, off);
-        key = o > key ? o : key;
-    }
-    if ((threadIdx.x & 31) == 0) s_key[threadIdx.x >> 5] = key;
-    __syncthreads();
+    // The block that stores a sequence's last argmax searches its tree.
+    __shared__ int s_last;
+    const int b = blockIdx.x / N;
     if (threadIdx.x == 0) {
-        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) key = s_key[w] > key ? s_key[w] : key;
-        const int len = (int)(key >> 32);
-        const int node = (int)(0xFFFFFFFFu - (unsigned)(key & 0xFFFFFFFFu));
-        if (len > max_path) {
-            status[b] = HT_STATUS_PATH_TOO_LONG;
-            accept_len[b] = 0;
-            next_token[b] = -1;
-        } else {
-            status[b] = HT_STATUS_OK;
-            accept_len[b] = len;
-            if (len == 0) {
-                next_token[b] = has_root ? rp : -1;
-            } else {
-                int j = len - 1;
-                for (int c = node; c >= 0; c = par[c]) path[j--] = c;
-                next_token[b] = prd[node];
-            }
-        }
+        __threadfence();
+        s_last = atomicAdd(reinterpret_cast<unsigned int *>(accept_len + b), 1u) == (unsigned)(N - 1);
     }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    accept_sequence(b, tokens, parent, root_pred, pred, N, Tn, max_path, accept_len, accept_path, next_token, status);
 }
 
 int launch_verify(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
@@ -157,23 +171,24 @@ int launch_verify(const void *logits, int dtype, const int32_t *tokens, const in
                   int32_t *accept_len, int32_t *accept_path, int32_t *next_token, int32_t *status,
                   cudaStream_t s) {
     const int rows = B * N;
+    // accept_len doubles as the per-sequence ticket until the sequence's last block overwrites it
+    const cudaError_t e = cudaMemsetAsync(accept_len, 0, (size_t)B * sizeof(int32_t), s);
+    if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
     switch (dtype) {
         case HT_F32:
-            row_argmax_kernel<float><<<rows, 256, 0, s>>>(static_cast<const float *>(logits), V, pred);
+            verify_kernel<float><<<rows, 256, 0, s>>>(static_cast<const float *>(logits), V, pred, tokens, parent, root_pred,
+                                                      N, T, max_path, accept_len, accept_path, next_token, status);
             break;
         case HT_F16:
-            row_argmax_kernel<__half><<<rows, 256, 0, s>>>(static_cast<const __half *>(logits), V, pred);
+            verify_kernel<__half><<<rows, 256, 0, s>>>(static_cast<const __half *>(logits), V, pred, tokens, parent, root_pred,
+                                                       N, T, max_path, accept_len, accept_path, next_token, status);
             break;
         default:
-            row_argmax_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>(
-                static_cast<const __nv_bfloat16 *>(logits), V, pred);
+            verify_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(logits), V, pred, tokens, parent,
+                                                              root_pred, N, T, max_path, accept_len, accept_path, next_token, status);
             break;
     }
-    int rc = check_launch("ht_verify_greedy (row argmax)");
-    if (rc != HT_OK) return rc;
-    accept_kernel<<<B, 128, 0, s>>>(tokens, parent, root_pred, pred, N, T, max_path, accept_len,
-                                    accept_path, next_token, status);
-    return check_launch("ht_verify_greedy (acceptance)");
+    return check_launch("ht_verify_greedy");
 }
 
 }  // namespace ht
