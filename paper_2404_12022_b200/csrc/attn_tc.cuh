@@ -289,8 +289,8 @@ __device__ __forceinline__ int tiles_per_cta(int total, int grid) { return (tota
 // Tiles per CTA.  An even share cuts nearly every unit in two, and every cut costs a partial
 // result in the workspace and a merge at the end.  While the cache is streamed at memory speed a
 // few idle SMs cost less than that, so when all sequences are equally long and some whole
-// multiple or whole fraction of a unit lies within 20 % above the even share, ranges of that
-// length are used and cuts fall on unit boundaries (or, for fractions, near them).
+// multiple or whole fraction of a unit lies within 20 % (or six tiles) above the even share, ranges
+// of that length are used and cuts fall on unit boundaries (or, for fractions, near them).
 __device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nkt, int B) {
     const int even = tiles_per_cta(total, grid);
     int n = 0;
@@ -307,7 +307,8 @@ __device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nk
     } else {
         cand = (even + n - 1) / n * n;                // whole units
     }
-    return (cand * 5 <= even * 6) ? cand : even;
+    // a cut costs about as much as half a dozen tiles (partial result, ticket, merge), whatever the size
+    return (cand * 5 <= even * 6 || cand - even <= 6) ? cand : even;
 }
 
 // Validates every sequence and fills len / nkt / pre.  Called by all threads of a block.
