@@ -41,81 +41,6 @@
 namespace ht {
 namespace tc {
 
-// Reduction of a unit's parts inside a thread-block cluster, by the 256 softmax threads of each CTA.
-// On entry this CTA's part (m, l, O in the layout of a workspace slot) lies at the start of its K / V
-// ring, which nothing else uses any more.  Every CTA owns 128 / k of the 128 output features: once all
-// peers have said that their rings are idle, each CTA copies, for every peer, that peer's feature
-// slice of its part (and m, l) into the peer's ring through distributed shared memory; after a
-// second round of arrivals each CTA merges the k slices it holds and writes its features of the
-// result.  No global memory, no atomics; both waits are bounded.
-constexpr int kXchgRecvOffset = (kSlotFloats * 4 + 1023) / 1024 * 1024;   // bytes from the ring's start
-
-template <bool kBf16>
-__device__ __noinline__ void cluster_exchange(const Params &p, Smem &sm, int rank, int b, int hk, bool valid,
-                                              int tid256, volatile int *abort_flag) {
-    const int k = p.cluster_k;
-    const int cg_per_slice = 32 / k;                    // 4-feature groups per CTA's slice
-    unsigned char *ring = &sm.ring[0][0];
-    const float4 *own4 = reinterpret_cast<const float4 *>(ring);
-    const float *own_ml = reinterpret_cast<const float *>(ring) + kRows * kD;
-    float4 *recv4 = reinterpret_cast<float4 *>(ring + kXchgRecvOffset);          // [sender][group in slice][row]
-    float *recv_ml = reinterpret_cast<float *>(ring + kXchgRecvOffset) + kRows * kD;   // [sender][m | l][row]
-    HT_TR(4, 30, 0);
-    softmax_groups_sync();                              // this CTA's part is complete
-    if (tid256 == 0)
-        for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&sm.xb[0]), (uint32_t)c));
-    mbar_wait_cluster(&sm.xb[0], 0, abort_flag);        // every peer's ring is idle
-    HT_TR(4, 31, 0);
-    if (!*abort_flag) {
-        // thread t moves rows t & 127 of feature groups (t >> 7) + 2 j; k is a power of two
-        const int sh = 5 - __ffs(k) + 1;                // log2(cg_per_slice)
-        const uint32_t recv_base = smem_u32(recv4 + rank * cg_per_slice * kRows + (tid256 & 127));
-#pragma unroll 4
-        for (int j = 0; j < 16; ++j) {
-            const int cg = (tid256 >> 7) + 2 * j, c = cg >> sh, x = cg & (cg_per_slice - 1);
-            st_peer_f4(map_to_peer(recv_base + x * kRows * 16, (uint32_t)c), own4[cg * kRows + (tid256 & 127)]);
-        }
-        const float ml = own_ml[tid256];                // 128 m then 128 l
-        for (int c = 0; c < k; ++c) st_peer_f1(map_to_peer(smem_u32(recv_ml + rank * 2 * kRows + tid256), (uint32_t)c), ml);
-    }
-    HT_TR(4, 32, 0);
-    asm volatile("fence.acq_rel.cluster;" ::: "memory");
-    softmax_groups_sync();
-    HT_TR(4, 33, 0);
-    if (tid256 == 0)
-        for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&sm.xb[1]), (uint32_t)c));
-    mbar_wait_cluster(&sm.xb[1], 0, abort_flag);        // every part has arrived here
-    HT_TR(4, 34, 0);
-    const int row = tid256 & 127, half = tid256 >> 7;
-    const int node = row / p.g;
-    if (!valid || node >= p.N || *abort_flag) return;
-    float M = -INFINITY;
-    for (int c = 0; c < k; ++c) M = fmaxf(M, recv_ml[c * 2 * kRows + row]);
-    float l = 0.f;
-    for (int c = 0; c < k; ++c) {
-        const float m = recv_ml[c * 2 * kRows + row];
-        if (m != -INFINITY) l = fmaf(exp2f(m - M), recv_ml[c * 2 * kRows + kRows + row], l);
-    }
-    const float inv = 1.f / l;
-    const int head = hk * p.g + row % p.g;
-    const int x_per_half = cg_per_slice / 2 > 0 ? cg_per_slice / 2 : 1;
-    for (int xi = 0; xi < x_per_half; ++xi) {
-        const int x = half * x_per_half + xi;
-        if (x >= cg_per_slice) break;
-        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int c = 0; c < k; ++c) {
-            const float m = recv_ml[c * 2 * kRows + row];
-            if (m == -INFINITY) continue;
-            const float f = exp2f(m - M);
-            const float4 v = recv4[(c * cg_per_slice + x) * kRows + row];
-            o.x = fmaf(f, v.x, o.x); o.y = fmaf(f, v.y, o.y); o.z = fmaf(f, v.z, o.z); o.w = fmaf(f, v.w, o.w);
-        }
-        unsigned char *dst = static_cast<unsigned char *>(p.out) +
-                             ((((size_t)b * p.N + node) * p.Hq + head) * kD + (rank * cg_per_slice + x) * 4) * 2;
-        *reinterpret_cast<uint2 *>(dst) = make_uint2(pack2<kBf16>(o.x * inv, o.y * inv), pack2<kBf16>(o.z * inv, o.w * inv));
-    }
-}
-
 template <bool kBf16>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -574,7 +499,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 pslot[kRows * kD + kRows + row] = 0.f;
             }
             const int unit = (int)blockIdx.x / p.cluster_k, b = unit / p.Hkv;
-            cluster_exchange<kBf16>(p, sm, (int)c_rank, b, unit - b * p.Hkv, sm.nkt[b] > 0, tid256, abort_flag);
+            cluster_exchange<kBf16>(p, &sm.ring[0][0], sm.xb, 0u, (int)c_rank, b, unit - b * p.Hkv, 0, sm.nkt[b] > 0, tid256, abort_flag);
         }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
         if (cut[0].valid || cut[1].valid) {
@@ -588,8 +513,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     merge_parts<kBf16>(p, cut[k], per, tid256, cut[k].rt, 0, 1);
                 }
         }
-        HT_TR(4, 39, 0);
-    }
+        }
 
     // ------------------------------- teardown -------------------------------
     tc_fence_before();
@@ -656,14 +580,17 @@ static int row_tiles(const ht_attn_desc &d) { return (d.N * (d.Hq / d.Hkv) + tc:
 static bool pair_mode(const ht_attn_desc &d) { return row_tiles(d) >= 2; }
 static int units_per_head(const ht_attn_desc &d) { return pair_mode(d) ? (row_tiles(d) + 1) / 2 : 1; }
 
-// Cluster size for the one-tile kernel when the (sequence, KV head) units are so few that a CTA
-// per unit would leave most SMs idle: the largest of 8, 4, 2 whose clusters fit the GPU at once.
+// Cluster size when the (sequence, KV head[, tile pair]) units are so few that a CTA per unit would
+// leave most SMs idle: the largest of 8, 4, 2 whose clusters fit the GPU at once.
 static int cluster_size(const ht_attn_desc &d) {
-    if (pair_mode(d)) return 0;
-    const long long units = (long long)d.B * d.Hkv;
+    const long long units = (long long)d.B * d.Hkv * units_per_head(d);
     const int sms = sm_count();
     for (int k = 8; k >= 2; k /= 2)
-        if (units * k <= sms) return k;
+        if (units * k <= sms) {
+            // Clusters leave SMs idle when units * k falls well short of the GPU; that only pays while the
+            // cache is short (the capacity bounds its length) and latency, not bandwidth, decides.
+            return (units * k * 4 >= 3ll * sms || d.cap <= 6144) ? k : 0;
+        }
     return 0;
 }
 
@@ -759,14 +686,16 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     cudaError_t e = cudaSuccess;
     if (k <= 1) e = cudaMemsetAsync(p.tickets, 0, (size_t)units * sizeof(unsigned int), s);   // clusters use no tickets
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    if (k > 1) {
+        p.cluster_k = k;
+        p.grid = (int)units * k;
+    }
     if (pair_mode(d)) return launch_attn_tc_pair_kernel(tm_q, tm_k, tm_v, p, d.dtype == HT_BF16, s);
     e = ensure_smem_attr(smem);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     // Few (sequence, KV head) units: one cluster of 8, 4 or 2 CTAs per unit, parts reduced through
     // distributed shared memory; otherwise one persistent CTA per SM.
     if (k > 1) {
-        p.cluster_k = k;
-        p.grid = (int)units * k;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)p.grid);
         cfg.blockDim = dim3(tc::kThreads);

@@ -413,5 +413,77 @@ __device__ __noinline__ void merge_parts(const Params &p, const CutUnit &cu, int
                        pack2<kBf16>(acc[8 * x + 4] * inv, acc[8 * x + 5] * inv), pack2<kBf16>(acc[8 * x + 6] * inv, acc[8 * x + 7] * inv));
 }
 
+// Reduction of a unit's parts inside a thread-block cluster, by the 256 softmax threads of each CTA.
+// On entry this CTA's part (m, l, O in the layout of a workspace slot) lies at `area`, a stretch of its
+// shared memory (Q and K / V buffers) that nothing else uses any more.  Every CTA owns 128 / k of the 128 output features: once all
+// peers have said that their rings are idle, each CTA copies, for every peer, that peer's feature
+// slice of its part (and m, l) into the peer's ring through distributed shared memory; after a
+// second round of arrivals each CTA merges the k slices it holds and writes its features of the
+// result.  No global memory, no atomics; both waits are bounded.
+constexpr int kXchgRecvOffset = (kSlotFloats * 4 + 1023) / 1024 * 1024;   // bytes from the area's start
+constexpr int kXchgBytes = kXchgRecvOffset + kRows * kD * 4 + 16 * 2 * kRows * 4;   // part + received slices + up to 16 senders' m, l
+
+template <bool kBf16>
+__device__ __noinline__ void cluster_exchange(const Params &p, unsigned char *area, unsigned long long *xb, uint32_t parity,
+                                              int rank, int b, int hk, int row_tile, bool valid, int tid256,
+                                              volatile int *abort_flag) {
+    const int k = p.cluster_k;
+    const int cg_per_slice = 32 / k;                    // 4-feature groups per CTA's slice
+    unsigned char *ring = area;
+    const float4 *own4 = reinterpret_cast<const float4 *>(ring);
+    const float *own_ml = reinterpret_cast<const float *>(ring) + kRows * kD;
+    float4 *recv4 = reinterpret_cast<float4 *>(ring + kXchgRecvOffset);          // [sender][group in slice][row]
+    float *recv_ml = reinterpret_cast<float *>(ring + kXchgRecvOffset) + kRows * kD;   // [sender][m | l][row]
+    softmax_groups_sync();                              // this CTA's part is complete
+    if (tid256 == 0)
+        for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&xb[0]), (uint32_t)c));
+    mbar_wait_cluster(&xb[0], parity, abort_flag);        // every peer's ring is idle
+    if (!*abort_flag) {
+        // thread t moves rows t & 127 of feature groups (t >> 7) + 2 j; k is a power of two
+        const int sh = 5 - __ffs(k) + 1;                // log2(cg_per_slice)
+        const uint32_t recv_base = smem_u32(recv4 + rank * cg_per_slice * kRows + (tid256 & 127));
+#pragma unroll 4
+        for (int j = 0; j < 16; ++j) {
+            const int cg = (tid256 >> 7) + 2 * j, c = cg >> sh, x = cg & (cg_per_slice - 1);
+            st_peer_f4(map_to_peer(recv_base + x * kRows * 16, (uint32_t)c), own4[cg * kRows + (tid256 & 127)]);
+        }
+        const float ml = own_ml[tid256];                // 128 m then 128 l
+        for (int c = 0; c < k; ++c) st_peer_f1(map_to_peer(smem_u32(recv_ml + rank * 2 * kRows + tid256), (uint32_t)c), ml);
+    }
+    asm volatile("fence.acq_rel.cluster;" ::: "memory");
+    softmax_groups_sync();
+    if (tid256 == 0)
+        for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&xb[1]), (uint32_t)c));
+    mbar_wait_cluster(&xb[1], parity, abort_flag);        // every part has arrived here
+    const int row = tid256 & 127, half = tid256 >> 7;
+    const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
+    if (!valid || node >= p.N || *abort_flag) return;
+    float M = -INFINITY;
+    for (int c = 0; c < k; ++c) M = fmaxf(M, recv_ml[c * 2 * kRows + row]);
+    float l = 0.f;
+    for (int c = 0; c < k; ++c) {
+        const float m = recv_ml[c * 2 * kRows + row];
+        if (m != -INFINITY) l = fmaf(exp2f(m - M), recv_ml[c * 2 * kRows + kRows + row], l);
+    }
+    const float inv = 1.f / l;
+    const int head = hk * p.g + row % p.g;
+    const int x_per_half = cg_per_slice / 2 > 0 ? cg_per_slice / 2 : 1;
+    for (int xi = 0; xi < x_per_half; ++xi) {
+        const int x = half * x_per_half + xi;
+        if (x >= cg_per_slice) break;
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = 0; c < k; ++c) {
+            const float m = recv_ml[c * 2 * kRows + row];
+            if (m == -INFINITY) continue;
+            const float f = exp2f(m - M);
+            const float4 v = recv4[(c * cg_per_slice + x) * kRows + row];
+            o.x = fmaf(f, v.x, o.x); o.y = fmaf(f, v.y, o.y); o.z = fmaf(f, v.z, o.z); o.w = fmaf(f, v.w, o.w);
+        }
+        unsigned char *dst = static_cast<unsigned char *>(p.out) +
+                             ((((size_t)b * p.N + node) * p.Hq + head) * kD + (rank * cg_per_slice + x) * 4) * 2;
+        *reinterpret_cast<uint2 *>(dst) = make_uint2(pack2<kBf16>(o.x * inv, o.y * inv), pack2<kBf16>(o.z * inv, o.w * inv));
+    }
+}
+
 }  // namespace tc
 }  // namespace ht

@@ -34,6 +34,7 @@ struct __align__(1024) PSmem {
     int32_t nkt[kMaxB];
     int32_t pre[kMaxB + 1];
     unsigned long long kv_full[kPStages], kv_empty[kPStages], q_full, q_empty, s_full[2][2], p_ready[2][2], o_done[2][2], mma_drain;
+    unsigned long long xb[2];          // cluster exchange: peers ready to receive / all parts delivered
     uint32_t tmem_base;
     int abort;
     int merge_here[2];
@@ -54,6 +55,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mbar_init(&sm.q_full, 1);
         mbar_init(&sm.q_empty, 2);          // one arrival per issuing thread
         mbar_init(&sm.mma_drain, 2);
+        for (int i = 0; i < 2; ++i) mbar_init(&sm.xb[i], p.cluster_k > 1 ? p.cluster_k : 1);
         for (int s = 0; s < 2; ++s)
             for (int h = 0; h < 2; ++h) {
                 mbar_init(&sm.s_full[s][h], 1);
@@ -80,8 +82,21 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     const int total = sm.pre[p.B];
     const int per = choose_per(total, p.grid, sm.nkt, p.B);
-    const int t_begin = min((int)blockIdx.x * per, total);
-    const int t_end = min(t_begin + per, total);
+    int t_begin = min((int)blockIdx.x * per, total);
+    int t_end = min(t_begin + per, total);
+    const bool clustered = p.cluster_k > 1;
+    uint32_t c_rank = 0;
+    if (clustered) {
+        // One cluster per (sequence, KV head, tile pair); its CTAs take equal shares of the unit's tiles.
+        cluster_sync_all();                             // the peers' barriers exist before anyone arrives on them
+        c_rank = cluster_ctarank();
+        const int unit = (int)blockIdx.x / p.cluster_k, b = unit / (p.Hkv * p.n_rt);
+        const int nk = sm.nkt[b], share = (nk + p.cluster_k - 1) / p.cluster_k;
+        const int t0 = sm.pre[b] + (unit - b * p.Hkv * p.n_rt) * nk;
+        t_begin = t0 + min((int)c_rank * share, nk);
+        t_end = t0 + min(((int)c_rank + 1) * share, nk);
+    }
+    unsigned char *const xarea = &sm.q[0][0];          // Q buffers and ring, idle once the CTA's tiles are done
 
     if (warp == 8) {
         // ------------------------------- TMA producer -------------------------------
@@ -267,7 +282,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int ih = 0; ih < 2 * sg.len; ++ih) {
                     const int i = ih >> 1, h = ih & 1;
                     const int kt = sg.kt0 + i;
-                    if (!complete && tid256 == 0 && h == 0) {
+                    if (!complete && !clustered && tid256 == 0 && h == 0) {
                         delivered_old = delivered;
                         delivered = ld_relaxed_gpu(&p.tickets[cut[cut_k].unit]);
                     }
@@ -401,18 +416,18 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tc_fence_after();
             }
             // --- segment epilogue: write the result, finish a cut unit, or leave a part ---
-            if (tid256 == 0) sm.direct = !complete && cut[cut_k].c_hi - cut[cut_k].c_lo == 1 && delivered_old == 1u;
+            if (tid256 == 0) sm.direct = !clustered && !complete && cut[cut_k].c_hi - cut[cut_k].c_lo == 1 && delivered_old == 1u;
             tc_fence_before();
             softmax_groups_sync();
             tc_fence_after();
             const bool direct = sm.direct;
-            const bool final = complete || direct;
-            if (active) {
+            const bool final = (complete && !clustered) || direct;
+            // this stream's rows: normalised to `out` (fin), merged with the one other part first (dir), or as a part to dst
+            auto emit = [&](float *dst, bool fin, bool dir) {
                 const int head = sg.hk * p.g + row % p.g;
-                float *pslot = p.part + ((size_t)(2 * (int)blockIdx.x + cut_k) * 2 + s) * kSlotFloats;
-                const float *oslot = pslot;            // the other part, when finishing the unit here
+                const float *oslot = dst;              // the other part, when finishing the unit here
                 float g0, gb = 0.f;
-                if (direct) {
+                if (dir) {
                     const CutUnit &cu = cut[cut_k];
                     const int oc = (cu.c_lo == (int)blockIdx.x) ? cu.c_hi : cu.c_lo;
                     oslot = p.part + ((size_t)(2 * oc + ((max(cu.t0, oc * per) == oc * per) ? 0 : 1)) * 2 + s) * kSlotFloats;
@@ -425,7 +440,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     g0 = fa * inv;
                     gb = fb * inv;
                 } else {
-                    g0 = complete ? 1.f / l_sum : 1.f;
+                    g0 = fin ? 1.f / l_sum : 1.f;
                 }
 #pragma unroll 1
                 for (int c4 = 0; c4 < (warp_real ? 4 : 0); ++c4) {
@@ -435,7 +450,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                     for (int c = 0; c < 32; ++c) xa[c] *= g0;
                     if (!real) continue;
-                    if (direct) {
+                    if (dir) {
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             const float4 v = __ldcg(reinterpret_cast<const float4 *>(oslot) + (col0 / 4 + c) * kRows + row);
@@ -445,29 +460,40 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                             xa[4 * c + 3] = fmaf(gb, v.w, xa[4 * c + 3]);
                         }
                     }
-                    if (final) {
+                    if (fin) {
                         uint32_t w[16];
 #pragma unroll
                         for (int c = 0; c < 16; ++c) w[c] = pack2<kBf16>(xa[2 * c], xa[2 * c + 1]);
-                        unsigned char *dst = static_cast<unsigned char *>(p.out) +
-                                             ((((size_t)sg.b * p.N + node) * p.Hq + head) * kD + col0) * 2;
+                        unsigned char *o = static_cast<unsigned char *>(p.out) +
+                                           ((((size_t)sg.b * p.N + node) * p.Hq + head) * kD + col0) * 2;
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
-                            *reinterpret_cast<uint4 *>(dst + c * 16) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+                            *reinterpret_cast<uint4 *>(o + c * 16) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
                     } else {
 #pragma unroll
                         for (int c = 0; c < 8; ++c)
-                            reinterpret_cast<float4 *>(pslot)[(col0 / 4 + c) * kRows + row] = make_float4(xa[4 * c], xa[4 * c + 1], xa[4 * c + 2], xa[4 * c + 3]);
+                            reinterpret_cast<float4 *>(dst)[(col0 / 4 + c) * kRows + row] = make_float4(xa[4 * c], xa[4 * c + 1], xa[4 * c + 2], xa[4 * c + 3]);
                     }
                 }
-                if (!final && real) {
-                    pslot[kRows * kD + row] = m_ref;
-                    pslot[kRows * kD + kRows + row] = l_sum;
+                if (!fin && real) {
+                    dst[kRows * kD + row] = m_ref;
+                    dst[kRows * kD + kRows + row] = l_sum;
                 }
+            };
+            if (clustered) {
+                // The unit's parts are reduced inside the cluster, one stream after the other through the
+                // same stretch of shared memory (the second stream's accumulator waits in TMEM meanwhile).
+                for (int x = 0; x < (two ? 2 : 1); ++x) {
+                    if (s == x) emit(reinterpret_cast<float *>(xarea), false, false);
+                    tc_fence_before();
+                    cluster_exchange<kBf16>(p, xarea, sm.xb, (uint32_t)x, (int)c_rank, sg.b, sg.hk, 2 * sg.rt + x, true, tid256, abort_flag);
+                }
+            } else if (active) {
+                emit(p.part + ((size_t)(2 * (int)blockIdx.x + cut_k) * 2 + s) * kSlotFloats, final || direct, direct);
             }
             tc_fence_before();
             softmax_groups_sync();                     // the accumulators are free for the next segment
-            if (!final) {
+            if (!final && !clustered) {
                 cut[cut_k].valid = two ? 3 : 1;         // which streams left a part
                 if (tid256 == 0) {
                     __threadfence();
@@ -476,6 +502,19 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
             J += sg.len;
             t += sg.len;
+        }
+        if (clustered && t_end <= t_begin) {
+            // an empty share still takes part in the cluster's exchanges, with parts that saw nothing
+            const int unit = (int)blockIdx.x / p.cluster_k, b = unit / (p.Hkv * p.n_rt);
+            const int rem = unit - b * p.Hkv * p.n_rt, hk = rem / p.n_rt, rt = rem - hk * p.n_rt;
+            for (int x = 0; x < ((2 * rt + 1 < p.n_row_tiles) ? 2 : 1); ++x) {
+                if (s == 0) {
+                    float *part = reinterpret_cast<float *>(xarea);
+                    part[kRows * kD + row] = -INFINITY;
+                    part[kRows * kD + kRows + row] = 0.f;
+                }
+                cluster_exchange<kBf16>(p, xarea, sm.xb, (uint32_t)x, (int)c_rank, b, hk, 2 * rt + x, sm.nkt[b] > 0, tid256, abort_flag);
+            }
         }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
         if (cut[0].valid || cut[1].valid) {
@@ -495,6 +534,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // ------------------------------- teardown -------------------------------
     tc_fence_before();
     __syncthreads();
+    if (clustered) cluster_sync_all();       // no CTA leaves while a peer may still write into its shared memory
     if (sm.abort && threadIdx.x == 0) {
         for (int b = 0; b < p.B; ++b)
             if (sm.nkt[b] > 0) p.status[b] = HT_STATUS_TIMEOUT;
@@ -521,6 +561,27 @@ int launch_attn_tc_pair_kernel(const CUtensorMap &tm_q, const CUtensorMap &tm_k,
             e = cudaFuncSetAttribute(tc::attn_tc_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         if (dev >= 0 && dev < 64) done[dev] = true;
+    }
+    if (p.cluster_k > 1) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)p.grid);
+        cfg.blockDim = dim3(tc::kPThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)p.cluster_k;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = bf16 ? cudaLaunchKernelEx(&cfg, tc::attn_tc_pair_kernel<true>, tm_q, tm_k, tm_v, p)
+                 : cudaLaunchKernelEx(&cfg, tc::attn_tc_pair_kernel<false>, tm_q, tm_k, tm_v, p);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(HT_ERR_CUDA, "ht_tree_attention (tcgen05, tile pairs, clusters of %d): %s", p.cluster_k, cudaGetErrorString(e));
+        }
+        return HT_OK;
     }
     if (bf16) tc::attn_tc_pair_kernel<true><<<p.grid, tc::kPThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
     else tc::attn_tc_pair_kernel<false><<<p.grid, tc::kPThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
