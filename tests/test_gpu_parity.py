@@ -175,6 +175,36 @@ def test_attention_every_work_split(hb, oracle, dtype, case):
     assert bool(((a - b2).abs() <= ulp * a.abs() + 1e-6).all())
 
 
+def test_attention_random_shapes_tensor_core_kernels_against_the_alu_kernel(hb, oracle):
+    """Forty seeded random shapes (batch, rows, head grouping, ragged lengths, tree kinds) through
+    whichever tensor-core kernel and work split they select, compared with the fp32-ALU kernel of
+    the same library on the GPU (itself checked against the oracle above); the first sequence and
+    KV head of every shape also against the oracle."""
+    rng = np.random.default_rng(2024)
+    for trial in range(40):
+        g = int(rng.choice([1, 1, 2, 4, 8, 16]))
+        Hkv = int(rng.choice([1, 2, 4, 8, 32]))
+        B = int(rng.choice([1, 1, 2, 3, 5, 12]))
+        N = int(rng.choice([1, 7, 19, 33, 64, 91, 130, 200]))
+        if N * g > 1100 or B * Hkv * g * N > 120000:
+            N = max(1, 1100 // g // 4)
+        lens = [int(x) for x in rng.choice([0, 1, 60, 127, 128, 300, 1000, 2500], size=B)]
+        cap = max(lens) + N + int(rng.integers(0, 200))
+        dtype = "bf16" if trial % 2 else "f16"
+        tree = str(rng.choice(["random", "chain", "roots"]))
+        q, k, v, kv_len, parent = make_attn_case(100 + trial, dtype, B, N, Hkv * g, Hkv, 128, lens, cap, tree)
+        out, status = hb.tree_attention(q, k, v, kv_len, parent)
+        ref, _ = hb.tree_attention(q, k, v, kv_len, parent, flags=hb.HT_ATTN_FORCE_SIMT)
+        torch.cuda.synchronize()
+        what = "trial %d: B=%d N=%d Hq=%d Hkv=%d lens=%s %s %s" % (trial, B, N, Hkv * g, Hkv, lens, tree, dtype)
+        assert status.cpu().tolist() == [0] * B, what
+        a, r = out.float(), ref.float()
+        eps = 2.0 ** -7 if dtype == "bf16" else 2.0 ** -10          # two roundings of the output plus P's rounding
+        assert torch.isfinite(a).all(), what
+        assert bool(((a - r).abs() <= 2e-3 + 2 * eps * r.abs() + 3 * eps).all()), what + ": max diff %.3e" % float((a - r).abs().max())
+        check_sampled_units(hb, oracle, q, k, v, kv_len.cpu().numpy(), parent, out, 1, DT[dtype], seed=trial, p_rounding=True)
+
+
 @pytest.mark.parametrize("shape", [(3, 9, 4, 2), (3, 40, 32, 8), (40, 9, 8, 4)], ids=lambda s: "B%dN%dHq%dHkv%d" % s)
 def test_attention_tensor_core_paths_skip_bad_sequences(hb, oracle, shape):
     """Status words and untouched rows on the 16-bit kernels (clusters, tile pairs, persistent)."""
