@@ -97,27 +97,31 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (warp == 8) {
         // ------------------------------- TMA producer -------------------------------
         if (lane == 0) {
-            int b_hint = 0, ring_i = 0, seg_i = 0;
+            int ring_i = 0, seg_i = 0;
             HT_TR_CTA(1);
-            for (int t = t_begin; t < t_end && !*abort_flag;) {
-                const Segment s = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
-                if (seg_i > 0 && !mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag)) break;
-                mbar_expect_tx(&sm.q_full, kEntryBytes);
-                tma_load_4d(sm.q, &tm_q, &sm.q_full, 0, s.hk * p.g, s.rt * p.rows_per_tile_nodes, s.b);
-                tma_load_4d(sm.q + kSlabBytes, &tm_q, &sm.q_full, 64, s.hk * p.g, s.rt * p.rows_per_tile_nodes, s.b);
-                ++seg_i;
-                for (int i = 0; i < 2 * s.len; ++i) {
-                    const int kt = s.kt0 + (i >> 1);
-                    const int slot = ring_i % kStages, use = ring_i / kStages;
-                    if (use > 0 && !mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag)) break;
-                    HT_TR(0, ring_i >> 1, ring_i & 1);
-                    const CUtensorMap *tm = (i & 1) ? &tm_v : &tm_k;
-                    mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
-                    tma_load_4d(sm.ring[slot], tm, &sm.kv_full[slot], 0, kt * kTile, s.hk, s.b);
-                    tma_load_4d(sm.ring[slot] + kSlabBytes, tm, &sm.kv_full[slot], 64, kt * kTile, s.hk, s.b);
-                    ++ring_i;
+            const int n = t_end - t_begin;
+            int hint_k = 0, hint_v = 0;
+            for (int e = 0; e < 2 * n && !*abort_flag; ++e) {
+                // entry e of the consumption order: K_0, K_1, V_0, K_2, V_1, ..., V_{n-1}
+                const bool is_v = e == 2 * n - 1 || (e != 0 && (e & 1) == 0);
+                const int j = e == 0 ? 0 : (e == 2 * n - 1 ? n - 1 : (is_v ? (e - 2) / 2 : (e + 1) / 2));
+                const Segment s = locate(sm.pre, sm.nkt, p.B, p.n_rt, t_begin + j, t_end, is_v ? hint_v : hint_k);
+                if (!is_v && (j == 0 || s.kt0 == 0)) {
+                    // first tile of a segment: its Q tile, once the previous segment's scores are done with Q
+                    if (seg_i > 0 && !mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag)) break;
+                    mbar_expect_tx(&sm.q_full, kEntryBytes);
+                    tma_load_4d(sm.q, &tm_q, &sm.q_full, 0, s.hk * p.g, s.rt * p.rows_per_tile_nodes, s.b);
+                    tma_load_4d(sm.q + kSlabBytes, &tm_q, &sm.q_full, 64, s.hk * p.g, s.rt * p.rows_per_tile_nodes, s.b);
+                    ++seg_i;
                 }
-                t += s.len;
+                const int slot = ring_i % kStages, use = ring_i / kStages;
+                if (use > 0 && !mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag)) break;
+                HT_TR(0, j, is_v ? 1 : 0);
+                const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
+                mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
+                tma_load_4d(sm.ring[slot], tm, &sm.kv_full[slot], 0, s.kt0 * kTile, s.hk, s.b);
+                tma_load_4d(sm.ring[slot] + kSlabBytes, tm, &sm.kv_full[slot], 64, s.kt0 * kTile, s.hk, s.b);
+                ++ring_i;
             }
             if (*abort_flag) {
                 // Every copy this thread issued must have landed before the CTA exits: wait, with the
@@ -138,7 +142,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int s = jj & 1;
                 mbar_wait(&sm.p_ready[s], (jj >> 1) & 1, abort_flag);
                 HT_TR(1, jj, 2);
-                const int e = 2 * jj + 1, slot = e % kStages;
+                const int e = ring_entry_v(jj, t_end - t_begin), slot = e % kStages;
                 mbar_wait(&sm.kv_full[slot], (e / kStages) & 1, abort_flag);
                 tc_fence_after();
                 if (!*abort_flag) {
@@ -160,7 +164,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 mbar_wait(&sm.q_full, seg_i & 1, abort_flag);
                 for (int i = 0; i < sg.len; ++i) {
                     const int s = j & 1;
-                    const int e = 2 * j, slot = e % kStages;
+                    const int e = ring_entry_k(j), slot = e % kStages;
                     mbar_wait(&sm.kv_full[slot], (e / kStages) & 1, abort_flag);
                     tc_fence_after();
                     HT_TR(1, j, 0);
@@ -371,7 +375,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (kt == sg.nkt - 1) {
                     const int valid = L + p.N - tile_lo;
                     if (valid < kTile) {
-                        const int e = 2 * jj + 1, slot = e % kStages;
+                        const int e = ring_entry_v(jj, t_end - t_begin), slot = e % kStages;
                         mbar_wait(&sm.kv_full[slot], (e / kStages) & 1, abort_flag);
                         const int vecs = (kTile - valid) * 8;               // 16-byte vectors per slab
                         for (int v = row; v < vecs; v += 128) {

@@ -348,6 +348,13 @@ __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, 
     __syncthreads();
 }
 
+
+// Ring order of the one-tile kernel: the tensor pipe consumes K_0, K_1, V_0, K_2, V_1, ... (the scores of
+// tile j+1 are issued before P V of tile j), so the tiles are fetched in that order and the ring is a FIFO:
+// a slot is handed back in the order it was filled.  n = tiles of this CTA.
+__device__ __forceinline__ int ring_entry_k(int j) { return j == 0 ? 0 : 2 * j - 1; }
+__device__ __forceinline__ int ring_entry_v(int j, int n) { return j == n - 1 ? 2 * n - 1 : 2 * j + 2; }
+
 // ---------------------------------------------------------------------------------------
 // Main kernel
 // ---------------------------------------------------------------------------------------
