@@ -198,6 +198,25 @@ int ht_draft_tree(const void *logits, int dtype, int B, int rows, int V, int fir
                   void *stream);
 
 /*
+ * Rotary position embedding at the tree's position ids, and placement of the rows' K / V behind
+ * the context -- the step ahead of ht_tree_attention.  Section "Tree attention": the flattened tree
+ * preserves "the original positional indices of each token"; Section "Training stage": a pseudo state
+ * of step i has position id j + i; Section "Setup": LLaMA-2 / Vicuna models, i.e. the rotary embedding
+ * in the half-split pairing (feature i with feature i + D/2, angle pos * rope_base^(-2i/D)).
+ *   desc     B, N, Hq, Hkv, D, cap, dtype and the cache strides are used (scale, num_splits, flags are not)
+ *   q_in     [B, N, Hq, D], k_in, v_in [B, N, Hkv, D]: the rows' projections before the rotation
+ *   pos      [B, N] int32 position ids (e.g. ht_draft_tree's `pos`, followed by the pseudo rows')
+ *   kv_len   [B] int32
+ *   q_out    [B, N, Hq, D]: q_in rotated (may alias q_in)
+ *   k_cache, v_cache [B, Hkv, cap, D]: row kv_len[b] + r receives k_in[b, r] rotated / v_in[b, r] as is
+ *   status   [B] out: HT_STATUS_BAD_LEN sequences are skipped (nothing of theirs is written)
+ * Angles are formed in fp64, products in fp32, one rounding to `dtype`.  D in {64, 128}.
+ */
+int ht_rope_kv_append(const ht_attn_desc *desc /* host */, const void *q_in, const void *k_in, const void *v_in,
+                      const int32_t *pos, const int32_t *kv_len, float rope_base, void *q_out, void *k_cache,
+                      void *v_cache, int32_t *status, void *stream);
+
+/*
  * Tree attention without a caller-provided workspace.  (The paper has no counterpart: this
  * entry point exists for integration, not for the method.)
  *

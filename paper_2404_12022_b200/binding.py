@@ -23,7 +23,7 @@ HT_STATUS_OK, HT_STATUS_BAD_TREE, HT_STATUS_BAD_LEN, HT_STATUS_BAD_PATH, HT_STAT
 HT_ATTN_FORCE_SIMT = 1
 
 EXPORTS = ("ht_version", "ht_last_error_string", "ht_transfer", "ht_tree_attention_workspace",
-           "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact", "ht_draft_tree", "ht_tree_attention_static")
+           "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact", "ht_draft_tree", "ht_rope_kv_append", "ht_tree_attention_static")
 HT_STATIC_SCRATCH_BYTES = 16 << 20
 
 _DTYPES = {torch.float32: HT_F32, torch.float16: HT_F16, torch.bfloat16: HT_BF16}
@@ -79,6 +79,8 @@ def load() -> ctypes.CDLL:
         lib.ht_kv_compact.argtypes = [vp, vp, ctypes.POINTER(CacheDesc), vp, vp, vp, i32, vp, vp, vp]
         lib.ht_draft_tree.restype = i32
         lib.ht_draft_tree.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
+        lib.ht_rope_kv_append.restype = i32
+        lib.ht_rope_kv_append.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
         _lib = lib
     return _lib
 
@@ -256,3 +258,20 @@ def draft_tree(logits, first_row: int, P: int, K: int, tmpl_parent, tmpl_rank, r
                                 _ptr(tmpl_rank), T, _ptr(root_token), _ptr(base_pos), _ptr(topk), _ptr(tokens),
                                 _ptr(pos), _ptr(status), _stream()))
     return topk, tokens, pos, status
+
+
+def rope_kv_append(q_in, k_in, v_in, pos, kv_len, k_cache, v_cache, rope_base: float = 10000.0, q_out=None):
+    """q_in [B, N, Hq, D]; k_in, v_in [B, N, Hkv, D]; pos [B, N] int32; kv_len [B] int32; caches
+    [B, Hkv, cap, D] (written in place at rows kv_len[b] + r).  Returns (q_out, status)."""
+    _need(q_in, name="q_in")
+    _need(k_in, q_in.dtype, "k_in")
+    _need(v_in, q_in.dtype, "v_in")
+    _need(pos, torch.int32, "pos")
+    _need(kv_len, torch.int32, "kv_len")
+    desc = make_attn_desc(q_in, k_cache)
+    if q_out is None:
+        q_out = torch.empty_like(q_in)
+    status = torch.empty(desc.B, dtype=torch.int32, device=q_in.device)
+    _check(load().ht_rope_kv_append(ctypes.byref(desc), _ptr(q_in), _ptr(k_in), _ptr(v_in), _ptr(pos), _ptr(kv_len),
+                                    float(rope_base), _ptr(q_out), _ptr(k_cache), _ptr(v_cache), _ptr(status), _stream()))
+    return q_out, status

@@ -158,4 +158,20 @@ int ht_draft_tree(const void *logits, int dtype, int B, int rows, int V, int fir
                         topk, tokens, pos, status, static_cast<cudaStream_t>(stream));
 }
 
+int ht_rope_kv_append(const ht_attn_desc *desc, const void *q_in, const void *k_in, const void *v_in, const int32_t *pos,
+                      const int32_t *kv_len, float rope_base, void *q_out, void *k_cache, void *v_cache, int32_t *status,
+                      void *stream) {
+    int rc = check_attn_desc(desc);
+    if (rc != HT_OK) return rc;
+    if (desc->B == 0 || desc->N == 0) return HT_OK;
+    if (!(rope_base > 1.f)) return fail(HT_ERR_INVALID_ARG, "rope_base must exceed 1");
+    if (!q_in || !k_in || !v_in || !pos || !kv_len || !q_out || !k_cache || !v_cache || !status)
+        return fail(HT_ERR_INVALID_ARG, "NULL pointer");
+    if (!aligned16(q_in) || !aligned16(k_in) || !aligned16(v_in) || !aligned16(q_out) || !aligned16(k_cache) || !aligned16(v_cache))
+        return fail(HT_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    if ((long long)desc->B * desc->N > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "B*N too large");
+    return launch_rope(*desc, q_in, k_in, v_in, pos, kv_len, rope_base, q_out, k_cache, v_cache, status,
+                       static_cast<cudaStream_t>(stream));
+}
+
 }  // extern "C"

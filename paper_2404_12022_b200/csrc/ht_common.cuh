@@ -85,6 +85,8 @@ int launch_verify(const void *logits, int dtype, const int32_t *tokens, const in
 int launch_draft(const void *logits, int dtype, int B, int rows, int V, int first_row, int P, int K,
                  const int32_t *tmpl_parent, const int32_t *tmpl_rank, int Tn, const int32_t *root_token,
                  const int32_t *base_pos, int32_t *topk, int32_t *tokens, int32_t *pos, int32_t *status, cudaStream_t s);
+int launch_rope(const ht_attn_desc &d, const void *q_in, const void *k_in, const void *v_in, const int32_t *pos,
+                const int32_t *kv_len, float base, void *q_out, void *kc, void *vc, int32_t *status, cudaStream_t s);
 int launch_compact(void *kc, void *vc, const ht_cache_desc &d, const int32_t *kv_len,
                    const int32_t *accept_len, const int32_t *accept_path, int max_path,
                    int32_t *new_kv_len, int32_t *status, cudaStream_t s);

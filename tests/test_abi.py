@@ -67,6 +67,12 @@ def test_host_side_rejections(lib):
     c = hb.CacheDesc(2, 1, 4, 64, 3, hb.HT_BF16, 8, 0, 0, 0)                   # 6-byte rows
     assert lib.ht_kv_compact(p, p, ctypes.byref(c), p, p, p, 8, p, p, None) == hb.HT_ERR_UNSUPPORTED
 
+    d = hb.AttnDesc(1, 4, 4, 4, 128, 64, hb.HT_BF16, 0.0, 0, 0, 0, 0)
+    lib.ht_rope_kv_append.argtypes = [ctypes.POINTER(hb.AttnDesc)] + [ctypes.c_void_p] * 5 + [ctypes.c_float] + [ctypes.c_void_p] * 5
+    assert lib.ht_rope_kv_append(ctypes.byref(d), p, p, p, p, p, 1.0, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG     # base must exceed 1
+    assert lib.ht_rope_kv_append(ctypes.byref(d), p, p, None, p, p, 10000.0, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG
+    assert lib.ht_rope_kv_append(ctypes.byref(d), p, p + 4, p, p, p, 10000.0, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG
+
     # ht_draft_tree(logits, dtype, B, rows, V, first_row, P, K, tmpl_parent, tmpl_rank, T, root, base, topk, tokens, pos, status, stream)
     assert lib.ht_draft_tree(p, hb.HT_F16, 1, 10, 100, 7, 3, 17, p, p, 5, None, p, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG   # K > 16
     assert lib.ht_draft_tree(p, hb.HT_F16, 1, 10, 100, 8, 3, 4, p, p, 5, None, p, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG    # rows 8..10 of 10

@@ -631,3 +631,83 @@ def test_draft_tree_closes_the_round_on_the_device(hb):
         assert np.array_equal(g.cpu().numpy(), r)
     assert got[1][0, 0].item() == nxt[0].item() and got[2][0, 0].item() == new_len[0].item()
 
+
+# ------------------------------------------------------------------------------------------
+# Rotary embedding at the tree's position ids + cache append (the step ahead of attention)
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("shape", [(1, 1, 2, 2, 64), (3, 18, 8, 2, 128), (4, 91, 32, 32, 128), (2, 67, 64, 8, 128)],
+                         ids=lambda s: "B%dN%dHq%dHkv%dD%d" % s)
+def test_rope_kv_append_matches_the_oracle(hb, dtype, shape):
+    from oracle import rope_oracle as ro
+    B, N, Hq, Hkv, D = shape
+    dt = DT[dtype]
+    rng = np.random.default_rng(B * 100 + N)
+    cap = 300 + N
+    q = wl.normal_tensor(51, 1, (B, N, Hq, D), "cuda", 1.0, dt)
+    k = wl.normal_tensor(51, 2, (B, N, Hkv, D), "cuda", 1.0, dt)
+    v = wl.normal_tensor(51, 3, (B, N, Hkv, D), "cuda", 1.0, dt)
+    big_k = wl.normal_tensor(51, 4, (B, Hkv + 1, cap, D), "cuda", 1.0, dt)      # a strided view over the heads
+    big_v = wl.normal_tensor(51, 5, (B, Hkv + 1, cap, D), "cuda", 1.0, dt)
+    kc, vc = big_k[:, :Hkv], big_v[:, :Hkv]
+    kv_len = rng.integers(0, 300, B).astype(np.int32)
+    if B >= 3:
+        kv_len[1] = 301                                        # does not fit: skipped
+    pos = (kv_len[:, None] + rng.integers(0, 7, (B, N))).astype(np.int32)
+    pos[0, 0] = 40000                                          # a large angle: fp32 angles would be off by 1e-3
+    k_before, v_before = f32np(kc), f32np(vc)
+    untouched = big_k[:, Hkv].clone()
+    view = torch.int32 if dt == torch.float32 else torch.int16
+    v_bits_in = v.view(view).cpu().numpy()
+    q_out, status = hb.rope_kv_append(q, k, v, torch.from_numpy(pos).cuda(), torch.from_numpy(kv_len).cuda(), kc, vc)
+    torch.cuda.synchronize()
+    q_ref, k_ref, v_ref, st_ref = ro.rope_kv_append(f32np(q), f32np(k), f32np(v), pos, kv_len, k_before, v_before)
+    assert np.array_equal(status.cpu().numpy(), st_ref)
+    tol = (lambda r: 1e-5) if dt == torch.float32 else (lambda r: 2e-3 + 1e-2 * np.abs(r))
+    for b in range(B):
+        if st_ref[b]:
+            assert np.array_equal(f32np(kc[b]), k_before[b]) and np.array_equal(f32np(vc[b]), v_before[b])
+            continue
+        assert (np.abs(f32np(q_out[b]) - q_ref[b]) <= tol(q_ref[b])).all()
+        assert (np.abs(f32np(kc[b]) - k_ref[b]) <= tol(k_ref[b])).all()
+        L = int(kv_len[b])
+        got_v = vc[b, :, L:L + N].contiguous().view(view).cpu().numpy()          # V rows are moved bit for bit
+        assert np.array_equal(got_v, np.transpose(v_bits_in[b], (1, 0, 2)))
+        keep = np.ones(cap, bool)
+        keep[L:L + N] = False
+        assert np.array_equal(f32np(kc[b])[:, keep], k_before[b][:, keep])       # nothing else is touched
+        assert np.array_equal(f32np(vc[b])[:, keep], v_before[b][:, keep])
+    assert torch.equal(big_k[:, Hkv], untouched)
+
+
+def test_rope_then_attention_equals_the_oracle_chain(hb, oracle):
+    """draft positions -> rotary embedding + cache append -> tree attention, against the same chain of oracles."""
+    from oracle import rope_oracle as ro
+    B, N, Hq, Hkv, D, cap = 2, 33, 8, 2, 128, 400
+    dt = torch.bfloat16
+    rng = np.random.default_rng(9)
+    q = wl.normal_tensor(52, 1, (B, N, Hq, D), "cuda", 1.0, dt)
+    k = wl.normal_tensor(52, 2, (B, N, Hkv, D), "cuda", 1.0, dt)
+    v = wl.normal_tensor(52, 3, (B, N, Hkv, D), "cuda", 1.0, dt)
+    kc = wl.normal_tensor(52, 4, (B, Hkv, cap, D), "cuda", 1.0, dt)
+    vc = wl.normal_tensor(52, 5, (B, Hkv, cap, D), "cuda", 1.0, dt)
+    parent = np.stack([rand_tree(rng, N, "random") for _ in range(B)])
+    depth = np.zeros((B, N), np.int32)
+    for b in range(B):
+        for r in range(N):
+            depth[b, r] = 0 if parent[b, r] < 0 else depth[b, parent[b, r]] + 1
+    kv_len = np.array([300, 17], np.int32)
+    pos = (kv_len[:, None] + depth).astype(np.int32)
+    k0, v0 = f32np(kc), f32np(vc)
+    q_out, st = hb.rope_kv_append(q, k, v, torch.from_numpy(pos).cuda(), torch.from_numpy(kv_len).cuda(), kc, vc)
+    out, st2 = hb.tree_attention(q_out, kc, vc, torch.from_numpy(kv_len).cuda(), torch.from_numpy(parent).cuda())
+    torch.cuda.synchronize()
+    assert st.cpu().tolist() == [0, 0] and st2.cpu().tolist() == [0, 0]
+    # oracle chain on the values the device holds after the rotation (its one rounding to bf16 included)
+    ref = oracle.tree_attention(f32np(q_out), f32np(kc), f32np(vc), kv_len, parent)
+    assert_close(f32np(out), ref, dt, "attention after rope")
+    q_ref, k_ref, v_ref, _ = ro.rope_kv_append(f32np(q), f32np(k), f32np(v), pos, kv_len, k0, v0)
+    assert (np.abs(f32np(q_out) - q_ref) <= 2e-3 + 1e-2 * np.abs(q_ref)).all()
+    assert (np.abs(f32np(kc) - k_ref) <= 2e-3 + 1e-2 * np.abs(k_ref)).all()
+
