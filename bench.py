@@ -242,6 +242,21 @@ def measured_peaks():
     return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
+def replica_aggregate(ms_total_local, steps, step_bytes, world, device):
+    """Whole-job figures of N independent replicas (the path does not shard): the step time is the
+    slowest rank's, the value is all ranks' bytes over that time.  Uses the default process group
+    when world > 1 (NCCL in the benchmark, gloo in the CPU test)."""
+    ms_total = ms_total_local
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        t = torch.tensor([ms_total_local], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / steps
+    return ms_step, world * step_bytes / (ms_step * 1e-3) / 1e9
+
+
 def run_native(args):
     import torch
     import torch.distributed as dist
@@ -286,13 +301,8 @@ def run_native(args):
     barrier()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop() if sampler else None
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-    ms_step = ms_total / args.steps
     step_bytes = step.step_bytes()
-    value = world * step_bytes / (ms_step * 1e-3) / 1e9
+    ms_step, value = replica_aggregate(ms_total, args.steps, step_bytes, world, "cuda")
 
     # correctness of what was just timed: status words and the seeded accepted lengths
     assert int(step.attn_status.abs().sum()) == 0 and int(step.verify_status.abs().sum()) == 0
