@@ -148,23 +148,37 @@ template <> struct MmaOp<__nv_bfloat16> {
     }
 };
 
-// A warp owns an equal, contiguous share of the groups of 16 weight rows.  Lane (g, t) = (lane / 4,
-// lane % 4) loads features [f + 8 t, f + 8 t + 8) of rows g and g + 8 of the group and of batch row
-// g of each 8-column batch tile; words 0 / 1 of those vectors fill k slots (2t, 2t+1) / (2t+8, 2t+9)
-// of one instruction, words 2 / 3 those of a second one.  U steps of 32 features are loaded before
-// the first is used.  The accumulator fragment holds rows g, g + 8 and batch columns 2t, 2t + 1.
-template <typename T, int NB, int U>
+// Work items are (group of 16 weight rows, one of S equal feature ranges); S = 1, 2 or 4 is chosen on
+// the host so that the items about fill the GPU's warp slots (with few row groups a warp per group
+// would leave most slots, and most of the memory system, idle).  A warp owns an equal, contiguous
+// share of the items; the S warps of a group sit in one block and the first of them adds up the
+// partial sums through shared memory.  Lane (g, t) = (lane / 4, lane % 4) loads features
+// [f + 8 t, f + 8 t + 8) of rows g and g + 8 of the group and of batch row g of each 8-column batch
+// tile; words 0 / 1 of those vectors fill k slots (2t, 2t+1) / (2t+8, 2t+9) of one instruction, words
+// 2 / 3 those of a second one.  U steps of 32 features are loaded before the first is used.  The
+// accumulator fragment holds rows g, g + 8 and batch columns 2t, 2t + 1.
+template <typename T, int NB, int U, bool kSplit>
 __global__ void __launch_bounds__(128, kTransferBlocksPerSm)
 transfer_mma_kernel(const T *__restrict__ h, const T *__restrict__ W, T *__restrict__ out,
-                    int rows_total, int d, int b0, int nb) {
-    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const long long warp = (long long)blockIdx.x * 4 + (threadIdx.x >> 5), n_warps = (long long)gridDim.x * 4;
+                    int rows_total, int d, int b0, int nb, int S) {
+    __shared__ float s_part[kSplit ? 4 : 1][NB * 4][32];
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
     const int groups = (rows_total + 15) / 16;
-    const int g_begin = (int)(warp * groups / n_warps), g_end = (int)((warp + 1) * groups / n_warps);
+    const int items = groups * S;
+    const int fchunk = ((d + 32 * S - 1) / (32 * S)) * 32;                   // features per range, a multiple of 32
     const uint4 zero = make_uint4(0, 0, 0, 0);
+    // With S > 1 every warp has exactly one item (block b holds items 4b .. 4b+3); with S = 1 the warps of a
+    // grid that just fills the GPU take equal contiguous shares of the groups (they differ by one at most).
+    const long long w = (long long)blockIdx.x * 4 + wib, n_warps = (long long)gridDim.x * 4;
+    const long long first = kSplit ? w : w * groups / n_warps;
+    const int count = kSplit ? 1 : (int)((w + 1) * groups / n_warps - first);
 
-    for (int grp = g_begin; grp < g_end; ++grp) {
+    for (int k = 0; k < count; ++k) {
+        const long long item = first + k;
+        const bool live = item < items;
+        const int grp = live ? (int)(kSplit ? item / S : item) : 0, part = kSplit ? (int)(item % S) : 0;   // `part` follows the warp's place in its block even past the last item
         const int r0 = grp * 16;
+        const int f_lo = part * fchunk, f_hi = live ? min(d, f_lo + fchunk) : 0;
         const T *wa_row = W + (size_t)min(r0 + g, rows_total - 1) * d;        // rows past the end repeat the last one
         const T *wb_row = W + (size_t)min(r0 + g + 8, rows_total - 1) * d;
         float acc[NB][4];
@@ -173,12 +187,12 @@ transfer_mma_kernel(const T *__restrict__ h, const T *__restrict__ W, T *__restr
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[n][i] = 0.f;
 
-        for (int fb = 0; fb < d; fb += 32 * U) {             // warp-uniform trip count: the products are warp-wide
+        for (int fb = f_lo; fb < f_hi; fb += 32 * U) {       // warp-uniform trip count: the products are warp-wide
             uint4 wa[U], wb[U], hb[U][NB];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int f = fb + u * 32 + t * 8;
-                const bool in = f < d;                                           // d is a multiple of 8
+                const bool in = f < f_hi;                                        // d is a multiple of 8
                 wa[u] = in ? ld_nc16(wa_row + f) : zero;
                 wb[u] = in ? ld_nc16(wb_row + f) : zero;
 #pragma unroll
@@ -195,20 +209,48 @@ transfer_mma_kernel(const T *__restrict__ h, const T *__restrict__ W, T *__restr
                     MmaOp<T>::run(acc[n], wa[u].z, wb[u].z, wa[u].w, wb[u].w, hb[u][n].z, hb[u][n].w);
                 }
         }
+        if (kSplit) {                                        // uniform over the block: one item per warp
 #pragma unroll
-        for (int n = 0; n < NB; ++n)
+            for (int n = 0; n < NB; ++n)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int row = r0 + g + (i >> 1) * 8, b = n * 8 + 2 * t + (i & 1);
-                if (row < rows_total && b < nb) out[(size_t)(b0 + b) * rows_total + row] = from_float<T>(acc[n][i]);
+                for (int i = 0; i < 4; ++i) s_part[wib][n * 4 + i][lane] = acc[n][i];
+            __syncthreads();
+            if (live && part == 0) {                     // part 0 sits S - 1 warps below the block's end: wib + o <= 3
+                for (int o = 1; o < S; ++o)
+#pragma unroll
+                    for (int n = 0; n < NB; ++n)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) acc[n][i] += s_part[wib + o][n * 4 + i][lane];
             }
+        }
+        if (live && part == 0) {
+#pragma unroll
+            for (int n = 0; n < NB; ++n)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = r0 + g + (i >> 1) * 8, b = n * 8 + 2 * t + (i & 1);
+                    if (row < rows_total && b < nb) out[(size_t)(b0 + b) * rows_total + row] = from_float<T>(acc[n][i]);
+                }
+        }
     }
 }
 
 template <typename T, int NB, int U>
 static int launch_mma(const void *h, const void *W, void *out, int rows_total, int d, int b0, int nb, cudaStream_t s) {
-    transfer_mma_kernel<T, NB, U><<<transfer_grid(rows_total, 16), 128, 0, s>>>(
-        static_cast<const T *>(h), static_cast<const T *>(W), static_cast<T *>(out), rows_total, d, b0, nb);
+    const int groups = (rows_total + 15) / 16;
+    const int full = transfer_grid(1 << 30, 16);               // blocks that fill the GPU once
+    int S = 1;
+    if (groups * 4ll <= full * 4ll && d >= 4 * 32 * U) S = 4;
+    else if (groups * 2ll <= full * 4ll && d >= 2 * 32 * U) S = 2;
+    if (S > 1) {
+        const int blocks = (groups * S + 3) / 4;                // S divides 4: a group's warps share a block
+        transfer_mma_kernel<T, NB, U, true><<<blocks, 128, 0, s>>>(static_cast<const T *>(h), static_cast<const T *>(W),
+                                                                   static_cast<T *>(out), rows_total, d, b0, nb, S);
+    } else {
+        const int blocks = (groups + 3) / 4 < full ? (groups + 3) / 4 : full;
+        transfer_mma_kernel<T, NB, U, false><<<blocks, 128, 0, s>>>(static_cast<const T *>(h), static_cast<const T *>(W),
+                                                                    static_cast<T *>(out), rows_total, d, b0, nb, 1);
+    }
     return check_launch("ht_transfer");
 }
 
