@@ -218,9 +218,9 @@ class ClockSampler:
 # DRAM traffic per launch of the attention kernel on a c3 layer, from the ncu capture summarised in
 # profiles/attn_tc_kernel_c3_layer.md (dram__bytes_read.sum + dram__bytes_write.sum).  It is only
 # reported while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.8e6,
+NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 290.4e6,
                "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh"],
-               "sha256": "d76973c628f86da03769293b941ef571a75d3782f42af551f63984b184db5c73"}
+               "sha256": "5ea1da2f6bd14ec46bccef71e658d6df28292457d9c55d2d70a1dece032940f1"}
 
 
 def ncu_traffic(w):
@@ -338,7 +338,9 @@ def kernels_per_attention(step):
 
 
 def per_kernel_pass(args, step, stream, torch):
-    """Same steps again with CUDA events around every library call, on the launching stream."""
+    """Same steps again with CUDA events on the launching stream: one pair around every run of
+    consecutive attention calls (an event between two launches would add its own gap to each of them),
+    one pair around each of the other calls."""
     n = min(args.steps, 10)
     names = ["attention", "transfer", "verify", "compact"]
     ev = {k: [] for k in names}
@@ -346,21 +348,30 @@ def per_kernel_pass(args, step, stream, torch):
     def pair():
         return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
+    def timed(name, fn):
+        a, b = pair(); a.record(); fn(); b.record(); ev[name].append((a, b))
+
+    def attention_run(lo, hi):
+        if hi > lo:
+            a, b = pair(); a.record()
+            for i in range(lo, hi):
+                step.attention(i, stream)
+            b.record(); ev["attention"].append((a, b, list(range(lo, hi))))
+
+    cut = min(step.transfer_at, step.layers)
     for _ in range(n):
-        for i in range(step.layers):
-            if i == step.transfer_at:
-                a, b = pair(); a.record(); step.transfer(stream); b.record(); ev["transfer"].append((a, b))
-            a, b = pair(); a.record(); step.attention(i, stream); b.record(); ev["attention"].append((a, b, i))
-        if step.transfer_at >= step.layers:
-            a, b = pair(); a.record(); step.transfer(stream); b.record(); ev["transfer"].append((a, b))
-        a, b = pair(); a.record(); step.verify(stream); b.record(); ev["verify"].append((a, b))
-        a, b = pair(); a.record(); step.compact(stream); b.record(); ev["compact"].append((a, b))
+        attention_run(0, cut)
+        timed("transfer", lambda: step.transfer(stream))
+        attention_run(cut, step.layers)
+        timed("verify", lambda: step.verify(stream))
+        timed("compact", lambda: step.compact(stream))
     torch.cuda.synchronize()
     tot = {k: sum(x[0].elapsed_time(x[1]) for x in v) for k, v in ev.items()}
     all_ms = sum(tot.values())
-    attn_ms = tot["attention"] / len(ev["attention"])
-    attn_bytes = sum(step.attention_bytes(x[2]) for x in ev["attention"]) / len(ev["attention"])
-    attn_flops = sum(step.attention_flops(x[2]) for x in ev["attention"]) / len(ev["attention"])
+    layers = [i for x in ev["attention"] for i in x[2]]
+    attn_ms = tot["attention"] / len(layers)
+    attn_bytes = sum(step.attention_bytes(i) for i in layers) / len(layers)
+    attn_flops = sum(step.attention_flops(i) for i in layers) / len(layers)
     peak, how = measured_peaks()
     achieved = attn_bytes / (attn_ms * 1e-3) / 1e9
     roofline = {"kernel": "ht_tree_attention", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
