@@ -48,7 +48,8 @@ def parse_args():
     ap.add_argument("--no-extras", action="store_true", help="skip e2e, cpu baseline and per-kernel timing")
     ap.add_argument("--sweep", default="", help="instead of the step benchmark, time ht_tree_attention alone on a set of "
                     "workloads and print one JSON line per point: 'configs' (c2, c2 at KV 2048, a c3 layer, c4) or "
-                    "'c5' (the 48 grouped-query points) or 'c5-quick' (12 of them)")
+                    "'c5' (the 48 grouped-query points) or 'c5-quick' (12 of them); 'transfer' times ht_transfer alone, with a "
+                    "pseudo state per sequence (B rows) and per tree node (B x T rows)")
     ap.add_argument("--only", default="", help="with --sweep: keep the workloads whose name contains this text")
     ap.add_argument("--sweep-reps", type=int, default=0, help="with --sweep: calls per graph (profiling small cases)")
     return ap.parse_args()
@@ -536,8 +537,65 @@ def run_sweep(args):
         del ks, vs, inp, ws, graph
 
 
+# (name, source rows, k, d): the configurations' projections with pseudo states hanging off one node per
+# sequence (B rows) and off every tree node (B x T rows)
+TRANSFER_POINTS = [("c2_per_sequence", 1, 3, 4096), ("c3_per_sequence", 4, 3, 4096), ("c4_per_sequence", 8, 4, 5120),
+                   ("c5_per_sequence_b16", 16, 3, 8192), ("c2_per_node", 88, 3, 4096), ("c3_per_node", 352, 3, 4096),
+                   ("c4_per_node", 512, 4, 5120), ("c5_per_node_b4_t256", 1024, 3, 8192),
+                   ("c5_per_node_b16_t256", 4096, 3, 8192)]
+
+
+def run_transfer_sweep(args):
+    """CUDA-event time of ht_transfer per call, replayed from a CUDA graph whose calls rotate over
+    enough copies of W to exceed twice the L2."""
+    import torch
+    from paper_2404_12022_b200 import binding as hb
+    from paper_2404_12022_b200 import workloads as wl
+    torch.cuda.set_device(0)
+    peak, how = measured_peaks()
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    tensor_peak = None
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        tensor_peak = float(json.load(open(path)).get("bf16_tflops", 0.0)) or None
+    for name, B, k, d in [x for x in TRANSFER_POINTS if args.only in x[0]]:
+        wbytes = k * d * d * 2
+        ncopy = int(max(2, -(-2 * l2 // wbytes)))
+        h = wl.normal_tensor(31, 1, (B, d), "cuda", 1.0, torch.bfloat16)
+        Ws = [wl.normal_tensor(31, 2 + i, (k, d, d), "cuda", 0.02, torch.bfloat16) for i in range(ncopy)]
+        out = torch.empty((B, k, d), dtype=torch.bfloat16, device="cuda")
+        for i in range(3):
+            hb.transfer(h, Ws[i % ncopy], out)
+        torch.cuda.synchronize()
+        reps = args.sweep_reps or ncopy * (4 if B <= 512 else 1)
+        graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side), torch.cuda.graph(graph, stream=side):
+            for i in range(reps):
+                hb.transfer(h, Ws[i % ncopy], out)
+        torch.cuda.synchronize()
+        graph.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        times = []
+        for _ in range(5):
+            e0.record(); graph.replay(); e1.record(); torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1) / reps * 1e3)
+        us = statistics.median(times)
+        byts = wbytes + B * d * 2 + B * k * d * 2
+        flops = 2.0 * B * k * d * d
+        line = {"workload": "transfer_" + name, "rows": B, "k": k, "d": d, "dtype": "bf16", "us": round(us, 2),
+                "hbm_gbs": round(byts / us / 1e3, 1), "frac_of_measured_hbm": round(byts / us / 1e3 / peak, 3),
+                "tflops": round(flops / us / 1e6, 1), "flop_per_byte": round(flops / byts, 1), "cold_l2_copies": ncopy}
+        if tensor_peak:
+            line["frac_of_measured_bf16"] = round(flops / us / 1e6 / tensor_peak, 3)
+        print(json.dumps(line), flush=True)
+        del Ws, graph
+
+
 def main():
     args = parse_args()
+    if args.sweep == "transfer":
+        return run_transfer_sweep(args)
     if args.sweep:
         return run_sweep(args)
     if args.impl == "reference":

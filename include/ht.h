@@ -94,6 +94,12 @@ const char *ht_last_error_string(void);
  *   out   [B, k, d]   out[b][i][r] = sum_c W[i][r][c] * h_src[b][c]
  * fp32 accumulation, result rounded once to `dtype`.  d must be a multiple of 4 (fp32)
  * or 8 (fp16 / bf16).  B*k*d == 0 is a no-op.
+ * B is the number of source rows, whatever they are: one per sequence (pseudo states
+ * hanging off one node), or one per tree node of every sequence (the reading in which
+ * every token gets its pseudo states), B x T rows, for which the 16-bit types run as a
+ * matrix product on the tensor cores in one pass over W.  That kernel's waits are bounded
+ * (about a second); should one run out, the outputs of the affected tile are NaN.
+ * All pointers are device pointers, 16-byte aligned; nothing is retained after the call.
  */
 int ht_transfer(const void *h_src, const void *W, void *out, int B, int k, int d, int dtype,
                 void *stream);

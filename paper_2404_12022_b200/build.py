@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libht.so")
-SOURCES = ["ht_api.cu", "transfer.cu", "attn_simt.cu", "attn_tc.cu", "attn_tc_pair.cu", "verify.cu", "compact.cu", "draft.cu", "rope.cu", "attn_static.cu"]
+SOURCES = ["ht_api.cu", "transfer.cu", "transfer_tc.cu", "attn_simt.cu", "attn_tc.cu", "attn_tc_pair.cu", "verify.cu", "compact.cu", "draft.cu", "rope.cu", "attn_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

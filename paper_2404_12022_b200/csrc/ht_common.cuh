@@ -70,6 +70,9 @@ __device__ __forceinline__ uint4 ld_nc16(const void *p) {   // streaming 16-byte
 
 // Entry points of the individual kernels' host launchers (defined in the .cu files).
 int launch_transfer(const void *h, const void *W, void *out, int B, int k, int d, int dtype, cudaStream_t s);
+bool transfer_tc_applicable(int B, int k, int d, int dtype);
+int transfer_tc_tile(int B, int R, int sms);
+int launch_transfer_tc(const void *h, const void *W, void *out, int B, int k, int d, int dtype, cudaStream_t s);
 size_t attn_simt_workspace(const ht_attn_desc &d, int *splits_out);
 int launch_attn_simt(const ht_attn_desc &d, const void *q, const void *kc, const void *vc,
                      const int32_t *kv_len, const int32_t *parent, void *out, void *ws, size_t ws_bytes,

@@ -3,8 +3,9 @@
 // Shape of the work: k*d output rows, each a dot product of one row of W (d elements,
 // read exactly once from HBM) with B hidden vectors (tiny, L1/L2 resident).  The kernel
 // is a weight stream: arithmetic intensity is B flop per weight byte, far below the
-// ridge for the batch sizes of decoding, so tensor cores are not used here and the
-// design goal is 16-byte coalesced loads with enough of them in flight.
+// ridge for the batch sizes of decoding, so the design goal is 16-byte coalesced loads
+// with enough of them in flight.  (Up to 16 source rows per pass: this file.  More rows,
+// 16-bit types: the tcgen05 kernel of transfer_tc.cu.)
 //
 // Every warp of a grid that just fills the GPU owns an equal, contiguous share of the k*d rows of
 // the flattened [k*d, d] weight and walks it R rows at a time.  Its lanes stride over the input
@@ -21,6 +22,9 @@
 // batch row) and the pairs of those vectors are dealt to the instruction's k slots in place:
 // no shuffles, no shared memory.  (tcgen05 would stage both operands through shared memory for
 // an M = 128 tile; with 4 to 16 batch columns this skinny product gains nothing from it.)
+#include <cstdlib>
+#include <cstring>
+
 #include "ht_common.cuh"
 
 namespace ht {
@@ -266,8 +270,20 @@ static int launch_typed16(const void *h, const void *W, void *out, int B, int k,
     return HT_OK;
 }
 
+// Which kernel takes a 16-bit call: up to 16 source rows the warp-level instruction on the words as
+// loaded, above that the tcgen05 kernel (one pass over W for any number of rows).  HT_TRANSFER_KERNEL =
+// "tc" or "mma" in the environment overrides the choice, for cross-checks of one against the other.
+static bool use_tc(int B, int k, int d, int dtype) {
+    if (!transfer_tc_applicable(B, k, d, dtype)) return false;
+    const char *e = getenv("HT_TRANSFER_KERNEL");
+    if (e && !strcmp(e, "tc")) return true;
+    if (e && !strcmp(e, "mma")) return false;
+    return B > 16;
+}
+
 int launch_transfer(const void *h, const void *W, void *out, int B, int k, int d, int dtype,
                     cudaStream_t s) {
+    if (use_tc(B, k, d, dtype)) return launch_transfer_tc(h, W, out, B, k, d, dtype, s);
     switch (dtype) {
         case HT_F32: return launch_typed<float>(h, W, out, B, k, d, s);
         case HT_F16: return launch_typed16<__half>(h, W, out, B, k, d, s);

@@ -431,6 +431,59 @@ def test_transfer_c5_shape(hb, oracle):
     assert_close(f32np(out), oracle.transfer(f32np(h), f32np(W)), torch.bfloat16, "transfer c5")
 
 
+# A pseudo state per tree node (Section "Hidden Transfer": every token of the sequence gets its pseudo
+# states) makes the batch B x T rows: the tensor-core kernel.  Shapes cover one and several 128-row tiles
+# with a ragged last one, a ragged last weight tile, a feature count that is not a multiple of 64, a
+# single 64-feature step, and the per-node batches of configs 2 and 3.
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("shape", [(17, 1, 64), (40, 2, 520), (88, 3, 1024), (128, 1, 256), (129, 2, 512),
+                                   (352, 3, 1024), (300, 1, 2056)],
+                         ids=lambda s: "B%dk%dd%d" % s)
+def test_transfer_many_rows(hb, oracle, dtype, shape):
+    B, k, d = shape
+    dt = DT[dtype]
+    h = wl.normal_tensor(24, 1, (B, d), "cuda", 1.0, dt)
+    W = wl.normal_tensor(24, 2, (k, d, d), "cuda", 1.0 / np.sqrt(d), dt)
+    out = hb.transfer(h, W)
+    assert_close(f32np(out), oracle.transfer(f32np(h), f32np(W)), dt, "transfer, many rows")
+
+
+def test_transfer_per_node_rows_of_config_3(hb, oracle):
+    B, k, d = 4 * 88, 3, 4096
+    h = wl.normal_tensor(25, 1, (B, d), "cuda", 1.0, torch.bfloat16)
+    W = wl.normal_tensor(25, 2, (k, d, d), "cuda", 0.02, torch.bfloat16)
+    out = hb.transfer(h, W)
+    rows = np.random.default_rng(25).choice(B, 24, replace=False)          # the oracle on a sample of rows
+    want = oracle.transfer(f32np(h)[rows], f32np(W))
+    assert_close(f32np(out)[rows], want, torch.bfloat16, "transfer, per-node rows")
+    # the rest against the warp-level kernel, sixteen rows at a time
+    other = torch.cat([_transfer_with(hb, "mma", h[i:i + 16], W) for i in range(0, B, 16)])
+    assert_close(f32np(out), f32np(other), torch.bfloat16, "tcgen05 against m16n8k16")
+
+
+def _transfer_with(hb, kernel, h, W):
+    import os
+    old = os.environ.get("HT_TRANSFER_KERNEL")
+    os.environ["HT_TRANSFER_KERNEL"] = kernel
+    try:
+        return hb.transfer(h, W)
+    finally:
+        if old is None:
+            del os.environ["HT_TRANSFER_KERNEL"]
+        else:
+            os.environ["HT_TRANSFER_KERNEL"] = old
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 32), (4, 3, 4096), (5, 2, 520), (16, 3, 1024)], ids=lambda s: "B%dk%dd%d" % s)
+def test_transfer_few_rows_on_either_kernel(hb, oracle, shape):
+    B, k, d = shape
+    h = wl.normal_tensor(26, 1, (B, d), "cuda", 1.0, torch.bfloat16)
+    W = wl.normal_tensor(26, 2, (k, d, d), "cuda", 1.0 / np.sqrt(d), torch.bfloat16)
+    want = oracle.transfer(f32np(h), f32np(W))
+    for kernel in ("tc", "mma"):
+        assert_close(f32np(_transfer_with(hb, kernel, h, W)), want, torch.bfloat16, "transfer on " + kernel)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
 @pytest.mark.parametrize("V", [50, 1000, 32000, 32003])
 def test_row_argmax_with_ties_and_nans(hb, oracle, dtype, V):
