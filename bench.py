@@ -50,6 +50,8 @@ def parse_args():
                     "workloads and print one JSON line per point: 'configs' (c2, c2 at KV 2048, a c3 layer, c4) or "
                     "'c5' (the 48 grouped-query points) or 'c5-quick' (12 of them); 'transfer' times ht_transfer alone, with a "
                     "pseudo state per sequence (B rows) and per tree node (B x T rows)")
+    ap.add_argument("--paged", type=int, default=0, help="with --sweep configs / c5: the same workloads with the cache cut into pages "
+                    "of this many rows, placed in a seeded random order in a pool (ht_tree_attention_paged)")
     ap.add_argument("--only", default="", help="with --sweep: keep the workloads whose name contains this text")
     ap.add_argument("--sweep-reps", type=int, default=0, help="with --sweep: calls per graph (profiling small cases)")
     return ap.parse_args()
@@ -509,6 +511,22 @@ def run_sweep(args):
         ws = torch.empty(max(hb.tree_attention_workspace(desc), 16), dtype=torch.uint8, device="cuda")
         reps = args.sweep_reps or max(nbuf, 16)
         call = lambda i: hb.tree_attention(q, ks[i % nbuf], vs[i % nbuf], kv_len, parent, out=out, workspace=ws, status=st)
+        if args.paged:
+            ps = args.paged
+            B, Hkv, cap, D = ks[0].shape
+            per = cap // ps
+            assert per * ps == cap, "--paged must divide the cache capacity %d" % cap
+            g = torch.Generator(device="cpu").manual_seed(w.seed)
+            table = torch.randperm(B * per, generator=g).to(torch.int32).reshape(B, per).cuda()
+
+            def to_pool(c):      # page table[b][i] of the pool holds rows [i ps, (i + 1) ps) of sequence b
+                pool = torch.empty((B * per, Hkv, ps, D), dtype=c.dtype, device="cuda")
+                pool[table.reshape(-1).long()] = c.view(B, Hkv, per, ps, D).permute(0, 2, 1, 3, 4).reshape(B * per, Hkv, ps, D)
+                return pool
+            ks = [to_pool(c) for c in ks]
+            vs = [to_pool(c) for c in vs]
+            call = lambda i: hb.tree_attention_paged(q, ks[i % nbuf], vs[i % nbuf], table, kv_len, parent, out=out,
+                                                     workspace=ws, status=st)
         for i in range(3):
             call(i)
         torch.cuda.synchronize()
@@ -533,7 +551,8 @@ def run_sweep(args):
                           "rows": rows, "q_heads": w.Hq, "kv_heads": w.Hkv, "dtype": w.dtype, "us": round(us, 2),
                           "hbm_gbs": round(byts / us / 1e3, 1), "frac_of_measured_hbm": round(byts / us / 1e3 / peak, 3),
                           "frac_of_8tbs": round(byts / us / 1e3 / 8000.0, 3), "tflops": round(flops / us / 1e6, 1),
-                          "flop_per_byte": round(flops / byts, 1), "cold_l2_copies": nbuf}), flush=True)
+                          "flop_per_byte": round(flops / byts, 1), "cold_l2_copies": nbuf,
+                          "cache": ("pages of %d rows" % args.paged) if args.paged else "contiguous"}), flush=True)
         del ks, vs, inp, ws, graph
 
 

@@ -54,6 +54,7 @@ enum {
     HT_STATUS_BAD_LEN = 2,       /* kv_len[b] < 0 or kv_len[b] + N > cap */
     HT_STATUS_BAD_PATH = 3,      /* accepted path not increasing / out of range */
     HT_STATUS_PATH_TOO_LONG = 4, /* the accepted path has more than max_path nodes */
+    HT_STATUS_BAD_PAGE = 5,      /* paged cache: a block-table entry the sequence needs is outside the pool */
     HT_STATUS_TIMEOUT = 6
 };
 
@@ -130,6 +131,38 @@ size_t ht_tree_attention_workspace(const ht_attn_desc *desc /* host */);
 int ht_tree_attention(const ht_attn_desc *desc /* host */, const void *q, const void *k_cache,
                       const void *v_cache, const int32_t *kv_len, const int32_t *parent, void *out,
                       void *workspace, size_t workspace_bytes, int32_t *status, void *stream);
+
+/*
+ * Tree attention over a paged cache: the same operation as ht_tree_attention (Section "Tree
+ * attention"), with the K / V rows of a sequence scattered over fixed-size pages of a shared pool,
+ * the layout serving systems keep their caches in.
+ *   pages->page_size   rows per page: a power of two >= 16
+ *   pages->max_pages   block-table entries per sequence; the capacity of a sequence is
+ *                      max_pages * page_size rows (desc->cap and desc's cache strides are ignored)
+ *   pages->n_pages     pages in the pool
+ *   pages->page_stride, head_stride   elements between pages / between the KV heads of a page;
+ *                      0 = Hkv * page_size * D / page_size * D.  Rows are D apart.
+ *   k_pages, v_pages   [n_pages, Hkv, page_size, D]
+ *   block_table        [B, max_pages] int32: cache row r of sequence b is row r % page_size of page
+ *                      block_table[b][r / page_size].  As in ht_tree_attention the K / V of query
+ *                      row r must already sit at cache row kv_len[b] + r.  Entries of pages wholly
+ *                      past row kv_len[b] + N are not consulted for a result and may hold anything.
+ *   status             as in ht_tree_attention, plus HT_STATUS_BAD_PAGE for a sequence one of whose
+ *                      needed entries lies outside [0, n_pages): page 0 is read in its place (no
+ *                      access outside the pool) and the sequence's rows of `out` are meaningless.
+ * q, kv_len, parent, out, workspace (ht_tree_attention_workspace(desc) bytes) as in
+ * ht_tree_attention.  Supported: fp16 / bf16, D = 128, Hq / Hkv a power of two, N <= 512,
+ * B <= 256 (the tensor-core kernels); anything else returns HT_ERR_UNSUPPORTED.
+ */
+typedef struct {
+    int32_t page_size, max_pages, n_pages;
+    int64_t page_stride, head_stride;
+} ht_paged_desc;
+int ht_tree_attention_paged(const ht_attn_desc *desc /* host */, const ht_paged_desc *pages /* host */,
+                            const void *q, const void *k_pages, const void *v_pages,
+                            const int32_t *block_table, const int32_t *kv_len, const int32_t *parent,
+                            void *out, void *workspace, size_t workspace_bytes, int32_t *status,
+                            void *stream);
 
 /*
  * Greedy verification -- Fig. 2 caption ("find the last accepted token position"),

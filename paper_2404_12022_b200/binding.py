@@ -23,7 +23,8 @@ HT_STATUS_OK, HT_STATUS_BAD_TREE, HT_STATUS_BAD_LEN, HT_STATUS_BAD_PATH, HT_STAT
 HT_ATTN_FORCE_SIMT = 1
 
 EXPORTS = ("ht_version", "ht_last_error_string", "ht_transfer", "ht_tree_attention_workspace",
-           "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact", "ht_draft_tree", "ht_rope_kv_append", "ht_tree_attention_static")
+           "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact", "ht_draft_tree", "ht_rope_kv_append", "ht_tree_attention_static",
+           "ht_tree_attention_paged")
 HT_STATIC_SCRATCH_BYTES = 16 << 20
 
 _DTYPES = {torch.float32: HT_F32, torch.float16: HT_F16, torch.bfloat16: HT_BF16}
@@ -35,6 +36,11 @@ class AttnDesc(ctypes.Structure):
                 ("dtype", ctypes.c_int32), ("scale", ctypes.c_float),
                 ("kv_stride_b", ctypes.c_int64), ("kv_stride_h", ctypes.c_int64),
                 ("num_splits", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class PagedDesc(ctypes.Structure):
+    _fields_ = [("page_size", ctypes.c_int32), ("max_pages", ctypes.c_int32), ("n_pages", ctypes.c_int32),
+                ("page_stride", ctypes.c_int64), ("head_stride", ctypes.c_int64)]
 
 
 class CacheDesc(ctypes.Structure):
@@ -73,6 +79,8 @@ def load() -> ctypes.CDLL:
         lib.ht_tree_attention.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         lib.ht_tree_attention_static.restype = i32
         lib.ht_tree_attention_static.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.ht_tree_attention_paged.restype = i32
+        lib.ht_tree_attention_paged.argtypes = [ctypes.POINTER(AttnDesc), ctypes.POINTER(PagedDesc), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         lib.ht_verify_greedy.restype = i32
         lib.ht_verify_greedy.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         lib.ht_kv_compact.restype = i32
@@ -164,6 +172,42 @@ def tree_attention(q, k_cache, v_cache, kv_len, parent, out=None, workspace=None
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(load().ht_tree_attention(ctypes.byref(desc), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(kv_len),
                                     _ptr(parent), _ptr(out), _ptr(workspace), ws_bytes, _ptr(status), _stream()))
+    return out, status
+
+
+def tree_attention_paged(q, k_pages, v_pages, block_table, kv_len, parent, out=None, workspace=None, status=None,
+                         scale: float = 0.0):
+    """q [B, N, Hq, D]; page pools [n_pages, Hkv, page_size, D] (may be strided over page / head);
+    block_table [B, max_pages] int32; kv_len [B] int32; parent [B, N] int32.  Returns (out, status)."""
+    _need(q, name="q")
+    _need(block_table, torch.int32, "block_table")
+    _need(kv_len, torch.int32, "kv_len")
+    _need(parent, torch.int32, "parent")
+    if not (k_pages.is_cuda and v_pages.is_cuda) or k_pages.dtype != q.dtype or v_pages.dtype != q.dtype:
+        raise ValueError("page pools must be CUDA tensors of q's dtype")
+    if k_pages.stride() != v_pages.stride() or k_pages.shape != v_pages.shape:
+        raise ValueError("k_pages and v_pages must share shape and strides")
+    B, N, Hq, D = q.shape
+    n_pages, Hkv, page_size, Dp = k_pages.shape
+    if Dp != D or k_pages.stride(3) != 1 or k_pages.stride(2) != D:
+        raise ValueError("page rows must be contiguous and D apart")
+    if block_table.dim() != 2 or block_table.shape[0] != B or tuple(parent.shape) != (B, N) or tuple(kv_len.shape) != (B,):
+        raise ValueError("block_table must be [B, max_pages], parent [B, N], kv_len [B]")
+    max_pages = block_table.shape[1]
+    desc = AttnDesc(B, N, Hq, Hkv, D, max_pages * page_size, _DTYPES[q.dtype], scale, 0, 0, 0, 0)
+    pages = PagedDesc(page_size, max_pages, n_pages, k_pages.stride(0), k_pages.stride(1))
+    if out is None:
+        out = torch.empty_like(q)
+    _need(out, q.dtype, "out")
+    if status is None:
+        status = torch.empty(B, dtype=torch.int32, device=q.device)
+    need = tree_attention_workspace(desc)
+    if workspace is None and need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().ht_tree_attention_paged(ctypes.byref(desc), ctypes.byref(pages), _ptr(q), _ptr(k_pages), _ptr(v_pages),
+                                          _ptr(block_table), _ptr(kv_len), _ptr(parent), _ptr(out), _ptr(workspace),
+                                          ws_bytes, _ptr(status), _stream()))
     return out, status
 
 

@@ -41,10 +41,11 @@
 namespace ht {
 namespace tc {
 
-template <bool kBf16>
+// kPaged: the cache is a pool of pages (separate instantiations, so that the contiguous kernels carry none of that code).
+template <bool kBf16, bool kPaged>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-               const __grid_constant__ CUtensorMap tm_v, const Params p) {
+               const __grid_constant__ CUtensorMap tm_v, const Params p, const PagedParams pp) {
     extern __shared__ unsigned char smem_raw[];
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -70,7 +71,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0);
+    plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0, kPaged);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -100,13 +101,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             int ring_i = 0, seg_i = 0;
             HT_TR_CTA(1);
             const int n = t_end - t_begin;
-            int hint_k = 0, hint_v = 0;
+            TileCursor cur_k, cur_v, cur_p;          // the K and V streams of the ring order, and the page-id lookahead
+            cur_k.init(t_begin, t_end);
+            cur_v.init(t_begin, t_end);
+            cur_p.init(t_begin, t_end);
+            if (kPaged)
+                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p);
             for (int e = 0; e < 2 * n && !*abort_flag; ++e) {
                 // entry e of the consumption order: K_0, K_1, V_0, K_2, V_1, ..., V_{n-1}
                 const bool is_v = e == 2 * n - 1 || (e != 0 && (e & 1) == 0);
                 const int j = e == 0 ? 0 : (e == 2 * n - 1 ? n - 1 : (is_v ? (e - 2) / 2 : (e + 1) / 2));
-                const Segment s = locate(sm.pre, sm.nkt, p.B, p.n_rt, t_begin + j, t_end, is_v ? hint_v : hint_k);
-                if (!is_v && (j == 0 || s.kt0 == 0)) {
+                if (is_v) cur_v.next(sm.pre, sm.nkt, p.B, p.n_rt);   // tile j of its stream
+                else cur_k.next(sm.pre, sm.nkt, p.B, p.n_rt);
+                struct { int b, hk, rt; } s;
+                s.b = is_v ? cur_v.s.b : cur_k.s.b;
+                s.hk = is_v ? cur_v.s.hk : cur_k.s.hk;
+                s.rt = is_v ? cur_v.s.rt : cur_k.s.rt;
+                const int kt = is_v ? cur_v.kt() : cur_k.kt();
+                if (!is_v && cur_k.first()) {
                     // first tile of a segment: its Q tile, once the previous segment's scores are done with Q
                     if (seg_i > 0 && !mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag)) break;
                     mbar_expect_tx(&sm.q_full, kEntryBytes);
@@ -118,11 +130,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (use > 0 && !mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag)) break;
                 HT_TR(0, j, is_v ? 1 : 0);
                 const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
+                if (kPaged && !is_v) {
+                    // the ids of tile j were asked for kPgAhead tiles ago; ask for those of tile j + kPgAhead
+                    pages_request(p, pp, sm.pre, sm.nkt, sm.pg, j + kPgAhead, cur_p);
+                    cp_async_wait<kPgAhead>();
+                }
                 mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
-                tma_load_4d(sm.ring[slot], tm, &sm.kv_full[slot], 0, s.kt0 * kTile, s.hk, s.b);
-                tma_load_4d(sm.ring[slot] + kSlabBytes, tm, &sm.kv_full[slot], 64, s.kt0 * kTile, s.hk, s.b);
+                fetch_kv_tile<kPaged>(p, pp, sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt, sm.len[s.b] + p.N, sm.pg[j % kPgTiles]);
                 ++ring_i;
             }
+            if (kPaged) cp_async_wait<0>();
             if (*abort_flag) {
                 // Every copy this thread issued must have landed before the CTA exits: wait, with the
                 // usual bound, for the latest armed phase of each ring slot and of the Q buffer.
@@ -609,6 +626,12 @@ size_t attn_tc_workspace(const ht_attn_desc &d) {
     return ticket_bytes(d) + (size_t)2 * sm_count() * (pair_mode(d) ? 2 : 1) * tc::kSlotFloats * sizeof(float);
 }
 
+typedef void (*AttnKernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const tc::Params, const tc::PagedParams);
+static AttnKernelFn attn_tc_fn(bool bf16, bool paged) {
+    return bf16 ? (paged ? tc::attn_tc_kernel<true, true> : tc::attn_tc_kernel<true, false>)
+                : (paged ? tc::attn_tc_kernel<false, true> : tc::attn_tc_kernel<false, false>);
+}
+
 // The kernels' dynamic shared memory limit is raised once per device.
 static cudaError_t ensure_smem_attr(size_t smem) {
     static bool done[64];
@@ -616,10 +639,10 @@ static cudaError_t ensure_smem_attr(size_t smem) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
-    e = cudaFuncSetAttribute(tc::attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(tc::attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+    for (int i = 0; i < 4; ++i) {
+        e = cudaFuncSetAttribute(attn_tc_fn(i & 1, i >> 1), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
     if (dev >= 0 && dev < 64) done[dev] = true;
     return cudaSuccess;
 }
@@ -642,10 +665,11 @@ extern "C" void ht_set_trace(void *ptr) { g_trace = static_cast<long long *>(ptr
 #endif
 
 int launch_attn_tc_pair_kernel(const CUtensorMap &tm_q, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const tc::Params &p,
-                               bool bf16, cudaStream_t s);
+                               const tc::PagedParams &pp, bool bf16, bool paged, cudaStream_t s);
 
 int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const void *vc, const int32_t *kv_len,
-                   const int32_t *parent, void *out, void *ws, size_t ws_bytes, int32_t *status, cudaStream_t s) {
+                   const int32_t *parent, void *out, void *ws, size_t ws_bytes, int32_t *status, cudaStream_t s,
+                   const ht_paged_desc *pages, const int32_t *block_table) {
     if (ws_bytes < attn_tc_workspace(d) || !ws)
         return fail(HT_ERR_WORKSPACE, "workspace holds %zu bytes, %zu needed", ws ? ws_bytes : 0, attn_tc_workspace(d));
     const int g = d.Hq / d.Hkv;
@@ -659,7 +683,18 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
         int rc = make_map(&tm_q, q, d.dtype, dims, strides, box);
         if (rc != HT_OK) return rc;
     }
-    {
+    if (pages) {
+        // [page][head][row][D]: a box is the rows of one tile that one page holds
+        const long long ph = pages->head_stride ? pages->head_stride : (long long)pages->page_size * d.D;
+        const long long pp = pages->page_stride ? pages->page_stride : (long long)d.Hkv * pages->page_size * d.D;
+        const cuuint64_t dims[4] = {(cuuint64_t)d.D, (cuuint64_t)pages->page_size, (cuuint64_t)d.Hkv, (cuuint64_t)pages->n_pages};
+        const cuuint64_t strides[3] = {(cuuint64_t)d.D * 2, (cuuint64_t)ph * 2, (cuuint64_t)pp * 2};
+        const cuuint32_t box[4] = {64, (cuuint32_t)(pages->page_size < tc::kTile ? pages->page_size : tc::kTile), 1, 1};
+        int rc = make_map(&tm_k, kc, d.dtype, dims, strides, box);
+        if (rc != HT_OK) return rc;
+        rc = make_map(&tm_v, vc, d.dtype, dims, strides, box);
+        if (rc != HT_OK) return rc;
+    } else {
         const cuuint64_t dims[4] = {(cuuint64_t)d.D, (cuuint64_t)d.cap, (cuuint64_t)d.Hkv, (cuuint64_t)d.B};
         const cuuint64_t strides[3] = {(cuuint64_t)d.D * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
         const cuuint32_t box[4] = {64, (cuuint32_t)tc::kTile, 1, 1};
@@ -680,6 +715,13 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     p.is_bf16 = d.dtype == HT_BF16;
     p.grid = sm_count();
     p.cluster_k = 0;
+    tc::PagedParams pp;
+    pp.block_table = pages ? block_table : nullptr;
+    pp.page_size = pages ? pages->page_size : 0;
+    pp.page_shift = 0;
+    while (pages && (1 << pp.page_shift) < pages->page_size) ++pp.page_shift;
+    pp.max_pages = pages ? pages->max_pages : 0;
+    pp.n_pages = pages ? pages->n_pages : 0;
 #ifdef HT_TC_TRACE
     p.trace = g_trace;
 #endif
@@ -689,12 +731,13 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     const int k = cluster_size(d);
     cudaError_t e = cudaSuccess;
     if (k <= 1) e = cudaMemsetAsync(p.tickets, 0, (size_t)units * sizeof(unsigned int), s);   // clusters use no tickets
+    if (e == cudaSuccess && pages) e = cudaMemsetAsync(status, 0, (size_t)d.B * sizeof(int32_t), s);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
     if (k > 1) {
         p.cluster_k = k;
         p.grid = (int)units * k;
     }
-    if (pair_mode(d)) return launch_attn_tc_pair_kernel(tm_q, tm_k, tm_v, p, d.dtype == HT_BF16, s);
+    if (pair_mode(d)) return launch_attn_tc_pair_kernel(tm_q, tm_k, tm_v, p, pp, d.dtype == HT_BF16, pages != nullptr, s);
     e = ensure_smem_attr(smem);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     // Few (sequence, KV head) units: one cluster of 8, 4 or 2 CTAs per unit, parts reduced through
@@ -712,16 +755,14 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        e = d.dtype == HT_BF16 ? cudaLaunchKernelEx(&cfg, tc::attn_tc_kernel<true>, tm_q, tm_k, tm_v, p)
-                               : cudaLaunchKernelEx(&cfg, tc::attn_tc_kernel<false>, tm_q, tm_k, tm_v, p);
+        e = cudaLaunchKernelEx(&cfg, attn_tc_fn(d.dtype == HT_BF16, pages != nullptr), tm_q, tm_k, tm_v, p, pp);
         if (e != cudaSuccess) {
             cudaGetLastError();
             return fail(HT_ERR_CUDA, "ht_tree_attention (tcgen05, clusters of %d): %s", k, cudaGetErrorString(e));
         }
         return HT_OK;
     }
-    if (d.dtype == HT_BF16) tc::attn_tc_kernel<true><<<p.grid, tc::kThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
-    else tc::attn_tc_kernel<false><<<p.grid, tc::kThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
+    attn_tc_fn(d.dtype == HT_BF16, pages != nullptr)<<<p.grid, tc::kThreads, smem, s>>>(tm_q, tm_k, tm_v, p, pp);
     return check_launch("ht_tree_attention (tcgen05)");
 }
 

@@ -20,6 +20,9 @@ constexpr int kMaxWords = 16;              // ancestor words per row -> N <= 512
 constexpr int kSlotFloats = kRows * kD + 2 * kRows;   // one partial result: O as [32 feature groups][128 rows][4], m[128], l[128]
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;  // log2 domain
+constexpr int kPgTiles = 8;                // paged cache: tiles whose page ids are held (4 in use or on their way + 4 being fetched)
+constexpr int kPgAhead = 4;                // ... and how many tiles ahead of the fetch the ids are asked for
+constexpr int kPgSub = 8;                  // pages per tile at the smallest page size (16 rows)
 
 struct Params {
     const int32_t *kv_len, *parent;
@@ -36,6 +39,14 @@ struct Params {
 #ifdef HT_TC_TRACE
     long long *trace;
 #endif
+};
+
+// Paged cache: cache row r of sequence b is row r % page_size of page block_table[b * max_pages + r / page_size];
+// the K / V maps then describe [page][head][row][D].  A kernel parameter of its own, read by the paged
+// instantiations only.
+struct PagedParams {
+    const int32_t *block_table;
+    int page_size, page_shift, max_pages, n_pages;      // page_size = 1 << page_shift
 };
 
 // Optional timeline of one CTA (clock64 stamps per role / tile / event) for tuning builds.
@@ -62,6 +73,7 @@ struct __align__(1024) Smem {
     int abort;
     int merge_here[2];
     int direct;
+    int32_t pg[kPgTiles][kPgSub];      // paged cache: page ids of the tiles about to be fetched
 };
 
 // ---------------------------------------------------------------------------------------
@@ -105,6 +117,14 @@ __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, v
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+
+// Asynchronous 4-byte copy global -> shared by the calling thread, and the group bookkeeping around it.
+__device__ __forceinline__ void cp_async4(void *dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
 
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -284,6 +304,30 @@ __device__ __forceinline__ Segment locate(const int32_t *pre, const int32_t *nkt
     return s;
 }
 
+// Walks the tiles of a CTA's range one by one; `locate` (two divisions) runs once per segment only.
+struct TileCursor {
+    Segment s;       // segment of the tile last returned
+    int i;           // tiles of it returned so far
+    int t, t_end, b_hint;
+    __device__ __forceinline__ void init(int t_begin, int t_end_) {
+        t = t_begin; t_end = t_end_; b_hint = 0; i = 0; s.len = 0; s.kt0 = 0;
+    }
+    // Moves to the next tile; false past the end of the range.  Afterwards s.b / s.hk / s.rt are the tile's
+    // unit, kt() its index within the unit's tiles and first() tells whether it opens a segment.
+    __device__ __forceinline__ bool next(const int32_t *pre, const int32_t *nkt, int B, int n_rt) {
+        if (i == s.len) {
+            if (t >= t_end) return false;
+            s = locate(pre, nkt, B, n_rt, t, t_end, b_hint);
+            i = 0;
+        }
+        ++i;
+        ++t;
+        return true;
+    }
+    __device__ __forceinline__ int kt() const { return s.kt0 + i - 1; }
+    __device__ __forceinline__ bool first() const { return i == 1; }
+};
+
 __device__ __forceinline__ int tiles_per_cta(int total, int grid) { return (total + grid - 1) / grid; }
 
 // Tiles per CTA.  An even share cuts nearly every unit in two, and every cut costs a partial
@@ -314,7 +358,7 @@ __device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nk
 // Validates every sequence and fills len / nkt / pre.  Called by all threads of a block.
 template <int NT>
 __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, int32_t *s_nkt, int32_t *s_pre,
-                                               bool write_status) {
+                                               bool write_status, bool errors_only = false) {
     // The lengths are asked for first and used last, so that their round trip to memory overlaps
     // the scan of the parent arrays (B <= kMaxB <= NT: one sequence per thread).
     const int my_b = threadIdx.x;
@@ -334,7 +378,9 @@ __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, 
         if (L < 0 || (long long)L + p.N > p.cap) code = HT_STATUS_BAD_LEN;
         s_len[b] = L;
         s_nkt[b] = code == HT_STATUS_OK ? (L + p.N + kTile - 1) / kTile : 0;
-        if (write_status) p.status[b] = code;
+        // paged cache: the status words were zeroed ahead of the launch, and a fetch may already have
+        // reported a bad page for this sequence, so only errors are written
+        if (write_status && (code != HT_STATUS_OK || !errors_only)) p.status[b] = code;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -348,6 +394,53 @@ __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, 
     __syncthreads();
 }
 
+
+// ---------------------------------------------------------------------------------------
+// Paged cache, producer side (one thread).  The page ids of tile jt of this CTA's range are asked for
+// kPgAhead tiles before the tile is fetched, by asynchronous 4-byte copies into a small ring in shared
+// memory, one copy group per tile (empty past the end of the range), so that the lookup's round trip
+// never stalls the fetches.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void pages_request(const Params &p, const PagedParams &pp, const int32_t *pre, const int32_t *nkt,
+                                              int32_t (*pg)[kPgSub], int jt, TileCursor &cur) {
+    if (cur.next(pre, nkt, p.B, p.n_rt)) {               // `cur` walks the range one tile per call: this is tile jt
+        const int sub = pp.page_size >= kTile ? 1 : kTile >> pp.page_shift;
+        const int first = (cur.kt() * kTile) >> pp.page_shift;
+        const int32_t *row = pp.block_table + (size_t)cur.s.b * pp.max_pages;
+        for (int x = 0; x < sub; ++x) {
+            if (first + x < pp.max_pages) cp_async4(&pg[jt % kPgTiles][x], row + first + x);
+            else pg[jt % kPgTiles][x] = -1;
+        }
+    }
+    cp_async_commit();
+}
+
+// Fetch of one K or V tile (two 64-feature slabs) into a ring entry.  Contiguous cache: rows kt * 128 ...
+// of (sequence b, head hk).  Paged cache: the tile's pages, whose ids `pg` holds; an id outside the pool
+// is replaced by page 0 (no access outside the pool), and reported in the sequence's status word if any of
+// the page's rows is a key of the sequence (rows past kv_len + N are masked and zeroed anyway).
+template <bool kPaged>
+__device__ __forceinline__ void fetch_kv_tile(const Params &p, const PagedParams &pp, unsigned char *dst, const CUtensorMap *tm,
+                                              void *bar, int b, int hk, int kt, int keys, const int32_t *pg) {
+    if (!kPaged) {
+        tma_load_4d(dst, tm, bar, 0, kt * kTile, hk, b);
+        tma_load_4d(dst + kSlabBytes, tm, bar, 64, kt * kTile, hk, b);
+        return;
+    }
+    const int ps = pp.page_size;
+    const int sub = ps >= kTile ? 1 : kTile >> pp.page_shift;
+    const int row0 = ps >= kTile ? (kt * kTile) & (ps - 1) : 0;
+    for (int x = 0; x < sub; ++x) {
+        int page = pg[x];
+        if ((unsigned)page >= (unsigned)pp.n_pages) {
+            if (kt * kTile + (x << pp.page_shift) < keys) p.status[b] = HT_STATUS_BAD_PAGE;
+            page = 0;
+        }
+        const int off = (x << pp.page_shift) * 128;         // rows of a slab are 128 bytes apart
+        tma_load_4d(dst + off, tm, bar, 0, row0, hk, page);
+        tma_load_4d(dst + kSlabBytes + off, tm, bar, 64, row0, hk, page);
+    }
+}
 
 // Ring order of the one-tile kernel: the tensor pipe consumes K_0, K_1, V_0, K_2, V_1, ... (the scores of
 // tile j+1 are issued before P V of tile j), so the tiles are fetched in that order and the ring is a FIFO:

@@ -39,12 +39,13 @@ struct __align__(1024) PSmem {
     int abort;
     int merge_here[2];
     int direct;
+    int32_t pg[kPgTiles][kPgSub];      // paged cache: page ids of the tiles about to be fetched
 };
 
-template <bool kBf16>
+template <bool kBf16, bool kPaged>
 __global__ void __launch_bounds__(kPThreads, 1)
 attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                    const __grid_constant__ CUtensorMap tm_v, const Params p) {
+                    const __grid_constant__ CUtensorMap tm_v, const Params p, const PagedParams pp) {
     extern __shared__ unsigned char smem_raw[];
     PSmem &sm = *reinterpret_cast<PSmem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -74,7 +75,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0);
+    plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0, kPaged);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -102,6 +103,10 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // ------------------------------- TMA producer -------------------------------
         if (lane == 0) {
             int b_hint = 0, ring_i = 0, seg_i = 0;
+            TileCursor cur_p;                         // page-id lookahead
+            cur_p.init(t_begin, t_end);
+            if (kPaged)
+                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p);
             for (int t = t_begin; t < t_end && !*abort_flag;) {
                 const Segment s = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
                 const bool two = 2 * s.rt + 1 < p.n_row_tiles;
@@ -119,13 +124,18 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (use > 0 && !mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag)) break;
                     HT_TR(0, ring_i >> 1, ring_i & 1);
                     const CUtensorMap *tm = (i & 1) ? &tm_v : &tm_k;
+                    const int jt = t - t_begin + (i >> 1);            // tile of this CTA's range
+                    if (kPaged && !(i & 1)) {
+                        pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt + kPgAhead, cur_p);
+                        cp_async_wait<kPgAhead>();
+                    }
                     mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
-                    tma_load_4d(sm.ring[slot], tm, &sm.kv_full[slot], 0, kt * kTile, s.hk, s.b);
-                    tma_load_4d(sm.ring[slot] + kSlabBytes, tm, &sm.kv_full[slot], 64, kt * kTile, s.hk, s.b);
+                    fetch_kv_tile<kPaged>(p, pp, sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt, sm.len[s.b] + p.N, sm.pg[jt % kPgTiles]);
                     ++ring_i;
                 }
                 t += s.len;
             }
+            if (kPaged) cp_async_wait<0>();
             if (*abort_flag) {
                 // Every copy this thread issued must have landed before the CTA exits.
                 for (int e = max(0, ring_i - kPStages); e < ring_i; ++e)
@@ -549,16 +559,19 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
 // Raises the kernels' dynamic shared memory limit (once per device) and launches.
 int launch_attn_tc_pair_kernel(const CUtensorMap &tm_q, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const tc::Params &p,
-                               bool bf16, cudaStream_t s) {
+                               const tc::PagedParams &pp, bool bf16, bool paged, cudaStream_t s) {
+    typedef void (*Fn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const tc::Params, const tc::PagedParams);
+    const Fn fns[4] = {tc::attn_tc_pair_kernel<false, false>, tc::attn_tc_pair_kernel<true, false>,
+                       tc::attn_tc_pair_kernel<false, true>, tc::attn_tc_pair_kernel<true, true>};
+    const Fn fn = fns[(bf16 ? 1 : 0) + (paged ? 2 : 0)];
     static bool done[64];
     const size_t smem = sizeof(tc::PSmem) + 1024;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
     if (!(dev >= 0 && dev < 64 && done[dev])) {
-        e = cudaFuncSetAttribute(tc::attn_tc_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tc::attn_tc_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        for (int i = 0; i < 4 && e == cudaSuccess; ++i)
+            e = cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         if (dev >= 0 && dev < 64) done[dev] = true;
     }
@@ -575,16 +588,14 @@ int launch_attn_tc_pair_kernel(const CUtensorMap &tm_q, const CUtensorMap &tm_k,
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        e = bf16 ? cudaLaunchKernelEx(&cfg, tc::attn_tc_pair_kernel<true>, tm_q, tm_k, tm_v, p)
-                 : cudaLaunchKernelEx(&cfg, tc::attn_tc_pair_kernel<false>, tm_q, tm_k, tm_v, p);
+        e = cudaLaunchKernelEx(&cfg, fn, tm_q, tm_k, tm_v, p, pp);
         if (e != cudaSuccess) {
             cudaGetLastError();
             return fail(HT_ERR_CUDA, "ht_tree_attention (tcgen05, tile pairs, clusters of %d): %s", p.cluster_k, cudaGetErrorString(e));
         }
         return HT_OK;
     }
-    if (bf16) tc::attn_tc_pair_kernel<true><<<p.grid, tc::kPThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
-    else tc::attn_tc_pair_kernel<false><<<p.grid, tc::kPThreads, smem, s>>>(tm_q, tm_k, tm_v, p);
+    fn<<<p.grid, tc::kPThreads, smem, s>>>(tm_q, tm_k, tm_v, p, pp);
     return check_launch("ht_tree_attention (tcgen05, tile pairs)");
 }
 

@@ -98,6 +98,41 @@ int ht_tree_attention(const ht_attn_desc *desc, const void *q, const void *k_cac
                             status, static_cast<cudaStream_t>(stream));
 }
 
+int ht_tree_attention_paged(const ht_attn_desc *desc, const ht_paged_desc *pages, const void *q, const void *k_pages,
+                            const void *v_pages, const int32_t *block_table, const int32_t *kv_len,
+                            const int32_t *parent, void *out, void *workspace, size_t workspace_bytes,
+                            int32_t *status, void *stream) {
+    if (!desc || !pages) return fail(HT_ERR_INVALID_ARG, "NULL descriptor");
+    const int ps = pages->page_size;
+    if (ps < 16 || (ps & (ps - 1)) != 0) return fail(HT_ERR_INVALID_ARG, "page_size must be a power of two >= 16");
+    if (pages->max_pages <= 0 || pages->n_pages <= 0) return fail(HT_ERR_INVALID_ARG, "max_pages and n_pages must be positive");
+    if ((long long)pages->max_pages * ps > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "max_pages * page_size too large");
+    if (pages->page_stride < 0 || pages->head_stride < 0 || pages->page_stride % 8 != 0 || pages->head_stride % 8 != 0)
+        return fail(HT_ERR_INVALID_ARG, "page strides must be non-negative multiples of 8 elements");
+    ht_attn_desc d = *desc;                      // the capacity of a sequence is what its table can hold
+    d.cap = pages->max_pages * ps;
+    d.kv_stride_b = 0;
+    d.kv_stride_h = 0;
+    int rc = check_attn_desc(&d);
+    if (rc != HT_OK) return rc;
+    if (pages->head_stride && pages->head_stride < (long long)ps * d.D)
+        return fail(HT_ERR_INVALID_ARG, "head_stride smaller than a page's rows of one head");
+    if (pages->page_stride && pages->page_stride < (long long)d.Hkv * ps * d.D)
+        return fail(HT_ERR_INVALID_ARG, "page_stride smaller than a page");
+    if (d.B == 0 || d.N == 0) return HT_OK;
+    if (!q || !k_pages || !v_pages || !block_table || !kv_len || !parent || !out || !status)
+        return fail(HT_ERR_INVALID_ARG, "NULL pointer");
+    if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out) || (workspace && !aligned16(workspace)))
+        return fail(HT_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    if (!attn_tc_applicable(d))
+        return fail(HT_ERR_UNSUPPORTED, "paged cache: fp16 / bf16, D = 128, Hq / Hkv a power of two, N <= 512, B <= 256, no flags or splits");
+    const size_t need = attn_tc_workspace(d);      // does not depend on the capacity
+    if (need > 0 && (!workspace || workspace_bytes < need))
+        return fail(HT_ERR_WORKSPACE, "workspace holds %zu bytes, %zu needed", workspace ? workspace_bytes : 0, need);
+    return launch_attn_tc(d, q, k_pages, v_pages, kv_len, parent, out, workspace, workspace_bytes, status,
+                          static_cast<cudaStream_t>(stream), pages, block_table);
+}
+
 int ht_verify_greedy(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
                      const int32_t *root_pred, int B, int N, int T, int V, int max_path, int32_t *pred,
                      int32_t *accept_len, int32_t *accept_path, int32_t *next_token, int32_t *status,

@@ -79,8 +79,10 @@ int launch_attn_simt(const ht_attn_desc &d, const void *q, const void *kc, const
                      int32_t *status, cudaStream_t s);
 bool attn_tc_applicable(const ht_attn_desc &d);
 size_t attn_tc_workspace(const ht_attn_desc &d);
+// `pages` / `block_table` null: contiguous cache (kc, vc as in ht_tree_attention); else the page pools.
 int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const void *vc, const int32_t *kv_len,
-                   const int32_t *parent, void *out, void *ws, size_t ws_bytes, int32_t *status, cudaStream_t s);
+                   const int32_t *parent, void *out, void *ws, size_t ws_bytes, int32_t *status, cudaStream_t s,
+                   const ht_paged_desc *pages = nullptr, const int32_t *block_table = nullptr);
 int launch_verify(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
                   const int32_t *root_pred, int B, int N, int T, int V, int max_path, int32_t *pred,
                   int32_t *accept_len, int32_t *accept_path, int32_t *next_token, int32_t *status,

@@ -431,6 +431,99 @@ def test_transfer_c5_shape(hb, oracle):
     assert_close(f32np(out), oracle.transfer(f32np(h), f32np(W)), torch.bfloat16, "transfer c5")
 
 
+# ---------------------------------------------------------------------------------------
+# Paged cache: the same attention with the rows of every sequence scattered over pages of a pool
+# ---------------------------------------------------------------------------------------
+def make_paged_case(seed, dtype, B, N, Hq, Hkv, lens, page_size, tree="random", extra_pages=1):
+    """A contiguous case whose caches are cut into pages and placed in a seeded random order; pages wholly
+    past a sequence's rows are not allocated (their table entries are -1) and unused pages hold NaN."""
+    from oracle import paged_oracle
+    per = (max(lens) + N + page_size - 1) // page_size + extra_pages
+    cap = per * page_size
+    q, k, v, kv_len, parent = make_attn_case(seed, dtype, B, N, Hq, Hkv, 128, lens, cap, tree, garbage=False)
+    kn, vn = k.float().cpu().numpy(), v.float().cpu().numpy()
+    pool_k, table = paged_oracle.scatter_to_pages(kn, page_size, seed + 1, fill=np.nan)
+    pool_v, _ = paged_oracle.scatter_to_pages(vn, page_size, seed + 1, fill=np.inf)
+    for b in range(B):
+        first_unused = (lens[b] + N + page_size - 1) // page_size
+        for i in range(first_unused, per):
+            pool_k[table[b, i]] = np.nan                       # "freed" pages: anything may be in them
+            pool_v[table[b, i]] = np.inf
+            table[b, i] = -1
+        used_rows = lens[b] + N                                # rows of the last page past the sequence
+        if used_rows % page_size:
+            pool_k[table[b, first_unused - 1], :, used_rows % page_size:] = np.nan
+            pool_v[table[b, first_unused - 1], :, used_rows % page_size:] = np.inf
+    dt = DT[dtype]
+    return (q, torch.from_numpy(pool_k).to(dt).cuda(), torch.from_numpy(pool_v).to(dt).cuda(),
+            torch.from_numpy(table).cuda(), kv_len, parent, k, v)
+
+
+PAGED_CASES = [
+    # (B, N, Hq, Hkv, lens, page_size): one-tile kernel, tile-pair kernel, clusters (B = 1), cut units
+    (2, 19, 8, 8, [37, 300], 16),
+    (3, 40, 32, 8, [0, 129, 515], 32),
+    (2, 91, 32, 32, [1000, 77], 64),
+    (4, 91, 32, 32, [500, 640, 128, 129], 128),
+    (2, 26, 16, 2, [700, 90], 256),
+    (1, 91, 32, 32, [1024], 16),
+    (1, 67, 64, 8, [2048], 128),
+    (2, 67, 64, 8, [3000, 4100], 64),
+    (1, 259, 64, 8, [600], 32),
+    (1, 30, 8, 1, [20000], 128),
+    (1, 30, 8, 1, [9000], 16),
+]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+@pytest.mark.parametrize("case", PAGED_CASES, ids=lambda c: "B%dN%dq%dkv%d_ps%d" % (c[0], c[1], c[2], c[3], c[5]))
+def test_paged_attention_against_the_oracle(hb, oracle, dtype, case):
+    from oracle import paged_oracle
+    B, N, Hq, Hkv, lens, ps = case
+    if dtype == "f16" and ps not in (16, 128):
+        pytest.skip("fp16 runs two page sizes")
+    q, pk, pv, table, kv_len, parent, k, v = make_paged_case(300 + ps + N, dtype, B, N, Hq, Hkv, lens, ps)
+    out, status = hb.tree_attention_paged(q, pk, pv, table, kv_len, parent)
+    assert status.cpu().tolist() == [0] * B
+    dt = DT[dtype]
+    # the contiguous entry point on the contiguous copy of the same data: same kernels, same tiles, so the
+    # results agree to the last bit whenever the work split is the same; compare within rounding
+    ref_out, _ = hb.tree_attention(q, k, v, kv_len, parent)
+    assert_close(f32np(out), f32np(ref_out), dt, "paged against contiguous")
+    if sum(lens) * N * Hq <= 40_000_000:
+        pkn, pvn = f32np(pk), f32np(pv)
+        pkn[~np.isfinite(pkn)] = 0.0
+        pvn[~np.isfinite(pvn)] = 0.0
+        args = (table.cpu().numpy(), kv_len.cpu().numpy(), parent.cpu().numpy())
+        want, ost = paged_oracle.tree_attention_paged(f32np(q), pkn, pvn, *args)
+        assert ost.tolist() == [0] * B
+        # rows with a handful of visible keys (a sequence without context): the weights' rounding to the
+        # input type shows, bounded by that fraction of the attention output of |V|
+        want_abs, _ = paged_oracle.tree_attention_paged(f32np(q), pkn, np.abs(pvn), *args)
+        assert_close_with_p_rounding(f32np(out), want, want_abs, dt, "paged attention")
+    else:
+        assert_close(f32np(out), oracle_attn(oracle, q, k, v, kv_len, parent), dt, "paged attention")
+
+
+def test_paged_attention_reports_bad_pages_and_lengths(hb):
+    from oracle import paged_oracle
+    B, N, Hq, Hkv, lens, ps = 3, 19, 8, 8, [100, 200, 300], 32
+    q, pk, pv, table, kv_len, parent, k, v = make_paged_case(77, "bf16", B, N, Hq, Hkv, lens, ps)
+    good, status = hb.tree_attention_paged(q, pk, pv, table, kv_len, parent)
+    assert status.cpu().tolist() == [0, 0, 0]
+    t2 = table.clone()
+    t2[1, 2] = pk.shape[0] + 5                     # a page sequence 1 needs, outside the pool
+    out, status = hb.tree_attention_paged(q, pk, pv, t2, kv_len, parent)
+    assert status.cpu().tolist() == [0, 5, 0]
+    assert torch.equal(out[0], good[0]) and torch.equal(out[2], good[2])
+    long = kv_len.clone()
+    long[2] = table.shape[1] * ps - N + 1          # one row more than the table can address
+    out = torch.full_like(good, 7.0)
+    out, status = hb.tree_attention_paged(q, pk, pv, table, long, parent, out=out)
+    assert status.cpu().tolist() == [0, 0, 2]
+    assert torch.equal(out[0], good[0]) and bool((out[2] == 7.0).all())
+
+
 # A pseudo state per tree node (Section "Hidden Transfer": every token of the sequence gets its pseudo
 # states) makes the batch B x T rows: the tensor-core kernel.  Shapes cover one and several 128-row tiles
 # with a ragged last one, a ragged last weight tile, a feature count that is not a multiple of 64, a
