@@ -97,17 +97,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
     if (warp == 8) {
         // ------------------------------- TMA producer -------------------------------
-        if (lane == 0) {
+        // Contiguous cache: one thread.  Paged cache: the whole warp walks the same loop (identical state in
+        // every lane), so that the pages of a tile are looked up and fetched by one lane each, in one
+        // instruction, instead of one after the other; lane 0 alone arms the barriers and fetches Q.
+        if (kPaged || lane == 0) {
             int ring_i = 0, seg_i = 0;
-            HT_TR_CTA(1);
+            if (lane == 0) HT_TR_CTA(1);
             const int n = t_end - t_begin;
             TileCursor cur_k, cur_v, cur_p;          // the K and V streams of the ring order, and the page-id lookahead
             cur_k.init(t_begin, t_end);
             cur_v.init(t_begin, t_end);
             cur_p.init(t_begin, t_end);
             if (kPaged)
-                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p);
-            for (int e = 0; e < 2 * n && !*abort_flag; ++e) {
+                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p, lane);
+            for (int e = 0; e < 2 * n; ++e) {
+                if (kPaged ? __any_sync(0xFFFFFFFFu, *abort_flag != 0) : (*abort_flag != 0)) break;
                 // entry e of the consumption order: K_0, K_1, V_0, K_2, V_1, ..., V_{n-1}
                 const bool is_v = e == 2 * n - 1 || (e != 0 && (e & 1) == 0);
                 const int j = e == 0 ? 0 : (e == 2 * n - 1 ? n - 1 : (is_v ? (e - 2) / 2 : (e + 1) / 2));
@@ -120,28 +124,45 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int kt = is_v ? cur_v.kt() : cur_k.kt();
                 if (!is_v && cur_k.first()) {
                     // first tile of a segment: its Q tile, once the previous segment's scores are done with Q
-                    if (seg_i > 0 && !mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag)) break;
-                    mbar_expect_tx(&sm.q_full, kEntryBytes);
-                    tma_load_4d(sm.q, &tm_q, &sm.q_full, 0, s.hk * p.g, s.rt * p.rows_per_tile_nodes, s.b);
-                    tma_load_4d(sm.q + kSlabBytes, &tm_q, &sm.q_full, 64, s.hk * p.g, s.rt * p.rows_per_tile_nodes, s.b);
+                    bool ok = seg_i == 0 || mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag);
+                    if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        mbar_expect_tx(&sm.q_full, kEntryBytes);
+                        tma_load_4d(sm.q, &tm_q, &sm.q_full, 0, s.hk * p.g, s.rt * p.rows_per_tile_nodes, s.b);
+                        tma_load_4d(sm.q + kSlabBytes, &tm_q, &sm.q_full, 64, s.hk * p.g, s.rt * p.rows_per_tile_nodes, s.b);
+                    }
                     ++seg_i;
                 }
                 const int slot = ring_i % kStages, use = ring_i / kStages;
-                if (use > 0 && !mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag)) break;
+                {
+                    bool ok = use == 0 || mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag);
+                    if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                }
                 HT_TR(0, j, is_v ? 1 : 0);
                 const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
                 if (kPaged && !is_v) {
                     // the ids of tile j were asked for kPgAhead tiles ago; ask for those of tile j + kPgAhead
-                    pages_request(p, pp, sm.pre, sm.nkt, sm.pg, j + kPgAhead, cur_p);
+                    pages_request(p, pp, sm.pre, sm.nkt, sm.pg, j + kPgAhead, cur_p, lane);
                     cp_async_wait<kPgAhead>();
                 }
-                mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
-                fetch_kv_tile<kPaged>(p, pp, sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt, sm.len[s.b] + p.N, sm.pg[j % kPgTiles]);
+                if (lane == 0) mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
+                if (kPaged) {
+                    __syncwarp();                                     // the barrier is armed before any lane's copy can complete
+                    fetch_kv_tile_paged(p, pp, sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt, sm.len[s.b] + p.N,
+                                        sm.pg[j % kPgTiles], lane);
+                } else {
+                    fetch_kv_tile(sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt);
+                }
                 ++ring_i;
             }
-            if (kPaged) cp_async_wait<0>();
-            if (*abort_flag) {
-                // Every copy this thread issued must have landed before the CTA exits: wait, with the
+            if (kPaged) {
+                cp_async_wait<0>();
+                __syncwarp();
+            }
+            if (lane == 0 && *abort_flag) {
+                // Every copy this warp issued must have landed before the CTA exits: wait, with the
                 // usual bound, for the latest armed phase of each ring slot and of the Q buffer.
                 for (int e = max(0, ring_i - kStages); e < ring_i; ++e)
                     mbar_wait(&sm.kv_full[e % kStages], (e / kStages) & 1, abort_flag, false);

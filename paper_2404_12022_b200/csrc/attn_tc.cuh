@@ -402,41 +402,42 @@ __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, 
 // never stalls the fetches.
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ void pages_request(const Params &p, const PagedParams &pp, const int32_t *pre, const int32_t *nkt,
-                                              int32_t (*pg)[kPgSub], int jt, TileCursor &cur) {
+                                              int32_t (*pg)[kPgSub], int jt, TileCursor &cur, int lane) {
     if (cur.next(pre, nkt, p.B, p.n_rt)) {               // `cur` walks the range one tile per call: this is tile jt
         const int sub = pp.page_size >= kTile ? 1 : kTile >> pp.page_shift;
         const int first = (cur.kt() * kTile) >> pp.page_shift;
-        const int32_t *row = pp.block_table + (size_t)cur.s.b * pp.max_pages;
-        for (int x = 0; x < sub; ++x) {
-            if (first + x < pp.max_pages) cp_async4(&pg[jt % kPgTiles][x], row + first + x);
-            else pg[jt % kPgTiles][x] = -1;
+        if (lane < sub) {                                // lane x: page x of the tile
+            if (first + lane < pp.max_pages)
+                cp_async4(&pg[jt % kPgTiles][lane], pp.block_table + (size_t)cur.s.b * pp.max_pages + first + lane);
+            else
+                pg[jt % kPgTiles][lane] = -1;
         }
     }
     cp_async_commit();
 }
 
-// Fetch of one K or V tile (two 64-feature slabs) into a ring entry.  Contiguous cache: rows kt * 128 ...
-// of (sequence b, head hk).  Paged cache: the tile's pages, whose ids `pg` holds; an id outside the pool
-// is replaced by page 0 (no access outside the pool), and reported in the sequence's status word if any of
-// the page's rows is a key of the sequence (rows past kv_len + N are masked and zeroed anyway).
-template <bool kPaged>
-__device__ __forceinline__ void fetch_kv_tile(const Params &p, const PagedParams &pp, unsigned char *dst, const CUtensorMap *tm,
-                                              void *bar, int b, int hk, int kt, int keys, const int32_t *pg) {
-    if (!kPaged) {
-        tma_load_4d(dst, tm, bar, 0, kt * kTile, hk, b);
-        tma_load_4d(dst + kSlabBytes, tm, bar, 64, kt * kTile, hk, b);
-        return;
-    }
+// Fetch of one K or V tile (two 64-feature slabs) into a ring entry.  Contiguous cache (one thread): rows
+// kt * 128 ... of (sequence b, head hk).
+__device__ __forceinline__ void fetch_kv_tile(unsigned char *dst, const CUtensorMap *tm, void *bar, int b, int hk, int kt) {
+    tma_load_4d(dst, tm, bar, 0, kt * kTile, hk, b);
+    tma_load_4d(dst + kSlabBytes, tm, bar, 64, kt * kTile, hk, b);
+}
+// Paged cache (the whole producer warp): lane x fetches the rows that page x of the tile holds, whose id
+// it asked for itself.  An id outside the pool is replaced by page 0 (no access outside the pool), and
+// reported in the sequence's status word if any of the page's rows is a key of the sequence (rows past
+// kv_len + N are masked and zeroed anyway).
+__device__ __forceinline__ void fetch_kv_tile_paged(const Params &p, const PagedParams &pp, unsigned char *dst, const CUtensorMap *tm,
+                                                    void *bar, int b, int hk, int kt, int keys, const int32_t *pg, int lane) {
     const int ps = pp.page_size;
     const int sub = ps >= kTile ? 1 : kTile >> pp.page_shift;
-    const int row0 = ps >= kTile ? (kt * kTile) & (ps - 1) : 0;
-    for (int x = 0; x < sub; ++x) {
-        int page = pg[x];
+    if (lane < sub) {
+        const int row0 = ps >= kTile ? (kt * kTile) & (ps - 1) : 0;
+        int page = pg[lane];
         if ((unsigned)page >= (unsigned)pp.n_pages) {
-            if (kt * kTile + (x << pp.page_shift) < keys) p.status[b] = HT_STATUS_BAD_PAGE;
+            if (kt * kTile + (lane << pp.page_shift) < keys) p.status[b] = HT_STATUS_BAD_PAGE;
             page = 0;
         }
-        const int off = (x << pp.page_shift) * 128;         // rows of a slab are 128 bytes apart
+        const int off = (lane << pp.page_shift) * 128;      // rows of a slab are 128 bytes apart
         tma_load_4d(dst + off, tm, bar, 0, row0, hk, page);
         tma_load_4d(dst + kSlabBytes + off, tm, bar, 64, row0, hk, page);
     }

@@ -101,43 +101,64 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     if (warp == 8) {
         // ------------------------------- TMA producer -------------------------------
-        if (lane == 0) {
+        // Contiguous cache: one thread.  Paged cache: the whole warp walks the loop with identical state and
+        // lane x looks up and fetches page x of a tile; lane 0 alone arms the barriers and fetches Q.
+        if (kPaged || lane == 0) {
             int b_hint = 0, ring_i = 0, seg_i = 0;
             TileCursor cur_p;                         // page-id lookahead
             cur_p.init(t_begin, t_end);
             if (kPaged)
-                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p);
-            for (int t = t_begin; t < t_end && !*abort_flag;) {
+                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p, lane);
+            bool stop = false;
+            for (int t = t_begin; t < t_end && !stop;) {
+                if (kPaged ? __any_sync(0xFFFFFFFFu, *abort_flag != 0) : (*abort_flag != 0)) break;
                 const Segment s = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
                 const bool two = 2 * s.rt + 1 < p.n_row_tiles;
-                if (seg_i > 0 && !mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag)) break;
-                mbar_expect_tx(&sm.q_full, two ? 2 * kEntryBytes : kEntryBytes);
-                for (int x = 0; x < (two ? 2 : 1); ++x) {
-                    const int node0 = (2 * s.rt + x) * p.rows_per_tile_nodes;
-                    tma_load_4d(sm.q[x], &tm_q, &sm.q_full, 0, s.hk * p.g, node0, s.b);
-                    tma_load_4d(sm.q[x] + kSlabBytes, &tm_q, &sm.q_full, 64, s.hk * p.g, node0, s.b);
+                {
+                    bool ok = seg_i == 0 || mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag);
+                    if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                }
+                if (lane == 0) {
+                    mbar_expect_tx(&sm.q_full, two ? 2 * kEntryBytes : kEntryBytes);
+                    for (int x = 0; x < (two ? 2 : 1); ++x) {
+                        const int node0 = (2 * s.rt + x) * p.rows_per_tile_nodes;
+                        tma_load_4d(sm.q[x], &tm_q, &sm.q_full, 0, s.hk * p.g, node0, s.b);
+                        tma_load_4d(sm.q[x] + kSlabBytes, &tm_q, &sm.q_full, 64, s.hk * p.g, node0, s.b);
+                    }
                 }
                 ++seg_i;
                 for (int i = 0; i < 2 * s.len; ++i) {
                     const int kt = s.kt0 + (i >> 1);
                     const int slot = ring_i % kPStages, use = ring_i / kPStages;
-                    if (use > 0 && !mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag)) break;
+                    bool ok = use == 0 || mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag);
+                    if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) { stop = true; break; }
                     HT_TR(0, ring_i >> 1, ring_i & 1);
                     const CUtensorMap *tm = (i & 1) ? &tm_v : &tm_k;
                     const int jt = t - t_begin + (i >> 1);            // tile of this CTA's range
                     if (kPaged && !(i & 1)) {
-                        pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt + kPgAhead, cur_p);
+                        pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt + kPgAhead, cur_p, lane);
                         cp_async_wait<kPgAhead>();
                     }
-                    mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
-                    fetch_kv_tile<kPaged>(p, pp, sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt, sm.len[s.b] + p.N, sm.pg[jt % kPgTiles]);
+                    if (lane == 0) mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
+                    if (kPaged) {
+                        __syncwarp();                                 // the barrier is armed before any lane's copy can complete
+                        fetch_kv_tile_paged(p, pp, sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt, sm.len[s.b] + p.N,
+                                            sm.pg[jt % kPgTiles], lane);
+                    } else {
+                        fetch_kv_tile(sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt);
+                    }
                     ++ring_i;
                 }
                 t += s.len;
             }
-            if (kPaged) cp_async_wait<0>();
-            if (*abort_flag) {
-                // Every copy this thread issued must have landed before the CTA exits.
+            if (kPaged) {
+                cp_async_wait<0>();
+                __syncwarp();
+            }
+            if (lane == 0 && *abort_flag) {
+                // Every copy this warp issued must have landed before the CTA exits.
                 for (int e = max(0, ring_i - kPStages); e < ring_i; ++e)
                     mbar_wait(&sm.kv_full[e % kPStages], (e / kPStages) & 1, abort_flag, false);
                 if (seg_i > 0) mbar_wait(&sm.q_full, (seg_i - 1) & 1, abort_flag, false);
