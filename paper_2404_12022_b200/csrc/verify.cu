@@ -22,6 +22,12 @@ __device__ __forceinline__ Best better(Best a, Best b) {
     return (b.v > a.v || (b.v == a.v && b.i < a.i)) ? b : a;
 }
 
+// pred is written by other blocks of the same launch: read through L2 when it is read from global memory
+// (a generic load works for the staged copy in shared memory as well).
+__device__ __forceinline__ int ld_pred(const int32_t *p) {
+    return __isGlobal(p) ? __ldcg(p) : *p;
+}
+
 // Path search of one sequence by one block.  Every thread walks the root path of its nodes (parent[c] < c
 // makes the walk finite), checks the match rule on the way and proposes (depth, node);
 // the block keeps the deepest valid node, lowest index on ties.
@@ -35,10 +41,25 @@ __device__ __forceinline__ void accept_sequence(const int b, const int32_t *__re
     int32_t *path = accept_path + (size_t)b * max_path;
     __shared__ int s_bad;
     __shared__ unsigned long long s_key[8];
+    // The walks below are chains of dependent reads: with the tree's three arrays in shared memory they
+    // cost one round trip to L2 in all instead of one per level (trees of up to kStage rows).
+    constexpr int kStage = 1024;
+    __shared__ int32_t s_par[kStage], s_tok[kStage], s_prd[kStage];
     if (threadIdx.x == 0) s_bad = 0;
     __syncthreads();
-    for (int c = threadIdx.x; c < N; c += blockDim.x)
-        if (par[c] < -1 || par[c] >= c) s_bad = 1;
+    if (N <= kStage) {
+        for (int c = threadIdx.x; c < N; c += blockDim.x) {
+            const int pc = par[c];
+            s_par[c] = pc;
+            s_prd[c] = __ldcg(prd + c);
+            if (c < T) s_tok[c] = tok[c];
+            if (pc < -1 || pc >= c) s_bad = 1;
+        }
+        par = s_par; tok = s_tok; prd = s_prd;
+    } else {
+        for (int c = threadIdx.x; c < N; c += blockDim.x)
+            if (par[c] < -1 || par[c] >= c) s_bad = 1;
+    }
     for (int j = threadIdx.x; j < max_path; j += blockDim.x) path[j] = -1;
     __syncthreads();
     if (s_bad) {
@@ -58,7 +79,7 @@ __device__ __forceinline__ void accept_sequence(const int b, const int32_t *__re
         bool ok = true;
         for (int c = n; c >= 0; c = par[c]) {
             const int p = par[c];
-            const bool m = p < 0 ? (!has_root || tok[c] == rp) : (tok[c] == __ldcg(prd + p));
+            const bool m = p < 0 ? (!has_root || tok[c] == rp) : (tok[c] == ld_pred(prd + p));
             ok = ok && m;
             ++depth;
         }
@@ -90,7 +111,7 @@ __device__ __forceinline__ void accept_sequence(const int b, const int32_t *__re
             } else {
                 int j = len - 1;
                 for (int c = node; c >= 0; c = par[c]) path[j--] = c;
-                next_token[b] = __ldcg(prd + node);
+                next_token[b] = ld_pred(prd + node);
             }
         }
     }
@@ -123,16 +144,17 @@ verify_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pred, c
                 unpack16<T>(raw[u], f);
 #pragma unroll
                 for (int e = 0; e < VE; ++e) {
-                    // NaN compares false both ways and is skipped; -inf at a lower index than
-                    // the current -inf candidate is taken through the equality branch.
-                    if (f[e] > best.v || (f[e] == best.v && j * VE + e < best.i)) best = Best{f[e], j * VE + e};
+                    // A thread meets its elements in increasing index order, so "larger value, lower index
+                    // on ties" is "strictly larger than the best so far".  NaN compares false and is
+                    // skipped; so is -inf, which a row without anything larger settles below.
+                    if (f[e] > best.v) best = Best{f[e], j * VE + e};
                 }
             }
         }
     } else {
         for (int j = threadIdx.x; j < V; j += blockDim.x) {
             const float x = to_float<T>(row[j]);
-            if (x > best.v || (x == best.v && j < best.i)) best = Best{x, j};
+            if (x > best.v) best = Best{x, j};
         }
     }
 #pragma unroll
@@ -151,8 +173,26 @@ verify_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pred, c
             Best o{__shfl_xor_sync(0xffffffffu, best.v, off), __shfl_xor_sync(0xffffffffu, best.i, off)};
             best = better(best, o);
         }
-        if (lane == 0) pred[blockIdx.x] = best.i == INT_MAX ? 0 : best.i;
+        if (lane == 0) warp_best[0] = best;
     }
+    __syncthreads();
+    best = warp_best[0];
+    if (best.i == INT_MAX) {
+        // Nothing in the row exceeds -inf: the answer is the first -inf, or 0 in a row of NaNs only.
+        int first = INT_MAX;
+        for (int j = threadIdx.x; j < V; j += blockDim.x)
+            if (to_float<T>(row[j]) == -INFINITY) { first = j; break; }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) first = min(first, __shfl_xor_sync(0xffffffffu, first, off));
+        __shared__ int warp_first[8];
+        if (lane == 0) warp_first[warp] = first;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int w = 1; w < (int)(blockDim.x >> 5); ++w) first = min(first, warp_first[w]);
+            best.i = first == INT_MAX ? 0 : first;
+        }
+    }
+    if (threadIdx.x == 0) pred[blockIdx.x] = best.i;
     // The block that stores a sequence's last argmax searches its tree.
     __shared__ int s_last;
     const int b = blockIdx.x / N;
