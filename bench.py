@@ -221,9 +221,9 @@ class ClockSampler:
 # DRAM traffic per launch of the attention kernel on a c3 layer, from the ncu capture summarised in
 # profiles/attn_tc_kernel_c3_layer.md (dram__bytes_read.sum + dram__bytes_write.sum).  It is only
 # reported while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 290.4e6,
+NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 291.8e6,
                "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh"],
-               "sha256": "5ea1da2f6bd14ec46bccef71e658d6df28292457d9c55d2d70a1dece032940f1"}
+               "sha256": "fb447c2e5d2e1f2b5508bf7acee7f899d77dffa4a26ddb59c33f2dcafc5062ed"}
 
 
 def ncu_traffic(w):
