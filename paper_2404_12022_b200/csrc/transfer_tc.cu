@@ -24,7 +24,7 @@ constexpr int kBK = 64;                    // features per stage: one swizzled 1
 constexpr int kHBytes = kBM * kBK * 2;     // h tile of a stage
 constexpr int kTThreads = 192;             // warps 0-3 read the accumulator, warp 4 TMA, warp 5 MMA
 constexpr int kMaxStages = 24;
-constexpr uint32_t kAccCols = 256;         // TMEM columns: bn <= 256
+constexpr uint32_t kAccCols = 256;         // TMEM columns of one accumulator: bn <= 256
 
 struct TParams {
     void *out;
@@ -32,6 +32,7 @@ struct TParams {
     int bn, n_m, stages;    // weight rows per tile, 128-row tiles of the batch, ring depth
     int h_rows;             // rows of the h box: 128, or fewer when the whole batch is smaller
     int kc;                 // 64-feature chunks per stage (one TMA instruction per operand fetches them all)
+    int mt;                 // 128-row tiles of h per CTA: 1, or 2 (two accumulators, one W tile for both)
     uint32_t stage_bytes;
 };
 
@@ -66,10 +67,11 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
                    const __grid_constant__ CUtensorMap tm_h_tail, const __grid_constant__ CUtensorMap tm_w_tail, const TParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *base = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    TBars &bar = *reinterpret_cast<TBars *>(base + (size_t)p.stages * p.stage_bytes + (kBM - p.h_rows) * kBK * 2);
+    TBars &bar = *reinterpret_cast<TBars *>(base + (size_t)p.stages * p.stage_bytes + (kBM * p.mt - p.h_rows) * kBK * 2);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &bar.abort;
-    const int m0 = ((int)blockIdx.x % p.n_m) * kBM, n0 = ((int)blockIdx.x / p.n_m) * p.bn;
+    const int m0 = ((int)blockIdx.x % p.n_m) * kBM * p.mt, n0 = ((int)blockIdx.x / p.n_m) * p.bn;
+    const uint32_t acc_cols = kAccCols * (uint32_t)p.mt;
     const int n_main = p.kc > 1 ? (p.d / kBK) / p.kc : 0;             // steps of kc whole chunks through the chunked view
     const int f_rest = n_main * p.kc * kBK;                           // first feature after them
     const int nk = n_main + (p.d - f_rest + kBK - 1) / kBK;           // + single chunks (the last one may be ragged)
@@ -91,7 +93,7 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         }
     }
     if (warp == 4) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bar.tmem_base)), "r"(kAccCols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bar.tmem_base)), "r"(acc_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -136,10 +138,13 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
                 const uint32_t a_addr = smem_u32(base + (size_t)slot * p.stage_bytes), b_addr = a_addr + chunk_h * p.kc;
                 const int chunks = ks < n_main ? p.kc : 1;
                 for (int c = 0; c < chunks; ++c) {
+                    for (int i = 0; i < p.mt; ++i) {           // a second 128-row tile of h, if it has rows at all
+                        if (i > 0 && m0 + i * kBM >= p.B) break;
 #pragma unroll
-                    for (int kk = 0; kk < kBK / 16; ++kk)      // 16 features = 32 bytes inside the swizzled line
-                        mma_ss(tmem, smem_desc(a_addr + c * chunk_h + kk * 32, 1, 1024 >> 4),
-                               smem_desc(b_addr + c * chunk_w + kk * 32, 1, 1024 >> 4), idesc, (ks | c | kk) != 0 ? 1u : 0u);
+                        for (int kk = 0; kk < kBK / 16; ++kk)  // 16 features = 32 bytes inside the swizzled line
+                            mma_ss(tmem + i * kAccCols, smem_desc(a_addr + c * chunk_h + i * kHBytes + kk * 32, 1, 1024 >> 4),
+                                   smem_desc(b_addr + c * chunk_w + kk * 32, 1, 1024 >> 4), idesc, (ks | c | kk) != 0 ? 1u : 0u);
+                    }
                 }
                 tc_commit(&bar.empty[slot]);
             }
@@ -150,30 +155,33 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         }
     } else {
         // ------------------------------- accumulator -> out -------------------------------
-        const int row = m0 + (int)threadIdx.x;             // TMEM lane = source row of the tile
         const bool waited = mbar_wait(&bar.acc_full, 0, abort_flag);
         const bool ok = __all_sync(0xFFFFFFFFu, waited);
         tc_fence_after();
-        unsigned char *dst_row = static_cast<unsigned char *>(p.out) + ((size_t)min(row, p.B - 1) * p.R + n0) * 2;
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        for (int i = 0; i < p.mt; ++i) {
+            const int row = m0 + i * kBM + (int)threadIdx.x;   // TMEM lane = source row of the tile
+            if (m0 + i * kBM >= p.B) break;
+            unsigned char *dst_row = static_cast<unsigned char *>(p.out) + ((size_t)min(row, p.B - 1) * p.R + n0) * 2;
 #pragma unroll 1
-        for (int c = 0; c < p.bn; c += 32) {
-            float v[32];
-            if (ok) {
-                tmem_ld32(tmem + lane_base + c, v);
-                tmem_ld_wait();
-            } else {
-                // a wait ran out: the tile's results are marked as not-a-number instead of left stale
+            for (int c = 0; c < p.bn; c += 32) {
+                float v[32];
+                if (ok) {
+                    tmem_ld32(tmem + lane_base + i * kAccCols + c, v);
+                    tmem_ld_wait();
+                } else {
+                    // a wait ran out: the tile's results are marked as not-a-number instead of left stale
 #pragma unroll
-                for (int x = 0; x < 32; ++x) v[x] = __int_as_float(0x7FC00000);
-            }
-            if (row < p.B) {
+                    for (int x = 0; x < 32; ++x) v[x] = __int_as_float(0x7FC00000);
+                }
+                if (row < p.B) {
 #pragma unroll
-                for (int x = 0; x < 32; x += 8) {
-                    if (c + x < p.bn && n0 + c + x < p.R)  // R and n0 are multiples of 8: a group of 8 is in or out as a whole
-                        *reinterpret_cast<uint4 *>(dst_row + (c + x) * 2) =
-                            make_uint4(pack2<kBf16>(v[x], v[x + 1]), pack2<kBf16>(v[x + 2], v[x + 3]),
-                                       pack2<kBf16>(v[x + 4], v[x + 5]), pack2<kBf16>(v[x + 6], v[x + 7]));
+                    for (int x = 0; x < 32; x += 8) {
+                        if (c + x < p.bn && n0 + c + x < p.R)  // R and n0 are multiples of 8: a group of 8 is in or out as a whole
+                            *reinterpret_cast<uint4 *>(dst_row + (c + x) * 2) =
+                                make_uint4(pack2<kBf16>(v[x], v[x + 1]), pack2<kBf16>(v[x + 2], v[x + 3]),
+                                           pack2<kBf16>(v[x + 4], v[x + 5]), pack2<kBf16>(v[x + 6], v[x + 7]));
+                    }
                 }
             }
         }
@@ -183,7 +191,7 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     __syncthreads();
     if (warp == 4) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kAccCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(acc_cols) : "memory");
     }
 }
 
@@ -273,19 +281,22 @@ int launch_transfer_tc(const void *h, const void *W, void *out, int B, int k, in
     p.out = out;
     p.B = B; p.R = R; p.d = d;
     p.bn = transfer_tc_tile(B, R, device_sms());
-    p.n_m = (B + ttc::kBM - 1) / ttc::kBM;
+    // Two 128-row tiles of h per CTA (two accumulators fed by one W tile) once there are enough rows: a third
+    // less traffic from L2 into shared memory per product, which is what bounds the large shapes.
+    p.mt = B > 3 * ttc::kBM ? 2 : 1;
+    p.n_m = (B + ttc::kBM * p.mt - 1) / (ttc::kBM * p.mt);
     // Fewer than 128 source rows: only those are fetched and held.  The tensor pipe still reads 128 rows
     // from the h tile's address on, i.e. on into the W tile and the next stage (the ring is followed by that
     // much padding); row m of the product depends on row m of h alone, and rows past B are not stored.
-    p.h_rows = B >= ttc::kBM ? ttc::kBM : (B + 7) / 8 * 8;
+    p.h_rows = p.mt == 2 ? 2 * ttc::kBM : (B >= ttc::kBM ? ttc::kBM : (B + 7) / 8 * 8);
     const int n_full = d / ttc::kBK;
-    const size_t pad = (size_t)(ttc::kBM - p.h_rows) * ttc::kBK * 2;
+    const size_t pad = (size_t)(ttc::kBM * p.mt - p.h_rows) * ttc::kBK * 2;
     const size_t budget = 227 * 1024 - 1024 - pad - sizeof(ttc::TBars) - 64;
     const size_t chunk_bytes = (size_t)(p.h_rows + p.bn) * ttc::kBK * 2;
     // Chunks per step: as many as leave two stages, for the streaming shapes (one 128-row tile of h, W tiles
     // well below the maximum); one for the others.
     p.kc = 1;
-    if (p.n_m == 1 && p.bn < 192)
+    if (p.mt == 1 && p.n_m == 1 && p.bn < 192)
         for (int kc = 8; kc > 1; kc /= 2)
             if (kc <= n_full && chunk_bytes * kc * 2 <= budget) { p.kc = kc; break; }
     p.stage_bytes = (uint32_t)((p.h_rows + p.bn) * ttc::kBK * 2 * p.kc);

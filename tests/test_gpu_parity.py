@@ -527,10 +527,11 @@ def test_paged_attention_reports_bad_pages_and_lengths(hb):
 # A pseudo state per tree node (Section "Hidden Transfer": every token of the sequence gets its pseudo
 # states) makes the batch B x T rows: the tensor-core kernel.  Shapes cover one and several 128-row tiles
 # with a ragged last one, a ragged last weight tile, a feature count that is not a multiple of 64, a
-# single 64-feature step, and the per-node batches of configs 2 and 3.
+# single 64-feature step, the per-node batches of configs 2 and 3, and (above 384 rows) CTAs that hold two 128-row
+# tiles, the second of them full, ragged or empty.
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 @pytest.mark.parametrize("shape", [(17, 1, 64), (40, 2, 520), (88, 3, 1024), (128, 1, 256), (129, 2, 512),
-                                   (352, 3, 1024), (300, 1, 2056)],
+                                   (352, 3, 1024), (300, 1, 2056), (400, 2, 520), (513, 1, 256), (777, 1, 1024)],
                          ids=lambda s: "B%dk%dd%d" % s)
 def test_transfer_many_rows(hb, oracle, dtype, shape):
     B, k, d = shape
