@@ -165,6 +165,27 @@ int ht_tree_attention_paged(const ht_attn_desc *desc /* host */, const ht_paged_
                             void *stream);
 
 /*
+ * The two row-moving steps on a paged cache (same pools, block table and descriptor as
+ * ht_tree_attention_paged; one block table serves all layers):
+ *   ht_rope_kv_append_paged  as ht_rope_kv_append, the rows of sequence b landing at logical cache rows
+ *       kv_len[b] + r through the block table.  A row whose page entry lies outside the pool is
+ *       not stored (its q row is still rotated) and marks the sequence HT_STATUS_BAD_PAGE.
+ *   ht_kv_compact_paged      as ht_kv_compact on pools [layers, n_pages, Hkv, page_size, D];
+ *       desc->cap, stride_b and stride_h are ignored (the capacity is max_pages * page_size, the strides
+ *       are those of `pages`), desc->stride_layer is the distance between the layers' pools in
+ *       elements (0 = n_pages * page_stride).  Rows move between pages as the table says; a
+ *       needed entry outside the pool leaves the sequence unchanged with HT_STATUS_BAD_PAGE.
+ */
+int ht_rope_kv_append_paged(const ht_attn_desc *desc /* host */, const ht_paged_desc *pages /* host */,
+                            const void *q_in, const void *k_in, const void *v_in, const int32_t *pos,
+                            const int32_t *kv_len, const int32_t *block_table, float rope_base,
+                            void *q_out, void *k_pages, void *v_pages, int32_t *status, void *stream);
+int ht_kv_compact_paged(void *k_pages, void *v_pages, const ht_cache_desc *desc /* host */,
+                        const ht_paged_desc *pages /* host */, const int32_t *block_table,
+                        const int32_t *kv_len, const int32_t *accept_len, const int32_t *accept_path,
+                        int max_path, int32_t *new_kv_len, int32_t *status, void *stream);
+
+/*
  * Greedy verification -- Fig. 2 caption ("find the last accepted token position"),
  * Section "Inference stage", Section "Setup" (greedy sampling; output identical to
  * auto-regressive decoding).

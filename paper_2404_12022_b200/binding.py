@@ -24,7 +24,7 @@ HT_ATTN_FORCE_SIMT = 1
 
 EXPORTS = ("ht_version", "ht_last_error_string", "ht_transfer", "ht_tree_attention_workspace",
            "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact", "ht_draft_tree", "ht_rope_kv_append", "ht_tree_attention_static",
-           "ht_tree_attention_paged")
+           "ht_tree_attention_paged", "ht_rope_kv_append_paged", "ht_kv_compact_paged")
 HT_STATIC_SCRATCH_BYTES = 16 << 20
 
 _DTYPES = {torch.float32: HT_F32, torch.float16: HT_F16, torch.bfloat16: HT_BF16}
@@ -81,6 +81,12 @@ def load() -> ctypes.CDLL:
         lib.ht_tree_attention_static.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.ht_tree_attention_paged.restype = i32
         lib.ht_tree_attention_paged.argtypes = [ctypes.POINTER(AttnDesc), ctypes.POINTER(PagedDesc), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        lib.ht_rope_kv_append_paged.restype = i32
+        lib.ht_rope_kv_append_paged.argtypes = [ctypes.POINTER(AttnDesc), ctypes.POINTER(PagedDesc), vp, vp, vp, vp, vp, vp,
+                                                ctypes.c_float, vp, vp, vp, vp, vp]
+        lib.ht_kv_compact_paged.restype = i32
+        lib.ht_kv_compact_paged.argtypes = [vp, vp, ctypes.POINTER(CacheDesc), ctypes.POINTER(PagedDesc), vp, vp, vp, vp, i32,
+                                            vp, vp, vp]
         lib.ht_verify_greedy.restype = i32
         lib.ht_verify_greedy.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         lib.ht_kv_compact.restype = i32
@@ -319,3 +325,59 @@ def rope_kv_append(q_in, k_in, v_in, pos, kv_len, k_cache, v_cache, rope_base: f
     _check(load().ht_rope_kv_append(ctypes.byref(desc), _ptr(q_in), _ptr(k_in), _ptr(v_in), _ptr(pos), _ptr(kv_len),
                                     float(rope_base), _ptr(q_out), _ptr(k_cache), _ptr(v_cache), _ptr(status), _stream()))
     return q_out, status
+
+
+def rope_kv_append_paged(q_in, k_in, v_in, pos, kv_len, block_table, k_pages, v_pages, rope_base: float = 10000.0,
+                         q_out=None):
+    """As ``rope_kv_append`` with the caches as page pools [n_pages, Hkv, page_size, D] (written in place at the
+    logical rows kv_len[b] + r through block_table [B, max_pages]).  Returns (q_out, status)."""
+    _need(q_in, name="q_in")
+    _need(k_in, q_in.dtype, "k_in")
+    _need(v_in, q_in.dtype, "v_in")
+    _need(pos, torch.int32, "pos")
+    _need(kv_len, torch.int32, "kv_len")
+    _need(block_table, torch.int32, "block_table")
+    B, N, Hq, D = q_in.shape
+    n_pages, Hkv, page_size, Dp = k_pages.shape
+    if Dp != D or k_pages.stride(3) != 1 or k_pages.stride(2) != D or k_pages.stride() != v_pages.stride():
+        raise ValueError("page rows must be contiguous and D apart, K and V pools alike")
+    max_pages = block_table.shape[1]
+    desc = AttnDesc(B, N, Hq, Hkv, D, max_pages * page_size, _DTYPES[q_in.dtype], 0.0, 0, 0, 0, 0)
+    pages = PagedDesc(page_size, max_pages, n_pages, k_pages.stride(0), k_pages.stride(1))
+    if q_out is None:
+        q_out = torch.empty_like(q_in)
+    status = torch.empty(B, dtype=torch.int32, device=q_in.device)
+    _check(load().ht_rope_kv_append_paged(ctypes.byref(desc), ctypes.byref(pages), _ptr(q_in), _ptr(k_in), _ptr(v_in),
+                                          _ptr(pos), _ptr(kv_len), _ptr(block_table), float(rope_base), _ptr(q_out),
+                                          _ptr(k_pages), _ptr(v_pages), _ptr(status), _stream()))
+    return q_out, status
+
+
+def kv_compact_paged(k_pages, v_pages, block_table, n_rows: int, kv_len, accept_len, accept_path, new_kv_len=None,
+                     status=None):
+    """In-place compaction of page pools [layers, n_pages, Hkv, page_size, D] that share block_table
+    [B, max_pages].  Returns (new_kv_len, status)."""
+    if not (k_pages.is_cuda and v_pages.is_cuda) or k_pages.dtype != v_pages.dtype:
+        raise ValueError("pools must be CUDA tensors of one dtype")
+    if k_pages.stride() != v_pages.stride() or k_pages.shape != v_pages.shape:
+        raise ValueError("k_pages and v_pages must share shape and strides")
+    layers, n_pages, Hkv, page_size, D = k_pages.shape
+    if k_pages.stride(4) != 1 or k_pages.stride(3) != D:
+        raise ValueError("page rows must be contiguous and D apart")
+    _need(block_table, torch.int32, "block_table")
+    _need(kv_len, torch.int32, "kv_len")
+    _need(accept_len, torch.int32, "accept_len")
+    _need(accept_path, torch.int32, "accept_path")
+    B, max_pages = block_table.shape
+    max_path = accept_path.shape[1]
+    desc = CacheDesc(layers, B, Hkv, max_pages * page_size, D, _DTYPES[k_pages.dtype], int(n_rows), k_pages.stride(0), 0, 0)
+    pages = PagedDesc(page_size, max_pages, n_pages, k_pages.stride(1), k_pages.stride(2))
+    dev = k_pages.device
+    if new_kv_len is None:
+        new_kv_len = torch.empty(B, dtype=torch.int32, device=dev)
+    if status is None:
+        status = torch.empty(B, dtype=torch.int32, device=dev)
+    _check(load().ht_kv_compact_paged(_ptr(k_pages), _ptr(v_pages), ctypes.byref(desc), ctypes.byref(pages),
+                                      _ptr(block_table), _ptr(kv_len), _ptr(accept_len), _ptr(accept_path), max_path,
+                                      _ptr(new_kv_len), _ptr(status), _stream()))
+    return new_kv_len, status

@@ -26,8 +26,10 @@ compact_kernel(unsigned char *__restrict__ k_cache, unsigned char *__restrict__ 
                int layers, int B, int Hkv, int cap, int N, int row_bytes, long long stride_layer_b,
                long long stride_b_b, long long stride_h_b, const int32_t *__restrict__ kv_len,
                const int32_t *__restrict__ accept_len, const int32_t *__restrict__ accept_path,
-               int max_path, int groups, int32_t *__restrict__ new_kv_len, int32_t *__restrict__ status) {
+               int max_path, int groups, int32_t *__restrict__ new_kv_len, int32_t *__restrict__ status, const PageMap pm) {
     __shared__ int32_t s_path[kCompactMaxPath];
+    __shared__ long long s_src[kCompactMaxPath], s_dst[kCompactMaxPath];   // byte offsets of the rows within (layer, tensor), short of the head's
+    __shared__ int s_bad_page;
     int idx = blockIdx.x;
     const int grp = idx % groups;
     idx /= groups;
@@ -52,6 +54,27 @@ compact_kernel(unsigned char *__restrict__ k_cache, unsigned char *__restrict__ 
             if (p < j || p >= N || (j > 0 && p <= s_path[j - 1])) code = HT_STATUS_BAD_PATH;
         }
     }
+    // Where the path's source and destination rows lie.  Paged cache: through the block table; an entry
+    // outside the pool leaves the sequence untouched, and every block of the sequence sees the same entries.
+    if (threadIdx.x == 0) s_bad_page = 0;
+    __syncthreads();
+    if (code == HT_STATUS_OK && threadIdx.x < a) {
+        const int j = threadIdx.x, rows[2] = {L + s_path[j], L + j};
+        long long off[2];
+        for (int x = 0; x < 2; ++x) {
+            if (pm.table) {
+                const int page = pm.table[(size_t)b * pm.max_pages + (rows[x] >> pm.shift)];
+                if ((unsigned)page >= (unsigned)pm.n_pages) s_bad_page = 1;
+                off[x] = (long long)page * pm.page_stride + (long long)(rows[x] & ((1 << pm.shift) - 1)) * row_bytes;   // strides of `pm` in bytes here
+            } else {
+                off[x] = (long long)b * stride_b_b + (long long)rows[x] * row_bytes;
+            }
+        }
+        s_src[j] = off[0];
+        s_dst[j] = off[1];
+    }
+    __syncthreads();
+    if (code == HT_STATUS_OK && s_bad_page) code = HT_STATUS_BAD_PAGE;
     if (layer == 0 && grp == 0 && threadIdx.x == 0) {
         status[b] = code;
         new_kv_len[b] = code == HT_STATUS_OK ? L + a : L;
@@ -63,8 +86,8 @@ compact_kernel(unsigned char *__restrict__ k_cache, unsigned char *__restrict__ 
     const int vec_per_row = row_bytes / 16;
     const int per_pair = a * vec_per_row;                        // <= 4096 (checked by the caller)
     const int pairs_per_pass = max(1, kCompactPerThread * kCompactThreads / per_pair);
-    unsigned char *const base_k = k_cache + (long long)layer * stride_layer_b + (long long)b * stride_b_b;
-    unsigned char *const base_v = v_cache + (long long)layer * stride_layer_b + (long long)b * stride_b_b;
+    unsigned char *const base_k = k_cache + (long long)layer * stride_layer_b;
+    unsigned char *const base_v = v_cache + (long long)layer * stride_layer_b;
 
     for (int p0 = pair_lo; p0 < pair_hi; p0 += pairs_per_pass) {
         const int total = min(pairs_per_pass, pair_hi - p0) * per_pair;
@@ -78,7 +101,7 @@ compact_kernel(unsigned char *__restrict__ k_cache, unsigned char *__restrict__ 
                 const int pair = p0 + pr, src = s_path[j];
                 const unsigned char *base = ((pair & 1) ? base_v : base_k) + (long long)(pair >> 1) * stride_h_b;
                 if (src != j)
-                    regs[i] = *reinterpret_cast<const uint4 *>(base + (size_t)(L + src) * row_bytes + (size_t)v * 16);
+                    regs[i] = *reinterpret_cast<const uint4 *>(base + s_src[j] + (size_t)v * 16);
             }
         }
         __syncthreads();
@@ -91,7 +114,7 @@ compact_kernel(unsigned char *__restrict__ k_cache, unsigned char *__restrict__ 
                 const int pair = p0 + pr;
                 unsigned char *base = ((pair & 1) ? base_v : base_k) + (long long)(pair >> 1) * stride_h_b;
                 if (s_path[j] != j)
-                    *reinterpret_cast<uint4 *>(base + (size_t)(L + j) * row_bytes + (size_t)v * 16) = regs[i];
+                    *reinterpret_cast<uint4 *>(base + s_dst[j] + (size_t)v * 16) = regs[i];
             }
         }
         __syncthreads();     // the next pass of this block may touch rows this pass has written only after all of it has
@@ -100,11 +123,14 @@ compact_kernel(unsigned char *__restrict__ k_cache, unsigned char *__restrict__ 
 
 int launch_compact(void *kc, void *vc, const ht_cache_desc &d, const int32_t *kv_len,
                    const int32_t *accept_len, const int32_t *accept_path, int max_path,
-                   int32_t *new_kv_len, int32_t *status, cudaStream_t s) {
+                   int32_t *new_kv_len, int32_t *status, cudaStream_t s, const PageMap &pm_elems) {
     const long long e = elem_bytes(d.dtype);
-    const long long stride_h = (d.stride_h ? d.stride_h : (long long)d.cap * d.D) * e;
+    PageMap pm = pm_elems;                 // the kernel takes the page strides in bytes
+    pm.page_stride *= e;
+    pm.head_stride *= e;
+    const long long stride_h = pm.table ? pm.head_stride : (d.stride_h ? d.stride_h : (long long)d.cap * d.D) * e;
     const long long stride_b = (d.stride_b ? d.stride_b : (long long)d.Hkv * d.cap * d.D) * e;
-    const long long stride_l = (d.stride_layer ? d.stride_layer : (long long)d.B * d.Hkv * d.cap * d.D) * e;
+    const long long stride_l = (d.stride_layer ? d.stride_layer : (pm.table ? (long long)pm.n_pages * pm_elems.page_stride : (long long)d.B * d.Hkv * d.cap * d.D)) * e;
     const int row_bytes = d.D * (int)e;
     // Enough blocks to occupy the GPU about twice over, at most one per (head, tensor) pair.
     const long long lb = (long long)d.layers * d.B;
@@ -114,7 +140,7 @@ int launch_compact(void *kc, void *vc, const ht_cache_desc &d, const int32_t *kv
     compact_kernel<<<(unsigned)(lb * groups), kCompactThreads, 0, s>>>(
         static_cast<unsigned char *>(kc), static_cast<unsigned char *>(vc), d.layers, d.B, d.Hkv, d.cap,
         d.N, row_bytes, stride_l, stride_b, stride_h, kv_len, accept_len, accept_path, max_path, (int)groups,
-        new_kv_len, status);
+        new_kv_len, status, pm);
     return check_launch("ht_kv_compact");
 }
 

@@ -209,4 +209,70 @@ int ht_rope_kv_append(const ht_attn_desc *desc, const void *q_in, const void *k_
                        static_cast<cudaStream_t>(stream));
 }
 
+static int check_paged_desc(const ht_paged_desc *pages, int Hkv, int D) {
+    if (!pages) return fail(HT_ERR_INVALID_ARG, "NULL descriptor");
+    const int ps = pages->page_size;
+    if (ps < 16 || (ps & (ps - 1)) != 0) return fail(HT_ERR_INVALID_ARG, "page_size must be a power of two >= 16");
+    if (pages->max_pages <= 0 || pages->n_pages <= 0) return fail(HT_ERR_INVALID_ARG, "max_pages and n_pages must be positive");
+    if ((long long)pages->max_pages * ps > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "max_pages * page_size too large");
+    if (pages->page_stride < 0 || pages->head_stride < 0 || pages->page_stride % 8 != 0 || pages->head_stride % 8 != 0)
+        return fail(HT_ERR_INVALID_ARG, "page strides must be non-negative multiples of 8 elements");
+    if (pages->head_stride && pages->head_stride < (long long)ps * D)
+        return fail(HT_ERR_INVALID_ARG, "head_stride smaller than a page's rows of one head");
+    if (pages->page_stride && pages->page_stride < (long long)Hkv * ps * D)
+        return fail(HT_ERR_INVALID_ARG, "page_stride smaller than a page");
+    return HT_OK;
+}
+
+int ht_rope_kv_append_paged(const ht_attn_desc *desc, const ht_paged_desc *pages, const void *q_in, const void *k_in,
+                            const void *v_in, const int32_t *pos, const int32_t *kv_len, const int32_t *block_table,
+                            float rope_base, void *q_out, void *k_pages, void *v_pages, int32_t *status, void *stream) {
+    if (!desc) return fail(HT_ERR_INVALID_ARG, "NULL descriptor");
+    int rc = check_paged_desc(pages, desc->Hkv, desc->D);
+    if (rc != HT_OK) return rc;
+    ht_attn_desc d = *desc;
+    d.cap = pages->max_pages * pages->page_size;
+    d.kv_stride_b = 0;
+    d.kv_stride_h = 0;
+    rc = check_attn_desc(&d);
+    if (rc != HT_OK) return rc;
+    if (d.B == 0 || d.N == 0) return HT_OK;
+    if (!(rope_base > 1.f)) return fail(HT_ERR_INVALID_ARG, "rope_base must exceed 1");
+    if (!q_in || !k_in || !v_in || !pos || !kv_len || !block_table || !q_out || !k_pages || !v_pages || !status)
+        return fail(HT_ERR_INVALID_ARG, "NULL pointer");
+    if (!aligned16(q_in) || !aligned16(k_in) || !aligned16(v_in) || !aligned16(q_out) || !aligned16(k_pages) || !aligned16(v_pages))
+        return fail(HT_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    if ((long long)d.B * d.N > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "B*N too large");
+    return launch_rope(d, q_in, k_in, v_in, pos, kv_len, rope_base, q_out, k_pages, v_pages, status,
+                       static_cast<cudaStream_t>(stream), make_page_map(pages, block_table, d.Hkv, d.D));
+}
+
+int ht_kv_compact_paged(void *k_pages, void *v_pages, const ht_cache_desc *desc, const ht_paged_desc *pages,
+                        const int32_t *block_table, const int32_t *kv_len, const int32_t *accept_len,
+                        const int32_t *accept_path, int max_path, int32_t *new_kv_len, int32_t *status, void *stream) {
+    if (!desc) return fail(HT_ERR_INVALID_ARG, "desc is NULL");
+    if (desc->layers <= 0 || desc->B < 0 || desc->Hkv <= 0 || desc->D <= 0 || desc->N < 0)
+        return fail(HT_ERR_INVALID_ARG, "bad cache sizes");
+    int rc = check_paged_desc(pages, desc->Hkv, desc->D);
+    if (rc != HT_OK) return rc;
+    if (!valid_dtype(desc->dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", desc->dtype);
+    if (max_path <= 0 || max_path > 64) return fail(HT_ERR_INVALID_ARG, "max_path must be in 1..64");
+    if (desc->B == 0) return HT_OK;
+    const int row_bytes = desc->D * elem_bytes(desc->dtype);
+    if (row_bytes % 16) return fail(HT_ERR_UNSUPPORTED, "a cache row must be a multiple of 16 bytes");
+    if ((long long)max_path * (row_bytes / 16) > 4096)
+        return fail(HT_ERR_UNSUPPORTED, "max_path * row size too large for one block");
+    if (!kv_len || !accept_len || !accept_path || !new_kv_len || !status || !k_pages || !v_pages || !block_table)
+        return fail(HT_ERR_INVALID_ARG, "NULL pointer");
+    if (!aligned16(k_pages) || !aligned16(v_pages)) return fail(HT_ERR_INVALID_ARG, "pools must be 16-byte aligned");
+    const long long e = elem_bytes(desc->dtype);
+    if (desc->stride_layer < 0 || (desc->stride_layer * e) % 16) return fail(HT_ERR_INVALID_ARG, "stride_layer must be a multiple of 16 bytes");
+    if (2ll * desc->layers * desc->B * desc->Hkv > 0x7fffffffLL)
+        return fail(HT_ERR_UNSUPPORTED, "too many (layer, sequence, head) units");
+    ht_cache_desc d = *desc;
+    d.cap = pages->max_pages * pages->page_size;
+    return launch_compact(k_pages, v_pages, d, kv_len, accept_len, accept_path, max_path, new_kv_len, status,
+                          static_cast<cudaStream_t>(stream), make_page_map(pages, block_table, d.Hkv, d.D));
+}
+
 }  // extern "C"

@@ -68,6 +68,25 @@ __device__ __forceinline__ uint4 ld_nc16(const void *p) {   // streaming 16-byte
     return v;
 }
 
+// Paged cache as the row-moving kernels see it: cache row r of sequence b is row r & (page_size - 1) of page
+// table[b * max_pages + (r >> shift)].  table == nullptr: contiguous cache.  Strides in elements.
+struct PageMap {
+    const int32_t *table;
+    int shift, max_pages, n_pages;
+    long long page_stride, head_stride;
+};
+inline PageMap make_page_map(const ht_paged_desc *pg, const int32_t *table, int Hkv, int D) {
+    PageMap m{};
+    if (!pg) return m;
+    m.table = table;
+    while ((1 << m.shift) < pg->page_size) ++m.shift;
+    m.max_pages = pg->max_pages;
+    m.n_pages = pg->n_pages;
+    m.head_stride = pg->head_stride ? pg->head_stride : (long long)pg->page_size * D;
+    m.page_stride = pg->page_stride ? pg->page_stride : (long long)Hkv * pg->page_size * D;
+    return m;
+}
+
 // Entry points of the individual kernels' host launchers (defined in the .cu files).
 int launch_transfer(const void *h, const void *W, void *out, int B, int k, int d, int dtype, cudaStream_t s);
 bool transfer_tc_applicable(int B, int k, int d, int dtype);
@@ -91,9 +110,10 @@ int launch_draft(const void *logits, int dtype, int B, int rows, int V, int firs
                  const int32_t *tmpl_parent, const int32_t *tmpl_rank, int Tn, const int32_t *root_token,
                  const int32_t *base_pos, int32_t *topk, int32_t *tokens, int32_t *pos, int32_t *status, cudaStream_t s);
 int launch_rope(const ht_attn_desc &d, const void *q_in, const void *k_in, const void *v_in, const int32_t *pos,
-                const int32_t *kv_len, float base, void *q_out, void *kc, void *vc, int32_t *status, cudaStream_t s);
+                const int32_t *kv_len, float base, void *q_out, void *kc, void *vc, int32_t *status, cudaStream_t s,
+                const PageMap &pm = PageMap{});
 int launch_compact(void *kc, void *vc, const ht_cache_desc &d, const int32_t *kv_len,
                    const int32_t *accept_len, const int32_t *accept_path, int max_path,
-                   int32_t *new_kv_len, int32_t *status, cudaStream_t s);
+                   int32_t *new_kv_len, int32_t *status, cudaStream_t s, const PageMap &pm = PageMap{});
 
 }  // namespace ht

@@ -19,14 +19,24 @@ __global__ void __launch_bounds__(128)
 rope_kv_append_kernel(const T *__restrict__ q_in, const T *__restrict__ k_in, const T *__restrict__ v_in,
                       const int32_t *__restrict__ pos, const int32_t *__restrict__ kv_len, double log2_base,
                       T *__restrict__ q_out, T *__restrict__ k_cache, T *__restrict__ v_cache, int N, int Hq, int Hkv,
-                      int cap, long long stride_b, long long stride_h, int32_t *__restrict__ status) {
+                      int cap, long long stride_b, long long stride_h, int32_t *__restrict__ status, const PageMap pm) {
     constexpr int VE = Vec16<T>::n, HALF = D / 2, VPH = HALF / VE;     // 16-byte vectors per half row
     __shared__ float s_cos[HALF], s_sin[HALF];
     const int b = blockIdx.x / N, r = blockIdx.x - b * N;
     const int L = kv_len[b];
     const bool bad = L < 0 || (long long)L + N > cap;
-    if (r == 0 && threadIdx.x == 0) status[b] = bad ? HT_STATUS_BAD_LEN : HT_STATUS_OK;
+    // paged cache: the status words were zeroed ahead of the launch and any block may report a bad page
+    if (r == 0 && threadIdx.x == 0 && (bad || !pm.table)) status[b] = bad ? HT_STATUS_BAD_LEN : HT_STATUS_OK;
     if (bad) return;
+    // where cache row L + r of this sequence starts, short of the head's offset
+    long long row_off = (long long)b * stride_b + (long long)(L + r) * D;
+    bool no_page = false;
+    if (pm.table) {
+        const int page = pm.table[(size_t)b * pm.max_pages + ((L + r) >> pm.shift)];
+        no_page = (unsigned)page >= (unsigned)pm.n_pages;
+        if (no_page && threadIdx.x == 0) status[b] = HT_STATUS_BAD_PAGE;   // the row's K and V are not stored; its q is rotated
+        row_off = (long long)page * pm.page_stride + (long long)((L + r) & ((1 << pm.shift) - 1)) * D;
+    }
     const double p = (double)pos[(size_t)b * N + r];
     for (int i = threadIdx.x; i < HALF; i += blockDim.x) {
         double s, c;
@@ -45,12 +55,14 @@ rope_kv_append_kernel(const T *__restrict__ q_in, const T *__restrict__ k_in, co
         if (h < Hq) {
             src = q_in + (((size_t)b * N + r) * Hq + h) * D;
             dst = q_out + (((size_t)b * N + r) * Hq + h) * D;
+        } else if (no_page) {
+            continue;
         } else if (h < Hq + Hkv) {
             src = k_in + (((size_t)b * N + r) * Hkv + (h - Hq)) * D;
-            dst = k_cache + (size_t)b * stride_b + (size_t)(h - Hq) * stride_h + (size_t)(L + r) * D;
+            dst = k_cache + row_off + (size_t)(h - Hq) * stride_h;
         } else {
             src = v_in + (((size_t)b * N + r) * Hkv + (h - Hq - Hkv)) * D;
-            dst = v_cache + (size_t)b * stride_b + (size_t)(h - Hq - Hkv) * stride_h + (size_t)(L + r) * D;
+            dst = v_cache + row_off + (size_t)(h - Hq - Hkv) * stride_h;
             rotate = false;
         }
         const uint4 lo_raw = *reinterpret_cast<const uint4 *>(src + vx * VE);
@@ -77,15 +89,16 @@ rope_kv_append_kernel(const T *__restrict__ q_in, const T *__restrict__ k_in, co
 
 template <typename T>
 static int launch_t(const ht_attn_desc &d, const void *q_in, const void *k_in, const void *v_in, const int32_t *pos,
-                    const int32_t *kv_len, float base, void *q_out, void *kc, void *vc, int32_t *status, cudaStream_t s) {
-    const long long sh = d.kv_stride_h ? d.kv_stride_h : (long long)d.cap * d.D;
+                    const int32_t *kv_len, float base, void *q_out, void *kc, void *vc, int32_t *status, cudaStream_t s,
+                    const PageMap &pm) {
+    const long long sh = pm.table ? pm.head_stride : (d.kv_stride_h ? d.kv_stride_h : (long long)d.cap * d.D);
     const long long sb = d.kv_stride_b ? d.kv_stride_b : (long long)d.Hkv * d.cap * d.D;
     const double l2b = log2((double)base);
     const unsigned blocks = (unsigned)(d.B * d.N);
 #define HT_ROPE_LAUNCH(DD)                                                                                                   \
     rope_kv_append_kernel<T, DD><<<blocks, 128, 0, s>>>(static_cast<const T *>(q_in), static_cast<const T *>(k_in),         \
                                                         static_cast<const T *>(v_in), pos, kv_len, l2b, static_cast<T *>(q_out), \
-                                                        static_cast<T *>(kc), static_cast<T *>(vc), d.N, d.Hq, d.Hkv, d.cap, sb, sh, status)
+                                                        static_cast<T *>(kc), static_cast<T *>(vc), d.N, d.Hq, d.Hkv, d.cap, sb, sh, status, pm)
     if (d.D == 64) HT_ROPE_LAUNCH(64);
     else HT_ROPE_LAUNCH(128);
 #undef HT_ROPE_LAUNCH
@@ -93,11 +106,16 @@ static int launch_t(const ht_attn_desc &d, const void *q_in, const void *k_in, c
 }
 
 int launch_rope(const ht_attn_desc &d, const void *q_in, const void *k_in, const void *v_in, const int32_t *pos,
-                const int32_t *kv_len, float base, void *q_out, void *kc, void *vc, int32_t *status, cudaStream_t s) {
+                const int32_t *kv_len, float base, void *q_out, void *kc, void *vc, int32_t *status, cudaStream_t s,
+                const PageMap &pm) {
+    if (pm.table) {
+        const cudaError_t e = cudaMemsetAsync(status, 0, (size_t)d.B * sizeof(int32_t), s);
+        if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    }
     switch (d.dtype) {
-        case HT_F32: return launch_t<float>(d, q_in, k_in, v_in, pos, kv_len, base, q_out, kc, vc, status, s);
-        case HT_F16: return launch_t<__half>(d, q_in, k_in, v_in, pos, kv_len, base, q_out, kc, vc, status, s);
-        default: return launch_t<__nv_bfloat16>(d, q_in, k_in, v_in, pos, kv_len, base, q_out, kc, vc, status, s);
+        case HT_F32: return launch_t<float>(d, q_in, k_in, v_in, pos, kv_len, base, q_out, kc, vc, status, s, pm);
+        case HT_F16: return launch_t<__half>(d, q_in, k_in, v_in, pos, kv_len, base, q_out, kc, vc, status, s, pm);
+        default: return launch_t<__nv_bfloat16>(d, q_in, k_in, v_in, pos, kv_len, base, q_out, kc, vc, status, s, pm);
     }
 }
 

@@ -858,3 +858,134 @@ def test_rope_then_attention_equals_the_oracle_chain(hb, oracle):
     assert (np.abs(f32np(q_out) - q_ref) <= 2e-3 + 1e-2 * np.abs(q_ref)).all()
     assert (np.abs(f32np(kc) - k_ref) <= 2e-3 + 1e-2 * np.abs(k_ref)).all()
 
+
+
+# ---------------------------------------------------------------------------------------
+# Paged cache: append and compaction through the block table, and the whole round on pages
+# ---------------------------------------------------------------------------------------
+def _paged_pools(seed, dt, layers, B, Hkv, D, ps, per, spare=2):
+    """Seeded pools [layers, n_pages, Hkv, ps, D] and a shuffled block table [B, per] shared by the layers."""
+    n_pages = B * per + spare
+    pk = wl.normal_tensor(seed, 1, (layers, n_pages, Hkv, ps, D), "cuda", 1.0, dt)
+    pv = wl.normal_tensor(seed, 2, (layers, n_pages, Hkv, ps, D), "cuda", 1.0, dt)
+    table = np.random.default_rng(seed).permutation(n_pages)[:B * per].astype(np.int32).reshape(B, per)
+    return pk, pv, table
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("ps", [16, 128])
+def test_paged_rope_kv_append_matches_the_oracle(hb, dtype, ps):
+    from oracle import paged_oracle
+    dt = DT[dtype]
+    B, N, Hq, Hkv, D = 3, 21, 8, 2, 128
+    per = 512 // ps
+    pk, pv, table = _paged_pools(61, dt, 1, B, Hkv, D, ps, per)
+    pk, pv = pk[0], pv[0]
+    rng = np.random.default_rng(ps)
+    q = wl.normal_tensor(62, 1, (B, N, Hq, D), "cuda", 1.0, dt)
+    k = wl.normal_tensor(62, 2, (B, N, Hkv, D), "cuda", 1.0, dt)
+    v = wl.normal_tensor(62, 3, (B, N, Hkv, D), "cuda", 1.0, dt)
+    kv_len = np.array([5, 512 - N + 1, 300], np.int32)         # sequence 1 does not fit its table
+    pos = (kv_len[:, None] + rng.integers(0, 6, (B, N))).astype(np.int32)
+    t_bad = table.copy()
+    t_bad[2, (300 + 7) // ps] = -3                             # a page of sequence 2 outside the pool
+    view = torch.int32 if dt == torch.float32 else torch.int16
+    for tbl, want_status in ((table, [0, 2, 0]), (t_bad, [0, 2, 5])):
+        k0, v0 = pk.clone(), pv.clone()
+        q_out, status = hb.rope_kv_append_paged(q, k, v, torch.from_numpy(pos).cuda(), torch.from_numpy(kv_len).cuda(),
+                                                torch.from_numpy(tbl).cuda(), k0, v0)
+        torch.cuda.synchronize()
+        q_ref, k_ref, v_ref, st_ref = paged_oracle.rope_kv_append_paged(f32np(q), f32np(k), f32np(v), pos, kv_len, tbl,
+                                                                      f32np(pk), f32np(pv))
+        assert status.cpu().tolist() == st_ref.tolist() == want_status
+        tol = (lambda r: 1e-5) if dt == torch.float32 else (lambda r: 2e-3 + 1e-2 * np.abs(r))
+        for b in range(B):
+            if st_ref[b] != 2:
+                assert (np.abs(f32np(q_out)[b] - q_ref[b]) <= tol(q_ref[b])).all()
+        assert (np.abs(f32np(k0) - k_ref) <= tol(k_ref)).all()            # rotated K rows where the oracle put them
+        # V rows are copies, bit for bit
+        v_want = torch.from_numpy(v_ref).to(dt).cuda()
+        assert torch.equal(v0.view(view), v_want.view(view))
+        # (page, row) pairs the oracle left alone are untouched, bit for bit
+        same = (v_ref == f32np(pv)).all(axis=(1, 3))                      # [n_pages, ps]
+        assert same.sum() == same.size - sum(N for b in range(B) if st_ref[b] == 0) - \
+            (sum(1 for r in range(N) if (300 + r) // ps != (300 + 7) // ps) if st_ref[2] == 5 else 0)
+        k_dev, k_old = k0.view(view).cpu().numpy().transpose(0, 2, 1, 3), pk.view(view).cpu().numpy().transpose(0, 2, 1, 3)
+        assert np.array_equal(k_dev[same], k_old[same])
+
+
+@pytest.mark.parametrize("ps", [16, 64])
+def test_paged_compaction_matches_the_oracle(hb, ps):
+    from oracle import paged_oracle
+    dt = torch.bfloat16
+    layers, B, Hkv, D, N = 3, 4, 2, 128, 12
+    per = 128 // ps
+    pk, pv, table = _paged_pools(63, dt, layers, B, Hkv, D, ps, per)
+    kv_len = np.array([7, 0, 100, 128 - N + 1], np.int32)     # the last one does not fit
+    alen = np.array([3, 4, 2, 1], np.int32)
+    apath = np.array([[0, 2, 5, -1, -1], [0, 1, 2, 3, -1], [4, 11, -1, -1, -1], [0, -1, -1, -1, -1]], np.int32)
+    bits = lambda t: t.view(torch.int16).cpu().numpy()
+    for tbl, want in ((table, [0, 0, 0, 2]), (np.where(np.arange(per)[None, :] == (100 + 11) // ps, np.int32(10 ** 6), table), None)):
+        k0, v0 = pk.clone(), pv.clone()
+        new_len, status = hb.kv_compact_paged(k0, v0, torch.from_numpy(tbl).cuda(), N, torch.from_numpy(kv_len).cuda(),
+                                              torch.from_numpy(alen).cuda(), torch.from_numpy(apath).cuda())
+        k_ref, v_ref, len_ref, st_ref = paged_oracle.kv_compact_paged(bits(pk), bits(pv), tbl, N, kv_len, alen, apath)
+        assert status.cpu().tolist() == st_ref.tolist() and new_len.cpu().tolist() == len_ref.tolist()
+        if want is not None:
+            assert st_ref.tolist() == want
+        else:
+            assert 5 in st_ref.tolist()
+        # every logical row below the new length, bit for bit; rows of untouched pages too
+        for b in range(B):
+            for r in range(int(len_ref[b])):
+                page = tbl[b, r // ps]
+                if 0 <= page < pk.shape[1]:
+                    assert np.array_equal(bits(k0)[:, page, :, r % ps], k_ref[:, page, :, r % ps])
+                    assert np.array_equal(bits(v0)[:, page, :, r % ps], v_ref[:, page, :, r % ps])
+        used = set(int(x) for x in tbl.reshape(-1) if 0 <= x < pk.shape[1])
+        for page in range(pk.shape[1]):
+            if page not in used:
+                assert torch.equal(k0[:, page], pk[:, page])
+
+
+def test_a_round_on_pages_equals_the_round_on_a_contiguous_cache(hb):
+    """append -> attention -> (acceptance given) -> compaction, on pages and on the contiguous layout holding the same
+    data: identical outputs, and identical cache contents below the new lengths."""
+    from oracle import paged_oracle
+    dt = torch.bfloat16
+    B, N, Hq, Hkv, D, ps = 2, 40, 16, 4, 128, 32
+    per = 640 // ps
+    cap = per * ps
+    rng = np.random.default_rng(17)
+    kc = wl.normal_tensor(71, 1, (1, B, Hkv, cap, D), "cuda", 1.0, dt)
+    vc = wl.normal_tensor(71, 2, (1, B, Hkv, cap, D), "cuda", 1.0, dt)
+    pool_k, table = paged_oracle.scatter_to_pages(f32np(kc[0]), ps, 72)
+    pool_v, _ = paged_oracle.scatter_to_pages(f32np(vc[0]), ps, 72)
+    pk = torch.from_numpy(pool_k).to(dt).cuda()[None].contiguous()
+    pv = torch.from_numpy(pool_v).to(dt).cuda()[None].contiguous()
+    tbl = torch.from_numpy(table).cuda()
+    q = wl.normal_tensor(71, 3, (B, N, Hq, D), "cuda", 1.0, dt)
+    k = wl.normal_tensor(71, 4, (B, N, Hkv, D), "cuda", 1.0, dt)
+    v = wl.normal_tensor(71, 5, (B, N, Hkv, D), "cuda", 1.0, dt)
+    parent = torch.from_numpy(np.stack([rand_tree(rng, N, "random") for _ in range(B)])).cuda()
+    kv_len = torch.tensor([500, 77], dtype=torch.int32, device="cuda")
+    pos = (kv_len[:, None] + torch.arange(N, device="cuda", dtype=torch.int32)[None] % 5).to(torch.int32).contiguous()
+    alen = torch.tensor([3, 2], dtype=torch.int32, device="cuda")
+    apath = torch.tensor([[0, 7, 30, -1], [5, 6, -1, -1]], dtype=torch.int32, device="cuda")
+
+    q1, s1 = hb.rope_kv_append(q, k, v, pos, kv_len, kc[0], vc[0])
+    o1, s2 = hb.tree_attention(q1, kc[0], vc[0], kv_len, parent)
+    n1, s3 = hb.kv_compact(kc, vc, N, kv_len, alen, apath)
+    q2, t1 = hb.rope_kv_append_paged(q, k, v, pos, kv_len, tbl, pk[0], pv[0])
+    o2, t2 = hb.tree_attention_paged(q2, pk[0], pv[0], tbl, kv_len, parent)
+    n2, t3 = hb.kv_compact_paged(pk, pv, tbl, N, kv_len, alen, apath)
+    torch.cuda.synchronize()
+    for st in (s1, s2, s3, t1, t2, t3):
+        assert st.cpu().tolist() == [0, 0]
+    assert torch.equal(q1, q2) and torch.equal(n1, n2)
+    assert_close(f32np(o2), f32np(o1), dt, "attention on pages against contiguous")
+    for b in range(B):
+        for r in range(int(n1[b])):
+            page = int(table[b, r // ps])
+            assert torch.equal(pk[0, page, :, r % ps], kc[0, b, :, r])
+            assert torch.equal(pv[0, page, :, r % ps], vc[0, b, :, r])
