@@ -505,6 +505,35 @@ def test_paged_attention_against_the_oracle(hb, oracle, dtype, case):
         assert_close(f32np(out), oracle_attn(oracle, q, k, v, kv_len, parent), dt, "paged attention")
 
 
+def test_paged_attention_random_shapes_against_the_contiguous_entry_point(hb):
+    """Thirty seeded random shapes (batch, rows, head grouping, ragged lengths, tree kinds, page sizes from 16 to 512)
+    through the paged entry point, against the contiguous entry point on the same data (whose kernels the tests above
+    hold to the oracle): the two run the same tiles in the same order, so they agree to the rounding of the output."""
+    rng = np.random.default_rng(4048)
+    for trial in range(30):
+        g = int(rng.choice([1, 1, 2, 4, 8, 16]))
+        Hkv = int(rng.choice([1, 2, 4, 8, 32]))
+        B = int(rng.choice([1, 1, 2, 3, 5, 12]))
+        N = int(rng.choice([1, 7, 19, 33, 64, 91, 130, 200]))
+        if N * g > 1100 or B * Hkv * g * N > 120000:
+            N = max(1, 1100 // g // 4)
+        lens = [int(x) for x in rng.choice([0, 1, 60, 127, 128, 300, 1000, 2500], size=B)]
+        ps = int(rng.choice([16, 32, 64, 128, 256, 512]))
+        dtype = "bf16" if trial % 2 else "f16"
+        tree = str(rng.choice(["random", "chain", "roots"]))
+        q, pk, pv, table, kv_len, parent, k, v = make_paged_case(500 + trial, dtype, B, N, Hkv * g, Hkv, lens, ps, tree,
+                                                                extra_pages=int(rng.integers(0, 3)))
+        out, status = hb.tree_attention_paged(q, pk, pv, table, kv_len, parent)
+        ref, _ = hb.tree_attention(q, k, v, kv_len, parent)
+        torch.cuda.synchronize()
+        what = "trial %d: B=%d N=%d Hq=%d Hkv=%d lens=%s %s %s pages of %d" % (trial, B, N, Hkv * g, Hkv, lens, tree, dtype, ps)
+        assert status.cpu().tolist() == [0] * B, what
+        a, r = out.float(), ref.float()
+        eps = 2.0 ** -7 if dtype == "bf16" else 2.0 ** -10
+        assert torch.isfinite(a).all(), what
+        assert bool(((a - r).abs() <= 1e-3 + 2 * eps * r.abs()).all()), what + ": max diff %.3e" % float((a - r).abs().max())
+
+
 def test_paged_attention_reports_bad_pages_and_lengths(hb):
     from oracle import paged_oracle
     B, N, Hq, Hkv, lens, ps = 3, 19, 8, 8, [100, 200, 300], 32
