@@ -61,17 +61,17 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, v
 // steps stream faster than many small ones.  That view only has whole chunks; what is left after the
 // last whole step goes chunk by chunk through plain [row][feature] maps, whose box may end past d and
 // is zero-filled there.  With kc = 1 (large tiles: the ring needs its depth more) every step is such a one.
-template <bool kBf16>
+template <bool kBf16, int kMT>           // kMT = p.mt: 128-row tiles of h per CTA
 __global__ void __launch_bounds__(kTThreads, 1)
 transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_h_tail, const __grid_constant__ CUtensorMap tm_w_tail, const TParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *base = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    TBars &bar = *reinterpret_cast<TBars *>(base + (size_t)p.stages * p.stage_bytes + (kBM * p.mt - p.h_rows) * kBK * 2);
+    TBars &bar = *reinterpret_cast<TBars *>(base + (size_t)p.stages * p.stage_bytes + (kBM * kMT - p.h_rows) * kBK * 2);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &bar.abort;
-    const int m0 = ((int)blockIdx.x % p.n_m) * kBM * p.mt, n0 = ((int)blockIdx.x / p.n_m) * p.bn;
-    const uint32_t acc_cols = kAccCols * (uint32_t)p.mt;
+    const int m0 = ((int)blockIdx.x % p.n_m) * kBM * kMT, n0 = ((int)blockIdx.x / p.n_m) * p.bn;
+    constexpr uint32_t acc_cols = kAccCols * (uint32_t)kMT;
     const int n_main = p.kc > 1 ? (p.d / kBK) / p.kc : 0;             // steps of kc whole chunks through the chunked view
     const int f_rest = n_main * p.kc * kBK;                           // first feature after them
     const int nk = n_main + (p.d - f_rest + kBK - 1) / kBK;           // + single chunks (the last one may be ragged)
@@ -93,7 +93,7 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         }
     }
     if (warp == 4) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bar.tmem_base)), "r"(acc_cols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bar.tmem_base)), "r"((uint32_t)acc_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -104,9 +104,9 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     if (warp == 4) {
         // ------------------------------- TMA producer -------------------------------
         if (lane == 0) {
-            int issued = 0;
-            for (int ks = 0; ks < nk && !*abort_flag; ++ks) {
-                const int slot = ks % p.stages, use = ks / p.stages;
+            int issued = 0, slot = 0, use = 0;         // slot and round of the ring, kept by counting (no division per step)
+            for (int ks = 0; ks < nk; ++ks, ++slot) {
+                if (slot == p.stages) { slot = 0; ++use; }
                 if (use > 0 && !mbar_wait(&bar.empty[slot], (use - 1) & 1, abort_flag)) break;
                 unsigned char *a = base + (size_t)slot * p.stage_bytes;
                 if (ks < n_main) {
@@ -130,20 +130,27 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         // ------------------------------- MMA issuer -------------------------------
         if (lane == 0) {
             const uint32_t idesc = instr_desc(kBf16, 0, (uint32_t)p.bn);
+            const uint64_t a_desc0 = smem_desc(smem_u32(base), 1, 1024 >> 4), b_desc0 = a_desc0;
+            const uint32_t stage16 = p.stage_bytes >> 4, h16 = chunk_h >> 4, w16 = chunk_w >> 4;
+            const bool second = kMT > 1 && m0 + kBM < p.B;
             bool all = true;
-            for (int ks = 0; ks < nk; ++ks) {
-                const int slot = ks % p.stages, use = ks / p.stages;
+            int slot = 0, use = 0;
+            for (int ks = 0; ks < nk; ++ks, ++slot) {
+                if (slot == p.stages) { slot = 0; ++use; }
                 if (!mbar_wait(&bar.full[slot], use & 1, abort_flag)) { all = false; break; }
                 tc_fence_after();
-                const uint32_t a_addr = smem_u32(base + (size_t)slot * p.stage_bytes), b_addr = a_addr + chunk_h * p.kc;
+                // The descriptors differ in their address field only (16-byte units in the low bits, never
+                // carrying out of it inside this CTA's shared memory): one template each, then additions.
+                const uint32_t a16 = (uint32_t)slot * stage16, b16 = a16 + h16 * p.kc;
                 const int chunks = ks < n_main ? p.kc : 1;
                 for (int c = 0; c < chunks; ++c) {
-                    for (int i = 0; i < p.mt; ++i) {           // a second 128-row tile of h, if it has rows at all
-                        if (i > 0 && m0 + i * kBM >= p.B) break;
+#pragma unroll
+                    for (int i = 0; i < kMT; ++i) {            // a second 128-row tile of h, if it has rows at all
+                        if (i > 0 && !second) break;
 #pragma unroll
                         for (int kk = 0; kk < kBK / 16; ++kk)  // 16 features = 32 bytes inside the swizzled line
-                            mma_ss(tmem + i * kAccCols, smem_desc(a_addr + c * chunk_h + i * kHBytes + kk * 32, 1, 1024 >> 4),
-                                   smem_desc(b_addr + c * chunk_w + kk * 32, 1, 1024 >> 4), idesc, (ks | c | kk) != 0 ? 1u : 0u);
+                            mma_ss(tmem + i * kAccCols, a_desc0 + (a16 + c * h16 + i * (kHBytes >> 4) + kk * 2),
+                                   b_desc0 + (b16 + c * w16 + kk * 2), idesc, (ks | c | kk) != 0 ? 1u : 0u);
                     }
                 }
                 tc_commit(&bar.empty[slot]);
@@ -159,7 +166,8 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         const bool ok = __all_sync(0xFFFFFFFFu, waited);
         tc_fence_after();
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        for (int i = 0; i < p.mt; ++i) {
+#pragma unroll
+        for (int i = 0; i < kMT; ++i) {
             const int row = m0 + i * kBM + (int)threadIdx.x;   // TMEM lane = source row of the tile
             if (m0 + i * kBM >= p.B) break;
             unsigned char *dst_row = static_cast<unsigned char *>(p.out) + ((size_t)min(row, p.B - 1) * p.R + n0) * 2;
@@ -191,7 +199,7 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
     __syncthreads();
     if (warp == 4) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(acc_cols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)acc_cols) : "memory");
     }
 }
 
@@ -323,24 +331,23 @@ int launch_transfer_tc(const void *h, const void *W, void *out, int B, int k, in
         tm_w = tm_w_tail;
     }
 
+    typedef void (*Fn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const ttc::TParams);
+    const Fn fns[4] = {ttc::transfer_tc_kernel<false, 1>, ttc::transfer_tc_kernel<true, 1>, ttc::transfer_tc_kernel<false, 2>,
+                       ttc::transfer_tc_kernel<true, 2>};
     static bool attr_done[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
     if (!(dev >= 0 && dev < 64 && attr_done[dev])) {
-        e = cudaFuncSetAttribute(ttc::transfer_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(ttc::transfer_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        for (int i = 0; i < 4 && e == cudaSuccess; ++i)
+            e = cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         if (dev >= 0 && dev < 64) attr_done[dev] = true;
     }
     const long long n_n = (R + p.bn - 1) / p.bn;
     const long long grid = n_n * p.n_m;
     if (grid > 0x7FFFFFFFll) return fail(HT_ERR_INVALID_ARG, "ht_transfer: too many tiles");
-    if (dtype == HT_BF16)
-        ttc::transfer_tc_kernel<true><<<(unsigned)grid, ttc::kTThreads, smem, s>>>(tm_h, tm_w, tm_h_tail, tm_w_tail, p);
-    else
-        ttc::transfer_tc_kernel<false><<<(unsigned)grid, ttc::kTThreads, smem, s>>>(tm_h, tm_w, tm_h_tail, tm_w_tail, p);
+    fns[(dtype == HT_BF16 ? 1 : 0) + (p.mt == 2 ? 2 : 0)]<<<(unsigned)grid, ttc::kTThreads, smem, s>>>(tm_h, tm_w, tm_h_tail, tm_w_tail, p);
     return check_launch("ht_transfer");
 }
 
