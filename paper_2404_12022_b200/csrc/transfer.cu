@@ -270,15 +270,17 @@ static int launch_typed16(const void *h, const void *W, void *out, int B, int k,
     return HT_OK;
 }
 
-// Which kernel takes a 16-bit call: up to 16 source rows the warp-level instruction on the words as
-// loaded, above that the tcgen05 kernel (one pass over W for any number of rows).  HT_TRANSFER_KERNEL =
+// Which kernel takes a 16-bit call: few source rows the warp-level instruction on the words as
+// loaded, more the tcgen05 kernel (one pass over W for any number of rows).  HT_TRANSFER_KERNEL =
 // "tc" or "mma" in the environment overrides the choice, for cross-checks of one against the other.
 static bool use_tc(int B, int k, int d, int dtype) {
     if (!transfer_tc_applicable(B, k, d, dtype)) return false;
     const char *e = getenv("HT_TRANSFER_KERNEL");
     if (e && !strcmp(e, "tc")) return true;
     if (e && !strcmp(e, "mma")) return false;
-    return B > 16;
+    // 9 to 16 rows take the warp-level kernel's two-tile form (24.5 us on config 3's W against 19.3 with up to 8
+    // rows); the tcgen05 kernel is ahead of that once W is large enough to amortise its set-up (21.6 us there).
+    return B > 16 || (B > 8 && (long long)k * d * d * 2 >= (64ll << 20));
 }
 
 int launch_transfer(const void *h, const void *W, void *out, int B, int k, int d, int dtype,
