@@ -71,6 +71,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    // Launched with programmatic stream serialization (the cluster launches are: nothing but kernels precedes them in
+    // the stream), the CTA has set itself up while the kernel before it was still finishing; everything that kernel
+    // may have written is read from here on.  Without that launch attribute both instructions do nothing.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0, kPaged);
     tc_fence_before();
     __syncthreads();
@@ -769,13 +774,15 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
         cfg.blockDim = dim3(tc::kThreads);
         cfg.dynamicSmemBytes = smem;
         cfg.stream = s;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = (unsigned)k;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = 2;
         e = cudaLaunchKernelEx(&cfg, attn_tc_fn(d.dtype == HT_BF16, pages != nullptr), tm_q, tm_k, tm_v, p, pp);
         if (e != cudaSuccess) {
             cudaGetLastError();
