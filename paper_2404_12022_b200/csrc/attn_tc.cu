@@ -71,9 +71,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // Launched with programmatic stream serialization (the cluster launches are: nothing but kernels precedes them in
-    // the stream), the CTA has set itself up while the kernel before it was still finishing; everything that kernel
-    // may have written is read from here on.  Without that launch attribute both instructions do nothing.
+    // The launch is serialized programmatically behind the kernel before it in the stream: the CTA has set itself
+    // up while that kernel was still finishing, and everything it may have written is read from here on.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0, kPaged);
@@ -577,6 +576,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
 }
 
+// What must be zero when the attention kernel starts: the units' arrival counters (and, for a paged cache, the
+// status words).  A kernel rather than a memset node so that the launches can be chained by programmatic stream
+// serialization: this one is in place, waiting, before the previous kernel of the stream has finished, and the
+// attention kernel behind it has its CTAs set up by the time this one is done.
+__global__ void attn_prepare_kernel(unsigned int *tickets, int n_tickets, int32_t *status, int n_status) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int stride = gridDim.x * blockDim.x, first = blockIdx.x * blockDim.x + threadIdx.x;
+    for (int i = first; i < n_tickets; i += stride) tickets[i] = 0u;
+    for (int i = first; i < n_status; i += stride) status[i] = 0;
+}
+
 }  // namespace tc
 
 // ---------------------------------------------------------------------------------------
@@ -756,9 +767,24 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     if (units > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "too many (sequence, head, row tile) units");
     const int k = cluster_size(d);
     cudaError_t e = cudaSuccess;
-    if (k <= 1) e = cudaMemsetAsync(p.tickets, 0, (size_t)units * sizeof(unsigned int), s);   // clusters use no tickets
-    if (e == cudaSuccess && pages) e = cudaMemsetAsync(status, 0, (size_t)d.B * sizeof(int32_t), s);
-    if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    if (k <= 1 || pages) {                        // clusters use no tickets; the paged kernels report bad pages from any CTA
+        const int n_t = k <= 1 ? (int)units : 0, n_s = pages ? d.B : 0;
+        const int n = n_t > n_s ? n_t : n_s;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)((n + 255) / 256 < 64 ? (n + 255) / 256 : 64));
+        cfg.blockDim = dim3(256);
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, tc::attn_prepare_kernel, p.tickets, n_t, status, n_s);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(HT_ERR_CUDA, "ht_tree_attention (preparation): %s", cudaGetErrorString(e));
+        }
+    }
     if (k > 1) {
         p.cluster_k = k;
         p.grid = (int)units * k;
@@ -767,31 +793,28 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     e = ensure_smem_attr(smem);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     // Few (sequence, KV head) units: one cluster of 8, 4 or 2 CTAs per unit, parts reduced through
-    // distributed shared memory; otherwise one persistent CTA per SM.
-    if (k > 1) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)p.grid);
-        cfg.blockDim = dim3(tc::kThreads);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = s;
-        cudaLaunchAttribute attr[2];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = (unsigned)k;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 2;
-        e = cudaLaunchKernelEx(&cfg, attn_tc_fn(d.dtype == HT_BF16, pages != nullptr), tm_q, tm_k, tm_v, p, pp);
-        if (e != cudaSuccess) {
-            cudaGetLastError();
-            return fail(HT_ERR_CUDA, "ht_tree_attention (tcgen05, clusters of %d): %s", k, cudaGetErrorString(e));
-        }
-        return HT_OK;
+    // distributed shared memory; otherwise one persistent CTA per SM.  Either way the launch is serialized
+    // programmatically behind the kernel before it.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.grid);
+    cfg.blockDim = dim3(tc::kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)(k > 1 ? k : 1);
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = k > 1 ? 2 : 1;
+    e = cudaLaunchKernelEx(&cfg, attn_tc_fn(d.dtype == HT_BF16, pages != nullptr), tm_q, tm_k, tm_v, p, pp);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(HT_ERR_CUDA, "ht_tree_attention (tcgen05, clusters of %d): %s", k > 1 ? k : 1, cudaGetErrorString(e));
     }
-    attn_tc_fn(d.dtype == HT_BF16, pages != nullptr)<<<p.grid, tc::kThreads, smem, s>>>(tm_q, tm_k, tm_v, p, pp);
-    return check_launch("ht_tree_attention (tcgen05)");
+    return HT_OK;
 }
 
 }  // namespace ht

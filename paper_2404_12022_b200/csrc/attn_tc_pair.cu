@@ -75,9 +75,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // Launched with programmatic stream serialization (the cluster launches are: nothing but kernels precedes them in
-    // the stream), the CTA has set itself up while the kernel before it was still finishing; everything that kernel
-    // may have written is read from here on.  Without that launch attribute both instructions do nothing.
+    // The launch is serialized programmatically behind the kernel before it in the stream: the CTA has set itself
+    // up while that kernel was still finishing, and everything it may have written is read from here on.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0, kPaged);
@@ -601,30 +600,27 @@ int launch_attn_tc_pair_kernel(const CUtensorMap &tm_q, const CUtensorMap &tm_k,
         if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         if (dev >= 0 && dev < 64) done[dev] = true;
     }
-    if (p.cluster_k > 1) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)p.grid);
-        cfg.blockDim = dim3(tc::kPThreads);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = s;
-        cudaLaunchAttribute attr[2];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = (unsigned)p.cluster_k;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 2;
-        e = cudaLaunchKernelEx(&cfg, fn, tm_q, tm_k, tm_v, p, pp);
-        if (e != cudaSuccess) {
-            cudaGetLastError();
-            return fail(HT_ERR_CUDA, "ht_tree_attention (tcgen05, tile pairs, clusters of %d): %s", p.cluster_k, cudaGetErrorString(e));
-        }
-        return HT_OK;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.grid);
+    cfg.blockDim = dim3(tc::kPThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // see launch_attn_tc
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)(p.cluster_k > 1 ? p.cluster_k : 1);
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p.cluster_k > 1 ? 2 : 1;
+    e = cudaLaunchKernelEx(&cfg, fn, tm_q, tm_k, tm_v, p, pp);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(HT_ERR_CUDA, "ht_tree_attention (tcgen05, tile pairs, clusters of %d): %s", p.cluster_k > 1 ? p.cluster_k : 1,
+                    cudaGetErrorString(e));
     }
-    fn<<<p.grid, tc::kPThreads, smem, s>>>(tm_q, tm_k, tm_v, p, pp);
-    return check_launch("ht_tree_attention (tcgen05, tile pairs)");
+    return HT_OK;
 }
 
 }  // namespace ht
