@@ -318,8 +318,7 @@ def run_native(args):
             "launch": "eager C-ABI calls" if args.eager else "CUDA graph of the step's C-ABI calls"}
     # launches of this library's kernels per step: one per attention call, transfer (one per batch
     # slice of 16), verification (argmax and acceptance in one), compaction
-    attn_launches = sum(1 for _ in range(step.layers))
-    line["gpu_launches"] = args.steps * (attn_launches * kernels_per_attention(step) + ((w.B + 15) // 16) + 1 + 1)
+    line["gpu_launches"] = args.steps * (sum(kernels_per_attention(step, i) for i in range(step.layers)) + ((w.B + 15) // 16) + 1 + 1)
 
     if rank == 0 and not args.no_extras:
         line["roofline"], line["kernels"] = per_kernel_pass(args, step, stream, torch)
@@ -336,8 +335,10 @@ def run_native(args):
         print(json.dumps(line), flush=True)
 
 
-def kernels_per_attention(step):
-    return 1      # one kernel per call (the ticket memset before it is not a kernel)
+def kernels_per_attention(step, i):
+    """Kernels layer i's attention call enqueues (the attention kernel, and with it the one that zeroes its tickets)."""
+    from paper_2404_12022_b200 import binding as hb
+    return hb.tree_attention_launches(step.descs[i])
 
 
 def per_kernel_pass(args, step, stream, torch):

@@ -128,6 +128,10 @@ int ht_transfer(const void *h_src, const void *W, void *out, int B, int k, int d
  * Supported: D in {64, 128}; N <= 1024.  B == 0 or N == 0 is a no-op.
  */
 size_t ht_tree_attention_workspace(const ht_attn_desc *desc /* host */);
+/* Number of this library's kernels that one ht_tree_attention call with this descriptor enqueues (1 or 2:
+ * a kernel that zeroes arrival counters, or one that merges split partials, may accompany the attention
+ * kernel); 0 for a descriptor the call would reject or that has nothing to do. */
+int ht_tree_attention_launches(const ht_attn_desc *desc /* host */);
 int ht_tree_attention(const ht_attn_desc *desc /* host */, const void *q, const void *k_cache,
                       const void *v_cache, const int32_t *kv_len, const int32_t *parent, void *out,
                       void *workspace, size_t workspace_bytes, int32_t *status, void *stream);

@@ -24,7 +24,7 @@ HT_ATTN_FORCE_SIMT = 1
 
 EXPORTS = ("ht_version", "ht_last_error_string", "ht_transfer", "ht_tree_attention_workspace",
            "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact", "ht_draft_tree", "ht_rope_kv_append", "ht_tree_attention_static",
-           "ht_tree_attention_paged", "ht_rope_kv_append_paged", "ht_kv_compact_paged")
+           "ht_tree_attention_paged", "ht_rope_kv_append_paged", "ht_kv_compact_paged", "ht_tree_attention_launches")
 HT_STATIC_SCRATCH_BYTES = 16 << 20
 
 _DTYPES = {torch.float32: HT_F32, torch.float16: HT_F16, torch.bfloat16: HT_BF16}
@@ -75,6 +75,8 @@ def load() -> ctypes.CDLL:
         lib.ht_transfer.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
         lib.ht_tree_attention_workspace.restype = sz
         lib.ht_tree_attention_workspace.argtypes = [ctypes.POINTER(AttnDesc)]
+        lib.ht_tree_attention_launches.restype = i32
+        lib.ht_tree_attention_launches.argtypes = [ctypes.POINTER(AttnDesc)]
         lib.ht_tree_attention.restype = i32
         lib.ht_tree_attention.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         lib.ht_tree_attention_static.restype = i32
@@ -146,6 +148,11 @@ def make_attn_desc(q: torch.Tensor, k_cache: torch.Tensor, scale: float = 0.0, n
         raise ValueError("cache rows must be contiguous and D apart")
     return AttnDesc(B, N, Hq, Hkv, D, cap, _DTYPES[q.dtype], float(scale), k_cache.stride(0),
                     k_cache.stride(1), num_splits, flags)
+
+
+def tree_attention_launches(desc: AttnDesc) -> int:
+    """Kernels of this library that one ``tree_attention`` call with this descriptor enqueues."""
+    return int(load().ht_tree_attention_launches(ctypes.byref(desc)))
 
 
 def tree_attention_workspace(desc: AttnDesc) -> int:

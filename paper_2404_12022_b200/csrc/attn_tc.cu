@@ -669,6 +669,9 @@ static AttnKernelFn attn_tc_fn(bool bf16, bool paged) {
                 : (paged ? tc::attn_tc_kernel<false, true> : tc::attn_tc_kernel<false, false>);
 }
 
+// Kernels per call: the attention kernel, and ahead of it the one that zeroes the tickets unless clusters are used.
+int attn_tc_launches(const ht_attn_desc &d) { return cluster_size(d) > 1 ? 1 : 2; }
+
 // The kernels' dynamic shared memory limit is raised once per device.
 static cudaError_t ensure_smem_attr(size_t smem) {
     static bool done[64];

@@ -77,6 +77,15 @@ size_t ht_tree_attention_workspace(const ht_attn_desc *desc) {
     return (need + 255) / 256 * 256;
 }
 
+int ht_tree_attention_launches(const ht_attn_desc *desc) {
+    if (check_attn_desc(desc) != HT_OK) return 0;
+    if (desc->B == 0 || desc->N == 0) return 0;
+    if (attn_tc_applicable(*desc)) return attn_tc_launches(*desc);
+    int splits = 1;
+    attn_simt_workspace(*desc, &splits);
+    return splits > 1 ? 2 : 1;
+}
+
 int ht_tree_attention(const ht_attn_desc *desc, const void *q, const void *k_cache, const void *v_cache,
                       const int32_t *kv_len, const int32_t *parent, void *out, void *workspace,
                       size_t workspace_bytes, int32_t *status, void *stream) {

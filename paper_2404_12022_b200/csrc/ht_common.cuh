@@ -98,6 +98,7 @@ int launch_attn_simt(const ht_attn_desc &d, const void *q, const void *kc, const
                      int32_t *status, cudaStream_t s);
 bool attn_tc_applicable(const ht_attn_desc &d);
 size_t attn_tc_workspace(const ht_attn_desc &d);
+int attn_tc_launches(const ht_attn_desc &d);      // kernels one call enqueues (contiguous cache)
 // `pages` / `block_table` null: contiguous cache (kc, vc as in ht_tree_attention); else the page pools.
 int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const void *vc, const int32_t *kv_len,
                    const int32_t *parent, void *out, void *ws, size_t ws_bytes, int32_t *status, cudaStream_t s,
