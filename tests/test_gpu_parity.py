@@ -205,6 +205,34 @@ def test_attention_random_shapes_tensor_core_kernels_against_the_alu_kernel(hb, 
         check_sampled_units(hb, oracle, q, k, v, kv_len.cpu().numpy(), parent, out, 1, DT[dtype], seed=trial, p_rounding=True)
 
 
+@pytest.mark.parametrize("shape", [(4, 91, 32, 32, 1500), (1, 91, 32, 32, 1024), (2, 40, 32, 4, 700), (3, 19, 16, 16, 3000)],
+                         ids=lambda s: "B%dN%dHq%dHkv%dL%d" % s)
+def test_attention_calls_in_a_row_see_each_others_results(hb, shape):
+    """The launches of consecutive calls overlap at their edges (a call's CTAs set themselves up while the call before
+    it finishes).  Six calls, each taking the previous call's output as its queries and sharing one workspace, must give
+    what the same calls give with the device drained between them."""
+    B, N, Hq, Hkv, L = shape
+    q0, k, v, kv_len, parent = make_attn_case(91, "bf16", B, N, Hq, Hkv, 128, [L - 13 * b for b in range(B)], L + N, garbage=False)
+    desc = hb.make_attn_desc(q0, k)
+    ws = torch.empty(max(hb.tree_attention_workspace(desc), 16), dtype=torch.uint8, device="cuda")
+
+    def chain(drain):
+        q = q0
+        for _ in range(6):
+            out, status = hb.tree_attention(q, k, v, kv_len, parent, workspace=ws)
+            if drain:
+                torch.cuda.synchronize()
+            q = out
+        torch.cuda.synchronize()
+        assert status.cpu().tolist() == [0] * B
+        return q
+
+    a, b = chain(True), chain(False)
+    # the work split may merge parts in another order from call to call: last place or the one next to it
+    ulp = 2.0 ** -7
+    assert bool(((a.float() - b.float()).abs() <= ulp * a.float().abs() + 1e-6).all())
+
+
 @pytest.mark.parametrize("shape", [(3, 9, 4, 2), (3, 40, 32, 8), (40, 9, 8, 4)], ids=lambda s: "B%dN%dHq%dHkv%d" % s)
 def test_attention_tensor_core_paths_skip_bad_sequences(hb, oracle, shape):
     """Status words and untouched rows on the 16-bit kernels (clusters, tile pairs, persistent)."""
