@@ -343,8 +343,9 @@ def kernels_per_attention(step, i):
 
 def per_kernel_pass(args, step, stream, torch):
     """Same steps again with CUDA events on the launching stream: one pair around every run of
-    consecutive attention calls (an event between two launches would add its own gap to each of them),
-    one pair around each of the other calls."""
+    consecutive attention calls (an event between two launches would add its own gap to each of them, and
+    would break the chain in which a call is set up while the one before it finishes), one pair around
+    each of the other calls."""
     n = min(args.steps, 10)
     names = ["attention", "transfer", "verify", "compact"]
     ev = {k: [] for k in names}
@@ -355,12 +356,29 @@ def per_kernel_pass(args, step, stream, torch):
     def timed(name, fn):
         a, b = pair(); a.record(); fn(); b.record(); ev[name].append((a, b))
 
+    # In the launch mode of the timed steps: a run of attention calls is replayed from a CUDA graph of its own (or,
+    # with --eager, enqueued call by call).
+    run_graphs = {}
+
     def attention_run(lo, hi):
-        if hi > lo:
-            a, b = pair(); a.record()
+        if hi <= lo:
+            return
+        if not args.eager and (lo, hi) not in run_graphs:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side), torch.cuda.graph(g, stream=side):
+                for i in range(lo, hi):
+                    step.attention(i, side.cuda_stream)
+            torch.cuda.current_stream().wait_stream(side)
+            run_graphs[(lo, hi)] = g
+        a, b = pair(); a.record()
+        if args.eager:
             for i in range(lo, hi):
                 step.attention(i, stream)
-            b.record(); ev["attention"].append((a, b, list(range(lo, hi))))
+        else:
+            run_graphs[(lo, hi)].replay()
+        b.record(); ev["attention"].append((a, b, list(range(lo, hi))))
 
     cut = min(step.transfer_at, step.layers)
     for _ in range(n):
