@@ -331,11 +331,16 @@ struct TileCursor {
 __device__ __forceinline__ int tiles_per_cta(int total, int grid) { return (total + grid - 1) / grid; }
 
 // Tiles per CTA.  An even share cuts nearly every unit in two, and every cut costs a partial
-// result in the workspace and a merge at the end.  While the cache is streamed at memory speed a
-// few idle SMs cost less than that, so when all sequences are equally long and some whole
-// multiple or whole fraction of a unit lies within 20 % (or six tiles) above the even share, ranges
-// of that length are used and cuts fall on unit boundaries (or, for fractions, near them).
-__device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nkt, int B) {
+// result in the workspace and a merge at the end: about as much as half a dozen tiles, whatever the
+// unit's length.  So when all sequences are equally long and some whole multiple or whole fraction of a
+// unit lies at most eight tiles above the even share, ranges of that length are used and cuts fall on unit
+// boundaries (config 3: 33 tiles against 29, one unit per CTA on 128 of the SMs); beyond that the idle SMs
+// cost more than the cuts (16 sequences of 32768 keys, one unit each: 257 tiles against 223, 566 -> 509 us
+// with the even share).  Where several units share a KV head (n_rt > 1: row-tile pairs of grouped-query
+// attention) aligned ranges also keep the CTAs of a head in step, so that its tiles cross DRAM once and
+// reach the other CTAs from L2; there alignment is kept up to 5 % above the even share (4 x 32768 keys,
+// 259 rows: 1.31 ms aligned, 1.42 ms even).
+__device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nkt, int B, int n_rt) {
     const int even = tiles_per_cta(total, grid);
     int n = 0;
     for (int b = 0; b < B; ++b) {
@@ -351,8 +356,7 @@ __device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nk
     } else {
         cand = (even + n - 1) / n * n;                // whole units
     }
-    // a cut costs about as much as half a dozen tiles (partial result, ticket, merge), whatever the size
-    return (cand * 5 <= even * 6 || cand - even <= 6) ? cand : even;
+    return (cand - even <= 8 || (n_rt > 1 && cand * 20 <= even * 21)) ? cand : even;
 }
 
 // Validates every sequence and fills len / nkt / pre.  Called by all threads of a block.

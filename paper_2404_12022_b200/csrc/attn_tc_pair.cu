@@ -86,7 +86,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t tmem = sm.tmem_base;
 
     const int total = sm.pre[p.B];
-    const int per = choose_per(total, p.grid, sm.nkt, p.B);
+    const int per = choose_per(total, p.grid, sm.nkt, p.B, p.n_rt);
     int t_begin = min((int)blockIdx.x * per, total);
     int t_end = min(t_begin + per, total);
     const bool clustered = p.cluster_k > 1;
