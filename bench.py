@@ -221,9 +221,9 @@ class ClockSampler:
 # DRAM traffic per launch of the attention kernel on a c3 layer, from the ncu capture summarised in
 # profiles/attn_tc_kernel_c3_layer.md (dram__bytes_read.sum + dram__bytes_write.sum).  It is only
 # reported while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.6e6,
+NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.8e6,
                "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh"],
-               "sha256": "9a8f37b95303e5cc359227b507ad45f5248f88c610d79a34c940665b37668645"}
+               "sha256": "80c74cb993cd1e5216847cfbc44bf24367ea31a582dbdaa08546c8a42cc06fda"}
 
 
 def ncu_traffic(w):
