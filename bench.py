@@ -412,7 +412,11 @@ def e2e_pass(args, step, inp, torch, world):
     """The same step with its per-step inputs arriving from pinned host memory and its results
     read back: q of every layer, the new K/V rows of the tree, logits, tree structure and the
     source hidden state go host -> device; attention outputs, pseudo hidden states and the
-    acceptance results come back.  The KV cache and the transfer weights are resident state."""
+    acceptance results come back.  The KV cache and the transfer weights are resident state.
+    The new rows reach the cache tail through ht_rope_kv_append (position 0 for every row: the
+    rotation by angle 0 is exact, so the step computes on the same values as the device-resident
+    runs)."""
+    from paper_2404_12022_b200 import binding as hb
     w = step.w
     n = min(args.steps, 5)
     dev = inp.k_cache.device
@@ -420,25 +424,33 @@ def e2e_pass(args, step, inp, torch, world):
     host_q = [pin(q) for q in inp.q]
     L = torch.tensor(w.kv_len, device=dev)
     idx = (L[:, None] + torch.arange(w.N, device=dev)[None]).long()          # [B, N] cache rows of the tree
-    gather = lambda c: torch.stack([c[:, b][:, :, idx[b]] for b in range(w.B)], 1)   # [layers, B, Hkv, N, D]
-    host_k, host_v = pin(gather(inp.k_cache)), pin(gather(inp.v_cache))
+    gather = lambda c: torch.stack([c[:, b][:, :, idx[b]] for b in range(w.B)], 1).permute(0, 1, 3, 2, 4).contiguous()
+    all_k, all_v = gather(inp.k_cache), gather(inp.v_cache)                      # [layers, B, N, Hkv, D]
+    rows_of = [q.shape[1] for q in inp.q]                                        # layers ahead of the transfer have no pseudo rows
+    host_k = [pin(all_k[i][:, :r].contiguous()) for i, r in enumerate(rows_of)]
+    host_v = [pin(all_v[i][:, :r].contiguous()) for i, r in enumerate(rows_of)]
+    del all_k, all_v
+    dev_q = [torch.empty_like(q) for q in inp.q]
+    pos0 = [torch.zeros((w.B, r), dtype=torch.int32, device=dev) for r in rows_of]
     host_small = [pin(t) for t in (inp.logits, inp.parent, inp.parent_tree, inp.tokens, inp.h_src, inp.kv_len)]
     host_rp = pin(inp.root_pred) if inp.root_pred is not None else None
-    dev_k, dev_v = torch.empty_like(host_k, device=dev), torch.empty_like(host_v, device=dev)
+    dev_k = [torch.empty_like(t, device=dev) for t in host_k]
+    dev_v = [torch.empty_like(t, device=dev) for t in host_v]
     small_targets = [inp.logits, inp.parent, inp.parent_tree, inp.tokens, inp.h_src, inp.kv_len]
     host_out = [torch.empty_like(o, device="cpu").pin_memory() for o in step.outs]
     host_res = [torch.empty_like(t, device="cpu").pin_memory() for t in
                 (step.pseudo, step.pred, step.accept_len, step.accept_path, step.next_token, step.new_kv_len)]
     res_src = [step.pseudo, step.pred, step.accept_len, step.accept_path, step.next_token, step.new_kv_len]
-    h2d = sum(t.numel() * t.element_size() for t in host_q + [host_k, host_v] + host_small + ([host_rp] if host_rp is not None else []))
+    h2d = sum(t.numel() * t.element_size() for t in host_q + host_k + host_v + host_small + ([host_rp] if host_rp is not None else []))
     d2h = sum(t.numel() * t.element_size() for t in host_out + host_res)
     stream = torch.cuda.current_stream().cuda_stream
 
-    copy_in, copy_out = torch.cuda.Stream(), torch.cuda.Stream()
+    copy_in, copy_out, place = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
     comp = torch.cuda.current_stream()
-    k_per_layer = host_k.shape[0]
+    k_per_layer = len(host_k)
     ev_in = [torch.cuda.Event() for _ in range(step.layers)]
     ev_out = [torch.cuda.Event() for _ in range(step.layers)]
+    ev_copied = [torch.cuda.Event() for _ in range(step.layers)]
     ev_small, ev_done = torch.cuda.Event(), torch.cuda.Event()
     assert k_per_layer == step.layers
 
@@ -453,13 +465,17 @@ def e2e_pass(args, step, inp, torch, world):
                 inp.root_pred.copy_(host_rp, non_blocking=True)
             ev_small.record(copy_in)
             for i in range(step.layers):
-                inp.q[i].copy_(host_q[i], non_blocking=True)
+                dev_q[i].copy_(host_q[i], non_blocking=True)
                 dev_k[i].copy_(host_k[i], non_blocking=True)
                 dev_v[i].copy_(host_v[i], non_blocking=True)
-                for b in range(w.B):                           # new K/V rows into the cache tail
-                    inp.k_cache[i, b, :, w.kv_len[b]:w.kv_len[b] + w.N] = dev_k[i, b]
-                    inp.v_cache[i, b, :, w.kv_len[b]:w.kv_len[b] + w.N] = dev_v[i, b]
-                ev_in[i].record(copy_in)
+                ev_copied[i].record(copy_in)
+        with torch.cuda.stream(place):                     # the rows' placement runs beside the next layer's copies
+            place.wait_event(ev_small)
+            for i in range(step.layers):
+                place.wait_event(ev_copied[i])
+                hb.rope_kv_append(dev_q[i], dev_k[i], dev_v[i], pos0[i], inp.kv_len, inp.k_cache[i], inp.v_cache[i],
+                                  q_out=inp.q[i])
+                ev_in[i].record(place)
         comp.wait_event(ev_small)
         for i in range(step.layers):
             comp.wait_event(ev_in[i])
