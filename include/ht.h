@@ -126,6 +126,10 @@ int ht_transfer(const void *h_src, const void *W, void *out, int B, int k, int d
  *            (their rows of `out` are left untouched).
  * Cache rows at or beyond kv_len[b] + N are never used for a result, whatever they hold.
  * Supported: D in {64, 128}; N <= 1024.  B == 0 or N == 0 is a no-op.
+ * Stream behaviour (fp16 / bf16, D = 128): the call's kernels are launched with programmatic
+ * stream serialization, i.e. their thread blocks may be set up while the kernel before them in
+ * `stream` is still finishing; they read inputs, workspace and outputs only after that kernel
+ * has completed, so the results are those of plain stream order.
  */
 size_t ht_tree_attention_workspace(const ht_attn_desc *desc /* host */);
 /* Number of this library's kernels that one ht_tree_attention call with this descriptor enqueues (1 or 2:
