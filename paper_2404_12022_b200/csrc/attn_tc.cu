@@ -458,8 +458,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const bool has0 = sg.len >= 2 || (J & 1) == 0;
             const bool has1 = sg.len >= 2 || (J & 1) == 1;
             const int head = sg.hk * p.g + row % p.g;
-            // a part goes to the workspace -- or, in a cluster, to this CTA's own (by now idle) K / V ring
-            float *pslot = clustered ? reinterpret_cast<float *>(&sm.ring[0][0]) : p.part + (size_t)(2 * (int)blockIdx.x + cut_k) * kSlotFloats;
+            // a part goes to the workspace -- or, in a cluster, to this CTA's own (by now idle) Q buffer and K / V ring
+            float *pslot = clustered ? reinterpret_cast<float *>(&sm.q[0]) : p.part + (size_t)(2 * (int)blockIdx.x + cut_k) * kSlotFloats;
             const float *oslot = pslot;                // the other part, when finishing the unit here
             float g0, g1, gb = 0.f;
             if (direct) {
@@ -540,12 +540,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (clustered) {
             const bool had_tiles = t_end > t_begin;
             if (!had_tiles && s == 0) {                // an empty share still delivers a part: nothing seen
-                float *pslot = reinterpret_cast<float *>(&sm.ring[0][0]);
+                float *pslot = reinterpret_cast<float *>(&sm.q[0]);
                 pslot[kRows * kD + row] = -INFINITY;
                 pslot[kRows * kD + kRows + row] = 0.f;
             }
             const int unit = (int)blockIdx.x / p.cluster_k, b = unit / p.Hkv;
-            cluster_exchange<kBf16>(p, &sm.ring[0][0], sm.xb, 0u, (int)c_rank, b, unit - b * p.Hkv, 0, sm.nkt[b] > 0, tid256, abort_flag);
+            cluster_exchange<kBf16>(p, &sm.q[0], sm.xb, 0u, (int)c_rank, b, unit - b * p.Hkv, 0, sm.nkt[b] > 0, tid256, abort_flag);
         }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
         if (cut[0].valid || cut[1].valid) {

@@ -11,7 +11,7 @@ namespace tc {
 constexpr int kTile = 128;                 // keys per tile
 constexpr int kRows = 128;                 // query rows per tile (UMMA M)
 constexpr int kD = 128;
-constexpr int kStages = 5;                 // ring entries (each one K or one V tile)
+constexpr int kStages = 4;                 // ring entries (each one K or one V tile)
 constexpr int kEntryBytes = kTile * kD * 2;
 constexpr int kSlabBytes = kEntryBytes / 2;   // [128 rows][64 elements] = 16 KiB
 constexpr int kThreads = 320;
@@ -527,6 +527,7 @@ __device__ __noinline__ void merge_parts(const Params &p, const CutUnit &cu, int
 // result.  No global memory, no atomics; both waits are bounded.
 constexpr int kXchgRecvOffset = (kSlotFloats * 4 + 1023) / 1024 * 1024;   // bytes from the area's start
 constexpr int kXchgBytes = kXchgRecvOffset + kRows * kD * 4 + 16 * 2 * kRows * 4;   // part + received slices + up to 16 senders' m, l
+static_assert(kXchgBytes <= (1 + kStages) * kEntryBytes, "the exchange area is the Q buffer and the ring");
 
 template <bool kBf16>
 __device__ __noinline__ void cluster_exchange(const Params &p, unsigned char *area, unsigned long long *xb, uint32_t parity,
