@@ -12,7 +12,8 @@
 //   - the unit of softmax / MMA work is half a K/V tile (64 keys).  Each stream has two 64-column
 //     score buffers in TMEM, so Q K^T of the next half is computed while the softmax of the
 //     current one runs, and P V follows as soon as P is written.  TMEM: 4 x 64 (S/P) + 2 x 128 (O).
-//   - shared memory: two Q tiles and a ring of four 32 KiB K / V tiles.
+//   - shared memory: two Q tiles and a ring of three 32 KiB K / V tiles (a fourth bought nothing and its
+//     32 KB of footprint cost 1-4 %).
 //   - a unit (sequence, KV head, tile pair) whose second tile does not exist runs with stream 1 idle.
 // Work split, cut units, tickets and merges are those of the one-tile kernel; a workspace slot
 // holds one part per stream.  Every wait is bounded.
@@ -21,7 +22,7 @@
 namespace ht {
 namespace tc {
 
-constexpr int kPStages = 4;
+constexpr int kPStages = 3;
 constexpr int kPThreads = kThreads + 32;      // + the second MMA-issuing warp
 constexpr int kHalf = 64;                     // keys per softmax / MMA step
 
