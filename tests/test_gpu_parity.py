@@ -205,6 +205,26 @@ def test_attention_random_shapes_tensor_core_kernels_against_the_alu_kernel(hb, 
         check_sampled_units(hb, oracle, q, k, v, kv_len.cpu().numpy(), parent, out, 1, DT[dtype], seed=trial, p_rounding=True)
 
 
+@pytest.mark.parametrize("shape", [(256, 7, 2, 2, "random"), (256, 3, 8, 1, "chain"), (1, 512, 2, 2, "random"), (2, 512, 4, 1, "chain"),
+                                   (1, 513, 2, 2, "random")],
+                         ids=lambda s: "B%dN%dHq%dHkv%d%s" % s)
+def test_attention_at_the_largest_sizes_the_tensor_core_kernels_take(hb, oracle, shape):
+    """256 sequences and 512 rows (16 ancestor words per row) are the tensor-core kernels' limits; one row more goes to
+    the ALU kernel.  Against the ALU kernel everywhere and the oracle on sampled units; ragged lengths from 0 up."""
+    B, N, Hq, Hkv, tree = shape
+    lens = [(37 * b) % 300 for b in range(B)] if B > 1 else [700]
+    q, k, v, kv_len, parent = make_attn_case(93, "bf16", B, N, Hq, Hkv, 128, lens, max(lens) + N + 5, tree)
+    out, status = hb.tree_attention(q, k, v, kv_len, parent)
+    ref, _ = hb.tree_attention(q, k, v, kv_len, parent, flags=hb.HT_ATTN_FORCE_SIMT)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0] * B
+    a, r = out.float(), ref.float()
+    eps = 2.0 ** -7
+    assert torch.isfinite(a).all()
+    assert bool(((a - r).abs() <= 2e-3 + 2 * eps * r.abs() + 3 * eps).all()), "max diff %.3e" % float((a - r).abs().max())
+    check_sampled_units(hb, oracle, q, k, v, kv_len.cpu().numpy(), parent, out, 2, torch.bfloat16, seed=N, p_rounding=True)
+
+
 @pytest.mark.parametrize("shape", [(4, 91, 32, 32, 1500), (1, 91, 32, 32, 1024), (2, 40, 32, 4, 700), (3, 19, 16, 16, 3000)],
                          ids=lambda s: "B%dN%dHq%dHkv%dL%d" % s)
 def test_attention_calls_in_a_row_see_each_others_results(hb, shape):
