@@ -42,7 +42,8 @@ namespace ht {
 namespace tc {
 
 // kPaged: the cache is a pool of pages (separate instantiations, so that the contiguous kernels carry none of that code).
-template <bool kBf16, bool kPaged>
+// kClustered: launched as clusters (p.cluster_k > 1); a template parameter so that the persistent form carries no cluster code.
+template <bool kBf16, bool kPaged, bool kClustered>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const Params p, const PagedParams pp) {
@@ -85,12 +86,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const int per = choose_per(total, p.grid, sm.nkt, p.B, p.n_rt);
     int t_begin = min((int)blockIdx.x * per, total);
     int t_end = min(t_begin + per, total);
-    const bool clustered = p.cluster_k > 1;
+    constexpr bool clustered = kClustered;
     uint32_t c_rank = 0;
     if (clustered) {
-        // One cluster per (sequence, KV head); the cluster's CTAs take equal shares of its tiles.  The
-        // peers' barriers must exist before anyone arrives on them.
-        cluster_sync_all();
+        // One cluster per (sequence, KV head); the cluster's CTAs take equal shares of its tiles.  (No cluster
+        // barrier here: the first remote access comes after the one all threads pass ahead of the exchange.)
         c_rank = cluster_ctarank();
         const int unit = (int)blockIdx.x / p.cluster_k, b = unit / p.Hkv, hk = unit - b * p.Hkv;
         const int nk = sm.nkt[b], share = (nk + p.cluster_k - 1) / p.cluster_k;
@@ -173,6 +173,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (seg_i > 0) mbar_wait(&sm.q_full, (seg_i - 1) & 1, abort_flag, false);
             }
         }
+        if (clustered) cluster_sync_all();             // the barrier ahead of the exchange (whole warp)
     } else if (warp == 9) {
         // ------------------------------- MMA issuer -------------------------------
         if (lane == 0) {
@@ -236,6 +237,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             tc_commit(&sm.mma_drain);
             mbar_wait(&sm.mma_drain, 0, abort_flag, false);
         }
+        if (clustered) cluster_sync_all();             // the barrier ahead of the exchange (whole warp)
     } else {
         // ------------------------------- softmax groups -------------------------------
         const int s = warp >> 2;                       // stream of this group
@@ -545,7 +547,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 pslot[kRows * kD + kRows + row] = 0.f;
             }
             const int unit = (int)blockIdx.x / p.cluster_k, b = unit / p.Hkv;
-            cluster_exchange<kBf16>(p, &sm.q[0], sm.xb, 0u, (int)c_rank, b, unit - b * p.Hkv, 0, sm.nkt[b] > 0, tid256, abort_flag);
+            cluster_exchange<kBf16>(p, &sm.q[0], sm.xb, 0u, (int)c_rank, b, unit - b * p.Hkv, 0, sm.nkt[b] > 0, tid256, abort_flag, true);
         }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
         if (cut[0].valid || cut[1].valid) {
@@ -664,9 +666,12 @@ size_t attn_tc_workspace(const ht_attn_desc &d) {
 }
 
 typedef void (*AttnKernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const tc::Params, const tc::PagedParams);
-static AttnKernelFn attn_tc_fn(bool bf16, bool paged) {
-    return bf16 ? (paged ? tc::attn_tc_kernel<true, true> : tc::attn_tc_kernel<true, false>)
-                : (paged ? tc::attn_tc_kernel<false, true> : tc::attn_tc_kernel<false, false>);
+static AttnKernelFn attn_tc_fn(bool bf16, bool paged, bool clustered) {
+    static const AttnKernelFn fns[8] = {
+        tc::attn_tc_kernel<false, false, false>, tc::attn_tc_kernel<true, false, false>, tc::attn_tc_kernel<false, true, false>,
+        tc::attn_tc_kernel<true, true, false>,   tc::attn_tc_kernel<false, false, true>, tc::attn_tc_kernel<true, false, true>,
+        tc::attn_tc_kernel<false, true, true>,   tc::attn_tc_kernel<true, true, true>};
+    return fns[(bf16 ? 1 : 0) + (paged ? 2 : 0) + (clustered ? 4 : 0)];
 }
 
 // Kernels per call: the attention kernel, and ahead of it the one that zeroes the tickets unless clusters are used.
@@ -679,8 +684,8 @@ static cudaError_t ensure_smem_attr(size_t smem) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
-    for (int i = 0; i < 4; ++i) {
-        e = cudaFuncSetAttribute(attn_tc_fn(i & 1, i >> 1), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    for (int i = 0; i < 8; ++i) {
+        e = cudaFuncSetAttribute(attn_tc_fn(i & 1, (i >> 1) & 1, i >> 2), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
     if (dev >= 0 && dev < 64) done[dev] = true;
@@ -812,7 +817,7 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = k > 1 ? 2 : 1;
-    e = cudaLaunchKernelEx(&cfg, attn_tc_fn(d.dtype == HT_BF16, pages != nullptr), tm_q, tm_k, tm_v, p, pp);
+    e = cudaLaunchKernelEx(&cfg, attn_tc_fn(d.dtype == HT_BF16, pages != nullptr, k > 1), tm_q, tm_k, tm_v, p, pp);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return fail(HT_ERR_CUDA, "ht_tree_attention (tcgen05, clusters of %d): %s", k > 1 ? k : 1, cudaGetErrorString(e));

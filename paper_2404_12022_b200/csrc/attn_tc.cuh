@@ -532,7 +532,7 @@ static_assert(kXchgBytes <= (1 + kStages) * kEntryBytes, "the exchange area is t
 template <bool kBf16>
 __device__ __noinline__ void cluster_exchange(const Params &p, unsigned char *area, unsigned long long *xb, uint32_t parity,
                                               int rank, int b, int hk, int row_tile, bool valid, int tid256,
-                                              volatile int *abort_flag) {
+                                              volatile int *abort_flag, bool whole_cluster_barrier = false) {
     const int k = p.cluster_k;
     const int cg_per_slice = 32 / k;                    // 4-feature groups per CTA's slice
     unsigned char *ring = area;
@@ -540,10 +540,18 @@ __device__ __noinline__ void cluster_exchange(const Params &p, unsigned char *ar
     const float *own_ml = reinterpret_cast<const float *>(ring) + kRows * kD;
     float4 *recv4 = reinterpret_cast<float4 *>(ring + kXchgRecvOffset);          // [sender][group in slice][row]
     float *recv_ml = reinterpret_cast<float *>(ring + kXchgRecvOffset) + kRows * kD;   // [sender][m | l][row]
-    softmax_groups_sync();                              // this CTA's part is complete
-    if (tid256 == 0)
-        for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&xb[0]), (uint32_t)c));
-    mbar_wait_cluster(&xb[0], parity, abort_flag);        // every peer's ring is idle
+    if (whole_cluster_barrier) {
+        // Every thread of every CTA of the cluster takes part in this barrier -- the softmax threads here, the
+        // producer and issuer warps once their work is done -- so behind it all parts are complete and no
+        // ring is in use any more.  It also stands in for a barrier at kernel start: the peers' mbarriers,
+        // initialised before anything else, exist by now.
+        cluster_sync_all();
+    } else {
+        softmax_groups_sync();                          // this CTA's part is complete
+        if (tid256 == 0)
+            for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&xb[0]), (uint32_t)c));
+        mbar_wait_cluster(&xb[0], parity, abort_flag);    // every peer's ring is idle
+    }
     if (!*abort_flag) {
         // thread t moves rows t & 127 of feature groups (t >> 7) + 2 j; k is a power of two
         const int sh = 5 - __ffs(k) + 1;                // log2(cg_per_slice)
