@@ -173,7 +173,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (seg_i > 0) mbar_wait(&sm.q_full, (seg_i - 1) & 1, abort_flag, false);
             }
         }
-        if (clustered) cluster_sync_all();             // the barrier ahead of the exchange (whole warp)
+        if (clustered) {                               // the two barriers of the exchange (whole warp)
+            cluster_sync_all();
+            cluster_sync_all();
+        }
     } else if (warp == 9) {
         // ------------------------------- MMA issuer -------------------------------
         if (lane == 0) {
@@ -237,7 +240,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             tc_commit(&sm.mma_drain);
             mbar_wait(&sm.mma_drain, 0, abort_flag, false);
         }
-        if (clustered) cluster_sync_all();             // the barrier ahead of the exchange (whole warp)
+        if (clustered) {                               // the two barriers of the exchange (whole warp)
+            cluster_sync_all();
+            cluster_sync_all();
+        }
     } else {
         // ------------------------------- softmax groups -------------------------------
         const int s = warp >> 2;                       // stream of this group
@@ -566,7 +572,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // ------------------------------- teardown -------------------------------
     tc_fence_before();
     __syncthreads();
-    if (clustered) cluster_sync_all();       // no CTA leaves while a peer may still write into its shared memory
+    // (cluster mode: the exchange's second barrier already guarantees that no peer writes here any more)
     if (threadIdx.x == 0) HT_TR_CTA(3);
     if (sm.abort && threadIdx.x == 0) {
         for (int b = 0; b < p.B; ++b)

@@ -543,8 +543,7 @@ __device__ __noinline__ void cluster_exchange(const Params &p, unsigned char *ar
     if (whole_cluster_barrier) {
         // Every thread of every CTA of the cluster takes part in this barrier -- the softmax threads here, the
         // producer and issuer warps once their work is done -- so behind it all parts are complete and no
-        // ring is in use any more.  It also stands in for a barrier at kernel start: the peers' mbarriers,
-        // initialised before anything else, exist by now.
+        // ring is in use any more.
         cluster_sync_all();
     } else {
         softmax_groups_sync();                          // this CTA's part is complete
@@ -564,11 +563,17 @@ __device__ __noinline__ void cluster_exchange(const Params &p, unsigned char *ar
         const float ml = own_ml[tid256];                // 128 m then 128 l
         for (int c = 0; c < k; ++c) st_peer_f1(map_to_peer(smem_u32(recv_ml + rank * 2 * kRows + tid256), (uint32_t)c), ml);
     }
-    asm volatile("fence.acq_rel.cluster;" ::: "memory");
-    softmax_groups_sync();
-    if (tid256 == 0)
-        for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&xb[1]), (uint32_t)c));
-    mbar_wait_cluster(&xb[1], parity, abort_flag);        // every part has arrived here
+    if (whole_cluster_barrier) {
+        // a second barrier of the whole cluster: every part has arrived everywhere, and nobody writes into a
+        // peer's shared memory after it, so a CTA may leave as soon as it has merged what it holds
+        cluster_sync_all();
+    } else {
+        asm volatile("fence.acq_rel.cluster;" ::: "memory");
+        softmax_groups_sync();
+        if (tid256 == 0)
+            for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&xb[1]), (uint32_t)c));
+        mbar_wait_cluster(&xb[1], parity, abort_flag);    // every part has arrived here
+    }
     const int row = tid256 & 127, half = tid256 >> 7;
     const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
     if (!valid || node >= p.N || *abort_flag) return;
