@@ -93,8 +93,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const bool clustered = p.cluster_k > 1;
     uint32_t c_rank = 0;
     if (clustered) {
-        // One cluster per (sequence, KV head, tile pair); its CTAs take equal shares of the unit's tiles.
-        cluster_sync_all();                             // the peers' barriers exist before anyone arrives on them
+        // One cluster per (sequence, KV head, tile pair); its CTAs take equal shares of the unit's tiles.  (No
+        // cluster barrier here: the first remote access comes after the one all threads pass ahead of the exchange.)
         c_rank = cluster_ctarank();
         const int unit = (int)blockIdx.x / p.cluster_k, b = unit / (p.Hkv * p.n_rt);
         const int nk = sm.nkt[b], share = (nk + p.cluster_k - 1) / p.cluster_k;
@@ -103,6 +103,13 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         t_end = t0 + min(((int)c_rank + 1) * share, nk);
     }
     unsigned char *const xarea = &sm.q[0][0];          // Q buffers and ring, idle once the CTA's tiles are done
+    // Cluster mode: the unit's one or two streams are exchanged in turn, each exchange between two barriers of the
+    // whole cluster (the softmax threads pass them inside the exchange, the other warps once their work is done).
+    int n_exchanges = 0;
+    if (clustered) {
+        const int unit = (int)blockIdx.x / p.cluster_k, rt = unit % p.n_rt;
+        n_exchanges = (2 * rt + 1 < p.n_row_tiles) ? 2 : 1;
+    }
 
     if (warp == 8) {
         // ------------------------------- TMA producer -------------------------------
@@ -169,6 +176,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (seg_i > 0) mbar_wait(&sm.q_full, (seg_i - 1) & 1, abort_flag, false);
             }
         }
+        for (int x = 0; x < 2 * n_exchanges; ++x) cluster_sync_all();
     } else if (warp >= 9) {
         // ------------------------------- MMA issuers -------------------------------
         // One issuing thread per stream (warp 9: stream 0, warp 10: stream 1), so that neither stream
@@ -261,6 +269,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tc_commit(&sm.mma_drain);
             mbar_wait(&sm.mma_drain, 0, abort_flag, false);
         }
+        for (int x = 0; x < 2 * n_exchanges; ++x) cluster_sync_all();
     } else {
         // ------------------------------- softmax groups -------------------------------
         const int s = warp >> 2;                       // stream of this group = which tile of the pair
@@ -522,7 +531,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int x = 0; x < (two ? 2 : 1); ++x) {
                     if (s == x) emit(reinterpret_cast<float *>(xarea), false, false);
                     tc_fence_before();
-                    cluster_exchange<kBf16>(p, xarea, sm.xb, (uint32_t)x, (int)c_rank, sg.b, sg.hk, 2 * sg.rt + x, true, tid256, abort_flag);
+                    cluster_exchange<kBf16>(p, xarea, sm.xb, (uint32_t)x, (int)c_rank, sg.b, sg.hk, 2 * sg.rt + x, true, tid256, abort_flag, true);
                 }
             } else if (active) {
                 emit(p.part + ((size_t)(2 * (int)blockIdx.x + cut_k) * 2 + s) * kSlotFloats, final || direct, direct);
@@ -549,7 +558,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     part[kRows * kD + row] = -INFINITY;
                     part[kRows * kD + kRows + row] = 0.f;
                 }
-                cluster_exchange<kBf16>(p, xarea, sm.xb, (uint32_t)x, (int)c_rank, b, hk, 2 * rt + x, sm.nkt[b] > 0, tid256, abort_flag);
+                cluster_exchange<kBf16>(p, xarea, sm.xb, (uint32_t)x, (int)c_rank, b, hk, 2 * rt + x, sm.nkt[b] > 0, tid256, abort_flag, true);
             }
         }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
@@ -570,7 +579,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // ------------------------------- teardown -------------------------------
     tc_fence_before();
     __syncthreads();
-    if (clustered) cluster_sync_all();       // no CTA leaves while a peer may still write into its shared memory
+    // (cluster mode: the last exchange's second barrier already guarantees that no peer writes here any more)
     if (sm.abort && threadIdx.x == 0) {
         for (int b = 0; b < p.B; ++b)
             if (sm.nkt[b] > 0) p.status[b] = HT_STATUS_TIMEOUT;
