@@ -58,7 +58,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         mbar_init(&sm.q_full, 1);
         mbar_init(&sm.q_empty, 1);
         mbar_init(&sm.mma_drain, 1);
-        for (int i = 0; i < 2; ++i) mbar_init(&sm.xb[i], p.cluster_k > 1 ? p.cluster_k : 1);
         for (int i = 0; i < 2; ++i) { mbar_init(&sm.s_full[i], 1); mbar_init(&sm.p_ready[i], 128); mbar_init(&sm.o_done[i], 1); }
         sm.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -553,7 +552,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 pslot[kRows * kD + kRows + row] = 0.f;
             }
             const int unit = (int)blockIdx.x / p.cluster_k, b = unit / p.Hkv;
-            cluster_exchange<kBf16>(p, &sm.q[0], sm.xb, 0u, (int)c_rank, b, unit - b * p.Hkv, 0, sm.nkt[b] > 0, tid256, abort_flag, true);
+            cluster_exchange<kBf16>(p, &sm.q[0], (int)c_rank, b, unit - b * p.Hkv, 0, sm.nkt[b] > 0, tid256, abort_flag);
         }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
         if (cut[0].valid || cut[1].valid) {

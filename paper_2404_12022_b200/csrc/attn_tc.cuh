@@ -68,7 +68,6 @@ struct __align__(1024) Smem {
     int32_t nkt[kMaxB];
     int32_t pre[kMaxB + 1];
     unsigned long long kv_full[kStages], kv_empty[kStages], q_full, q_empty, s_full[2], p_ready[2], o_done[2], mma_drain;
-    unsigned long long xb[2];          // cluster exchange: peers ready to receive / all parts delivered
     uint32_t tmem_base;
     int abort;
     int merge_here[2];
@@ -198,7 +197,7 @@ __device__ __forceinline__ unsigned int ld_relaxed_gpu(const unsigned int *ptr) 
     return v;
 }
 
-// ---- thread-block cluster: rank, peer shared memory, barriers in a peer's shared memory ----
+// ---- thread-block cluster: rank, stores to a peer's shared memory, barrier of the whole cluster ----
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -214,28 +213,6 @@ __device__ __forceinline__ void st_peer_f4(uint32_t peer_addr, float4 v) {
 }
 __device__ __forceinline__ void st_peer_f1(uint32_t peer_addr, float v) {
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_addr), "f"(v) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_peer(uint32_t peer_bar_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(peer_bar_addr) : "memory");
-}
-// Bounded wait on a barrier of this CTA that peers arrive on.
-__device__ __forceinline__ bool mbar_wait_cluster(void *bar, uint32_t parity, volatile int *abort_flag) {
-    if (*abort_flag) return false;
-    const uint32_t addr = smem_u32(bar);
-    long long t0 = 0;
-    for (uint32_t it = 0;; ++it) {
-        uint32_t ok;
-        asm volatile(
-            "{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
-        if (ok) return true;
-        if ((it & 63u) == 63u) {
-            if (*abort_flag) return false;
-            const long long now = clock64();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > 2000000000ll) { *abort_flag = 1; return false; }
-        }
-    }
 }
 __device__ __forceinline__ void cluster_sync_all() {   // every thread of every CTA of the cluster
     asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -520,19 +497,19 @@ __device__ __noinline__ void merge_parts(const Params &p, const CutUnit &cu, int
 
 // Reduction of a unit's parts inside a thread-block cluster, by the 256 softmax threads of each CTA.
 // On entry this CTA's part (m, l, O in the layout of a workspace slot) lies at `area`, a stretch of its
-// shared memory (Q and K / V buffers) that nothing else uses any more.  Every CTA owns 128 / k of the 128 output features: once all
-// peers have said that their rings are idle, each CTA copies, for every peer, that peer's feature
-// slice of its part (and m, l) into the peer's ring through distributed shared memory; after a
-// second round of arrivals each CTA merges the k slices it holds and writes its features of the
-// result.  No global memory, no atomics; both waits are bounded.
+// shared memory (Q and K / V buffers) that nothing else uses any more.  Every CTA owns 128 / k of the 128
+// output features.  Behind a barrier of the whole cluster each CTA copies, for every peer, that peer's
+// feature slice of its part (and m, l) into the peer's area through distributed shared memory; behind a
+// second barrier each CTA merges the k slices it holds and writes its features of the result.  No global
+// memory, no atomics, no wait that could run out.  The other warps of every CTA of the cluster must
+// execute the same two barriers per call.
 constexpr int kXchgRecvOffset = (kSlotFloats * 4 + 1023) / 1024 * 1024;   // bytes from the area's start
 constexpr int kXchgBytes = kXchgRecvOffset + kRows * kD * 4 + 16 * 2 * kRows * 4;   // part + received slices + up to 16 senders' m, l
 static_assert(kXchgBytes <= (1 + kStages) * kEntryBytes, "the exchange area is the Q buffer and the ring");
 
 template <bool kBf16>
-__device__ __noinline__ void cluster_exchange(const Params &p, unsigned char *area, unsigned long long *xb, uint32_t parity,
-                                              int rank, int b, int hk, int row_tile, bool valid, int tid256,
-                                              volatile int *abort_flag, bool whole_cluster_barrier = false) {
+__device__ __noinline__ void cluster_exchange(const Params &p, unsigned char *area, int rank, int b, int hk, int row_tile,
+                                              bool valid, int tid256, volatile int *abort_flag) {
     const int k = p.cluster_k;
     const int cg_per_slice = 32 / k;                    // 4-feature groups per CTA's slice
     unsigned char *ring = area;
@@ -540,17 +517,10 @@ __device__ __noinline__ void cluster_exchange(const Params &p, unsigned char *ar
     const float *own_ml = reinterpret_cast<const float *>(ring) + kRows * kD;
     float4 *recv4 = reinterpret_cast<float4 *>(ring + kXchgRecvOffset);          // [sender][group in slice][row]
     float *recv_ml = reinterpret_cast<float *>(ring + kXchgRecvOffset) + kRows * kD;   // [sender][m | l][row]
-    if (whole_cluster_barrier) {
-        // Every thread of every CTA of the cluster takes part in this barrier -- the softmax threads here, the
-        // producer and issuer warps once their work is done -- so behind it all parts are complete and no
-        // ring is in use any more.
-        cluster_sync_all();
-    } else {
-        softmax_groups_sync();                          // this CTA's part is complete
-        if (tid256 == 0)
-            for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&xb[0]), (uint32_t)c));
-        mbar_wait_cluster(&xb[0], parity, abort_flag);    // every peer's ring is idle
-    }
+    // Every thread of every CTA of the cluster takes part in this barrier -- the softmax threads here, the
+    // producer and issuer warps once their work is done -- so behind it all parts are complete and no
+    // ring is in use any more.
+    cluster_sync_all();
     if (!*abort_flag) {
         // thread t moves rows t & 127 of feature groups (t >> 7) + 2 j; k is a power of two
         const int sh = 5 - __ffs(k) + 1;                // log2(cg_per_slice)
@@ -563,17 +533,9 @@ __device__ __noinline__ void cluster_exchange(const Params &p, unsigned char *ar
         const float ml = own_ml[tid256];                // 128 m then 128 l
         for (int c = 0; c < k; ++c) st_peer_f1(map_to_peer(smem_u32(recv_ml + rank * 2 * kRows + tid256), (uint32_t)c), ml);
     }
-    if (whole_cluster_barrier) {
-        // a second barrier of the whole cluster: every part has arrived everywhere, and nobody writes into a
-        // peer's shared memory after it, so a CTA may leave as soon as it has merged what it holds
-        cluster_sync_all();
-    } else {
-        asm volatile("fence.acq_rel.cluster;" ::: "memory");
-        softmax_groups_sync();
-        if (tid256 == 0)
-            for (int c = 0; c < k; ++c) mbar_arrive_peer(map_to_peer(smem_u32(&xb[1]), (uint32_t)c));
-        mbar_wait_cluster(&xb[1], parity, abort_flag);    // every part has arrived here
-    }
+    // a second barrier of the whole cluster: every part has arrived everywhere, and nobody writes into a
+    // peer's shared memory after it, so a CTA may leave as soon as it has merged what it holds
+    cluster_sync_all();
     const int row = tid256 & 127, half = tid256 >> 7;
     const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
     if (!valid || node >= p.N || *abort_flag) return;

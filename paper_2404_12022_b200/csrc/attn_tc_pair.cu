@@ -35,7 +35,6 @@ struct __align__(1024) PSmem {
     int32_t nkt[kMaxB];
     int32_t pre[kMaxB + 1];
     unsigned long long kv_full[kPStages], kv_empty[kPStages], q_full, q_empty, s_full[2][2], p_ready[2][2], o_done[2][2], mma_drain;
-    unsigned long long xb[2];          // cluster exchange: peers ready to receive / all parts delivered
     uint32_t tmem_base;
     int abort;
     int merge_here[2];
@@ -57,7 +56,6 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mbar_init(&sm.q_full, 1);
         mbar_init(&sm.q_empty, 2);          // one arrival per issuing thread
         mbar_init(&sm.mma_drain, 2);
-        for (int i = 0; i < 2; ++i) mbar_init(&sm.xb[i], p.cluster_k > 1 ? p.cluster_k : 1);
         for (int s = 0; s < 2; ++s)
             for (int h = 0; h < 2; ++h) {
                 mbar_init(&sm.s_full[s][h], 1);
@@ -531,7 +529,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int x = 0; x < (two ? 2 : 1); ++x) {
                     if (s == x) emit(reinterpret_cast<float *>(xarea), false, false);
                     tc_fence_before();
-                    cluster_exchange<kBf16>(p, xarea, sm.xb, (uint32_t)x, (int)c_rank, sg.b, sg.hk, 2 * sg.rt + x, true, tid256, abort_flag, true);
+                    cluster_exchange<kBf16>(p, xarea, (int)c_rank, sg.b, sg.hk, 2 * sg.rt + x, true, tid256, abort_flag);
                 }
             } else if (active) {
                 emit(p.part + ((size_t)(2 * (int)blockIdx.x + cut_k) * 2 + s) * kSlotFloats, final || direct, direct);
@@ -558,7 +556,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     part[kRows * kD + row] = -INFINITY;
                     part[kRows * kD + kRows + row] = 0.f;
                 }
-                cluster_exchange<kBf16>(p, xarea, sm.xb, (uint32_t)x, (int)c_rank, b, hk, 2 * rt + x, sm.nkt[b] > 0, tid256, abort_flag, true);
+                cluster_exchange<kBf16>(p, xarea, (int)c_rank, b, hk, 2 * rt + x, sm.nkt[b] > 0, tid256, abort_flag);
             }
         }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
