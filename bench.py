@@ -221,9 +221,9 @@ class ClockSampler:
 # DRAM traffic per launch of the attention kernel on a c3 layer, from the ncu capture summarised in
 # profiles/attn_tc_kernel_c3_layer.md (dram__bytes_read.sum + dram__bytes_write.sum).  It is only
 # reported while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.5e6,
+NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.2e6,
                "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh"],
-               "sha256": "5adc226b8545bcea63114bff53e55d8f1f720f4c64552a1c71610764d99bd078"}
+               "sha256": "4edf36cdfa5fcf3160686cb4308991935f4621101f7203a70fcf4b7cc555d481"}
 
 
 def ncu_traffic(w):
