@@ -38,7 +38,7 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4"])
+    ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4"])
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling small cases)")
     ap.add_argument("--kv", type=int, default=0, help="override the KV length of c3 (profiling small cases)")
@@ -59,6 +59,8 @@ def parse_args():
 
 def make_workload(args):
     from paper_2404_12022_b200 import workloads as wl
+    if args.workload == "c1":
+        return wl.config_c1()
     if args.workload == "c2":
         return wl.config_c2()
     if args.workload == "c4":

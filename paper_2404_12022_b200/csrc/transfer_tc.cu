@@ -266,17 +266,31 @@ static int device_sms() {
     return cached[dev];
 }
 
+// Source-row tiles of 128 per CTA: two (two accumulators fed by one W tile) once there are enough rows -- a
+// third less traffic from L2 into shared memory per product, which is what bounds the large shapes.
+static int transfer_tc_mt(int B) { return B > 3 * ttc::kBM ? 2 : 1; }
+
 // Weight rows per tile.  While one wave of CTAs can hold all tiles, the tiles are made just small enough to
-// give every SM one (the stream over W is spread over the whole GPU); beyond that the largest tile, which
-// reads the h tile least often per product.
+// give every SM one (the stream over W is spread over the whole GPU).  Beyond that the tiles run in waves,
+// and a CTA's time follows the bytes it stages per step (source rows + weight rows): among the wave counts
+// that a tile of at most 256 rows can meet, the one with the least waves x (source rows + bn) is taken --
+// 512 x 20480: 286 tiles of 144 in two full waves instead of 160 tiles of 256 in a full and a thin one.
 int transfer_tc_tile(int B, int R, int sms) {
-    const int n_m = (B + ttc::kBM - 1) / ttc::kBM;
-    const int slots = sms / n_m;
-    if (slots >= 1) {
+    const int mt = transfer_tc_mt(B);
+    const int rows = ttc::kBM * mt;
+    const int n_m = (B + rows - 1) / rows;
+    int best_bn = 256;
+    long long best = ((((long long)(R + 255) / 256) * n_m + sms - 1) / sms) * (rows + 256);
+    for (int w = 1; w <= 16; ++w) {
+        const int slots = (int)((long long)sms * w / n_m);
+        if (slots < 1) continue;
         const int bn = ((R + slots - 1) / slots + 15) / 16 * 16;
-        if (bn <= 256) return bn;
+        if (bn > 256) continue;
+        if (w == 1) return bn;
+        const long long cost = (long long)w * (rows + bn);
+        if (cost < best) { best = cost; best_bn = bn; }
     }
-    return 256;
+    return best_bn;
 }
 
 bool transfer_tc_applicable(int B, int k, int d, int dtype) {
@@ -289,9 +303,7 @@ int launch_transfer_tc(const void *h, const void *W, void *out, int B, int k, in
     p.out = out;
     p.B = B; p.R = R; p.d = d;
     p.bn = transfer_tc_tile(B, R, device_sms());
-    // Two 128-row tiles of h per CTA (two accumulators fed by one W tile) once there are enough rows: a third
-    // less traffic from L2 into shared memory per product, which is what bounds the large shapes.
-    p.mt = B > 3 * ttc::kBM ? 2 : 1;
+    p.mt = transfer_tc_mt(B);
     p.n_m = (B + ttc::kBM * p.mt - 1) / (ttc::kBM * p.mt);
     // Fewer than 128 source rows: only those are fetched and held.  The tensor pipe still reads 128 rows
     // from the h tile's address on, i.e. on into the W tile and the next stage (the ring is followed by that

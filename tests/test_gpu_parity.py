@@ -619,8 +619,11 @@ def test_transfer_many_rows(hb, oracle, dtype, shape):
     assert_close(f32np(out), oracle.transfer(f32np(h), f32np(W)), dt, "transfer, many rows")
 
 
-def test_transfer_per_node_rows_of_config_3(hb, oracle):
-    B, k, d = 4 * 88, 3, 4096
+# (1025, 4, 2048): five two-tile CTAs per weight tile, more tiles than SMs -- the weight tiles are then sized for
+# whole waves (144 rows; the last one ragged), not for the widest accumulator
+@pytest.mark.parametrize("shape", [(4 * 88, 3, 4096), (1025, 4, 2048)], ids=lambda s: "B%dk%dd%d" % s)
+def test_transfer_per_node_rows_of_config_3(hb, oracle, shape):
+    B, k, d = shape
     h = wl.normal_tensor(25, 1, (B, d), "cuda", 1.0, torch.bfloat16)
     W = wl.normal_tensor(25, 2, (k, d, d), "cuda", 0.02, torch.bfloat16)
     out = hb.transfer(h, W)
