@@ -23,6 +23,10 @@ namespace ht {
 namespace tc {
 
 constexpr int kPStages = 3;
+#ifndef HT_POLY_EVERY
+#define HT_POLY_EVERY 4
+#endif
+constexpr int kPolyEvery = HT_POLY_EVERY;     // one pair of exponentials in this many goes to the FMA pipe (a power of two)
 constexpr int kPThreads = kThreads + 32;      // + the second MMA-issuing warp
 constexpr int kHalf = 64;                     // keys per softmax / MMA step
 
@@ -408,9 +412,14 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                         for (int c = 0; c < 16; ++c) {
                             float p0, p1;
-                            unpack_f32x2(fma_f32x2(pack_f32x2(xa[2 * c], xa[2 * c + 1]), scale2, nbase2), p0, p1);
-                            p0 = ex2(p0);
-                            p1 = ex2(p1);
+                            const unsigned long long x2 = fma_f32x2(pack_f32x2(xa[2 * c], xa[2 * c + 1]), scale2, nbase2);
+                            if ((c & (kPolyEvery - 1)) == kPolyEvery - 1) {
+                                ex2_poly_x2(x2, p0, p1);
+                            } else {
+                                unpack_f32x2(x2, p0, p1);
+                                p0 = ex2(p0);
+                                p1 = ex2(p1);
+                            }
                             acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
                             r[c] = pack2<kBf16>(p0, p1);
                         }
@@ -418,9 +427,14 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                         for (int c = 0; c < 16; ++c) {
                             float p0, p1;
-                            unpack_f32x2(fma_f32x2(pack_f32x2(xb[2 * c], xb[2 * c + 1]), scale2, nbase2), p0, p1);
-                            p0 = ex2(p0);
-                            p1 = ex2(p1);
+                            const unsigned long long x2 = fma_f32x2(pack_f32x2(xb[2 * c], xb[2 * c + 1]), scale2, nbase2);
+                            if ((c & (kPolyEvery - 1)) == kPolyEvery - 1) {
+                                ex2_poly_x2(x2, p0, p1);
+                            } else {
+                                unpack_f32x2(x2, p0, p1);
+                                p0 = ex2(p0);
+                                p1 = ex2(p1);
+                            }
                             acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
                             r[c] = pack2<kBf16>(p0, p1);
                         }
