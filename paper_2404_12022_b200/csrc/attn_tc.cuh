@@ -241,30 +241,6 @@ __device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, un
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
-// 2^x for a pair of values on the FMA pipe instead of the special-function unit (which does 16 a clock
-// per SM and is what the tile-pair kernel's exponential pass runs into): x = n + r with n the nearest
-// integer (read off the low mantissa bits of x + 1.5 * 2^23) and r in [-1/2, 1/2]; 2^r by a cubic (least
-// maximum relative error on that interval, 7.6e-5: a sixth of the rounding of a 16-bit P); n goes into
-// the exponent by an integer multiply-add.  x below -125 (masked scores are -inf) gives 2^-125 in place
-// of 0, which is 0 to everything it meets afterwards.
-__device__ __forceinline__ void ex2_poly_x2(unsigned long long x2, float &p0, float &p1) {
-    float x0, x1;
-    unpack_f32x2(x2, x0, x1);
-    const unsigned long long x = pack_f32x2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
-    const unsigned long long magic = pack_f32x2(12582912.f, 12582912.f);
-    const unsigned long long fi = add_f32x2(x, magic);
-    const unsigned long long xr = add_f32x2(fi, pack_f32x2(-12582912.f, -12582912.f));
-    const unsigned long long r = fma_f32x2(xr, pack_f32x2(-1.f, -1.f), x);
-    unsigned long long q = fma_f32x2(pack_f32x2(0.05516993626952171f, 0.05516993626952171f), r,
-                                     pack_f32x2(0.24260683357715607f, 0.24260683357715607f));
-    q = fma_f32x2(q, r, pack_f32x2(0.693260908126831f, 0.693260908126831f));
-    q = fma_f32x2(q, r, pack_f32x2(0.99992835521698f, 0.99992835521698f));
-    float q0, q1, f0, f1;
-    unpack_f32x2(q, q0, q1);
-    unpack_f32x2(fi, f0, f1);
-    p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(f0) << 23));
-    p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(f1) << 23));
-}
 
 __device__ __forceinline__ void softmax_groups_sync() {   // the 256 softmax threads
     asm volatile("bar.sync 1, 256;" ::: "memory");
