@@ -423,21 +423,32 @@ def e2e_pass(args, step, inp, torch, world):
     n = min(args.steps, 5)
     dev = inp.k_cache.device
     pin = lambda t: t.cpu().pin_memory()
-    host_q = [pin(q) for q in inp.q]
     L = torch.tensor(w.kv_len, device=dev)
     idx = (L[:, None] + torch.arange(w.N, device=dev)[None]).long()          # [B, N] cache rows of the tree
     gather = lambda c: torch.stack([c[:, b][:, :, idx[b]] for b in range(w.B)], 1).permute(0, 1, 3, 2, 4).contiguous()
     all_k, all_v = gather(inp.k_cache), gather(inp.v_cache)                      # [layers, B, N, Hkv, D]
     rows_of = [q.shape[1] for q in inp.q]                                        # layers ahead of the transfer have no pseudo rows
-    host_k = [pin(all_k[i][:, :r].contiguous()) for i, r in enumerate(rows_of)]
-    host_v = [pin(all_v[i][:, :r].contiguous()) for i, r in enumerate(rows_of)]
+    # One pinned buffer and one device buffer per layer hold q | k | v back to back, so a layer's inputs
+    # travel as one copy.
+    host_in, dev_in, host_q, host_k, host_v, dev_q, dev_k, dev_v = [], [], [], [], [], [], [], []
+    for i, r in enumerate(rows_of):
+        parts = [inp.q[i], all_k[i][:, :r].contiguous(), all_v[i][:, :r].contiguous()]
+        total = sum(t.numel() for t in parts)
+        hbuf = torch.empty(total, dtype=parts[0].dtype).pin_memory()
+        dbuf = torch.empty(total, dtype=parts[0].dtype, device=dev)
+        views_h, views_d, at = [], [], 0
+        for t in parts:
+            views_h.append(hbuf[at:at + t.numel()].view(t.shape))
+            views_d.append(dbuf[at:at + t.numel()].view(t.shape))
+            views_h[-1].copy_(t)
+            at += t.numel()
+        host_in.append(hbuf); dev_in.append(dbuf)
+        host_q.append(views_h[0]); host_k.append(views_h[1]); host_v.append(views_h[2])
+        dev_q.append(views_d[0]); dev_k.append(views_d[1]); dev_v.append(views_d[2])
     del all_k, all_v
-    dev_q = [torch.empty_like(q) for q in inp.q]
     pos0 = [torch.zeros((w.B, r), dtype=torch.int32, device=dev) for r in rows_of]
     host_small = [pin(t) for t in (inp.logits, inp.parent, inp.parent_tree, inp.tokens, inp.h_src, inp.kv_len)]
     host_rp = pin(inp.root_pred) if inp.root_pred is not None else None
-    dev_k = [torch.empty_like(t, device=dev) for t in host_k]
-    dev_v = [torch.empty_like(t, device=dev) for t in host_v]
     small_targets = [inp.logits, inp.parent, inp.parent_tree, inp.tokens, inp.h_src, inp.kv_len]
     host_out = [torch.empty_like(o, device="cpu").pin_memory() for o in step.outs]
     host_res = [torch.empty_like(t, device="cpu").pin_memory() for t in
@@ -467,9 +478,7 @@ def e2e_pass(args, step, inp, torch, world):
                 inp.root_pred.copy_(host_rp, non_blocking=True)
             ev_small.record(copy_in)
             for i in range(step.layers):
-                dev_q[i].copy_(host_q[i], non_blocking=True)
-                dev_k[i].copy_(host_k[i], non_blocking=True)
-                dev_v[i].copy_(host_v[i], non_blocking=True)
+                dev_in[i].copy_(host_in[i], non_blocking=True)
                 ev_copied[i].record(copy_in)
         with torch.cuda.stream(place):                     # the rows' placement runs beside the next layer's copies
             place.wait_event(ev_small)
