@@ -53,7 +53,7 @@ attn_simt_kernel(SimtParams p) {
     const int L = p.kv_len[b];
     const int32_t *par = p.parent + (size_t)b * N;
 
-    // Legality of this sequence's inputs; every block of the sequence reaches the same verdict.
+    // Legality of this sequence's inputs; every block of the sequence comes to the same decision.
     if (threadIdx.x == 0) s_bad = 0;
     __syncthreads();
     for (int c = threadIdx.x; c < N; c += blockDim.x)
