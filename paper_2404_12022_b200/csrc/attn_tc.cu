@@ -454,6 +454,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             tc_fence_before();
             softmax_groups_sync();
             tc_fence_after();
+            // In a cluster the part goes straight from the accumulators into the peers' shared memory (each
+            // peer owns a slice of the features), so the barrier that says "every CTA of the cluster is done with
+            // its Q buffer and ring" comes first: every thread of every CTA takes part in it, the producer and
+            // issuer warps once their work is done.
+            if (clustered) cluster_sync_all();
             const float m0 = sm.ml[0][row][0], l0 = sm.ml[0][row][1];
             const float m1 = sm.ml[1][row][0], l1 = sm.ml[1][row][1];
             const bool direct = sm.direct;
@@ -465,8 +470,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const bool has0 = sg.len >= 2 || (J & 1) == 0;
             const bool has1 = sg.len >= 2 || (J & 1) == 1;
             const int head = sg.hk * p.g + row % p.g;
-            // a part goes to the workspace -- or, in a cluster, to this CTA's own (by now idle) Q buffer and K / V ring
-            float *pslot = clustered ? reinterpret_cast<float *>(&sm.q[0]) : p.part + (size_t)(2 * (int)blockIdx.x + cut_k) * kSlotFloats;
+            // a part goes to the workspace -- or, in a cluster, slice by slice to the peers' (by now idle) Q buffers and rings
+            float *pslot = clustered ? nullptr : p.part + (size_t)(2 * (int)blockIdx.x + cut_k) * kSlotFloats;
+            const int xk_sh = clustered ? 5 - __ffs(p.cluster_k) + 1 : 0;        // log2 of the 4-feature groups per peer's slice
+            const uint32_t xrecv = smem_u32(&sm.q[0]) + kXchgRecvOffset;           // same offset in every CTA of the cluster
             const float *oslot = pslot;                // the other part, when finishing the unit here
             float g0, g1, gb = 0.f;
             if (direct) {
@@ -517,13 +524,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
                         *reinterpret_cast<uint4 *>(dst + c * 16) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+                } else if (clustered) {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {    // feature group cg belongs to peer cg >> xk_sh, as that slice's group x
+                        const int cg = col0 / 4 + c, x = cg & ((1 << xk_sh) - 1);
+                        st_peer_f4(map_to_peer(xrecv + (uint32_t)((((int)c_rank << xk_sh) + x) * kRows + row) * 16u, (uint32_t)(cg >> xk_sh)),
+                                   make_float4(xa_e[4 * c], xa_e[4 * c + 1], xa_e[4 * c + 2], xa_e[4 * c + 3]));
+                    }
                 } else {
 #pragma unroll
                     for (int c = 0; c < 8; ++c)      // 32 consecutive rows of one feature group: 512 contiguous bytes per warp
                         reinterpret_cast<float4 *>(pslot)[(col0 / 4 + c) * kRows + row] = make_float4(xa_e[4 * c], xa_e[4 * c + 1], xa_e[4 * c + 2], xa_e[4 * c + 3]);
                 }
             }
-            if (!final && s == 0 && real) {
+            if (clustered) {
+                // every peer gets this part's maximum (from stream 0's threads) and sum (from stream 1's)
+                if (real)
+                    for (int c = 0; c < p.cluster_k; ++c)
+                        st_peer_f1(map_to_peer(xrecv + (uint32_t)(kRows * kD + ((int)c_rank * 2 + s) * kRows + row) * 4u, (uint32_t)c), s == 0 ? M : l_tot);
+            } else if (!final && s == 0 && real) {
                 pslot[kRows * kD + row] = M;
                 pslot[kRows * kD + kRows + row] = l_tot;
             }
@@ -545,14 +564,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         if (tid256 == 0) HT_TR_CTA(2);
         if (clustered) {
-            const bool had_tiles = t_end > t_begin;
-            if (!had_tiles && s == 0) {                // an empty share still delivers a part: nothing seen
-                float *pslot = reinterpret_cast<float *>(&sm.q[0]);
-                pslot[kRows * kD + row] = -INFINITY;
-                pslot[kRows * kD + kRows + row] = 0.f;
+            if (t_end <= t_begin) {                    // an empty share still delivers a part: nothing seen
+                cluster_sync_all();
+                const uint32_t xrecv = smem_u32(&sm.q[0]) + kXchgRecvOffset;
+                for (int c = 0; c < p.cluster_k; ++c)
+                    st_peer_f1(map_to_peer(xrecv + (uint32_t)(kRows * kD + ((int)c_rank * 2 + s) * kRows + row) * 4u, (uint32_t)c), s == 0 ? -INFINITY : 0.f);
             }
             const int unit = (int)blockIdx.x / p.cluster_k, b = unit / p.Hkv;
-            cluster_exchange<kBf16>(p, &sm.q[0], (int)c_rank, b, unit - b * p.Hkv, 0, sm.nkt[b] > 0, tid256, abort_flag);
+            cluster_merge<kBf16>(p, &sm.q[0], (int)c_rank, b, unit - b * p.Hkv, 0, sm.nkt[b] > 0, tid256, abort_flag);
         }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
         if (cut[0].valid || cut[1].valid) {
