@@ -495,14 +495,13 @@ __device__ __noinline__ void merge_parts(const Params &p, const CutUnit &cu, int
                        pack2<kBf16>(acc[8 * x + 4] * inv, acc[8 * x + 5] * inv), pack2<kBf16>(acc[8 * x + 6] * inv, acc[8 * x + 7] * inv));
 }
 
-// Reduction of a unit's parts inside a thread-block cluster, by the 256 softmax threads of each CTA.
-// On entry this CTA's part (m, l, O in the layout of a workspace slot) lies at `area`, a stretch of its
-// shared memory (Q and K / V buffers) that nothing else uses any more.  Every CTA owns 128 / k of the 128
-// output features.  Behind a barrier of the whole cluster each CTA copies, for every peer, that peer's
-// feature slice of its part (and m, l) into the peer's area through distributed shared memory; behind a
-// second barrier each CTA merges the k slices it holds and writes its features of the result.  No global
-// memory, no atomics, no wait that could run out.  The other warps of every CTA of the cluster must
-// execute the same two barriers per call.
+// Reduction of a unit's parts inside a thread-block cluster, by the 256 softmax threads of each CTA.  Every CTA
+// owns 128 / k of the 128 output features.  Behind a barrier of the whole cluster (all parts complete, no Q
+// buffer or ring in use any more) each thread sends its row's feature groups straight from the accumulator
+// into the owners' shared memory, `area` + kXchgRecvOffset (Q buffer and ring), through distributed shared
+// memory; behind a second barrier each CTA merges the k slices it holds and writes its features of the result.
+// No global memory, no atomics, no wait that could run out.  The other warps of every CTA of the cluster execute
+// the same two barriers.
 constexpr int kXchgRecvOffset = (kSlotFloats * 4 + 1023) / 1024 * 1024;   // bytes from the area's start
 constexpr int kXchgBytes = kXchgRecvOffset + kRows * kD * 4 + 16 * 2 * kRows * 4;   // part + received slices + up to 16 senders' m, l
 static_assert(kXchgBytes <= (1 + kStages) * kEntryBytes, "the exchange area is the Q buffer and the ring");
@@ -547,36 +546,6 @@ __device__ __noinline__ void cluster_merge(const Params &p, unsigned char *area,
         *reinterpret_cast<uint2 *>(dst) = make_uint2(pack2<kBf16>(o.x * inv, o.y * inv), pack2<kBf16>(o.z * inv, o.w * inv));
     }
 }
-
-template <bool kBf16>
-__device__ __noinline__ void cluster_exchange(const Params &p, unsigned char *area, int rank, int b, int hk, int row_tile,
-                                              bool valid, int tid256, volatile int *abort_flag) {
-    const int k = p.cluster_k;
-    const int cg_per_slice = 32 / k;                    // 4-feature groups per CTA's slice
-    unsigned char *ring = area;
-    const float4 *own4 = reinterpret_cast<const float4 *>(ring);
-    const float *own_ml = reinterpret_cast<const float *>(ring) + kRows * kD;
-    float4 *recv4 = reinterpret_cast<float4 *>(ring + kXchgRecvOffset);          // [sender][group in slice][row]
-    float *recv_ml = reinterpret_cast<float *>(ring + kXchgRecvOffset) + kRows * kD;   // [sender][m | l][row]
-    // Every thread of every CTA of the cluster takes part in this barrier -- the softmax threads here, the
-    // producer and issuer warps once their work is done -- so behind it all parts are complete and no
-    // ring is in use any more.
-    cluster_sync_all();
-    if (!*abort_flag) {
-        // thread t moves rows t & 127 of feature groups (t >> 7) + 2 j; k is a power of two
-        const int sh = 5 - __ffs(k) + 1;                // log2(cg_per_slice)
-        const uint32_t recv_base = smem_u32(recv4 + rank * cg_per_slice * kRows + (tid256 & 127));
-#pragma unroll 4
-        for (int j = 0; j < 16; ++j) {
-            const int cg = (tid256 >> 7) + 2 * j, c = cg >> sh, x = cg & (cg_per_slice - 1);
-            st_peer_f4(map_to_peer(recv_base + x * kRows * 16, (uint32_t)c), own4[cg * kRows + (tid256 & 127)]);
-        }
-        const float ml = own_ml[tid256];                // 128 m then 128 l
-        for (int c = 0; c < k; ++c) st_peer_f1(map_to_peer(smem_u32(recv_ml + rank * 2 * kRows + tid256), (uint32_t)c), ml);
-    }
-    cluster_merge<kBf16>(p, area, rank, b, hk, row_tile, valid, tid256, abort_flag);
-}
-
 
 }  // namespace tc
 }  // namespace ht

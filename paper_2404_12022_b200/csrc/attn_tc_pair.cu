@@ -52,6 +52,47 @@ __device__ __forceinline__ void ex2_poly_x2(unsigned long long x2, float &p0, fl
     p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(f1) << 23));
 }
 
+// Cluster reduction of the tile-pair kernel: both streams' parts travel in one exchange.  Every CTA owns 128 / k of
+// the output features; thread (row, stream) sends its row's 32 feature groups straight from the accumulator into the
+// owners' shared memory (Q buffers and ring, idle by then), layout per stream [sender][group in slice][row] float4
+// followed by [sender][m | l][row]; behind the second barrier of the cluster the same thread merges the k slices of
+// its row and writes the CTA's features of the result.
+constexpr int kPXchgMl = kRows * kD * 4;                         // bytes from a stream's area to its m, l
+constexpr int kPXchgStream = kPXchgMl + 8 * 2 * kRows * 4;       // up to 8 senders
+static_assert(2 * kPXchgStream <= (2 + kPStages) * kEntryBytes, "the exchange area is the Q buffers and the ring");
+
+template <bool kBf16>
+__device__ __noinline__ void cluster_merge_pair(const Params &p, const unsigned char *area, int rank, int b, int hk, int row_tile,
+                                                bool valid, int row, volatile int *abort_flag) {
+    cluster_sync_all();                                 // every part has arrived everywhere; nobody writes to a peer any more
+    const int k = p.cluster_k, cgps = 32 / k;
+    const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
+    if (!valid || row_tile >= p.n_row_tiles || node >= p.N || *abort_flag) return;
+    const float4 *recv4 = reinterpret_cast<const float4 *>(area);
+    const float *recv_ml = reinterpret_cast<const float *>(area + kPXchgMl);
+    float M = -INFINITY;
+    for (int c = 0; c < k; ++c) M = fmaxf(M, recv_ml[c * 2 * kRows + row]);
+    float l = 0.f;
+    for (int c = 0; c < k; ++c) {
+        const float m = recv_ml[c * 2 * kRows + row];
+        if (m != -INFINITY) l = fmaf(exp2f(m - M), recv_ml[c * 2 * kRows + kRows + row], l);
+    }
+    const float inv = 1.f / l;
+    const int head = hk * p.g + row % p.g;
+    unsigned char *dst = static_cast<unsigned char *>(p.out) + ((((size_t)b * p.N + node) * p.Hq + head) * kD + rank * cgps * 4) * 2;
+    for (int x = 0; x < cgps; ++x) {
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = 0; c < k; ++c) {
+            const float m = recv_ml[c * 2 * kRows + row];
+            if (m == -INFINITY) continue;
+            const float f = exp2f(m - M);
+            const float4 v = recv4[(c * cgps + x) * kRows + row];
+            o.x = fmaf(f, v.x, o.x); o.y = fmaf(f, v.y, o.y); o.z = fmaf(f, v.z, o.z); o.w = fmaf(f, v.w, o.w);
+        }
+        *reinterpret_cast<uint2 *>(dst + x * 8) = make_uint2(pack2<kBf16>(o.x * inv, o.y * inv), pack2<kBf16>(o.z * inv, o.w * inv));
+    }
+}
+
 struct __align__(1024) PSmem {
     unsigned char q[2][kEntryBytes];
     unsigned char ring[kPStages][kEntryBytes];
@@ -127,13 +168,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         t_end = t0 + min(((int)c_rank + 1) * share, nk);
     }
     unsigned char *const xarea = &sm.q[0][0];          // Q buffers and ring, idle once the CTA's tiles are done
-    // Cluster mode: the unit's one or two streams are exchanged in turn, each exchange between two barriers of the
-    // whole cluster (the softmax threads pass them inside the exchange, the other warps once their work is done).
-    int n_exchanges = 0;
-    if (clustered) {
-        const int unit = (int)blockIdx.x / p.cluster_k, rt = unit % p.n_rt;
-        n_exchanges = (2 * rt + 1 < p.n_row_tiles) ? 2 : 1;
-    }
+    // Cluster mode: the unit's parts are exchanged between two barriers of the whole cluster (the softmax threads pass
+    // them around their sends, the other warps once their work is done).
 
     if (warp == 8) {
         // ------------------------------- TMA producer -------------------------------
@@ -200,7 +236,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (seg_i > 0) mbar_wait(&sm.q_full, (seg_i - 1) & 1, abort_flag, false);
             }
         }
-        for (int x = 0; x < 2 * n_exchanges; ++x) cluster_sync_all();
+        if (clustered) { cluster_sync_all(); cluster_sync_all(); }
     } else if (warp >= 9) {
         // ------------------------------- MMA issuers -------------------------------
         // One issuing thread per stream (warp 9: stream 0, warp 10: stream 1), so that neither stream
@@ -293,7 +329,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tc_commit(&sm.mma_drain);
             mbar_wait(&sm.mma_drain, 0, abort_flag, false);
         }
-        for (int x = 0; x < 2 * n_exchanges; ++x) cluster_sync_all();
+        if (clustered) { cluster_sync_all(); cluster_sync_all(); }
     } else {
         // ------------------------------- softmax groups -------------------------------
         const int s = warp >> 2;                       // stream of this group = which tile of the pair
@@ -502,7 +538,9 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const bool direct = sm.direct;
             const bool final = (complete && !clustered) || direct;
             // this stream's rows: normalised to `out` (fin), merged with the one other part first (dir), or as a part to dst
-            auto emit = [&](float *dst, bool fin, bool dir) {
+            const int xk_sh = clustered ? 5 - __ffs(p.cluster_k) + 1 : 0;        // log2 of the 4-feature groups per peer's slice
+            const uint32_t xrecv = smem_u32(xarea) + (uint32_t)(s * kPXchgStream);  // this stream's receive area: same offset in every CTA
+            auto emit = [&](float *dst, bool fin, bool dir, bool peer) {
                 const int head = sg.hk * p.g + row % p.g;
                 const float *oslot = dst;              // the other part, when finishing the unit here
                 float g0, gb = 0.f;
@@ -548,27 +586,41 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
                             *reinterpret_cast<uint4 *>(o + c * 16) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+                    } else if (peer) {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {    // feature group cg belongs to peer cg >> xk_sh, as that slice's group x
+                            const int cg = col0 / 4 + c, x = cg & ((1 << xk_sh) - 1);
+                            st_peer_f4(map_to_peer(xrecv + (uint32_t)((((int)c_rank << xk_sh) + x) * kRows + row) * 16u, (uint32_t)(cg >> xk_sh)),
+                                       make_float4(xa[4 * c], xa[4 * c + 1], xa[4 * c + 2], xa[4 * c + 3]));
+                        }
                     } else {
 #pragma unroll
                         for (int c = 0; c < 8; ++c)
                             reinterpret_cast<float4 *>(dst)[(col0 / 4 + c) * kRows + row] = make_float4(xa[4 * c], xa[4 * c + 1], xa[4 * c + 2], xa[4 * c + 3]);
                     }
                 }
-                if (!fin && real) {
+                if (peer) {
+                    if (real)
+                        for (int c = 0; c < p.cluster_k; ++c) {
+                            const uint32_t ml = map_to_peer(xrecv + (uint32_t)(kPXchgMl + ((int)c_rank * 2 * kRows + row) * 4), (uint32_t)c);
+                            st_peer_f1(ml, m_ref);
+                            st_peer_f1(ml + kRows * 4, l_sum);
+                        }
+                } else if (!fin && real) {
                     dst[kRows * kD + row] = m_ref;
                     dst[kRows * kD + kRows + row] = l_sum;
                 }
             };
             if (clustered) {
-                // The unit's parts are reduced inside the cluster, one stream after the other through the
-                // same stretch of shared memory (the second stream's accumulator waits in TMEM meanwhile).
-                for (int x = 0; x < (two ? 2 : 1); ++x) {
-                    if (s == x) emit(reinterpret_cast<float *>(xarea), false, false);
-                    tc_fence_before();
-                    cluster_exchange<kBf16>(p, xarea, (int)c_rank, sg.b, sg.hk, 2 * sg.rt + x, true, tid256, abort_flag);
-                }
+                // The unit's parts are reduced inside the cluster: behind a barrier that every thread of the cluster
+                // passes once its work is done (all parts complete, no ring in use) each stream's threads send
+                // their rows to the features' owners; the merge follows behind a second barrier.
+                cluster_sync_all();
+                if (active) emit(nullptr, false, false, true);
+                tc_fence_before();
+                cluster_merge_pair<kBf16>(p, xarea + s * kPXchgStream, (int)c_rank, sg.b, sg.hk, row_tile, true, row, abort_flag);
             } else if (active) {
-                emit(p.part + ((size_t)(2 * (int)blockIdx.x + cut_k) * 2 + s) * kSlotFloats, final || direct, direct);
+                emit(p.part + ((size_t)(2 * (int)blockIdx.x + cut_k) * 2 + s) * kSlotFloats, final || direct, direct, false);
             }
             tc_fence_before();
             softmax_groups_sync();                     // the accumulators are free for the next segment
@@ -583,17 +635,17 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             t += sg.len;
         }
         if (clustered && t_end <= t_begin) {
-            // an empty share still takes part in the cluster's exchanges, with parts that saw nothing
+            // an empty share still takes part in the cluster's exchange, with parts that saw nothing
             const int unit = (int)blockIdx.x / p.cluster_k, b = unit / (p.Hkv * p.n_rt);
             const int rem = unit - b * p.Hkv * p.n_rt, hk = rem / p.n_rt, rt = rem - hk * p.n_rt;
-            for (int x = 0; x < ((2 * rt + 1 < p.n_row_tiles) ? 2 : 1); ++x) {
-                if (s == 0) {
-                    float *part = reinterpret_cast<float *>(xarea);
-                    part[kRows * kD + row] = -INFINITY;
-                    part[kRows * kD + kRows + row] = 0.f;
+            cluster_sync_all();
+            if (2 * rt + s < p.n_row_tiles)
+                for (int c = 0; c < p.cluster_k; ++c) {
+                    const uint32_t ml = map_to_peer(smem_u32(xarea) + (uint32_t)(s * kPXchgStream + kPXchgMl + ((int)c_rank * 2 * kRows + row) * 4), (uint32_t)c);
+                    st_peer_f1(ml, -INFINITY);
+                    st_peer_f1(ml + kRows * 4, 0.f);
                 }
-                cluster_exchange<kBf16>(p, xarea, (int)c_rank, b, hk, 2 * rt + x, sm.nkt[b] > 0, tid256, abort_flag);
-            }
+            cluster_merge_pair<kBf16>(p, xarea + s * kPXchgStream, (int)c_rank, b, hk, 2 * rt + s, sm.nkt[b] > 0, row, abort_flag);
         }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
         if (cut[0].valid || cut[1].valid) {
