@@ -223,9 +223,9 @@ class ClockSampler:
 # DRAM traffic per launch of the attention kernel on a c3 layer, from the ncu capture summarised in
 # profiles/attn_tc_kernel_c3_layer.md (dram__bytes_read.sum + dram__bytes_write.sum).  It is only
 # reported while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.2e6,
+NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.4e6,
                "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh"],
-               "sha256": "4edf36cdfa5fcf3160686cb4308991935f4621101f7203a70fcf4b7cc555d481"}
+               "sha256": "5a5bef8714cfe0319aff1929eac0d7845a96d21bde1f4985a951d013302a6a9d"}
 
 
 def ncu_traffic(w):
