@@ -225,7 +225,7 @@ class ClockSampler:
 # reported while the kernel source is the one that was profiled.
 NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.4e6,
                "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh"],
-               "sha256": "5a5bef8714cfe0319aff1929eac0d7845a96d21bde1f4985a951d013302a6a9d"}
+               "sha256": "d66636ddd95c59df34ad061efdbffc6603c6424f70aa605dff8ee93e7b7a18d9"}
 
 
 def ncu_traffic(w):

@@ -672,8 +672,9 @@ static int cluster_size(const ht_attn_desc &d) {
     for (int k = 8; k >= 2; k /= 2)
         if (units * k <= sms) {
             // Clusters leave SMs idle when units * k falls well short of the GPU; that only pays while the
-            // cache is short (the capacity bounds its length) and latency, not bandwidth, decides.
-            return (units * k * 4 >= 3ll * sms || d.cap <= 6144) ? k : 0;
+            // cache is short (the capacity bounds its length) and latency, not bandwidth, decides: up to
+            // about a dozen tiles per CTA.
+            return (units * k * 4 >= 3ll * sms || d.cap <= (k == 8 ? 12288 : 6144)) ? k : 0;
         }
     return 0;
 }
