@@ -30,6 +30,10 @@ compact_kernel(unsigned char *__restrict__ k_cache, unsigned char *__restrict__ 
     __shared__ int32_t s_path[kCompactMaxPath];
     __shared__ long long s_src[kCompactMaxPath], s_dst[kCompactMaxPath];   // byte offsets of the rows within (layer, tensor), short of the head's
     __shared__ int s_bad_page;
+    // The launch is serialized programmatically behind the kernel before it in the stream (the verification, as a
+    // rule): the blocks are in place while that kernel finishes, and read what it wrote from here on.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int idx = blockIdx.x;
     const int grp = idx % groups;
     idx /= groups;
@@ -137,11 +141,23 @@ int launch_compact(void *kc, void *vc, const ht_cache_desc &d, const int32_t *kv
     long long groups = (2 * 148 + lb - 1) / lb;
     if (groups < 1) groups = 1;
     if (groups > 2ll * d.Hkv) groups = 2ll * d.Hkv;
-    compact_kernel<<<(unsigned)(lb * groups), kCompactThreads, 0, s>>>(
-        static_cast<unsigned char *>(kc), static_cast<unsigned char *>(vc), d.layers, d.B, d.Hkv, d.cap,
-        d.N, row_bytes, stride_l, stride_b, stride_h, kv_len, accept_len, accept_path, max_path, (int)groups,
-        new_kv_len, status, pm);
-    return check_launch("ht_kv_compact");
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(lb * groups));
+    cfg.blockDim = dim3(kCompactThreads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t le = cudaLaunchKernelEx(&cfg, compact_kernel, static_cast<unsigned char *>(kc), static_cast<unsigned char *>(vc),
+                                              d.layers, d.B, d.Hkv, d.cap, d.N, row_bytes, stride_l, stride_b, stride_h, kv_len,
+                                              accept_len, accept_path, max_path, (int)groups, new_kv_len, status, pm);
+    if (le != cudaSuccess) {
+        cudaGetLastError();
+        return fail(HT_ERR_CUDA, "ht_kv_compact: %s", cudaGetErrorString(le));
+    }
+    return HT_OK;
 }
 
 }  // namespace ht

@@ -35,6 +35,8 @@ template <typename T, int R, int BT, int U>
 __global__ void __launch_bounds__(128, kTransferBlocksPerSm)
 transfer_kernel(const T *__restrict__ h, const T *__restrict__ W, T *__restrict__ out,
                 int rows_total, int d, int b0, int nb) {
+    // lets a kernel that is serialized programmatically behind this one set itself up while this one runs
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     constexpr int VE = Vec16<T>::n;
     constexpr int BC = BT < 4 ? BT : 4;              // batch columns handled per pass over the loaded weights
     const int lane = threadIdx.x & 31;
@@ -166,6 +168,8 @@ __global__ void __launch_bounds__(128, kTransferBlocksPerSm)
 transfer_mma_kernel(const T *__restrict__ h, const T *__restrict__ W, T *__restrict__ out,
                     int rows_total, int d, int b0, int nb, int S) {
     __shared__ float s_part[kSplit ? 4 : 1][NB * 4][32];
+    // lets a kernel that is serialized programmatically behind this one set itself up while this one runs
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
     const int groups = (rows_total + 15) / 16;
     const int items = groups * S;

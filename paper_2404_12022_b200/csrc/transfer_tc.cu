@@ -65,6 +65,8 @@ template <bool kBf16, int kMT>           // kMT = p.mt: 128-row tiles of h per C
 __global__ void __launch_bounds__(kTThreads, 1)
 transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_h_tail, const __grid_constant__ CUtensorMap tm_w_tail, const TParams p) {
+    // lets a kernel that is serialized programmatically behind this one set itself up while this one runs
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     extern __shared__ unsigned char smem_raw[];
     unsigned char *base = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     TBars &bar = *reinterpret_cast<TBars *>(base + (size_t)p.stages * p.stage_bytes + (kBM * kMT - p.h_rows) * kBK * 2);

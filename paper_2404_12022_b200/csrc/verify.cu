@@ -123,6 +123,8 @@ verify_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pred, c
               const int32_t *__restrict__ parent, const int32_t *__restrict__ root_pred, int N, int Tn, int max_path,
               int32_t *__restrict__ accept_len, int32_t *__restrict__ accept_path, int32_t *__restrict__ next_token,
               int32_t *__restrict__ status) {
+    // lets a kernel that is serialized programmatically behind this one set itself up while this one runs
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     constexpr int VE = Vec16<T>::n;
     const T *row = logits + (size_t)blockIdx.x * V;
     Best best{-INFINITY, INT_MAX};
