@@ -231,6 +231,8 @@ int ht_verify_greedy(const void *logits, int dtype, const int32_t *tokens, const
  *   status [B] out: HT_STATUS_BAD_LEN / HT_STATUS_BAD_PATH sequences are left unchanged and
  *            new_kv_len[b] = kv_len[b].
  * max_path <= 64.  D * element size must be a multiple of 16 bytes.
+ * The kernel is launched with programmatic stream serialization and waits, at its first instruction, for
+ * the work ahead of it in the stream: ordering is that of an ordinary launch.
  */
 int ht_kv_compact(void *k_cache, void *v_cache, const ht_cache_desc *desc /* host */,
                   const int32_t *kv_len, const int32_t *accept_len, const int32_t *accept_path,
