@@ -320,7 +320,7 @@ def run_native(args):
             "launch": "eager C-ABI calls" if args.eager else "CUDA graph of the step's C-ABI calls"}
     # launches of this library's kernels per step: one per attention call, transfer (one per batch
     # slice of 16), verification (argmax and acceptance in one), compaction
-    line["gpu_launches"] = args.steps * (sum(kernels_per_attention(step, i) for i in range(step.layers)) + ((w.B + 15) // 16) + 1 + 1)
+    line["gpu_launches"] = args.steps * (sum(kernels_per_attention(step, i) for i in range(step.layers)) + ((w.B + 15) // 16) + 2 + 1)    # + transfer, verification (two kernels), compaction
 
     if rank == 0 and not args.no_extras:
         line["roofline"], line["kernels"] = per_kernel_pass(args, step, stream, torch)

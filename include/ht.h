@@ -212,6 +212,9 @@ int ht_kv_compact_paged(void *k_pages, void *v_pages, const ht_cache_desc *desc 
  *   next_token  [B] out: pred at the path's last node; root_pred[b] (or -1 without
  *             root_pred) when nothing is accepted
  *   status    [B] out: HT_STATUS_BAD_TREE, HT_STATUS_PATH_TOO_LONG (accept_len 0, next -1)
+ * Two kernels (one zeroes the per-sequence arrival counters kept in accept_len), both launched with programmatic
+ * stream serialization and waiting, at their first instruction, for the work ahead of them in the stream: ordering
+ * is that of ordinary launches.
  */
 int ht_verify_greedy(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
                      const int32_t *root_pred, int B, int N, int T, int V, int max_path,

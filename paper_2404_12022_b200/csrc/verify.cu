@@ -123,7 +123,10 @@ verify_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pred, c
               const int32_t *__restrict__ parent, const int32_t *__restrict__ root_pred, int N, int Tn, int max_path,
               int32_t *__restrict__ accept_len, int32_t *__restrict__ accept_path, int32_t *__restrict__ next_token,
               int32_t *__restrict__ status) {
-    // lets a kernel that is serialized programmatically behind this one set itself up while this one runs
+    // The launch is serialized programmatically behind the kernel that zeroes the tickets, which itself waits for the
+    // work ahead of it in the stream: from here on everything that work wrote may be read.  A kernel serialized
+    // behind this one (the compaction) may set itself up meanwhile.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     constexpr int VE = Vec16<T>::n;
     const T *row = logits + (size_t)blockIdx.x * V;
@@ -208,29 +211,56 @@ verify_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pred, c
     accept_sequence(b, tokens, parent, root_pred, pred, N, Tn, max_path, accept_len, accept_path, next_token, status);
 }
 
+// accept_len doubles as the per-sequence ticket until the sequence's last block overwrites it: zero at the start.
+// A kernel rather than a memset node, so that the launches chain by programmatic stream serialization: it is in
+// place, waiting, before the kernel ahead of it in the stream has finished.
+__global__ void verify_prepare_kernel(int32_t *accept_len, int B) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (int i = threadIdx.x; i < B; i += blockDim.x) accept_len[i] = 0;
+}
+
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 int launch_verify(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
                   const int32_t *root_pred, int B, int N, int T, int V, int max_path, int32_t *pred,
                   int32_t *accept_len, int32_t *accept_path, int32_t *next_token, int32_t *status,
                   cudaStream_t s) {
-    const int rows = B * N;
-    // accept_len doubles as the per-sequence ticket until the sequence's last block overwrites it
-    const cudaError_t e = cudaMemsetAsync(accept_len, 0, (size_t)B * sizeof(int32_t), s);
-    if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
-    switch (dtype) {
-        case HT_F32:
-            verify_kernel<float><<<rows, 256, 0, s>>>(static_cast<const float *>(logits), V, pred, tokens, parent, root_pred,
-                                                      N, T, max_path, accept_len, accept_path, next_token, status);
-            break;
-        case HT_F16:
-            verify_kernel<__half><<<rows, 256, 0, s>>>(static_cast<const __half *>(logits), V, pred, tokens, parent, root_pred,
-                                                       N, T, max_path, accept_len, accept_path, next_token, status);
-            break;
-        default:
-            verify_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(logits), V, pred, tokens, parent,
-                                                              root_pred, N, T, max_path, accept_len, accept_path, next_token, status);
-            break;
+    const unsigned rows = (unsigned)(B * N);
+    cudaError_t e = launch_chained(verify_prepare_kernel, 1u, 256u, s, accept_len, B);
+    if (e == cudaSuccess) {
+        switch (dtype) {
+            case HT_F32:
+                e = launch_chained(verify_kernel<float>, rows, 256u, s, static_cast<const float *>(logits), V, pred, tokens, parent, root_pred,
+                                   N, T, max_path, accept_len, accept_path, next_token, status);
+                break;
+            case HT_F16:
+                e = launch_chained(verify_kernel<__half>, rows, 256u, s, static_cast<const __half *>(logits), V, pred, tokens, parent, root_pred,
+                                   N, T, max_path, accept_len, accept_path, next_token, status);
+                break;
+            default:
+                e = launch_chained(verify_kernel<__nv_bfloat16>, rows, 256u, s, static_cast<const __nv_bfloat16 *>(logits), V, pred, tokens, parent,
+                                   root_pred, N, T, max_path, accept_len, accept_path, next_token, status);
+                break;
+        }
     }
-    return check_launch("ht_verify_greedy");
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(HT_ERR_CUDA, "ht_verify_greedy: %s", cudaGetErrorString(e));
+    }
+    return HT_OK;
 }
 
 }  // namespace ht
