@@ -20,6 +20,8 @@ rope_kv_append_kernel(const T *__restrict__ q_in, const T *__restrict__ k_in, co
                       const int32_t *__restrict__ pos, const int32_t *__restrict__ kv_len, double log2_base,
                       T *__restrict__ q_out, T *__restrict__ k_cache, T *__restrict__ v_cache, int N, int Hq, int Hkv,
                       int cap, long long stride_b, long long stride_h, int32_t *__restrict__ status, const PageMap pm) {
+    // lets a kernel that is serialized programmatically behind this one (the attention call) set itself up meanwhile
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     constexpr int VE = Vec16<T>::n, HALF = D / 2, VPH = HALF / VE;     // 16-byte vectors per half row
     __shared__ float s_cos[HALF], s_sin[HALF];
     const int b = blockIdx.x / N, r = blockIdx.x - b * N;
