@@ -234,6 +234,9 @@ int ht_verify_greedy(const void *logits, int dtype, const int32_t *tokens, const
  *   status [B] out: HT_STATUS_BAD_LEN / HT_STATUS_BAD_PATH sequences are left unchanged and
  *            new_kv_len[b] = kv_len[b].
  * max_path <= 64.  D * element size must be a multiple of 16 bytes.
+ * new_kv_len must not overlap kv_len or accept_len (HT_ERR_INVALID_ARG): the sequence's thread blocks
+ * read both throughout the kernel, so an update in place would be seen by some of them and not by
+ * others.  Keep two length arrays and swap them between rounds.
  * The kernel is launched with programmatic stream serialization and waits, at its first instruction, for
  * the work ahead of it in the stream: ordering is that of an ordinary launch.
  */
@@ -303,8 +306,10 @@ int ht_rope_kv_append(const ht_attn_desc *desc /* host */, const void *q_in, con
  *   - A problem whose partials exceed the array is refused with HT_ERR_WORKSPACE and a
  *     message giving both sizes; desc->num_splits = 1 never needs scratch.
  *   - The first call on each device looks up the array's device address (with the caller's
- *     current device, which must be the one the pointers and the stream belong to).  Make
- *     that first call outside any stream capture.
+ *     current device, which must be the one the pointers and the stream belong to; a q on
+ *     another device is refused with HT_ERR_INVALID_ARG).  Make that first call outside any
+ *     stream capture.  The address is kept for the life of the process: after
+ *     cudaDeviceReset the library's per-device state is stale and the process must reload it.
  *   - All calls share the array and it keeps the previous call's contents.  Nothing in it
  *     needs clearing, but calls that overlap on the GPU (two streams, two host threads)
  *     race on it: serialise them.

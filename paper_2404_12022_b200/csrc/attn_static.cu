@@ -67,6 +67,16 @@ extern "C" int ht_tree_attention_static(const ht_attn_desc *desc, const void *q,
                     "this problem needs %zu bytes of split scratch but the built-in scratch holds %zu: "
                     "lower num_splits (1 needs none) or call ht_tree_attention with a workspace",
                     need, (size_t)HT_STATIC_SCRATCH_BYTES);
+    // The array's address is looked up for the current device: the buffers must live there too (a kernel given
+    // another device's address would write through it into the wrong memory).
+    int dev = -1;
+    cudaPointerAttributes attr;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaPointerGetAttributes(&attr, q) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(HT_ERR_CUDA, "cannot tell which device the current one is, or which one holds q");
+    }
+    if (attr.type == cudaMemoryTypeDevice && attr.device != dev)
+        return fail(HT_ERR_INVALID_ARG, "q lives on device %d but device %d is current: make the buffers' device current", attr.device, dev);
     void *scratch = nullptr;
     rc = scratch_address(&scratch);
     if (rc != HT_OK) return rc;

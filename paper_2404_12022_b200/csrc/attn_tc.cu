@@ -36,10 +36,58 @@
 // Every wait on an mbarrier is bounded; when one runs out the CTA raises an abort flag,
 // reports HT_STATUS_TIMEOUT, runs to the end of its control flow without further waiting,
 // drains its own copies, frees its TMEM and returns.
+#include <stddef.h>
+
 #include "attn_tc.cuh"
 
 namespace ht {
 namespace tc {
+
+// Second softmax pass over the 128 scores of this thread's row: exponentials, row sum (into acc2), P to TMEM
+// as packed 16-bit pairs over scores already consumed.  On entry chunk 0 (32 scores) is on its way into xa.
+// kHiLo = false (tiles of context keys): P chunk c lands in columns [16 c, 16 c + 16).
+// kHiLo = true (tiles with tree keys: a row may see a handful of keys only, and then the rounding of its
+// weights to 16 bits is no longer averaged away): P goes to the tensor pipe as a pair hi + lo of 16-bit
+// values, P V is issued for both; chunk c's hi lands in columns [32 c, 32 c + 16) and its lo = P - hi in
+// [32 c + 16, 32 c + 32), i.e. every chunk's results take the chunk's own columns.
+template <bool kBf16, bool kHiLo>
+__device__ __forceinline__ void softmax_pass2(uint32_t s_addr, float *xa, float *xb, unsigned long long scale2,
+                                              unsigned long long nbase2, unsigned long long &acc2) {
+    constexpr int kStep = kHiLo ? 32 : 16;             // columns a chunk's results take
+    // 32 scores -> 16 packed pairs at column `col`; with kHiLo a second sweep forms the same exponentials again and
+    // stores what the rounding took away (no registers beyond the first sweep's: these tiles are few)
+    auto chunk = [&](const float *x, uint32_t col) {
+        uint32_t r[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+            float p0, p1;
+            unpack_f32x2(fma_f32x2(pack_f32x2(x[2 * c], x[2 * c + 1]), scale2, nbase2), p0, p1);
+            p0 = ex2(p0);
+            p1 = ex2(p1);
+            acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
+            r[c] = pack2<kBf16>(p0, p1);
+        }
+        tmem_st16(col, r);
+        if (kHiLo) {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                float p0, p1;
+                unpack_f32x2(fma_f32x2(pack_f32x2(x[2 * c], x[2 * c + 1]), scale2, nbase2), p0, p1);
+                r[c] = pack2_rest<kBf16>(ex2(p0), ex2(p1), r[c]);
+            }
+            tmem_st16(col + 16, r);
+        }
+    };
+#pragma unroll 1
+    for (int h = 0; h < 2; ++h) {
+        tmem_ld_wait();
+        tmem_ld32(s_addr + (2 * h + 1) * 32, xb);
+        chunk(xa, s_addr + (2 * h) * kStep);
+        tmem_ld_wait();
+        if (h == 0) tmem_ld32(s_addr + 2 * 32, xa);
+        chunk(xb, s_addr + (2 * h + 1) * kStep);
+    }
+}
 
 // kPaged: the cache is a pool of pages (separate instantiations, so that the contiguous kernels carry none of that code).
 // kClustered: launched as clusters (p.cluster_k > 1); a template parameter so that the persistent form carries no cluster code.
@@ -51,7 +99,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &sm.abort;
-    if (threadIdx.x == 0) HT_TR_CTA(0);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&sm.kv_full[i], 1); mbar_init(&sm.kv_empty[i], 1); }
@@ -105,7 +152,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // instruction, instead of one after the other; lane 0 alone arms the barriers and fetches Q.
         if (kPaged || lane == 0) {
             int ring_i = 0, seg_i = 0;
-            if (lane == 0) HT_TR_CTA(1);
             const int n = t_end - t_begin;
             TileCursor cur_k, cur_v, cur_p;          // the K and V streams of the ring order, and the page-id lookahead
             cur_k.init(t_begin, t_end);
@@ -143,7 +189,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                 }
-                HT_TR(0, j, is_v ? 1 : 0);
                 const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
                 if (kPaged && !is_v) {
                     // the ids of tile j were asked for kPgAhead tiles ago; ask for those of tile j + kPgAhead
@@ -183,10 +228,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const uint32_t q_addr = smem_u32(sm.q);
             int b_hint = 0, j = 0, seg_i = 0;
             int prev_first = 0;          // is tile j-1 the first of its stream within its segment?
-            auto issue_pv = [&](int jj, int first) {
+            bool prev_tree = false;      // does tile j-1 hold tree keys?  Its P is then a hi + lo pair (see the softmax)
+            auto issue_pv = [&](int jj, int first, bool tree) {
                 const int s = jj & 1;
                 mbar_wait(&sm.p_ready[s], (jj >> 1) & 1, abort_flag);
-                HT_TR(1, jj, 2);
                 const int e = ring_entry_v(jj, t_end - t_begin), slot = e % kStages;
                 mbar_wait(&sm.kv_full[slot], (e / kStages) & 1, abort_flag);
                 tc_fence_after();
@@ -198,7 +243,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         // line per key), the second 64-feature slab one slab further (LBO), groups of
                         // 8 keys 1 KiB apart (SBO); 16 keys per instruction = 2 KiB.
                         const uint64_t b_desc = smem_desc(v_addr + kk * 2048, kSlabBytes >> 4, 1024 >> 4);
-                        mma_ts(tmem + 256 + s * 128, tmem + s * 128 + kk * 8, b_desc, idesc_pv, (kk > 0 || !first) ? 1u : 0u);
+                        if (!tree) {
+                            mma_ts(tmem + 256 + s * 128, tmem + s * 128 + kk * 8, b_desc, idesc_pv, (kk > 0 || !first) ? 1u : 0u);
+                        } else {
+                            // P as hi + lo: the 16 keys of step kk are the half (kk & 1) of score chunk kk / 2
+                            const uint32_t a_hi = tmem + s * 128 + (kk >> 1) * 32 + (kk & 1) * 8;
+                            mma_ts(tmem + 256 + s * 128, a_hi, b_desc, idesc_pv, (kk > 0 || !first) ? 1u : 0u);
+                            mma_ts(tmem + 256 + s * 128, a_hi + 16, b_desc, idesc_pv, 1u);
+                        }
                     }
                 }
                 tc_commit(&sm.kv_empty[slot]);
@@ -212,7 +264,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     const int e = ring_entry_k(j), slot = e % kStages;
                     mbar_wait(&sm.kv_full[slot], (e / kStages) & 1, abort_flag);
                     tc_fence_after();
-                    HT_TR(1, j, 0);
                     if (!*abort_flag) {
                         const uint32_t k_addr = smem_u32(sm.ring[slot]);
 #pragma unroll
@@ -227,14 +278,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     tc_commit(&sm.s_full[s]);
                     tc_commit(&sm.kv_empty[slot]);
                     if (i == sg.len - 1) tc_commit(&sm.q_empty);
-                    if (j > 0) issue_pv(j - 1, prev_first);
+                    if (j > 0) issue_pv(j - 1, prev_first, prev_tree);
                     prev_first = i < 2;
+                    prev_tree = (sg.kt0 + i + 1) * kTile > sm.len[sg.b];
                     ++j;
                 }
                 t += sg.len;
                 ++seg_i;
             }
-            if (j > 0) issue_pv(j - 1, prev_first);
+            if (j > 0) issue_pv(j - 1, prev_first, prev_tree);
             // No tensor-core operation of this CTA may be in flight when its TMEM is freed.
             tc_commit(&sm.mma_drain);
             mbar_wait(&sm.mma_drain, 0, abort_flag, false);
@@ -305,10 +357,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     delivered_old = delivered;
                     delivered = ld_relaxed_gpu(&p.tickets[cut[cut_k].unit]);
                 }
-                HT_TR(2 + s, jj, 0);
                 mbar_wait(&sm.s_full[s], (jj >> 1) & 1, abort_flag);
                 tc_fence_after();
-                HT_TR(2 + s, jj, 1);
                 const uint32_t s_addr = tmem + lane_base + s * 128;
                 const int tile_lo = kt * kTile;
                 float *const xa = xa_e, *const xb = xb_e;
@@ -356,7 +406,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     }
                 }
                 const float mx = fmaxf(mx0, mx1) * p.scale_log2;   // scale > 0: max commutes with scaling
-                HT_TR(2 + s, jj, 2);
                 // --- running maximum, raised lazily ---
                 const float m_new = fmaxf(m_ref, mx);
                 const bool grow = (m_ref != -INFINITY) && (m_new > m_ref + kRescaleThreshold);
@@ -385,34 +434,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 // in columns [16 c, 16 c + 16), which hold scores already consumed. ---
                 const unsigned long long nbase2 = pack_f32x2(-base, -base);
                 unsigned long long acc2 = pack_f32x2(0.f, 0.f);
-#pragma unroll 1
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t r[16];
-                    tmem_ld_wait();
-                    tmem_ld32(s_addr + (2 * h + 1) * 32, xb);
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        float p0, p1;
-                        unpack_f32x2(fma_f32x2(pack_f32x2(xa[2 * c], xa[2 * c + 1]), scale2, nbase2), p0, p1);
-                        p0 = ex2(p0);
-                        p1 = ex2(p1);
-                        acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
-                        r[c] = pack2<kBf16>(p0, p1);
-                    }
-                    tmem_st16(s_addr + (2 * h) * 16, r);
-                    tmem_ld_wait();
-                    if (h == 0) tmem_ld32(s_addr + 2 * 32, xa);
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        float p0, p1;
-                        unpack_f32x2(fma_f32x2(pack_f32x2(xb[2 * c], xb[2 * c + 1]), scale2, nbase2), p0, p1);
-                        p0 = ex2(p0);
-                        p1 = ex2(p1);
-                        acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
-                        r[c] = pack2<kBf16>(p0, p1);
-                    }
-                    tmem_st16(s_addr + (2 * h + 1) * 16, r);
-                }
+                if (tile_lo + kTile > L) softmax_pass2<kBf16, true>(s_addr, xa, xb, scale2, nbase2, acc2);
+                else softmax_pass2<kBf16, false>(s_addr, xa, xb, scale2, nbase2, acc2);
                 {
                     float a0, a1;
                     unpack_f32x2(acc2, a0, a1);
@@ -435,7 +458,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     }
                 }
                 tc_fence_before();
-                HT_TR(2 + s, jj, 3);
                 mbar_arrive(&sm.p_ready[s]);
                 ++n_mine;
                 last_jj = jj;
@@ -445,7 +467,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 mbar_wait(&sm.o_done[s], (last_jj >> 1) & 1, abort_flag);
                 tc_fence_after();
             }
-            HT_TR(4, J, 0);
             sm.ml[s][row][0] = m_ref;
             sm.ml[s][row][1] = l_sum;
             // With one other part and that part already in the workspace, this CTA finishes the unit
@@ -558,11 +579,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     ticket[cut_k] = atomicAdd(&p.tickets[cut[cut_k].unit], 1u);
                 }
             }
-            HT_TR(4, J, 1);
             J += sg.len;
             t += sg.len;
         }
-        if (tid256 == 0) HT_TR_CTA(2);
         if (clustered) {
             if (t_end <= t_begin) {                    // an empty share still delivers a part: nothing seen
                 cluster_sync_all();
@@ -591,7 +610,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     tc_fence_before();
     __syncthreads();
     // (cluster mode: the exchange's second barrier already guarantees that no peer writes here any more)
-    if (threadIdx.x == 0) HT_TR_CTA(3);
     if (sm.abort && threadIdx.x == 0) {
         for (int b = 0; b < p.B; ++b)
             if (sm.nkt[b] > 0) p.status[b] = HT_STATUS_TIMEOUT;
@@ -729,10 +747,6 @@ static int make_map(CUtensorMap *map, const void *base, int dtype, const cuuint6
     return HT_OK;
 }
 
-#ifdef HT_TC_TRACE
-static long long *g_trace = nullptr;
-extern "C" void ht_set_trace(void *ptr) { g_trace = static_cast<long long *>(ptr); }
-#endif
 
 int launch_attn_tc_pair_kernel(const CUtensorMap &tm_q, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const tc::Params &p,
                                const tc::PagedParams &pp, bool bf16, bool paged, cudaStream_t s);
@@ -792,10 +806,7 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     while (pages && (1 << pp.page_shift) < pages->page_size) ++pp.page_shift;
     pp.max_pages = pages ? pages->max_pages : 0;
     pp.n_pages = pages ? pages->n_pages : 0;
-#ifdef HT_TC_TRACE
-    p.trace = g_trace;
-#endif
-    const size_t smem = sizeof(tc::Smem) + 1024;
+    const size_t smem = offsetof(tc::Smem, anc) + (size_t)((d.N + 31) / 32) * tc::kRows * sizeof(uint32_t) + 1024;
     const long long units = (long long)d.B * d.Hkv * p.n_rt;
     if (units > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "too many (sequence, head, row tile) units");
     const int k = cluster_size(d);
@@ -823,7 +834,7 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
         p.grid = (int)units * k;
     }
     if (pair_mode(d)) return launch_attn_tc_pair_kernel(tm_q, tm_k, tm_v, p, pp, d.dtype == HT_BF16, pages != nullptr, s);
-    e = ensure_smem_attr(smem);
+    e = ensure_smem_attr(sizeof(tc::Smem) + 1024);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     // Few (sequence, KV head) units: one cluster of 8, 4 or 2 CTAs per unit, parts reduced through
     // distributed shared memory; otherwise one persistent CTA per SM.  Either way the launch is serialized

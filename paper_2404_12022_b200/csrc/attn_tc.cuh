@@ -16,7 +16,7 @@ constexpr int kEntryBytes = kTile * kD * 2;
 constexpr int kSlabBytes = kEntryBytes / 2;   // [128 rows][64 elements] = 16 KiB
 constexpr int kThreads = 320;
 constexpr int kMaxB = 256;
-constexpr int kMaxWords = 16;              // ancestor words per row -> N <= 512
+constexpr int kMaxWords = 32;              // ancestor words per row -> N <= 1024
 constexpr int kSlotFloats = kRows * kD + 2 * kRows;   // one partial result: O as [32 feature groups][128 rows][4], m[128], l[128]
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;  // log2 domain
@@ -36,9 +36,6 @@ struct Params {
     int is_bf16;
     int grid;
     int cluster_k;         // > 1: launched as clusters of this many CTAs, one cluster per (sequence, KV head)
-#ifdef HT_TC_TRACE
-    long long *trace;
-#endif
 };
 
 // Paged cache: cache row r of sequence b is row r % page_size of page block_table[b * max_pages + r / page_size];
@@ -49,19 +46,9 @@ struct PagedParams {
     int page_size, page_shift, max_pages, n_pages;      // page_size = 1 << page_shift
 };
 
-// Optional timeline of one CTA (clock64 stamps per role / tile / event) for tuning builds.
-#ifdef HT_TC_TRACE
-#define HT_TR(role, j, ev) do { if (p.trace && blockIdx.x == HT_TC_TRACE && (threadIdx.x & 31) == 0 && ((role) < 2 || (threadIdx.x & 127) == 0) && (j) < 40) p.trace[((role) * 40 + (j)) * 4 + (ev)] = clock64(); } while (0)
-#define HT_TR_CTA(ev) do { if (p.trace && (threadIdx.x & 31) == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); p.trace[1000 + blockIdx.x * 4 + (ev)] = (long long)gt; } } while (0)
-#else
-#define HT_TR(role, j, ev) do { } while (0)
-#define HT_TR_CTA(ev) do { } while (0)
-#endif
-
 struct __align__(1024) Smem {
     unsigned char q[kEntryBytes];
     unsigned char ring[kStages][kEntryBytes];
-    uint32_t anc[kMaxWords][kRows];
     int32_t parent[kMaxWords * 32];
     float ml[2][kRows][2];
     int32_t len[kMaxB];
@@ -73,6 +60,7 @@ struct __align__(1024) Smem {
     int merge_here[2];
     int direct;
     int32_t pg[kPgTiles][kPgSub];      // paged cache: page ids of the tiles about to be fetched
+    uint32_t anc[kMaxWords][kRows];    // ancestor words of the tile's rows; last member: only ceil(N / 32) words are allocated
 };
 
 // ---------------------------------------------------------------------------------------
@@ -442,6 +430,22 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
         __half2 v = __floats2half2_rn(lo, hi);
         return *reinterpret_cast<uint32_t *>(&v);
     }
+}
+
+// What rounding (lo, hi) to the packed 16-bit word w took away, rounded likewise:
+// value = w + rest to about 2^-17 (bf16) / 2^-22 (fp16) of the value.
+template <bool kBf16>
+__device__ __forceinline__ uint32_t pack2_rest(float lo, float hi, uint32_t w) {
+    float wl, wh;
+    if (kBf16) {
+        wl = __uint_as_float(w << 16);
+        wh = __uint_as_float(w & 0xFFFF0000u);
+    } else {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w));
+        wl = f.x;
+        wh = f.y;
+    }
+    return pack2<kBf16>(lo - wl, hi - wh);
 }
 
 // A unit that was cut between CTAs: which one, and which CTAs hold its parts.

@@ -17,6 +17,8 @@
 //   - a unit (sequence, KV head, tile pair) whose second tile does not exist runs with stream 1 idle.
 // Work split, cut units, tickets and merges are those of the one-tile kernel; a workspace slot
 // holds one part per stream.  Every wait is bounded.
+#include <stddef.h>
+
 #include "attn_tc.cuh"
 
 namespace ht {
@@ -96,7 +98,6 @@ __device__ __noinline__ void cluster_merge_pair(const Params &p, const unsigned 
 struct __align__(1024) PSmem {
     unsigned char q[2][kEntryBytes];
     unsigned char ring[kPStages][kEntryBytes];
-    uint32_t anc[2][kMaxWords][kRows];
     int32_t parent[kMaxWords * 32];
     int32_t len[kMaxB];
     int32_t nkt[kMaxB];
@@ -107,6 +108,7 @@ struct __align__(1024) PSmem {
     int merge_here[2];
     int direct;
     int32_t pg[kPgTiles][kPgSub];      // paged cache: page ids of the tiles about to be fetched
+    uint32_t anc[2 * kMaxWords * kRows];   // ancestor words [stream][word][row]; last member: only 2 * ceil(N / 32) words are allocated
 };
 
 template <bool kBf16, bool kPaged>
@@ -206,7 +208,6 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     bool ok = use == 0 || mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag);
                     if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) { stop = true; break; }
-                    HT_TR(0, ring_i >> 1, ring_i & 1);
                     const CUtensorMap *tm = (i & 1) ? &tm_v : &tm_k;
                     const int jt = t - t_begin + (i >> 1);            // tile of this CTA's range
                     if (kPaged && !(i & 1)) {
@@ -252,13 +253,13 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             int b_hint = 0, j = 0, seg_i = 0;
             uint32_t uses[2] = {0, 0};                      // completed uses of p_ready[s][h]
             bool pend = false, pend_first = false;          // the half tile whose P V is still to be issued
+            bool pend_tree = false;                         // it holds tree keys: its P is a hi + lo pair (see the softmax)
             int pend_j = 0, pend_h = 0;
             auto issue_pv = [&]() {
                 const int e = 2 * pend_j + 1, slot = e % kPStages;
                 mbar_wait(&sm.kv_full[slot], (e / kPStages) & 1, abort_flag);
                 mbar_wait(&sm.p_ready[s][pend_h], uses[pend_h] & 1, abort_flag);
                 ++uses[pend_h];
-                if (s == 0) HT_TR(1, pend_j, 2 + pend_h);
                 tc_fence_after();
                 if (!*abort_flag) {
                     const uint32_t v_addr = smem_u32(sm.ring[slot]) + pend_h * (kHalf * 128);
@@ -270,6 +271,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         const uint64_t b_desc = smem_desc(v_addr + kk * 2048, kSlabBytes >> 4, 1024 >> 4);
                         mma_ts(tmem + 256 + s * 128, tmem + s * 128 + pend_h * kHalf + kk * 8, b_desc, idesc_pv,
                                (kk > 0 || !pend_first) ? 1u : 0u);
+                        if (pend_tree) mma_ts(tmem + 256 + s * 128, tmem + s * 128 + pend_h * kHalf + 32 + kk * 8, b_desc, idesc_pv, 1u);
                     }
                 }
                 tc_commit(&sm.o_done[s][pend_h]);
@@ -296,7 +298,6 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         continue;
                     }
                     for (int h = 0; h < 2; ++h) {
-                        if (s == 0) HT_TR(1, j, h);
                         if (!*abort_flag) {
                             const uint32_t k_addr = smem_u32(sm.ring[slot]) + h * (kHalf * 128);
 #pragma unroll
@@ -316,6 +317,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         if (pend) issue_pv();
                         pend = true;
                         pend_first = (i == 0 && h == 0);
+                        pend_tree = (sg.kt0 + i) * kTile + (h + 1) * kHalf > sm.len[sg.b];
                         pend_j = j;
                         pend_h = h;
                     }
@@ -360,9 +362,9 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 softmax_groups_sync();                 // previous segment no longer reads parent / anc
                 for (int c = tid256; c < p.N; c += 256) sm.parent[c] = p.parent[(size_t)sg.b * p.N + c];
                 softmax_groups_sync();
-                for (int w = 0; w < words; ++w) sm.anc[s][w][row] = 0u;   // padding rows see the context only; their results are dropped
+                for (int w = 0; w < words; ++w) sm.anc[(s * words + w) * kRows + row] = 0u;   // padding rows see the context only; their results are dropped
                 if (real)
-                    for (int c = node; c >= 0; c = sm.parent[c]) sm.anc[s][c >> 5][row] |= 1u << (c & 31);
+                    for (int c = node; c >= 0; c = sm.parent[c]) sm.anc[(s * words + (c >> 5)) * kRows + row] |= 1u << (c & 31);
                 softmax_groups_sync();
                 anc_b = sg.b;
                 anc_rt = sg.rt;
@@ -391,10 +393,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         delivered_old = delivered;
                         delivered = ld_relaxed_gpu(&p.tickets[cut[cut_k].unit]);
                     }
-                    if (h == 0) HT_TR(2 + s, J + i, 0);
                     mbar_wait(&sm.s_full[s][h], uses_s[h] & 1, abort_flag);
                     ++uses_s[h];
-                    HT_TR(2 + s, J + i, 1 + h);
                     tc_fence_after();
                     const uint32_t s_addr = tmem + lane_base + s * 128 + h * kHalf;
                     const int key_lo = kt * kTile + h * kHalf;
@@ -407,8 +407,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                             const int cc0 = key_lo + 32 * w - L;
                             if (cc0 <= -32) continue;
                             const int wi = cc0 >> 5, sh = cc0 & 31;
-                            const uint32_t lo = wi < 0 ? 0xFFFFFFFFu : (wi < words ? sm.anc[s][wi][row] : 0u);
-                            const uint32_t hi = (wi + 1 >= 0 && wi + 1 < words) ? sm.anc[s][wi + 1][row] : 0u;
+                            const uint32_t lo = wi < 0 ? 0xFFFFFFFFu : (wi < words ? sm.anc[(s * words + wi) * kRows + row] : 0u);
+                            const uint32_t hi = (wi + 1 >= 0 && wi + 1 < words) ? sm.anc[(s * words + wi + 1) * kRows + row] : 0u;
                             const uint32_t vis = __funnelshift_r(lo, hi, sh);
                             tmem_ld32(s_addr + w * 32, xa);
                             tmem_ld_wait();
@@ -465,12 +465,18 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     // --- pass 2: exponentials, row sum, P as packed 16-bit pairs over the consumed scores ---
                     const unsigned long long nbase2 = pack_f32x2(-base, -base);
                     unsigned long long acc2 = pack_f32x2(0.f, 0.f);
-                    {
+                    // 32 scores -> 16 packed pairs at column `col`.  Half tiles with tree keys (a row may see a handful
+                    // of keys only, and then the rounding of its weights to 16 bits is no longer averaged away) send P
+                    // to the tensor pipe as a pair hi + lo of 16-bit values: a second sweep forms the same exponentials
+                    // again and stores what the rounding took away 32 columns further (all 64 scores are in registers,
+                    // so the buffer's upper half is free), and P V is issued for both.
+                    const bool hi_lo = key_lo + kHalf > L;
+                    auto chunk = [&](const float *x, uint32_t col) {
                         uint32_t r[16];
 #pragma unroll
                         for (int c = 0; c < 16; ++c) {
                             float p0, p1;
-                            const unsigned long long x2 = fma_f32x2(pack_f32x2(xa[2 * c], xa[2 * c + 1]), scale2, nbase2);
+                            const unsigned long long x2 = fma_f32x2(pack_f32x2(x[2 * c], x[2 * c + 1]), scale2, nbase2);
                             if ((c & (kPolyEvery - 1)) == kPolyEvery - 1) {
                                 ex2_poly_x2(x2, p0, p1);
                             } else {
@@ -481,23 +487,26 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                             acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
                             r[c] = pack2<kBf16>(p0, p1);
                         }
-                        tmem_st16(s_addr, r);
+                        tmem_st16(col, r);
+                        if (hi_lo) {
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            float p0, p1;
-                            const unsigned long long x2 = fma_f32x2(pack_f32x2(xb[2 * c], xb[2 * c + 1]), scale2, nbase2);
-                            if ((c & (kPolyEvery - 1)) == kPolyEvery - 1) {
-                                ex2_poly_x2(x2, p0, p1);
-                            } else {
-                                unpack_f32x2(x2, p0, p1);
-                                p0 = ex2(p0);
-                                p1 = ex2(p1);
+                            for (int c = 0; c < 16; ++c) {
+                                float p0, p1;
+                                const unsigned long long x2 = fma_f32x2(pack_f32x2(x[2 * c], x[2 * c + 1]), scale2, nbase2);
+                                if ((c & (kPolyEvery - 1)) == kPolyEvery - 1) {
+                                    ex2_poly_x2(x2, p0, p1);
+                                } else {
+                                    unpack_f32x2(x2, p0, p1);
+                                    p0 = ex2(p0);
+                                    p1 = ex2(p1);
+                                }
+                                r[c] = pack2_rest<kBf16>(p0, p1, r[c]);
                             }
-                            acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
-                            r[c] = pack2<kBf16>(p0, p1);
+                            tmem_st16(col + 32, r);
                         }
-                        tmem_st16(s_addr + 16, r);
-                    }
+                    };
+                    chunk(xa, s_addr);
+                    chunk(xb, s_addr + 16);
                     {
                         float a0, a1;
                         unpack_f32x2(acc2, a0, a1);
@@ -521,7 +530,6 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         }
                     }
                     tc_fence_before();
-                    if (h == 1) HT_TR(2 + s, J + i, 3);
                     mbar_arrive(&sm.p_ready[s][h]);
                     ++uses_o[h];                        // the P V of this half will arrive on o_done[s][h]
                     last_h = h;
@@ -686,13 +694,14 @@ int launch_attn_tc_pair_kernel(const CUtensorMap &tm_q, const CUtensorMap &tm_k,
                        tc::attn_tc_pair_kernel<false, true>, tc::attn_tc_pair_kernel<true, true>};
     const Fn fn = fns[(bf16 ? 1 : 0) + (paged ? 2 : 0)];
     static bool done[64];
-    const size_t smem = sizeof(tc::PSmem) + 1024;
+    const size_t smem_max = sizeof(tc::PSmem) + 1024;
+    const size_t smem = offsetof(tc::PSmem, anc) + (size_t)2 * ((p.N + 31) / 32) * tc::kRows * sizeof(uint32_t) + 1024;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
     if (!(dev >= 0 && dev < 64 && done[dev])) {
         for (int i = 0; i < 4 && e == cudaSuccess; ++i)
-            e = cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            e = cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
         if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         if (dev >= 0 && dev < 64) done[dev] = true;
     }

@@ -9,6 +9,12 @@ namespace ht {
 
 static thread_local char g_err[512] = "no error";
 
+// Do the int32 arrays [a, a + n) and [b, b + n) share an element?
+static bool overlap_i32(const int32_t *a, const int32_t *b, long long n) {
+    const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b), len = (uintptr_t)n * sizeof(int32_t);
+    return x < y + len && y < x + len;
+}
+
 int fail(int code, const char *fmt, ...) {
     va_list ap;
     va_start(ap, fmt);
@@ -180,6 +186,8 @@ int ht_kv_compact(void *k_cache, void *v_cache, const ht_cache_desc *desc, const
         return fail(HT_ERR_INVALID_ARG, "cache strides must be multiples of 16 bytes");
     if (2ll * desc->layers * desc->B * desc->Hkv > 0x7fffffffLL)
         return fail(HT_ERR_UNSUPPORTED, "too many (layer, sequence, head) units");
+    if (overlap_i32(new_kv_len, kv_len, desc->B) || overlap_i32(new_kv_len, accept_len, desc->B))
+        return fail(HT_ERR_INVALID_ARG, "new_kv_len must not overlap kv_len or accept_len: every block of a sequence reads them");
     return launch_compact(k_cache, v_cache, *desc, kv_len, accept_len, accept_path, max_path, new_kv_len, status,
                           static_cast<cudaStream_t>(stream));
 }
@@ -278,6 +286,8 @@ int ht_kv_compact_paged(void *k_pages, void *v_pages, const ht_cache_desc *desc,
     if (desc->stride_layer < 0 || (desc->stride_layer * e) % 16) return fail(HT_ERR_INVALID_ARG, "stride_layer must be a multiple of 16 bytes");
     if (2ll * desc->layers * desc->B * desc->Hkv > 0x7fffffffLL)
         return fail(HT_ERR_UNSUPPORTED, "too many (layer, sequence, head) units");
+    if (overlap_i32(new_kv_len, kv_len, desc->B) || overlap_i32(new_kv_len, accept_len, desc->B))
+        return fail(HT_ERR_INVALID_ARG, "new_kv_len must not overlap kv_len or accept_len: every block of a sequence reads them");
     ht_cache_desc d = *desc;
     d.cap = pages->max_pages * pages->page_size;
     return launch_compact(k_pages, v_pages, d, kv_len, accept_len, accept_path, max_path, new_kv_len, status,

@@ -152,6 +152,18 @@ def append_pseudo_rows(parent_tree: np.ndarray, src: int, n_pseudo: int) -> np.n
     return np.concatenate([parent_tree, np.array(extra[:n_pseudo], dtype=np.int32)]).astype(np.int32)
 
 
+def append_pseudo_rows_per_node(parent_tree: np.ndarray, k: int) -> np.ndarray:
+    """Pseudo positions for EVERY tree node (each token of the input gets its pseudo states): behind
+    the T tree rows, node c owns rows T + c k ... T + c k + k - 1; the first hangs off c, each later
+    one off its predecessor.  T (1 + k) rows in all."""
+    T = len(parent_tree)
+    extra = []
+    for c in range(T):
+        for i in range(k):
+            extra.append(c if i == 0 else T + c * k + i - 1)
+    return np.concatenate([parent_tree, np.array(extra, dtype=np.int32)]).astype(np.int32)
+
+
 def node_depths(parent: np.ndarray) -> np.ndarray:
     depth = np.zeros(len(parent), dtype=np.int32)
     for i, p in enumerate(parent):
@@ -252,6 +264,7 @@ class Workload:
     want_len: Optional[List[int]]   # seeded accepted length per sequence (None: drawn 0..4)
     seed: int
     max_path: int = 8
+    per_node: bool = False          # pseudo rows hang off every tree node (P = T k) instead of one source node
 
     @property
     def N(self) -> int:
@@ -300,6 +313,12 @@ def config_c4(B: int = 8, lo: int = 512, hi: int = 8192) -> Workload:
                     5120, 4, 32000, 0.02, 0, True, None, _seed(4))
 
 
+def per_node_variant(w: Workload) -> Workload:
+    """The same configuration with pseudo states for every tree node: P = T k pseudo rows, N = T (1 + k)
+    query rows, and B T source rows for the projection."""
+    return dataclasses.replace(w, name=w.name + "_per_node", P=w.T * w.k, per_node=True)
+
+
 def config_c5(kv: int, T: int, B: int) -> Workload:
     point = [512, 2048, 8192, 32768].index(kv) * 16 + [16, 64, 128, 256].index(T) * 4 + [1, 4, 16].index(B)
     return Workload("c5_gqa70b_kv%d_t%d_b%d" % (kv, T, B), 1, B, 64, 8, 128, "bf16", [kv] * B,
@@ -337,7 +356,7 @@ class Inputs:
     tokens: torch.Tensor             # [B, T] int32
     logits: Optional[torch.Tensor]   # [B, N, V]
     root_pred: Optional[torch.Tensor]
-    h_src: torch.Tensor              # [B, d]
+    h_src: torch.Tensor              # [B, d] ([B T, d] with pseudo rows per node)
     W: Optional[torch.Tensor]        # [k, d, d]
     want_len: List[int]
     planted_path: List[List[int]]
@@ -353,7 +372,7 @@ def make_structure(w: Workload):
         assert len(tree) == w.T
         s = 0 if w.tree in ("binary3", "forest4322") else int(rng.integers(w.T))
         trees.append(tree)
-        parents.append(append_pseudo_rows(tree, s, w.P))
+        parents.append(append_pseudo_rows_per_node(tree, w.k) if w.per_node else append_pseudo_rows(tree, s, w.P))
         tokens.append(draft_tokens(tree, w.V, rng))
         src.append(s)
         want.append(int(w.want_len[b]) if w.want_len is not None else int(rng.integers(0, 5)))
@@ -395,7 +414,7 @@ def make_inputs(w: Workload, device="cpu", with_logits: bool = True, with_transf
             want[b] = len(path)
         if w.use_root_pred:
             root_pred = torch.tensor(rp, dtype=torch.int32, device=device)
-    h_src = normal_tensor(w.seed, 5, (w.B, w.d), device, 1.0, dt)
+    h_src = normal_tensor(w.seed, 5, (w.B * w.T if w.per_node else w.B, w.d), device, 1.0, dt)
     W = normal_tensor(w.seed, 6, (w.k, w.d, w.d), device, w.w_std, dt) if with_transfer else None
     return Inputs(
         w=w, q=q, k_cache=k_cache, v_cache=v_cache,

@@ -64,6 +64,9 @@ def test_host_side_rejections(lib):
     c = hb.CacheDesc(2, 1, 4, 64, 128, hb.HT_BF16, 8, 0, 0, 0)
     assert lib.ht_kv_compact(p, p, ctypes.byref(c), p, p, p, 65, p, p, None) == hb.HT_ERR_INVALID_ARG
     assert lib.ht_kv_compact(None, p, ctypes.byref(c), p, p, p, 8, p, p, None) == hb.HT_ERR_INVALID_ARG
+    assert lib.ht_kv_compact(p, p, ctypes.byref(c), p, p + 64, p + 128, 8, p, p + 192, None) == hb.HT_ERR_INVALID_ARG   # new_kv_len is kv_len
+    assert b"overlap" in lib.ht_last_error_string()
+    assert lib.ht_kv_compact(p, p, ctypes.byref(c), p, p + 64, p + 128, 8, p + 64, p + 192, None) == hb.HT_ERR_INVALID_ARG   # ... is accept_len
     c = hb.CacheDesc(2, 1, 4, 64, 3, hb.HT_BF16, 8, 0, 0, 0)                   # 6-byte rows
     assert lib.ht_kv_compact(p, p, ctypes.byref(c), p, p, p, 8, p, p, None) == hb.HT_ERR_UNSUPPORTED
 

@@ -6,7 +6,10 @@ inside the library.  The test calls it through the C ABI twice in a row, on diff
 inputs, so that the second call runs on an array still holding the first call's partials,
 and compares each result with what ``ht_tree_attention`` returns for the same inputs.
 Both run the same kernel, so the results must agree to well within the parity tolerance
-(1e-5 for fp32, 2e-3 + 1e-2 |ref| for bf16); sizes beyond the array must be refused.
+(1e-5 for fp32, 2e-3 + 1e-2 |ref| for bf16); each result is also held to the CPU oracle at
+that tolerance.  The second call must leave the device's free memory as it found it, must
+flag an illegal tree and a length that does not fit like the ordinary entry point does, and
+sizes beyond the array must be refused.
 """
 import numpy as np
 import pytest
@@ -33,22 +36,41 @@ def test_static_scratch_entry_point_matches_the_workspace_one_twice_in_a_row():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from paper_2404_12022_b200 import binding as hb
+    from oracle import ht_oracle
+    ht_oracle.build()
     cases = [(101, torch.float32, 2, 37, 4, 2, 64, [513, 64], 640, 4),
              (102, torch.bfloat16, 1, 91, 8, 8, 128, [1000], 1152, 3)]
-    for seed, dtype, B, N, Hq, Hkv, D, lens, cap, splits in cases:
+    for i, (seed, dtype, B, N, Hq, Hkv, D, lens, cap, splits) in enumerate(cases):
         q, k, v, kv_len, parent = _case(seed, dtype, B, N, Hq, Hkv, D, lens, cap)
         ref, st_ref = hb.tree_attention(q, k, v, kv_len, parent, num_splits=splits,
                                         flags=hb.HT_ATTN_FORCE_SIMT)
         out = torch.empty_like(q)
         status = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         hb.tree_attention_static(q, k, v, kv_len, parent, out=out, status=status, num_splits=splits)
         torch.cuda.synchronize()
+        if i > 0:                       # the first call may load the kernels' code; the second allocates nothing
+            assert torch.cuda.mem_get_info()[0] == free_before
         assert status.cpu().tolist() == st_ref.cpu().tolist() == [0] * B
-        err = (out.float() - ref.float()).abs()
-        if dtype == torch.float32:
-            assert float(err.max()) <= 1e-5
-        else:
-            assert bool((err <= 2e-3 + 1e-2 * ref.float().abs()).all())
+        want = ht_oracle.tree_attention(q.float().cpu().numpy(), k.float().cpu().numpy(), v.float().cpu().numpy(),
+                                        kv_len.cpu().numpy(), parent.cpu().numpy())
+        for other in (ref.float().cpu().numpy().astype(np.float64), want):
+            err = np.abs(out.float().cpu().numpy() - other)
+            if dtype == torch.float32:
+                assert float(err.max()) <= 1e-5
+            else:
+                assert bool((err <= 2e-3 + 1e-2 * np.abs(other)).all())
+    # sequences only the device can find fault with are skipped and flagged, their rows left alone
+    q, k, v, kv_len, parent = _case(104, torch.float32, 3, 9, 4, 2, 64, [10, 20, 30], 64)
+    parent[1, 4] = 4
+    kv_len[2] = 60
+    out = torch.full_like(q, 7.0)
+    out, status = hb.tree_attention_static(q, k, v, kv_len, parent, out=out, num_splits=2)
+    ref, st_ref = hb.tree_attention(q, k, v, kv_len, parent, out=torch.full_like(q, 7.0), num_splits=2, flags=hb.HT_ATTN_FORCE_SIMT)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == st_ref.cpu().tolist() == [hb.HT_STATUS_OK, hb.HT_STATUS_BAD_TREE, hb.HT_STATUS_BAD_LEN]
+    assert bool((out[1:] == 7.0).all()) and float((out[0] - ref[0]).abs().max()) <= 1e-5
     # a problem whose partials do not fit in the built-in array is refused, not truncated
     q, k, v, kv_len, parent = _case(103, torch.float32, 4, 200, 16, 16, 128, [300] * 4, 512)
     with pytest.raises(hb.HtError) as e:
