@@ -54,28 +54,38 @@ template <bool kBf16, bool kHiLo>
 __device__ __forceinline__ void softmax_pass2(uint32_t s_addr, float *xa, float *xb, unsigned long long scale2,
                                               unsigned long long nbase2, unsigned long long &acc2) {
     constexpr int kStep = kHiLo ? 32 : 16;             // columns a chunk's results take
-    // 32 scores -> 16 packed pairs at column `col`; with kHiLo a second sweep forms the same exponentials again and
-    // stores what the rounding took away (no registers beyond the first sweep's: these tiles are few)
+    // 32 scores -> 16 packed pairs at column `col`; with kHiLo eight pairs at a time, each with what its rounding
+    // took away (few registers: these tiles share the hot loop's allocation)
     auto chunk = [&](const float *x, uint32_t col) {
-        uint32_t r[16];
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-            float p0, p1;
-            unpack_f32x2(fma_f32x2(pack_f32x2(x[2 * c], x[2 * c + 1]), scale2, nbase2), p0, p1);
-            p0 = ex2(p0);
-            p1 = ex2(p1);
-            acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
-            r[c] = pack2<kBf16>(p0, p1);
-        }
-        tmem_st16(col, r);
-        if (kHiLo) {
+        if (!kHiLo) {
+            uint32_t r[16];
 #pragma unroll
             for (int c = 0; c < 16; ++c) {
                 float p0, p1;
                 unpack_f32x2(fma_f32x2(pack_f32x2(x[2 * c], x[2 * c + 1]), scale2, nbase2), p0, p1);
-                r[c] = pack2_rest<kBf16>(ex2(p0), ex2(p1), r[c]);
+                p0 = ex2(p0);
+                p1 = ex2(p1);
+                acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
+                r[c] = pack2<kBf16>(p0, p1);
             }
-            tmem_st16(col + 16, r);
+            tmem_st16(col, r);
+        } else {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t r[8], r_lo[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    float p0, p1;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(x[16 * half + 2 * c], x[16 * half + 2 * c + 1]), scale2, nbase2), p0, p1);
+                    p0 = ex2(p0);
+                    p1 = ex2(p1);
+                    acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
+                    r[c] = pack2<kBf16>(p0, p1);
+                    r_lo[c] = pack2_rest<kBf16>(p0, p1, r[c]);
+                }
+                tmem_st8(col + half * 8, r);
+                tmem_st8(col + 16 + half * 8, r_lo);
+            }
         }
     };
 #pragma unroll 1
@@ -223,64 +233,65 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
     } else if (warp == 9) {
         // ------------------------------- MMA issuer -------------------------------
+        // One thread: a chain of dependent instructions that shares its scheduler with two softmax warps, so the
+        // instructions per tile are kept few: ring slots and phases are counted (no division), barrier addresses
+        // and descriptor words are formed once, each product is one instruction sequence, and the abort flag is
+        // looked at only when a wait has to spin.
         if (lane == 0) {
             const uint32_t idesc_qk = instr_desc(kBf16, 0), idesc_pv = instr_desc(kBf16, 1);
-            const uint32_t q_addr = smem_u32(sm.q);
+            const uint32_t hi_k = desc_hi(1, 1024 >> 4), hi_v = desc_hi(kSlabBytes >> 4, 1024 >> 4);
+            const uint32_t q_lo = desc_lo_with_lbo(smem_u32(sm.q), 1);
+            const uint32_t ring_k_lo = desc_lo_with_lbo(smem_u32(sm.ring[0]), 1);            // slot x: + x * (kEntryBytes / 16)
+            const uint32_t ring_v_lo = desc_lo_with_lbo(smem_u32(sm.ring[0]), kSlabBytes >> 4);
+            const uint32_t bar_kv_full = smem_u32(&sm.kv_full[0]), bar_kv_empty = smem_u32(&sm.kv_empty[0]);
+            const uint32_t bar_s_full = smem_u32(&sm.s_full[0]), bar_p_ready = smem_u32(&sm.p_ready[0]), bar_o_done = smem_u32(&sm.o_done[0]);
+            const int n = t_end - t_begin;
             int b_hint = 0, j = 0, seg_i = 0;
             int prev_first = 0;          // is tile j-1 the first of its stream within its segment?
             bool prev_tree = false;      // does tile j-1 hold tree keys?  Its P is then a hi + lo pair (see the softmax)
-            auto issue_pv = [&](int jj, int first, bool tree) {
-                const int s = jj & 1;
-                mbar_wait(&sm.p_ready[s], (jj >> 1) & 1, abort_flag);
-                const int e = ring_entry_v(jj, t_end - t_begin), slot = e % kStages;
-                mbar_wait(&sm.kv_full[slot], (e / kStages) & 1, abort_flag);
-                tc_fence_after();
-                if (!*abort_flag) {
-                    const uint32_t v_addr = smem_u32(sm.ring[slot]);
-#pragma unroll
-                    for (int kk = 0; kk < kTile / 16; ++kk) {
-                        // V tile as B operand, MN-major: 64 features contiguous (one swizzled 128-byte
-                        // line per key), the second 64-feature slab one slab further (LBO), groups of
-                        // 8 keys 1 KiB apart (SBO); 16 keys per instruction = 2 KiB.
-                        const uint64_t b_desc = smem_desc(v_addr + kk * 2048, kSlabBytes >> 4, 1024 >> 4);
-                        if (!tree) {
-                            mma_ts(tmem + 256 + s * 128, tmem + s * 128 + kk * 8, b_desc, idesc_pv, (kk > 0 || !first) ? 1u : 0u);
-                        } else {
-                            // P as hi + lo: the 16 keys of step kk are the half (kk & 1) of score chunk kk / 2
-                            const uint32_t a_hi = tmem + s * 128 + (kk >> 1) * 32 + (kk & 1) * 8;
-                            mma_ts(tmem + 256 + s * 128, a_hi, b_desc, idesc_pv, (kk > 0 || !first) ? 1u : 0u);
-                            mma_ts(tmem + 256 + s * 128, a_hi + 16, b_desc, idesc_pv, 1u);
-                        }
-                    }
-                }
-                tc_commit(&sm.kv_empty[slot]);
-                tc_commit(&sm.o_done[s]);
+            bool alive = !*abort_flag;   // false once a wait of this thread has given up: no further waits or products
+            // ring entries in consumption order K_0, K_1, V_0, K_2, V_1, ...: slot and phase of the next K and V entry
+            uint32_t k_slot = 0, k_ph = 0, v_slot = 2 % kStages, v_ph = 0;
+            auto advance = [](uint32_t &slot, uint32_t &ph, uint32_t by) {
+                slot += by;
+                if (slot >= (uint32_t)kStages) { slot -= kStages; ph ^= 1u; }
             };
+            auto issue_pv = [&](int jj, int first, bool tree) {
+                const uint32_t s = jj & 1;
+                alive = alive && mbar_wait_quick(bar_p_ready + s * 8, (jj >> 1) & 1, abort_flag);
+                alive = alive && mbar_wait_quick(bar_kv_full + v_slot * 8, v_ph, abort_flag);
+                tc_fence_after();
+                if (alive) {
+                    // V tile as B operand, MN-major: 64 features contiguous (one swizzled 128-byte line per key), the
+                    // second 64-feature slab one slab further (LBO), groups of 8 keys 1 KiB apart (SBO); 16 keys per
+                    // instruction = 2 KiB.
+                    const uint32_t v_lo = ring_v_lo + v_slot * (kEntryBytes >> 4);
+                    if (!tree) mma_block_pv128(tmem + 256 + s * 128, tmem + s * 128, v_lo, hi_v, idesc_pv, first ? 0u : 1u);
+                    else mma_block_pv128_hilo(tmem + 256 + s * 128, tmem + s * 128, v_lo, hi_v, idesc_pv, first ? 0u : 1u);
+                }
+                tc_commit_addr(bar_kv_empty + v_slot * 8);
+                tc_commit_addr(bar_o_done + s * 8);
+                advance(v_slot, v_ph, jj + 2 == n ? 1 : 2);                  // V entries: 2, 4, ..., 2n - 2, then 2n - 1
+            };
+            if (n == 1) v_slot = 1;                                          // a single tile: K_0, V_0
             for (int t = t_begin; t < t_end;) {
                 const Segment sg = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
-                mbar_wait(&sm.q_full, seg_i & 1, abort_flag);
+                const int L = sm.len[sg.b];
+                alive = alive && mbar_wait_quick(smem_u32(&sm.q_full), seg_i & 1, abort_flag);
                 for (int i = 0; i < sg.len; ++i) {
-                    const int s = j & 1;
-                    const int e = ring_entry_k(j), slot = e % kStages;
-                    mbar_wait(&sm.kv_full[slot], (e / kStages) & 1, abort_flag);
+                    const uint32_t s = j & 1;
+                    alive = alive && mbar_wait_quick(bar_kv_full + k_slot * 8, k_ph, abort_flag);
                     tc_fence_after();
-                    if (!*abort_flag) {
-                        const uint32_t k_addr = smem_u32(sm.ring[slot]);
-#pragma unroll
-                        for (int kk = 0; kk < kD / 16; ++kk) {
-                            // K-major operands: 16 features = 32 bytes inside the 128-byte swizzled
-                            // line; the second 64-feature slab lies one slab further.
-                            const uint32_t off = (kk >> 2) * kSlabBytes + (kk & 3) * 32;
-                            mma_ss(tmem + s * 128, smem_desc(q_addr + off, 1, 1024 >> 4),
-                                   smem_desc(k_addr + off, 1, 1024 >> 4), idesc_qk, kk > 0 ? 1u : 0u);
-                        }
-                    }
-                    tc_commit(&sm.s_full[s]);
-                    tc_commit(&sm.kv_empty[slot]);
+                    // K-major operands: 16 features = 32 bytes inside the 128-byte swizzled line; the second
+                    // 64-feature slab lies one slab further.
+                    if (alive) mma_block_qk(tmem + s * 128, q_lo, ring_k_lo + k_slot * (kEntryBytes >> 4), hi_k, idesc_qk);
+                    tc_commit_addr(bar_s_full + s * 8);
+                    tc_commit_addr(bar_kv_empty + k_slot * 8);
                     if (i == sg.len - 1) tc_commit(&sm.q_empty);
+                    advance(k_slot, k_ph, j == 0 ? 1 : 2);                    // K entries: 0, 1, 3, 5, ...
                     if (j > 0) issue_pv(j - 1, prev_first, prev_tree);
                     prev_first = i < 2;
-                    prev_tree = (sg.kt0 + i + 1) * kTile > sm.len[sg.b];
+                    prev_tree = (sg.kt0 + i + 1) * kTile > L;
                     ++j;
                 }
                 t += sg.len;

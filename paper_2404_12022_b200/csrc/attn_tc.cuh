@@ -99,6 +99,35 @@ __device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, volatile i
     }
 }
 
+// The same wait for the roles that are one thread's chain of dependent instructions (the MMA issuers): the
+// common case -- the phase has completed or completes within the instruction's own suspension -- costs one
+// try_wait and a branch; the abort flag is looked at only once the wait has to spin (out of line).  The caller
+// remembers a false result and stops waiting and issuing from then on.
+static __device__ __noinline__ bool mbar_wait_spin(uint32_t addr, uint32_t parity, volatile int *abort_flag) {
+    long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 2000000000ll) { *abort_flag = 1; return false; }
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait_quick(uint32_t addr, uint32_t parity, volatile int *abort_flag) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+    if (ok) return true;
+    return mbar_wait_spin(addr, parity, abort_flag);
+}
+
 __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, void *bar, int c0, int c1, int c2, int c3) {
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
@@ -169,6 +198,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r) {
         ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
           "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
           "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t *r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -244,6 +278,87 @@ __device__ __forceinline__ uint32_t instr_desc(int is_bf16, int b_mn_major, uint
     const uint32_t fmt = is_bf16 ? 1u : 0u;
     return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)b_mn_major << 16) | ((n >> 3) << 17) |
            ((128u >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------------------
+// Whole products as one instruction sequence.  The MMA-issuing threads are chains of dependent instructions that
+// share their schedulers with the softmax warps, so every instruction between "operands landed" and "products
+// issued" shows in the tile time; here a descriptor costs one 32-bit addition (all descriptors of an operand
+// share their upper word, and the lower word is linear in the shared-memory address).
+// ---------------------------------------------------------------------------------------
+// Lower / upper word of the descriptor smem_desc(addr, lbo16, sbo16).
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr) { return (addr >> 4) & 0x3FFFu; }
+__device__ __forceinline__ uint32_t desc_hi(uint32_t lbo16, uint32_t sbo16) {
+    return (uint32_t)(smem_desc(0, lbo16, sbo16) >> 32);
+}
+// lbo16 sits in the lower word
+__device__ __forceinline__ uint32_t desc_lo_with_lbo(uint32_t addr, uint32_t lbo16) { return desc_lo(addr) | (lbo16 << 16); }
+
+#define HT_MMA_SS_STEP(off, pred) \
+    "add.u32 al, %1, " #off ";\nadd.u32 bl, %2, " #off ";\nmov.b64 a, {al, %3};\nmov.b64 b, {bl, %3};\n" \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %4, " #pred ";\n"
+// S[tmem] = Q K^T over the 128 features: both operands K-major in shared memory (a_lo / b_lo: lower descriptor
+// words of feature 0, lbo included; hi: the shared upper word); 16 features = 2 descriptor units inside a
+// 64-feature slab, the second slab kSlabBytes further.
+__device__ __forceinline__ void mma_block_qk(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc) {
+    asm volatile(
+        "{\n.reg .pred pf, pt;\n.reg .b32 al, bl;\n.reg .b64 a, b;\n"
+        "setp.ne.b32 pf, %0, %0;\nsetp.eq.b32 pt, %0, %0;\n"
+        HT_MMA_SS_STEP(0, pf) HT_MMA_SS_STEP(2, pt) HT_MMA_SS_STEP(4, pt) HT_MMA_SS_STEP(6, pt)
+        HT_MMA_SS_STEP(1024, pt) HT_MMA_SS_STEP(1026, pt) HT_MMA_SS_STEP(1028, pt) HT_MMA_SS_STEP(1030, pt)
+        "}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc) : "memory");
+}
+static_assert(kSlabBytes / 16 == 1024, "slab offset in descriptor units");
+
+#define HT_MMA_TS_STEP(acol, boff, pred) \
+    "add.u32 at, %1, " #acol ";\nadd.u32 bl, %2, " #boff ";\nmov.b64 b, {bl, %3};\n" \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], [at], b, %4, " #pred ";\n"
+// O[tmem] (+)= P V over 64 keys: P from TMEM (16 keys = 8 columns), V MN-major in shared memory (16 keys = 2 KiB
+// = 128 descriptor units).  accumulate = 0 starts the accumulator afresh.
+__device__ __forceinline__ void mma_block_pv64(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p0, pt;\n.reg .b32 at, bl;\n.reg .b64 b;\n"
+        "setp.ne.b32 p0, %5, 0;\nsetp.eq.b32 pt, %0, %0;\n"
+        HT_MMA_TS_STEP(0, 0, p0) HT_MMA_TS_STEP(8, 128, pt) HT_MMA_TS_STEP(16, 256, pt) HT_MMA_TS_STEP(24, 384, pt)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+// ... over 128 keys, P in columns [0, 64) of its buffer.
+__device__ __forceinline__ void mma_block_pv128(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p0, pt;\n.reg .b32 at, bl;\n.reg .b64 b;\n"
+        "setp.ne.b32 p0, %5, 0;\nsetp.eq.b32 pt, %0, %0;\n"
+        HT_MMA_TS_STEP(0, 0, p0) HT_MMA_TS_STEP(8, 128, pt) HT_MMA_TS_STEP(16, 256, pt) HT_MMA_TS_STEP(24, 384, pt)
+        HT_MMA_TS_STEP(32, 512, pt) HT_MMA_TS_STEP(40, 640, pt) HT_MMA_TS_STEP(48, 768, pt) HT_MMA_TS_STEP(56, 896, pt)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+// ... over 128 keys with P as a hi + lo pair: the 16 keys of step kk are the half (kk & 1) of score chunk kk / 2,
+// hi in the chunk's columns [0, 16), lo in [16, 32); both products are issued.
+__device__ __forceinline__ void mma_block_pv128_hilo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p0, pt;\n.reg .b32 at, bl;\n.reg .b64 b;\n"
+        "setp.ne.b32 p0, %5, 0;\nsetp.eq.b32 pt, %0, %0;\n"
+        HT_MMA_TS_STEP(0, 0, p0) HT_MMA_TS_STEP(16, 0, pt) HT_MMA_TS_STEP(8, 128, pt) HT_MMA_TS_STEP(24, 128, pt)
+        HT_MMA_TS_STEP(32, 256, pt) HT_MMA_TS_STEP(48, 256, pt) HT_MMA_TS_STEP(40, 384, pt) HT_MMA_TS_STEP(56, 384, pt)
+        HT_MMA_TS_STEP(64, 512, pt) HT_MMA_TS_STEP(80, 512, pt) HT_MMA_TS_STEP(72, 640, pt) HT_MMA_TS_STEP(88, 640, pt)
+        HT_MMA_TS_STEP(96, 768, pt) HT_MMA_TS_STEP(112, 768, pt) HT_MMA_TS_STEP(104, 896, pt) HT_MMA_TS_STEP(120, 896, pt)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+// ... over 64 keys with P as a hi + lo pair: hi in columns [0, 32) of the half's buffer, lo in [32, 64).
+__device__ __forceinline__ void mma_block_pv64_hilo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p0, pt;\n.reg .b32 at, bl;\n.reg .b64 b;\n"
+        "setp.ne.b32 p0, %5, 0;\nsetp.eq.b32 pt, %0, %0;\n"
+        HT_MMA_TS_STEP(0, 0, p0) HT_MMA_TS_STEP(32, 0, pt) HT_MMA_TS_STEP(8, 128, pt) HT_MMA_TS_STEP(40, 128, pt)
+        HT_MMA_TS_STEP(16, 256, pt) HT_MMA_TS_STEP(48, 256, pt) HT_MMA_TS_STEP(24, 384, pt) HT_MMA_TS_STEP(56, 384, pt)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_commit_addr(uint32_t bar_addr) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_addr) : "memory");
 }
 
 // ---------------------------------------------------------------------------------------

@@ -246,82 +246,88 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // issued.  A tcgen05.commit covers the issuing thread's own operations, so the K / V slots and the
         // Q buffers are released by one arrival from each of the two threads; in a unit without a second
         // tile the thread of stream 1 issues nothing and only keeps step with the ring.
+        // Each thread is a chain of dependent instructions that shares its scheduler with two softmax warps, so the
+        // instructions per half tile are kept few: ring slots and phases are counted (no division), barrier
+        // addresses and descriptor words are formed once, each product is one instruction sequence, and the
+        // abort flag is looked at only when a wait has to spin.
         if (lane == 0) {
             const int s = warp - 9;
             const uint32_t idesc_qk = instr_desc(kBf16, 0, kHalf), idesc_pv = instr_desc(kBf16, 1, 128);
-            const uint32_t q_addr = smem_u32(sm.q[s]);
-            int b_hint = 0, j = 0, seg_i = 0;
-            uint32_t uses[2] = {0, 0};                      // completed uses of p_ready[s][h]
+            const uint32_t hi_k = desc_hi(1, 1024 >> 4), hi_v = desc_hi(kSlabBytes >> 4, 1024 >> 4);
+            const uint32_t q_lo = desc_lo_with_lbo(smem_u32(sm.q[s]), 1);
+            const uint32_t ring_k_lo = desc_lo_with_lbo(smem_u32(sm.ring[0]), 1);            // slot x: + x * (kEntryBytes / 16)
+            const uint32_t ring_v_lo = desc_lo_with_lbo(smem_u32(sm.ring[0]), kSlabBytes >> 4);
+            const uint32_t bar_kv_full = smem_u32(&sm.kv_full[0]), bar_kv_empty = smem_u32(&sm.kv_empty[0]);
+            const uint32_t bar_s_full = smem_u32(&sm.s_full[s][0]), bar_p_ready = smem_u32(&sm.p_ready[s][0]), bar_o_done = smem_u32(&sm.o_done[s][0]);
+            const uint32_t s_tmem = tmem + s * 128, o_tmem = tmem + 256 + s * 128;
+            int b_hint = 0, seg_i = 0;
+            uint32_t uses0 = 0, uses1 = 0;                  // completed uses of p_ready[s][0 / 1]
             bool pend = false, pend_first = false;          // the half tile whose P V is still to be issued
             bool pend_tree = false;                         // it holds tree keys: its P is a hi + lo pair (see the softmax)
-            int pend_j = 0, pend_h = 0;
+            uint32_t pend_h = 0, pend_slot = 0, pend_ph = 0; // ... its half, and the slot and phase of its V tile
+            bool alive = !*abort_flag;                      // false once a wait of this thread has given up: no further waits or products
+            uint32_t slot = 0, ph = 0;                      // ring entries alternate K, V: slot and phase of the next entry
+            auto advance = [&]() {
+                if (++slot == (uint32_t)kPStages) { slot = 0; ph ^= 1u; }
+            };
             auto issue_pv = [&]() {
-                const int e = 2 * pend_j + 1, slot = e % kPStages;
-                mbar_wait(&sm.kv_full[slot], (e / kPStages) & 1, abort_flag);
-                mbar_wait(&sm.p_ready[s][pend_h], uses[pend_h] & 1, abort_flag);
-                ++uses[pend_h];
+                if (pend_h == 0) alive = alive && mbar_wait_quick(bar_kv_full + pend_slot * 8, pend_ph, abort_flag);
+                const uint32_t u = pend_h ? uses1 : uses0;
+                alive = alive && mbar_wait_quick(bar_p_ready + pend_h * 8, u & 1, abort_flag);
+                if (pend_h) ++uses1; else ++uses0;
                 tc_fence_after();
-                if (!*abort_flag) {
-                    const uint32_t v_addr = smem_u32(sm.ring[slot]) + pend_h * (kHalf * 128);
-#pragma unroll
-                    for (int kk = 0; kk < kHalf / 16; ++kk) {
-                        // V as B operand, MN-major: 64 features contiguous per key (one swizzled 128-byte
-                        // line), the second 64-feature slab one slab further (LBO), groups of 8 keys
-                        // 1 KiB apart (SBO); 16 keys per instruction = 2 KiB.
-                        const uint64_t b_desc = smem_desc(v_addr + kk * 2048, kSlabBytes >> 4, 1024 >> 4);
-                        mma_ts(tmem + 256 + s * 128, tmem + s * 128 + pend_h * kHalf + kk * 8, b_desc, idesc_pv,
-                               (kk > 0 || !pend_first) ? 1u : 0u);
-                        if (pend_tree) mma_ts(tmem + 256 + s * 128, tmem + s * 128 + pend_h * kHalf + 32 + kk * 8, b_desc, idesc_pv, 1u);
-                    }
+                if (alive) {
+                    // V as B operand, MN-major: 64 features contiguous per key (one swizzled 128-byte line), the
+                    // second 64-feature slab one slab further (LBO), groups of 8 keys 1 KiB apart (SBO); 16 keys
+                    // per instruction = 2 KiB.
+                    const uint32_t v_lo = ring_v_lo + pend_slot * (kEntryBytes >> 4) + pend_h * (kHalf * 128 >> 4);
+                    if (!pend_tree) mma_block_pv64(o_tmem, s_tmem + pend_h * kHalf, v_lo, hi_v, idesc_pv, pend_first ? 0u : 1u);
+                    else mma_block_pv64_hilo(o_tmem, s_tmem + pend_h * kHalf, v_lo, hi_v, idesc_pv, pend_first ? 0u : 1u);
                 }
-                tc_commit(&sm.o_done[s][pend_h]);
-                if (pend_h == 1) tc_commit(&sm.kv_empty[slot]);
+                tc_commit_addr(bar_o_done + pend_h * 8);
+                if (pend_h == 1) tc_commit_addr(bar_kv_empty + pend_slot * 8);
                 pend = false;
             };
             for (int t = t_begin; t < t_end;) {
                 const Segment sg = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
                 const bool act = s == 0 || 2 * sg.rt + 1 < p.n_row_tiles;
-                mbar_wait(&sm.q_full, seg_i & 1, abort_flag);
+                const int L = sm.len[sg.b];
+                alive = alive && mbar_wait_quick(smem_u32(&sm.q_full), seg_i & 1, abort_flag);
                 for (int i = 0; i < sg.len; ++i) {
-                    const int e = 2 * j, slot = e % kPStages;
-                    mbar_wait(&sm.kv_full[slot], (e / kPStages) & 1, abort_flag);
+                    const uint32_t k_slot = slot;
+                    alive = alive && mbar_wait_quick(bar_kv_full + slot * 8, ph, abort_flag);
                     tc_fence_after();
+                    advance();
+                    const uint32_t v_slot = slot, v_ph = ph;
+                    advance();
                     if (!act) {
                         // keep step with the ring: hand both slots of this tile back once they are loaded
                         if (pend) issue_pv();
-                        tc_commit(&sm.kv_empty[slot]);
+                        tc_commit_addr(bar_kv_empty + k_slot * 8);
                         if (i == sg.len - 1) tc_commit(&sm.q_empty);
-                        const int ev = e + 1, vslot = ev % kPStages;
-                        mbar_wait(&sm.kv_full[vslot], (ev / kPStages) & 1, abort_flag);
-                        tc_commit(&sm.kv_empty[vslot]);
-                        ++j;
+                        alive = alive && mbar_wait_quick(bar_kv_full + v_slot * 8, v_ph, abort_flag);
+                        tc_commit_addr(bar_kv_empty + v_slot * 8);
                         continue;
                     }
-                    for (int h = 0; h < 2; ++h) {
-                        if (!*abort_flag) {
-                            const uint32_t k_addr = smem_u32(sm.ring[slot]) + h * (kHalf * 128);
+                    const int key_hi = (sg.kt0 + i) * kTile + kHalf;        // end of the tile's first half
 #pragma unroll
-                            for (int kk = 0; kk < kD / 16; ++kk) {
-                                // K-major operands: 16 features = 32 bytes inside the 128-byte swizzled
-                                // line; the second 64-feature slab lies one slab further.
-                                const uint32_t off = (kk >> 2) * kSlabBytes + (kk & 3) * 32;
-                                mma_ss(tmem + s * 128 + h * kHalf, smem_desc(q_addr + off, 1, 1024 >> 4),
-                                       smem_desc(k_addr + off, 1, 1024 >> 4), idesc_qk, kk > 0 ? 1u : 0u);
-                            }
-                        }
-                        tc_commit(&sm.s_full[s][h]);
+                    for (int h = 0; h < 2; ++h) {
+                        // K-major operands: 16 features = 32 bytes inside the 128-byte swizzled line; the second
+                        // 64-feature slab lies one slab further.
+                        if (alive) mma_block_qk(s_tmem + h * kHalf, q_lo, ring_k_lo + k_slot * (kEntryBytes >> 4) + h * (kHalf * 128 >> 4), hi_k, idesc_qk);
+                        tc_commit_addr(bar_s_full + h * 8);
                         if (h == 1) {
-                            tc_commit(&sm.kv_empty[slot]);
+                            tc_commit_addr(bar_kv_empty + k_slot * 8);
                             if (i == sg.len - 1) tc_commit(&sm.q_empty);
                         }
                         if (pend) issue_pv();
                         pend = true;
                         pend_first = (i == 0 && h == 0);
-                        pend_tree = (sg.kt0 + i) * kTile + (h + 1) * kHalf > sm.len[sg.b];
-                        pend_j = j;
+                        pend_tree = key_hi + h * kHalf > L;
                         pend_h = h;
+                        pend_slot = v_slot;
+                        pend_ph = v_ph;
                     }
-                    ++j;
                 }
                 t += sg.len;
                 ++seg_i;
