@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--simt", action="store_true", help="force the fp32-ALU attention kernel")
     ap.add_argument("--eager", action="store_true", help="enqueue every library call from the host instead of replaying a CUDA graph of the step")
     ap.add_argument("--no-extras", action="store_true", help="skip e2e, cpu baseline and per-kernel timing")
+    ap.add_argument("--fused", choices=["auto", "on", "off"], default="auto",
+                    help="verification and compaction as one launch (ht_verify_greedy_compact) or as two calls; auto: one launch for few (layer, sequence) pairs")
     ap.add_argument("--sweep", default="", help="instead of the step benchmark, time ht_tree_attention alone on a set of "
                     "workloads and print one JSON line per point: 'configs' (c2, c2 at KV 2048, a c3 layer, c4) or "
                     "'c5' (the 48 grouped-query points) or 'c5-quick' (12 of them); 'transfer' times ht_transfer alone, with a "
@@ -280,7 +282,7 @@ def run_native(args):
 
     w = make_workload(args)
     inp = wl.make_inputs(w, "cuda")
-    step = VerifyStep(inp, num_splits=args.splits, flags=hb.HT_ATTN_FORCE_SIMT if args.simt else 0)
+    step = VerifyStep(inp, num_splits=args.splits, flags=hb.HT_ATTN_FORCE_SIMT if args.simt else 0, fused={"auto": None, "on": True, "off": False}[args.fused])
     stream = torch.cuda.current_stream().cuda_stream
 
     def barrier():
@@ -318,9 +320,9 @@ def run_native(args):
             "vs_baseline": None, "dtype": w.dtype, "data": "synthetic", "config": workload_config(w, world),
             "step_us": ms_step * 1e3, "step_bytes": step_bytes, "clocks": clocks,
             "launch": "eager C-ABI calls" if args.eager else "CUDA graph of the step's C-ABI calls"}
-    # launches of this library's kernels per step: one per attention call, transfer (one per batch
-    # slice of 16), verification (argmax and acceptance in one), compaction
-    line["gpu_launches"] = args.steps * (sum(kernels_per_attention(step, i) for i in range(step.layers)) + ((w.B + 15) // 16) + 2 + 1)    # + transfer, verification (two kernels), compaction
+    # launches of this library's kernels per step: the attention calls' (ht_tree_attention_launches), transfer (one
+    # per batch slice of 16), verification with the compaction in the same launch
+    line["gpu_launches"] = args.steps * (sum(kernels_per_attention(step, i) for i in range(step.layers)) + ((w.B + 15) // 16) + (1 if step.fused else 2))    # + transfer, verification and compaction (one kernel when fused)
 
     if rank == 0 and not args.no_extras:
         line["roofline"], line["kernels"] = per_kernel_pass(args, step, stream, torch)
@@ -349,7 +351,7 @@ def per_kernel_pass(args, step, stream, torch):
     would break the chain in which a call is set up while the one before it finishes), one pair around
     each of the other calls."""
     n = min(args.steps, 10)
-    names = ["attention", "transfer", "verify", "compact"]
+    names = ["attention", "transfer"] + (["verify_compact"] if step.fused else ["verify", "compact"])
     ev = {k: [] for k in names}
 
     def pair():
@@ -387,8 +389,11 @@ def per_kernel_pass(args, step, stream, torch):
         attention_run(0, cut)
         timed("transfer", lambda: step.transfer(stream))
         attention_run(cut, step.layers)
-        timed("verify", lambda: step.verify(stream))
-        timed("compact", lambda: step.compact(stream))
+        if step.fused:
+            timed("verify_compact", lambda: step.verify_compact(stream))
+        else:
+            timed("verify", lambda: step.verify(stream))
+            timed("compact", lambda: step.compact(stream))
     torch.cuda.synchronize()
     tot = {k: sum(x[0].elapsed_time(x[1]) for x in v) for k, v in ev.items()}
     all_ms = sum(tot.values())
@@ -402,9 +407,10 @@ def per_kernel_pass(args, step, stream, torch):
                 "frac": achieved / peak, "frac_of_nominal_8tbs": achieved / 8000.0, "peak_source": how,
                 "traffic": ncu_traffic(step.w), "bytes_per_launch": attn_bytes, "us_per_launch": attn_ms * 1e3,
                 "tflops": attn_flops / (attn_ms * 1e-3) / 1e12}
-    bytes_of = {"transfer": step.transfer_bytes(), "verify": step.verify_bytes(), "compact": step.compact_bytes()}
+    bytes_of = {"transfer": step.transfer_bytes(), "verify": step.verify_bytes(), "compact": step.compact_bytes(),
+                "verify_compact": step.verify_bytes() + step.compact_bytes()}
     kernels = {"attention": {"us": attn_ms * 1e3, "share": tot["attention"] / all_ms, "gbs": achieved}}
-    for k in ("transfer", "verify", "compact"):
+    for k in names[1:]:
         us = tot[k] / len(ev[k]) * 1e3
         kernels[k] = {"us": us, "share": tot[k] / all_ms, "gbs": bytes_of[k] / (us * 1e-6) / 1e9}
     return roofline, kernels
@@ -499,8 +505,11 @@ def e2e_pass(args, step, inp, torch, world):
                 host_out[i].copy_(step.outs[i], non_blocking=True)
         if step.transfer_at >= step.layers:
             step.transfer(stream)
-        step.verify(stream)
-        step.compact(stream)
+        if step.fused:
+            step.verify_compact(stream)
+        else:
+            step.verify(stream)
+            step.compact(stream)
         for s, h in zip(res_src, host_res):
             h.copy_(s, non_blocking=True)
         torch.cuda.synchronize()

@@ -212,14 +212,39 @@ int ht_kv_compact_paged(void *k_pages, void *v_pages, const ht_cache_desc *desc 
  *   next_token  [B] out: pred at the path's last node; root_pred[b] (or -1 without
  *             root_pred) when nothing is accepted
  *   status    [B] out: HT_STATUS_BAD_TREE, HT_STATUS_PATH_TOO_LONG (accept_len 0, next -1)
- * Two kernels (one zeroes the per-sequence arrival counters kept in accept_len), both launched with programmatic
- * stream serialization and waiting, at their first instruction, for the work ahead of them in the stream: ordering
- * is that of ordinary launches.
+ * max_path <= 255.
+ * accept_len is also where the kernel counts, in the bits above the low eight, the rows of a sequence that are
+ * done; the sequence's last thread block replaces the count by the length.  ON ENTRY every accept_len[b] must
+ * therefore hold a value in [0, 255]: zero before the first call (the caller clears it once), afterwards what
+ * the previous call left there will do.  Anything else (uninitialised memory, a buffer last used by a call that
+ * did not finish) makes the count come out wrong and the sequence's outputs are not written.
+ * One kernel, launched with programmatic stream serialization and waiting, at its first instruction, for the
+ * work ahead of it in the stream: ordering is that of an ordinary launch.
  */
 int ht_verify_greedy(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
                      const int32_t *root_pred, int B, int N, int T, int V, int max_path,
                      int32_t *pred, int32_t *accept_len, int32_t *accept_path,
                      int32_t *next_token, int32_t *status, void *stream);
+
+/*
+ * Greedy verification and KV compaction in one launch -- Fig. 2 caption and Section "Inference stage" (find the
+ * last accepted position, then go on from it): ht_verify_greedy followed by ht_kv_compact, with the same
+ * arguments, results and restrictions as the two calls (max_path <= 64; new_kv_len must not overlap kv_len or
+ * accept_len; accept_len[b] in [0, 255] on entry), and the same results bit for bit.
+ *   rows     logits rows per sequence whose argmax is taken, T <= rows <= N; 0 selects T, the rows
+ *            acceptance can consult.  pred[b][r] is written for r < rows only.
+ *   status, compact_status   [B] out: the status words of the verification and of the compaction.
+ *   desc     its B and N must equal B and N.
+ * The thread blocks first take the argmax of the rows; the block that completes a sequence searches its
+ * tree; then all blocks share out the compaction's (layer, sequence, head group) items, each waiting (bounded:
+ * about a second, then HT_STATUS_TIMEOUT in compact_status and the sequence's cache left as it is) until the
+ * sequence's accepted length has been stored.  The grid never exceeds what the GPU holds at once.
+ */
+int ht_verify_greedy_compact(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
+                             const int32_t *root_pred, int B, int N, int T, int V, int max_path, int rows,
+                             int32_t *pred, int32_t *accept_len, int32_t *accept_path, int32_t *next_token,
+                             int32_t *status, void *k_cache, void *v_cache, const ht_cache_desc *desc /* host */,
+                             const int32_t *kv_len, int32_t *new_kv_len, int32_t *compact_status, void *stream);
 
 /*
  * KV compaction -- implied by verifying under a KV cache (Fig. 1 caption; Section

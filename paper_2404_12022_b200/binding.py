@@ -24,7 +24,8 @@ HT_ATTN_FORCE_SIMT = 1
 
 EXPORTS = ("ht_version", "ht_last_error_string", "ht_transfer", "ht_tree_attention_workspace",
            "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact", "ht_draft_tree", "ht_rope_kv_append", "ht_tree_attention_static",
-           "ht_tree_attention_paged", "ht_rope_kv_append_paged", "ht_kv_compact_paged", "ht_tree_attention_launches")
+           "ht_tree_attention_paged", "ht_rope_kv_append_paged", "ht_kv_compact_paged", "ht_tree_attention_launches",
+           "ht_verify_greedy_compact")
 HT_STATIC_SCRATCH_BYTES = 16 << 20
 
 _DTYPES = {torch.float32: HT_F32, torch.float16: HT_F16, torch.bfloat16: HT_BF16}
@@ -91,6 +92,9 @@ def load() -> ctypes.CDLL:
                                             vp, vp, vp]
         lib.ht_verify_greedy.restype = i32
         lib.ht_verify_greedy.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        lib.ht_verify_greedy_compact.restype = i32
+        lib.ht_verify_greedy_compact.argtypes = [vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp,
+                                                 vp, vp, ctypes.POINTER(CacheDesc), vp, vp, vp, vp]
         lib.ht_kv_compact.restype = i32
         lib.ht_kv_compact.argtypes = [vp, vp, ctypes.POINTER(CacheDesc), vp, vp, vp, i32, vp, vp, vp]
         lib.ht_draft_tree.restype = i32
@@ -243,8 +247,10 @@ def tree_attention_static(q, k_cache, v_cache, kv_len, parent, out=None, status=
     return out, status
 
 
-def verify_greedy(logits, tokens, parent, root_pred=None, max_path: int = 8):
+def verify_greedy(logits, tokens, parent, root_pred=None, max_path: int = 8, accept_len=None):
     """logits [B, N, V]; tokens [B, T] int32; parent [B, N] int32; root_pred [B] int32 or None.
+    ``accept_len`` [B] int32, if given, must hold zeros or what an earlier call left in it (the kernel counts
+    arrivals in its upper bits); by default a zeroed tensor is made.
     Returns (pred [B, N], accept_len [B], accept_path [B, max_path], next_token [B], status [B])."""
     _need(logits, name="logits")
     _need(tokens, torch.int32, "tokens")
@@ -257,7 +263,10 @@ def verify_greedy(logits, tokens, parent, root_pred=None, max_path: int = 8):
         _need(root_pred, torch.int32, "root_pred")
     dev = logits.device
     pred = torch.empty((B, N), dtype=torch.int32, device=dev)
-    accept_len = torch.empty(B, dtype=torch.int32, device=dev)
+    if accept_len is None:
+        accept_len = torch.zeros(B, dtype=torch.int32, device=dev)
+    else:
+        _need(accept_len, torch.int32, "accept_len")
     accept_path = torch.empty((B, max_path), dtype=torch.int32, device=dev)
     next_token = torch.empty(B, dtype=torch.int32, device=dev)
     status = torch.empty(B, dtype=torch.int32, device=dev)
@@ -265,6 +274,47 @@ def verify_greedy(logits, tokens, parent, root_pred=None, max_path: int = 8):
                                    _ptr(root_pred), B, N, T, V, max_path, _ptr(pred), _ptr(accept_len),
                                    _ptr(accept_path), _ptr(next_token), _ptr(status), _stream()))
     return pred, accept_len, accept_path, next_token, status
+
+
+def verify_greedy_compact(logits, tokens, parent, root_pred, k_cache, v_cache, kv_len, max_path: int = 8, rows: int = 0,
+                          accept_len=None):
+    """Verification and compaction in one launch: ``verify_greedy`` followed by ``kv_compact`` on caches
+    [layers, B, Hkv, cap, D].  ``rows``: logits rows per sequence whose argmax is taken (0 = the T tree rows).
+    Returns (pred, accept_len, accept_path, next_token, status, new_kv_len, compact_status)."""
+    _need(logits, name="logits")
+    _need(tokens, torch.int32, "tokens")
+    _need(parent, torch.int32, "parent")
+    _need(kv_len, torch.int32, "kv_len")
+    B, N, V = logits.shape
+    T = tokens.shape[1]
+    if tuple(parent.shape) != (B, N) or tokens.shape[0] != B:
+        raise ValueError("parent must be [B, N] and tokens [B, T]")
+    if root_pred is not None:
+        _need(root_pred, torch.int32, "root_pred")
+    if not (k_cache.is_cuda and v_cache.is_cuda) or k_cache.dtype != v_cache.dtype:
+        raise ValueError("caches must be CUDA tensors of one dtype")
+    if k_cache.stride() != v_cache.stride() or k_cache.shape != v_cache.shape:
+        raise ValueError("k_cache and v_cache must share shape and strides")
+    layers, Bc, Hkv, cap, D = k_cache.shape
+    if k_cache.stride(4) != 1 or k_cache.stride(3) != D or Bc != B:
+        raise ValueError("cache rows must be contiguous and D apart, and the caches must hold B sequences")
+    desc = CacheDesc(layers, B, Hkv, cap, D, _DTYPES[k_cache.dtype], N, k_cache.stride(0), k_cache.stride(1), k_cache.stride(2))
+    dev = logits.device
+    pred = torch.full((B, N), -1, dtype=torch.int32, device=dev)
+    if accept_len is None:
+        accept_len = torch.zeros(B, dtype=torch.int32, device=dev)
+    else:
+        _need(accept_len, torch.int32, "accept_len")
+    accept_path = torch.empty((B, max_path), dtype=torch.int32, device=dev)
+    next_token = torch.empty(B, dtype=torch.int32, device=dev)
+    status = torch.empty(B, dtype=torch.int32, device=dev)
+    new_kv_len = torch.empty(B, dtype=torch.int32, device=dev)
+    compact_status = torch.empty(B, dtype=torch.int32, device=dev)
+    _check(load().ht_verify_greedy_compact(_ptr(logits), _DTYPES[logits.dtype], _ptr(tokens), _ptr(parent), _ptr(root_pred),
+                                           B, N, T, V, max_path, rows, _ptr(pred), _ptr(accept_len), _ptr(accept_path),
+                                           _ptr(next_token), _ptr(status), _ptr(k_cache), _ptr(v_cache), ctypes.byref(desc),
+                                           _ptr(kv_len), _ptr(new_kv_len), _ptr(compact_status), _stream()))
+    return pred, accept_len, accept_path, next_token, status, new_kv_len, compact_status
 
 
 def kv_compact(k_cache, v_cache, n_rows: int, kv_len, accept_len, accept_path, new_kv_len=None,

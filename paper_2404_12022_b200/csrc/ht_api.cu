@@ -3,7 +3,7 @@
 #include <stdarg.h>
 #include <stdio.h>
 
-#include "ht_common.cuh"
+#include "compact.cuh"
 
 namespace ht {
 
@@ -156,13 +156,62 @@ int ht_verify_greedy(const void *logits, int dtype, const int32_t *tokens, const
     if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     if (B == 0) return HT_OK;
     if (N == 0 || V <= 0) return fail(HT_ERR_INVALID_ARG, "N and V must be positive");
-    if (max_path <= 0) return fail(HT_ERR_INVALID_ARG, "max_path must be positive");
+    if (max_path <= 0 || max_path > 255) return fail(HT_ERR_INVALID_ARG, "max_path must be in 1..255");
     if (!logits || !parent || !pred || !accept_len || !accept_path || !next_token || !status || (T > 0 && !tokens))
         return fail(HT_ERR_INVALID_ARG, "NULL pointer");
     if (!aligned16(logits)) return fail(HT_ERR_INVALID_ARG, "logits must be 16-byte aligned");
     if ((long long)B * N > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "B*N too large");
-    return launch_verify(logits, dtype, tokens, parent, root_pred, B, N, T, V, max_path, pred, accept_len,
-                         accept_path, next_token, status, static_cast<cudaStream_t>(stream));
+    return launch_verify(logits, dtype, tokens, parent, root_pred, B, N, T, V, max_path, N, pred, accept_len,
+                         accept_path, next_token, status, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+static int check_cache_desc(const ht_cache_desc *desc, int max_path) {
+    if (!desc) return fail(HT_ERR_INVALID_ARG, "desc is NULL");
+    if (desc->layers <= 0 || desc->B < 0 || desc->Hkv <= 0 || desc->cap <= 0 || desc->D <= 0 || desc->N < 0)
+        return fail(HT_ERR_INVALID_ARG, "bad cache sizes");
+    if (!valid_dtype(desc->dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", desc->dtype);
+    if (max_path <= 0 || max_path > 64) return fail(HT_ERR_INVALID_ARG, "max_path must be in 1..64");
+    const int row_bytes = desc->D * elem_bytes(desc->dtype);
+    if (row_bytes % 16) return fail(HT_ERR_UNSUPPORTED, "a cache row must be a multiple of 16 bytes");
+    if ((long long)max_path * (row_bytes / 16) > 4096)
+        return fail(HT_ERR_UNSUPPORTED, "max_path * row size too large for one block");
+    const long long e = elem_bytes(desc->dtype);
+    if ((desc->stride_layer * e) % 16 || (desc->stride_b * e) % 16 || (desc->stride_h * e) % 16)
+        return fail(HT_ERR_INVALID_ARG, "cache strides must be multiples of 16 bytes");
+    if (2ll * desc->layers * desc->B * desc->Hkv > 0x7fffffffLL)
+        return fail(HT_ERR_UNSUPPORTED, "too many (layer, sequence, head) units");
+    return HT_OK;
+}
+
+int ht_verify_greedy_compact(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
+                             const int32_t *root_pred, int B, int N, int T, int V, int max_path, int rows,
+                             int32_t *pred, int32_t *accept_len, int32_t *accept_path, int32_t *next_token,
+                             int32_t *status, void *k_cache, void *v_cache, const ht_cache_desc *desc,
+                             const int32_t *kv_len, int32_t *new_kv_len, int32_t *compact_status, void *stream) {
+    if (B < 0 || N < 0 || T < 0 || T > N) return fail(HT_ERR_INVALID_ARG, "need 0 <= T <= N and B >= 0");
+    if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    int rc = check_cache_desc(desc, max_path);
+    if (rc != HT_OK) return rc;
+    if (desc->B != B || desc->N != N) return fail(HT_ERR_INVALID_ARG, "the cache descriptor's B and N must be those of the logits");
+    if (B == 0) return HT_OK;
+    if (N == 0 || V <= 0) return fail(HT_ERR_INVALID_ARG, "N and V must be positive");
+    if (rows == 0) rows = T > 0 ? T : 1;
+    if (rows < T || rows < 1 || rows > N) return fail(HT_ERR_INVALID_ARG, "rows = %d must lie in [max(T, 1), N]", rows);
+    if (!logits || !parent || !pred || !accept_len || !accept_path || !next_token || !status || (T > 0 && !tokens) ||
+        !k_cache || !v_cache || !kv_len || !new_kv_len || !compact_status)
+        return fail(HT_ERR_INVALID_ARG, "NULL pointer");
+    if (!aligned16(logits) || !aligned16(k_cache) || !aligned16(v_cache))
+        return fail(HT_ERR_INVALID_ARG, "logits and caches must be 16-byte aligned");
+    if ((long long)B * N > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "B*N too large");
+    if (overlap_i32(new_kv_len, kv_len, B) || overlap_i32(new_kv_len, accept_len, B))
+        return fail(HT_ERR_INVALID_ARG, "new_kv_len must not overlap kv_len or accept_len: every block of a sequence reads them");
+    // about one compaction item per thread block of the verification's grid (it holds B * rows blocks, or as many as
+    // the GPU takes at once, whichever is less: four per SM)
+    const long long grid_guess = (long long)B * rows < 4 * 148 ? (long long)B * rows : 4 * 148;
+    const CompactArgs c = make_compact_args(k_cache, v_cache, *desc, kv_len, accept_len, accept_path, max_path, new_kv_len,
+                                            compact_status, PageMap{}, (int)grid_guess);
+    return launch_verify(logits, dtype, tokens, parent, root_pred, B, N, T, V, max_path, rows, pred, accept_len,
+                         accept_path, next_token, status, &c, static_cast<cudaStream_t>(stream));
 }
 
 int ht_kv_compact(void *k_cache, void *v_cache, const ht_cache_desc *desc, const int32_t *kv_len,

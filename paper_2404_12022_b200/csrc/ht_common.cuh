@@ -103,10 +103,13 @@ int attn_tc_launches(const ht_attn_desc &d);      // kernels one call enqueues (
 int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const void *vc, const int32_t *kv_len,
                    const int32_t *parent, void *out, void *ws, size_t ws_bytes, int32_t *status, cudaStream_t s,
                    const ht_paged_desc *pages = nullptr, const int32_t *block_table = nullptr);
+struct CompactArgs;
+// rows: logits rows per sequence whose argmax is taken (T <= rows <= N); compact: the compaction to run in the same
+// launch, or null.
 int launch_verify(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
-                  const int32_t *root_pred, int B, int N, int T, int V, int max_path, int32_t *pred,
+                  const int32_t *root_pred, int B, int N, int T, int V, int max_path, int rows, int32_t *pred,
                   int32_t *accept_len, int32_t *accept_path, int32_t *next_token, int32_t *status,
-                  cudaStream_t s);
+                  const CompactArgs *compact, cudaStream_t s);
 int launch_draft(const void *logits, int dtype, int B, int rows, int V, int first_row, int P, int K,
                  const int32_t *tmpl_parent, const int32_t *tmpl_rank, int Tn, const int32_t *root_token,
                  const int32_t *base_pos, int32_t *topk, int32_t *tokens, int32_t *pos, int32_t *status, cudaStream_t s);

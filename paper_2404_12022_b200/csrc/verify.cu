@@ -1,14 +1,20 @@
 // Greedy verification (Fig. 2 caption; Sections "Inference stage" and "Setup"):
 // row argmax of the logits, then the longest root path of the draft tree whose tokens
-// are the ones greedy decoding would emit.
+// are the ones greedy decoding would emit -- and, in the fused form, the compaction of the
+// accepted path's K/V rows (Fig. 1 caption) in the same launch.
 //
-// One launch: a block per logits row streams it once (16-byte loads, eight in flight per thread,
-// shuffle reductions) and stores the row's argmax; the block that finishes a sequence's last row
-// (a ticket per sequence, drawn on the accept_len word, which a memset clears ahead of the launch)
-// runs the path search for that sequence -- a few hundred integer operations.  Nobody waits.
+// One launch, a grid no larger than the GPU holds at once.  A block streams logits rows
+// (16-byte loads, all of a row in flight at once, shuffle reductions) and stores each row's
+// argmax; the block that finishes a sequence's last row runs the path search for that
+// sequence -- a few hundred integer operations.  Arrivals are counted in the upper bits of the
+// sequence's accept_len word: the caller hands it over holding a small value (zero, or the
+// length an earlier call left there), the last block overwrites it with the new length, so
+// that no kernel has to clear anything ahead of the launch.  In the fused form the blocks then
+// share out the (layer, sequence, head group) items of the compaction; a block waits (bounded)
+// for the sequence's length to appear before it moves that sequence's rows.
 #include <limits.h>
 
-#include "ht_common.cuh"
+#include "compact.cuh"
 
 namespace ht {
 
@@ -28,13 +34,22 @@ __device__ __forceinline__ int ld_pred(const int32_t *p) {
     return __isGlobal(p) ? __ldcg(p) : *p;
 }
 
+__device__ __forceinline__ void st_release(int32_t *p, int v) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire(const int32_t *p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
 // Path search of one sequence by one block.  Every thread walks the root path of its nodes (parent[c] < c
 // makes the walk finite), checks the match rule on the way and proposes (depth, node);
 // the block keeps the deepest valid node, lowest index on ties.
 __device__ __forceinline__ void accept_sequence(const int b, const int32_t *__restrict__ tokens, const int32_t *__restrict__ parent,
               const int32_t *__restrict__ root_pred, const int32_t *pred, int N, int T,
               int max_path, int32_t *accept_len, int32_t *__restrict__ accept_path,
-              int32_t *__restrict__ next_token, int32_t *__restrict__ status) {
+              int32_t *__restrict__ next_token, int32_t *__restrict__ status, const int done_mark) {
     const int32_t *par = parent + (size_t)b * N;
     const int32_t *tok = tokens + (size_t)b * T;
     const int32_t *prd = pred + (size_t)b * N;
@@ -65,8 +80,8 @@ __device__ __forceinline__ void accept_sequence(const int b, const int32_t *__re
     if (s_bad) {
         if (threadIdx.x == 0) {
             status[b] = HT_STATUS_BAD_TREE;
-            accept_len[b] = 0;
             next_token[b] = -1;
+            st_release(accept_len + b, done_mark);
         }
         return;
     }
@@ -99,13 +114,14 @@ __device__ __forceinline__ void accept_sequence(const int b, const int32_t *__re
         for (int w = 1; w < (int)(blockDim.x >> 5); ++w) key = s_key[w] > key ? s_key[w] : key;
         const int len = (int)(key >> 32);
         const int node = (int)(0xFFFFFFFFu - (unsigned)(key & 0xFFFFFFFFu));
+        // the length goes last, with release semantics: it is also the word other blocks wait on (fused form: marked
+        // "done", since a small value is also what the word held before the sequence's first row arrived)
         if (len > max_path) {
             status[b] = HT_STATUS_PATH_TOO_LONG;
-            accept_len[b] = 0;
             next_token[b] = -1;
+            st_release(accept_len + b, done_mark);
         } else {
             status[b] = HT_STATUS_OK;
-            accept_len[b] = len;
             if (len == 0) {
                 next_token[b] = has_root ? rp : -1;
             } else {
@@ -113,38 +129,35 @@ __device__ __forceinline__ void accept_sequence(const int b, const int32_t *__re
                 for (int c = node; c >= 0; c = par[c]) path[j--] = c;
                 next_token[b] = ld_pred(prd + node);
             }
+            st_release(accept_len + b, done_mark | len);
         }
     }
 }
 
+constexpr int kVerifyThreads = 256;
+constexpr unsigned kTicket = 256u;           // arrivals are counted in units of this on the accept_len word: lengths stay below it
+constexpr int kDoneMark = 1 << 30;           // fused form: the length is in the word's low bits, the compaction may begin
+
+// Argmax of one logits row by the block: lowest index on ties, NaN never wins, a row of NaNs gives 0.  All threads
+// return the same index.
 template <typename T>
-__global__ void __launch_bounds__(256)
-verify_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pred, const int32_t *__restrict__ tokens,
-              const int32_t *__restrict__ parent, const int32_t *__restrict__ root_pred, int N, int Tn, int max_path,
-              int32_t *__restrict__ accept_len, int32_t *__restrict__ accept_path, int32_t *__restrict__ next_token,
-              int32_t *__restrict__ status) {
-    // The launch is serialized programmatically behind the kernel that zeroes the tickets, which itself waits for the
-    // work ahead of it in the stream: from here on everything that work wrote may be read.  A kernel serialized
-    // behind this one (the compaction) may set itself up meanwhile.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+__device__ __forceinline__ int row_argmax(const T *__restrict__ row, int V) {
     constexpr int VE = Vec16<T>::n;
-    const T *row = logits + (size_t)blockIdx.x * V;
     Best best{-INFINITY, INT_MAX};
     const bool vec_ok = ((size_t)V * sizeof(T)) % 16 == 0;
     if (vec_ok) {
         const int nvec = V / VE;
-        constexpr int U = 8;                       // independent 16-byte loads in flight per thread
-        for (int j0 = threadIdx.x; j0 < nvec; j0 += U * blockDim.x) {
+        constexpr int U = 16;                      // independent 16-byte loads in flight per thread: 64 KB per block and pass
+        for (int j0 = threadIdx.x; j0 < nvec; j0 += U * kVerifyThreads) {
             uint4 raw[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const int j = j0 + u * blockDim.x;
-                raw[u] = ld_nc16(row + (size_t)min(j, nvec - 1) * VE);   // past the end: the last vector again
+                const int j = j0 + u * kVerifyThreads;
+                raw[u] = __ldcs(reinterpret_cast<const uint4 *>(row + (size_t)min(j, nvec - 1) * VE));   // past the end: the last vector again
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const int j = min(j0 + u * (int)blockDim.x, nvec - 1);
+                const int j = min(j0 + u * kVerifyThreads, nvec - 1);
                 float f[VE];
                 unpack16<T>(raw[u], f);
 #pragma unroll
@@ -157,7 +170,7 @@ verify_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pred, c
             }
         }
     } else {
-        for (int j = threadIdx.x; j < V; j += blockDim.x) {
+        for (int j = threadIdx.x; j < V; j += kVerifyThreads) {
             const float x = to_float<T>(row[j]);
             if (x > best.v) best = Best{x, j};
         }
@@ -167,57 +180,107 @@ verify_kernel(const T *__restrict__ logits, int V, int32_t *__restrict__ pred, c
         Best o{__shfl_xor_sync(0xffffffffu, best.v, off), __shfl_xor_sync(0xffffffffu, best.i, off)};
         best = better(best, o);
     }
-    __shared__ Best warp_best[8];
+    __shared__ Best warp_best[kVerifyThreads / 32];
+    __shared__ int warp_first[kVerifyThreads / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();                               // the previous row's readers of these arrays are done
     if (lane == 0) warp_best[warp] = best;
     __syncthreads();
-    if (warp == 0) {
-        best = lane < (int)(blockDim.x >> 5) ? warp_best[lane] : Best{-INFINITY, INT_MAX};
-#pragma unroll
-        for (int off = 4; off > 0; off >>= 1) {
-            Best o{__shfl_xor_sync(0xffffffffu, best.v, off), __shfl_xor_sync(0xffffffffu, best.i, off)};
-            best = better(best, o);
-        }
-        if (lane == 0) warp_best[0] = best;
-    }
-    __syncthreads();
     best = warp_best[0];
+#pragma unroll
+    for (int w = 1; w < kVerifyThreads / 32; ++w) best = better(best, warp_best[w]);
     if (best.i == INT_MAX) {
         // Nothing in the row exceeds -inf: the answer is the first -inf, or 0 in a row of NaNs only.
         int first = INT_MAX;
-        for (int j = threadIdx.x; j < V; j += blockDim.x)
+        for (int j = threadIdx.x; j < V; j += kVerifyThreads)
             if (to_float<T>(row[j]) == -INFINITY) { first = j; break; }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) first = min(first, __shfl_xor_sync(0xffffffffu, first, off));
-        __shared__ int warp_first[8];
         if (lane == 0) warp_first[warp] = first;
         __syncthreads();
-        if (threadIdx.x == 0) {
-            for (int w = 1; w < (int)(blockDim.x >> 5); ++w) first = min(first, warp_first[w]);
-            best.i = first == INT_MAX ? 0 : first;
-        }
+        first = warp_first[0];
+        for (int w = 1; w < kVerifyThreads / 32; ++w) first = min(first, warp_first[w]);
+        best.i = first == INT_MAX ? 0 : first;
     }
-    if (threadIdx.x == 0) pred[blockIdx.x] = best.i;
-    // The block that stores a sequence's last argmax searches its tree.
-    __shared__ int s_last;
-    const int b = blockIdx.x / N;
-    if (threadIdx.x == 0) {
-        __threadfence();
-        s_last = atomicAdd(reinterpret_cast<unsigned int *>(accept_len + b), 1u) == (unsigned)(N - 1);
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    accept_sequence(b, tokens, parent, root_pred, pred, N, Tn, max_path, accept_len, accept_path, next_token, status);
+    return best.i;
 }
 
-// accept_len doubles as the per-sequence ticket until the sequence's last block overwrites it: zero at the start.
-// A kernel rather than a memset node, so that the launches chain by programmatic stream serialization: it is in
-// place, waiting, before the kernel ahead of it in the stream has finished.
-__global__ void verify_prepare_kernel(int32_t *accept_len, int B) {
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+struct VerifyArgs {
+    const void *logits;
+    const int32_t *tokens, *parent, *root_pred;
+    int B, N, T, V, max_path;
+    int rows;                 // logits rows per sequence whose argmax is taken: T <= rows <= N
+    int32_t *pred, *accept_len, *accept_path, *next_token, *status;
+};
+
+// kFused: the blocks go on to the compaction once their rows are done.
+template <typename T, bool kFused>
+__global__ void __launch_bounds__(kVerifyThreads, 4)
+verify_kernel(const VerifyArgs v, const CompactArgs c) {
+    // The launch is serialized programmatically behind the kernel ahead of it in the stream: from here on everything
+    // that kernel wrote may be read.  A kernel serialized behind this one may set itself up meanwhile.
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    for (int i = threadIdx.x; i < B; i += blockDim.x) accept_len[i] = 0;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    __shared__ int s_last;
+    const int n_rows = v.B * v.rows;
+    for (int idx = blockIdx.x; idx < n_rows; idx += gridDim.x) {
+        const int b = idx / v.rows, r = idx - b * v.rows;
+        const int best = row_argmax<T>(static_cast<const T *>(v.logits) + ((size_t)b * v.N + r) * v.V, v.V);
+        if (threadIdx.x == 0) {
+            v.pred[(size_t)b * v.N + r] = best;
+            // The block that stores a sequence's last argmax searches its tree.
+            __threadfence();
+            const unsigned before = atomicAdd(reinterpret_cast<unsigned int *>(v.accept_len + b), kTicket);
+            s_last = before / kTicket == (unsigned)(v.rows - 1);
+        }
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            accept_sequence(b, v.tokens, v.parent, v.root_pred, v.pred, v.N, v.T, v.max_path, v.accept_len, v.accept_path,
+                            v.next_token, v.status, kFused ? kDoneMark : 0);
+        }
+        __syncthreads();
+    }
+    if (!kFused) return;
+    // ---- compaction: items (layer, sequence, head group) dealt out to the blocks.  The grid is no larger than the
+    // GPU holds at once and every block has finished its rows before it waits here, so the length it waits for is
+    // on its way; the wait is bounded all the same.  The sequence's word says "done | length" from the path search
+    // on; finished items are counted in it as the rows were, and the last one leaves the plain length there. ----
+    __shared__ CompactSmem csm;
+    __shared__ int s_len_b;
+    const int n_items = c.layers * c.B * c.groups;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        int x = item;
+        const int grp = x % c.groups;
+        x /= c.groups;
+        const int b = x % c.B, layer = x / c.B;
+        const int L = c.kv_len[b];                           // on its way while the length is waited for
+        if (threadIdx.x == 0) {
+            int a = ld_acquire(v.accept_len + b);
+            const long long t0 = clock64();
+            while (!(a & kDoneMark)) {                       // rows are still arriving, or have not begun to
+                if (clock64() - t0 > 2000000000ll) { a = -1; break; }
+                __nanosleep(64);
+                a = ld_acquire(v.accept_len + b);
+            }
+            s_len_b = a < 0 ? -1 : (a & (int)(kTicket - 1));
+        }
+        __syncthreads();
+        const int a = s_len_b;
+        if (a < 0) {                                         // gave up: the sequence is left as it is
+            if (layer == 0 && grp == 0 && threadIdx.x == 0) {
+                c.status[b] = HT_STATUS_TIMEOUT;
+                c.new_kv_len[b] = L;
+            }
+            __syncthreads();
+            continue;
+        }
+        compact_item<8>(c, csm, layer, b, grp, a, L);
+        if (threadIdx.x == 0) {
+            const unsigned before = atomicAdd(reinterpret_cast<unsigned int *>(v.accept_len + b), kTicket);
+            if ((before & ~(unsigned)kDoneMark) / kTicket == (unsigned)(c.layers * c.groups - 1)) v.accept_len[b] = a;
+        }
+    }
 }
 
 template <typename... KArgs, typename... Args>
@@ -234,27 +297,48 @@ static cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsig
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Blocks of a verification kernel the GPU holds at once.
+template <typename Kernel>
+static int resident_blocks(Kernel kernel) {
+    int dev = 0, sms = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kVerifyThreads, 0) != cudaSuccess || sms <= 0 || per_sm <= 0) {
+        cudaGetLastError();
+        return 148;
+    }
+    return sms * per_sm;
+}
+
+template <typename T>
+static cudaError_t launch_verify_t(const VerifyArgs &v, const CompactArgs *compact, cudaStream_t s) {
+    static int cap_plain[64], cap_fused[64];          // per device
+    int dev = 0;
+    cudaGetDevice(&dev);
+    int *slot = (dev >= 0 && dev < 64) ? (compact ? &cap_fused[dev] : &cap_plain[dev]) : nullptr;
+    int cap = slot ? *slot : 0;
+    if (cap == 0) {
+        cap = compact ? resident_blocks(verify_kernel<T, true>) : resident_blocks(verify_kernel<T, false>);
+        if (slot) *slot = cap;
+    }
+    const long long want = (long long)v.B * v.rows;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    if (compact) return launch_chained(verify_kernel<T, true>, grid, (unsigned)kVerifyThreads, s, v, *compact);
+    return launch_chained(verify_kernel<T, false>, grid, (unsigned)kVerifyThreads, s, v, CompactArgs{});
+}
+
 int launch_verify(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
-                  const int32_t *root_pred, int B, int N, int T, int V, int max_path, int32_t *pred,
+                  const int32_t *root_pred, int B, int N, int T, int V, int max_path, int rows, int32_t *pred,
                   int32_t *accept_len, int32_t *accept_path, int32_t *next_token, int32_t *status,
-                  cudaStream_t s) {
-    const unsigned rows = (unsigned)(B * N);
-    cudaError_t e = launch_chained(verify_prepare_kernel, 1u, 256u, s, accept_len, B);
-    if (e == cudaSuccess) {
-        switch (dtype) {
-            case HT_F32:
-                e = launch_chained(verify_kernel<float>, rows, 256u, s, static_cast<const float *>(logits), V, pred, tokens, parent, root_pred,
-                                   N, T, max_path, accept_len, accept_path, next_token, status);
-                break;
-            case HT_F16:
-                e = launch_chained(verify_kernel<__half>, rows, 256u, s, static_cast<const __half *>(logits), V, pred, tokens, parent, root_pred,
-                                   N, T, max_path, accept_len, accept_path, next_token, status);
-                break;
-            default:
-                e = launch_chained(verify_kernel<__nv_bfloat16>, rows, 256u, s, static_cast<const __nv_bfloat16 *>(logits), V, pred, tokens, parent,
-                                   root_pred, N, T, max_path, accept_len, accept_path, next_token, status);
-                break;
-        }
+                  const CompactArgs *compact, cudaStream_t s) {
+    VerifyArgs v{};
+    v.logits = logits; v.tokens = tokens; v.parent = parent; v.root_pred = root_pred;
+    v.B = B; v.N = N; v.T = T; v.V = V; v.max_path = max_path; v.rows = rows;
+    v.pred = pred; v.accept_len = accept_len; v.accept_path = accept_path; v.next_token = next_token; v.status = status;
+    cudaError_t e;
+    switch (dtype) {
+        case HT_F32: e = launch_verify_t<float>(v, compact, s); break;
+        case HT_F16: e = launch_verify_t<__half>(v, compact, s); break;
+        default: e = launch_verify_t<__nv_bfloat16>(v, compact, s); break;
     }
     if (e != cudaSuccess) {
         cudaGetLastError();

@@ -2,8 +2,9 @@
 
 ``VerifyStep`` owns the descriptors, outputs and workspace of a workload so that a step is
 nothing but C-ABI calls on the current stream: per layer ``ht_tree_attention`` (with the
-pseudo rows joining after the transfer layer), one ``ht_transfer``, one
-``ht_verify_greedy`` and one ``ht_kv_compact`` over all layers.  The dense parts of the
+pseudo rows joining after the transfer layer), one ``ht_transfer``, and verification plus
+compaction over all layers as one launch (``ht_verify_greedy_compact``; ``fused=False``: one
+``ht_verify_greedy`` and one ``ht_kv_compact``).  The dense parts of the
 transformer layer between those calls are outside this library; their outputs (q, the new
 K/V rows, the logits) are inputs here.
 """
@@ -19,7 +20,12 @@ from .workloads import Inputs
 
 
 class VerifyStep:
-    def __init__(self, inp: Inputs, num_splits: int = 0, flags: int = 0):
+    def __init__(self, inp: Inputs, num_splits: int = 0, flags: int = 0, fused: Optional[bool] = None):
+        # Verification and compaction as one launch (ht_verify_greedy_compact) or as two calls.  The chain of
+        # dependent steps is the same either way (argmax, count, path search, rows); measured behind an attention
+        # call, one launch is ahead for one sequence and one layer (16.1 against 17.1 us on config 2) and behind
+        # once the compaction has many (layer, sequence) items (21.5 against 19.9 us on config 3's 32 layers).
+        self.fused = (inp.k_cache.shape[0] * inp.w.B <= 4) if fused is None else fused
         w = inp.w
         self.inp = inp
         self.w = w
@@ -42,7 +48,7 @@ class VerifyStep:
         self.attn_status = torch.zeros((self.layers, w.B), dtype=torch.int32, device=dev)
         self.pseudo = torch.empty((w.B, w.k, w.d), dtype=inp.h_src.dtype, device=dev)
         self.pred = torch.empty((w.B, w.N), dtype=torch.int32, device=dev)
-        self.accept_len = torch.empty(w.B, dtype=torch.int32, device=dev)
+        self.accept_len = torch.zeros(w.B, dtype=torch.int32, device=dev)     # zero once: the kernel leaves a length in it each time
         self.accept_path = torch.empty((w.B, w.max_path), dtype=torch.int32, device=dev)
         self.next_token = torch.empty(w.B, dtype=torch.int32, device=dev)
         self.verify_status = torch.empty(w.B, dtype=torch.int32, device=dev)
@@ -84,6 +90,17 @@ class VerifyStep:
             inp.kv_len.data_ptr(), self.accept_len.data_ptr(), self.accept_path.data_ptr(), self.w.max_path,
             self.new_kv_len.data_ptr(), self.compact_status.data_ptr(), stream))
 
+    def verify_compact(self, stream: int) -> None:
+        """Verification (argmax of the tree rows only) and compaction as one launch."""
+        inp, w = self.inp, self.w
+        hb._check(self.lib.ht_verify_greedy_compact(
+            inp.logits.data_ptr(), hb._DTYPES[inp.logits.dtype], inp.tokens.data_ptr(), inp.parent.data_ptr(),
+            None if inp.root_pred is None else inp.root_pred.data_ptr(), w.B, w.N, w.T, w.V, w.max_path, 0,
+            self.pred.data_ptr(), self.accept_len.data_ptr(), self.accept_path.data_ptr(),
+            self.next_token.data_ptr(), self.verify_status.data_ptr(), inp.k_cache.data_ptr(), inp.v_cache.data_ptr(),
+            ctypes.byref(self.cache_desc), inp.kv_len.data_ptr(), self.new_kv_len.data_ptr(),
+            self.compact_status.data_ptr(), stream))
+
     def run(self, stream: Optional[int] = None, attn_hook=None) -> None:
         """Enqueue one whole step.  ``attn_hook(i, when)`` is called around each attention call
         (when = 0 before, 1 after) so that a caller can record events."""
@@ -98,8 +115,11 @@ class VerifyStep:
                 attn_hook(i, 1)
         if self.transfer_at >= self.layers:
             self.transfer(s)
-        self.verify(s)
-        self.compact(s)
+        if self.fused:
+            self.verify_compact(s)
+        else:
+            self.verify(s)
+            self.compact(s)
 
     def capture(self) -> None:
         """Record one whole step into a CUDA graph (after at least one eager ``run``, which does the
@@ -136,7 +156,7 @@ class VerifyStep:
 
     def verify_bytes(self) -> int:
         w = self.w
-        return w.B * w.N * w.V * w.elem_bytes()
+        return w.B * (w.T if self.fused else w.N) * w.V * w.elem_bytes()       # fused: the tree rows only
 
     def compact_bytes(self) -> int:
         w = self.w

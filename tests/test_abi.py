@@ -61,6 +61,20 @@ def test_host_side_rejections(lib):
     assert lib.ht_verify_greedy(p, hb.HT_F16, p, p, None, 1, 4, 3, 100, 8, None, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG
     assert lib.ht_verify_greedy(p, hb.HT_F16, p, p, None, 1, 4, 3, 100, 0, p, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG
 
+    assert lib.ht_verify_greedy(p, hb.HT_F16, p, p, None, 1, 4, 3, 100, 256, p, p, p, p, p, None) == hb.HT_ERR_INVALID_ARG   # lengths must stay below 256
+
+    # ht_verify_greedy_compact(logits, dtype, tokens, parent, root_pred, B, N, T, V, max_path, rows, pred, accept_len, accept_path,
+    #                          next_token, status, k_cache, v_cache, desc, kv_len, new_kv_len, compact_status, stream)
+    c = hb.CacheDesc(2, 1, 4, 64, 128, hb.HT_BF16, 4, 0, 0, 0)
+    fused = lambda rows, desc, new_len: lib.ht_verify_greedy_compact(p, hb.HT_F16, p, p, None, 1, 4, 3, 100, 8, rows, p, p + 64, p, p, p,
+                                                                     p, p, ctypes.byref(desc), p + 128, new_len, p, None)
+    assert fused(2, c, p + 192) == hb.HT_ERR_INVALID_ARG          # rows < T
+    assert fused(5, c, p + 192) == hb.HT_ERR_INVALID_ARG          # rows > N
+    assert fused(0, c, p + 128) == hb.HT_ERR_INVALID_ARG          # new_kv_len is kv_len
+    assert fused(0, c, p + 64) == hb.HT_ERR_INVALID_ARG           # new_kv_len is accept_len
+    assert fused(0, hb.CacheDesc(2, 1, 4, 64, 128, hb.HT_BF16, 5, 0, 0, 0), p + 192) == hb.HT_ERR_INVALID_ARG    # the descriptor's N is not the logits'
+    assert fused(0, hb.CacheDesc(2, 0, 4, 64, 128, hb.HT_BF16, 4, 0, 0, 0), p + 192) == hb.HT_ERR_INVALID_ARG    # nor its B
+
     c = hb.CacheDesc(2, 1, 4, 64, 128, hb.HT_BF16, 8, 0, 0, 0)
     assert lib.ht_kv_compact(p, p, ctypes.byref(c), p, p, p, 65, p, p, None) == hb.HT_ERR_INVALID_ARG
     assert lib.ht_kv_compact(None, p, ctypes.byref(c), p, p, p, 8, p, p, None) == hb.HT_ERR_INVALID_ARG

@@ -858,6 +858,93 @@ def test_compaction_of_32_layers_and_the_refused_update_in_place(hb, oracle):
         assert np.array_equal(ka[:, b, :, :n], k_ref[:, b, :, :n]) and np.array_equal(va[:, b, :, :n], v_ref[:, b, :, :n])
 
 
+def _fused_against_the_two_calls(hb, oracle, inp, rows, rounds=2):
+    """ht_verify_greedy_compact on a copy of the caches against the oracle and against the two separate calls, bit for
+    bit; called `rounds` times on the same accept_len buffer (the later calls start from the lengths the earlier left)."""
+    w = inp.w
+    view = torch.int32 if inp.k_cache.dtype == torch.float32 else torch.int16
+    k0, v0 = inp.k_cache.clone(), inp.v_cache.clone()
+    o_pred, o_alen, o_apath, o_nxt, o_status = oracle.verify_greedy(
+        f32np(inp.logits), inp.tokens.cpu().numpy(), inp.parent.cpu().numpy(),
+        None if inp.root_pred is None else inp.root_pred.cpu().numpy(), w.max_path)
+    k_ref, v_ref, len_ref, st_ref = oracle.kv_compact(k0.view(view).cpu().numpy(), v0.view(view).cpu().numpy(), w.N,
+                                                      inp.kv_len.cpu().numpy(), o_alen, o_apath)
+    alen = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+    for i in range(rounds):
+        k, v = k0.clone(), v0.clone()
+        pred, alen, apath, nxt, status, new_len, cstatus = hb.verify_greedy_compact(
+            inp.logits, inp.tokens, inp.parent, inp.root_pred, k, v, inp.kv_len, w.max_path, rows, accept_len=alen)
+        torch.cuda.synchronize()
+        n_scanned = rows if rows else w.T
+        assert np.array_equal(pred.cpu().numpy()[:, :n_scanned], o_pred[:, :n_scanned])
+        assert (pred[:, n_scanned:] == -1).all()                       # rows beyond are not touched
+        for g, r in ((alen, o_alen), (apath, o_apath), (nxt, o_nxt), (status, o_status), (new_len, len_ref), (cstatus, st_ref)):
+            assert np.array_equal(g.cpu().numpy(), r), "round %d" % i
+        ka, va = k.view(view).cpu().numpy(), v.view(view).cpu().numpy()
+        for b in range(w.B):
+            n = int(len_ref[b])
+            assert np.array_equal(ka[:, b, :, :n], k_ref[:, b, :, :n]) and np.array_equal(va[:, b, :, :n], v_ref[:, b, :, :n])
+            L = int(inp.kv_len[b])
+            assert np.array_equal(ka[:, b, :, :L], k0.view(view).cpu().numpy()[:, b, :, :L])
+    # the two separate calls on the same inputs leave the same bytes everywhere the result is specified
+    k2, v2 = k0.clone(), v0.clone()
+    p2, a2, ap2, n2, s2 = hb.verify_greedy(inp.logits, inp.tokens, inp.parent, inp.root_pred, w.max_path)
+    nl2, cs2 = hb.kv_compact(k2, v2, w.N, inp.kv_len, a2, ap2)
+    torch.cuda.synchronize()
+    assert torch.equal(a2, alen) and torch.equal(ap2, apath) and torch.equal(n2, nxt) and torch.equal(nl2, new_len)
+    for b in range(w.B):
+        n = int(len_ref[b])
+        assert torch.equal(k2[:, b, :, :n], k[:, b, :, :n]) and torch.equal(v2[:, b, :, :n], v[:, b, :, :n])
+
+
+@pytest.mark.parametrize("cfg", ["c1", "c2", "c3", "c4", "c5_b16", "c2_per_node"])
+def test_fused_verification_and_compaction(hb, oracle, cfg):
+    """One launch for row argmax, path search and compaction (the fused epilogue of the verification): the
+    configurations' shapes, with the argmax restricted to the tree rows (rows = 0) and over all rows."""
+    w = {"c1": lambda: wl.config_c1(2), "c2": wl.config_c2, "c3": lambda: wl.config_c3(layers=3, kv=700),
+         "c4": lambda: wl.config_c4(lo=100, hi=900), "c5_b16": lambda: wl.config_c5(512, 256, 16),
+         "c2_per_node": lambda: wl.per_node_variant(dataclasses.replace(wl.config_c2(), kv_len=[300], d=64))}[cfg]()
+    inp = wl.make_inputs(w, "cuda", with_transfer=False)
+    _fused_against_the_two_calls(hb, oracle, inp, 0)
+    _fused_against_the_two_calls(hb, oracle, inp, w.N, rounds=1)
+
+
+def test_fused_verification_many_layers_and_statuses(hb, oracle):
+    """32 layers (more compaction items than thread blocks), a sequence whose tree is illegal, one whose path is longer
+    than max_path and one whose length does not fit: the same status words and untouched caches as the two calls."""
+    rng = np.random.default_rng(8)
+    layers, B, Hkv, cap, D, T, P, V = 32, 5, 4, 64, 128, 12, 2, 64
+    N = T + P
+    k = wl.normal_tensor(34, 1, (layers, B, Hkv, cap, D), "cuda", 1.0, torch.bfloat16)
+    v = wl.normal_tensor(34, 2, (layers, B, Hkv, cap, D), "cuda", 1.0, torch.bfloat16)
+    parent = np.stack([rand_tree(rng, N, "chain" if b == 3 else "random") for b in range(B)])
+    parent[1, 5] = 7                                              # not an earlier row
+    tokens = rng.integers(0, 3, (B, T)).astype(np.int32)
+    logits = np.zeros((B, N, V), np.float32)
+    np.put_along_axis(logits, rng.integers(0, 3, (B, N))[..., None], 1.0, axis=2)
+    for r in range(N):                                            # sequence 3: a chain that matches all the way down
+        logits[3, r] = 0
+        if r + 1 < T:
+            logits[3, r, tokens[3, r + 1]] = 1.0
+    root_pred = tokens[:, 0].copy()
+    kv_len = np.array([10, 20, 30, 40, cap - N + 1], np.int32)    # the last one does not fit
+    args = [torch.from_numpy(x).cuda() for x in (logits, tokens, parent, root_pred)]
+    o = oracle.verify_greedy(logits, tokens, parent, root_pred, 8)
+    kb, vb = k.view(torch.int16).cpu().numpy(), v.view(torch.int16).cpu().numpy()
+    k_ref, v_ref, len_ref, st_ref = oracle.kv_compact(kb, vb, N, kv_len, o[1], o[2])
+    res = hb.verify_greedy_compact(args[0].to(torch.bfloat16), args[1], args[2], args[3], k, v, torch.from_numpy(kv_len).cuda(), 8, 0)
+    torch.cuda.synchronize()
+    pred, alen, apath, nxt, status, new_len, cstatus = res
+    for g, r in ((alen, o[1]), (apath, o[2]), (nxt, o[3]), (status, o[4]), (new_len, len_ref), (cstatus, st_ref)):
+        assert np.array_equal(g.cpu().numpy(), r)
+    assert status.cpu().tolist()[1] == hb.HT_STATUS_BAD_TREE and status.cpu().tolist()[3] == hb.HT_STATUS_PATH_TOO_LONG
+    assert cstatus.cpu().tolist()[4] == hb.HT_STATUS_BAD_LEN
+    ka, va = k.view(torch.int16).cpu().numpy(), v.view(torch.int16).cpu().numpy()
+    for b in range(B):
+        n = int(len_ref[b])
+        assert np.array_equal(ka[:, b, :, :n], k_ref[:, b, :, :n]) and np.array_equal(va[:, b, :, :n], v_ref[:, b, :, :n])
+
+
 def test_toy_lossless_loop_on_the_gpu(hb):
     """Draft-and-verify rounds through the library reproduce plain greedy decoding (fp32)."""
     from toy_lm import run_lossless_loop
