@@ -60,6 +60,12 @@ enum {
 
 /* ht_attn_desc.flags */
 #define HT_ATTN_FORCE_SIMT 1u /* use the fp32-ALU kernel even where a tensor-core kernel applies */
+/* Test hook, never to be set in production: the tensor-core kernels' device-side waits give up after about a
+ * microsecond instead of a second, so that their give-up path can be exercised: the call returns, the sequences'
+ * status words read HT_STATUS_TIMEOUT and `out` is meaningless.  Nothing faults and nothing is left in flight:
+ * a thread block that has given up still waits, with the full limit, for its own copies and tensor-core
+ * operations before it frees what they write to. */
+#define HT_ATTN_TEST_SHORT_WAITS 0x80000000u
 
 typedef struct {
     int32_t B, N, Hq, Hkv, D, cap;

@@ -21,6 +21,8 @@ HT_OK = 0
 HT_ERR_INVALID_ARG, HT_ERR_UNSUPPORTED, HT_ERR_BAD_TREE, HT_ERR_WORKSPACE, HT_ERR_CUDA, HT_ERR_TIMEOUT = range(1, 7)
 HT_STATUS_OK, HT_STATUS_BAD_TREE, HT_STATUS_BAD_LEN, HT_STATUS_BAD_PATH, HT_STATUS_PATH_TOO_LONG = range(5)
 HT_ATTN_FORCE_SIMT = 1
+HT_ATTN_TEST_SHORT_WAITS = 0x80000000
+HT_STATUS_BAD_PAGE, HT_STATUS_TIMEOUT = 5, 6
 
 EXPORTS = ("ht_version", "ht_last_error_string", "ht_transfer", "ht_tree_attention_workspace",
            "ht_tree_attention", "ht_verify_greedy", "ht_kv_compact", "ht_draft_tree", "ht_rope_kv_append", "ht_tree_attention_static",

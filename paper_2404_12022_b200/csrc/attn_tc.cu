@@ -117,6 +117,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         mbar_init(&sm.mma_drain, 1);
         for (int i = 0; i < 2; ++i) { mbar_init(&sm.s_full[i], 1); mbar_init(&sm.p_ready[i], 128); mbar_init(&sm.o_done[i], 1); }
         sm.abort = 0;
+        sm.wait_kcycles = p.wait_kcycles;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x == 32) {                 // descriptors on their way while the CTA sets itself up
@@ -810,6 +811,7 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     p.is_bf16 = d.dtype == HT_BF16;
     p.grid = sm_count();
     p.cluster_k = 0;
+    p.wait_kcycles = (d.flags & HT_ATTN_TEST_SHORT_WAITS) ? tc::kWaitKcyclesTest : tc::kWaitKcycles;
     tc::PagedParams pp;
     pp.block_table = pages ? block_table : nullptr;
     pp.page_size = pages ? pages->page_size : 0;

@@ -36,6 +36,11 @@ struct Params {
     int is_bf16;
     int grid;
     int cluster_k;         // > 1: launched as clusters of this many CTAs, one cluster per (sequence, KV head)
+    int wait_kcycles;      // how long a wait on an mbarrier may last, in units of 1024 clock cycles
+};
+enum : int {
+    kWaitKcycles = 2000000,            // about a second
+    kWaitKcyclesTest = 0               // HT_ATTN_TEST_SHORT_WAITS: a wait for anything not yet there runs out at once
 };
 
 // Paged cache: cache row r of sequence b is row r % page_size of page block_table[b * max_pages + r / page_size];
@@ -55,8 +60,8 @@ struct __align__(1024) Smem {
     int32_t nkt[kMaxB];
     int32_t pre[kMaxB + 1];
     unsigned long long kv_full[kStages], kv_empty[kStages], q_full, q_empty, s_full[2], p_ready[2], o_done[2], mma_drain;
+    int abort, wait_kcycles;           // the abort flag, and right behind it the limit of a wait (the waits read both as one 8-byte word)
     uint32_t tmem_base;
-    int abort;
     int merge_here[2];
     int direct;
     int32_t pg[kPgTiles][kPgSub];      // paged cache: page ids of the tiles about to be fetched
@@ -78,23 +83,37 @@ __device__ __forceinline__ void mbar_arrive(void *bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 // Bounded wait for the completion of the phase with the given parity.  Returns false (and
-// raises the CTA's abort flag) when about a second passes without it.
+// raises the CTA's abort flag) when the limit kept behind the abort flag (about a second) passes without it.
+// honor_abort = false is for the waits that must not be cut short once the CTA has given up: those for its
+// own copies in flight and for its own tensor-core operations, ahead of freeing what they write to; they
+// always get the full second.
 __device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, volatile int *abort_flag,
                                           bool honor_abort = true) {
-    if (honor_abort && *abort_flag) return false;
+    // one load for the flag and the limit behind it
+    const long long ctl = *reinterpret_cast<volatile long long *>(abort_flag);
+    const int limit_k = (int)(ctl >> 32);
+    if (honor_abort && (int)ctl) return false;
+    // limit 0 (the test hook): polls that do not suspend, and the clock looked at after every one of them, so that
+    // a wait for anything not yet there runs out at once
+    const bool instant = honor_abort && limit_k == 0;
     const uint32_t addr = smem_u32(bar);
     long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
         uint32_t ok;
-        asm volatile(
-            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+        if (instant)
+            asm volatile(
+                "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+        else
+            asm volatile(
+                "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
         if (ok) return true;
-        if ((it & 63u) == 63u) {
+        if ((it & 63u) == 63u || instant) {
             if (honor_abort && *abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > 2000000000ll) { *abort_flag = 1; return false; }
+            else if (now - t0 > ((long long)(honor_abort ? limit_k : kWaitKcycles) << 10)) { *abort_flag = 1; return false; }
         }
     }
 }
@@ -115,7 +134,7 @@ static __device__ __noinline__ bool mbar_wait_spin(uint32_t addr, uint32_t parit
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > 2000000000ll) { *abort_flag = 1; return false; }
+            else if (now - t0 > ((long long)abort_flag[1] << 10)) { *abort_flag = 1; return false; }
         }
     }
 }

@@ -103,8 +103,8 @@ struct __align__(1024) PSmem {
     int32_t nkt[kMaxB];
     int32_t pre[kMaxB + 1];
     unsigned long long kv_full[kPStages], kv_empty[kPStages], q_full, q_empty, s_full[2][2], p_ready[2][2], o_done[2][2], mma_drain;
+    int abort, wait_kcycles;           // the abort flag, and right behind it the limit of a wait (the waits read both as one 8-byte word)
     uint32_t tmem_base;
-    int abort;
     int merge_here[2];
     int direct;
     int32_t pg[kPgTiles][kPgSub];      // paged cache: page ids of the tiles about to be fetched
@@ -132,6 +132,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 mbar_init(&sm.o_done[s][h], 1);
             }
         sm.abort = 0;
+        sm.wait_kcycles = p.wait_kcycles;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x == 32) {                 // descriptors on their way while the CTA sets itself up

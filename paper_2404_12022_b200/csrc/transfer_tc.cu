@@ -38,8 +38,8 @@ struct TParams {
 
 struct TBars {
     unsigned long long full[kMaxStages], empty[kMaxStages], acc_full, mma_drain;
+    int abort, wait_kcycles;           // the abort flag, and right behind it the limit of a wait (the waits read both as one 8-byte word)
     uint32_t tmem_base;
-    int abort;
 };
 
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, void *bar, int c0, int c1) {
@@ -84,6 +84,7 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
         mbar_init(&bar.acc_full, 1);
         mbar_init(&bar.mma_drain, 1);
         bar.abort = 0;
+        bar.wait_kcycles = tc::kWaitKcycles;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x == 32) {

@@ -280,6 +280,29 @@ def test_attention_calls_in_a_row_see_each_others_results(hb, shape):
     assert bool(((a.float() - b.float()).abs() <= ulp * a.float().abs() + 1e-6).all())
 
 
+@pytest.mark.parametrize("shape", [(5, 37, 32, 32, [900, 640, 33, 1200, 512]), (2, 19, 64, 8, [3000, 2500])],
+                         ids=lambda s: "B%dN%dHq%dHkv%d" % s[:4])
+def test_attention_waits_that_run_out_are_reported_and_leave_the_device_usable(hb, oracle, shape):
+    """Failure detection without a fault: with the test hook the kernels' waits give up after about a microsecond,
+    which is less than the first tile takes to arrive (one-tile and tile-pair kernel, one persistent CTA per SM, no
+    clusters).  The call must return with HT_STATUS_TIMEOUT for every sequence, and the next ordinary call on the same
+    stream, workspace and output buffer must be correct: nothing was left in flight and no tensor memory was lost."""
+    B, N, Hq, Hkv, lens = shape
+    q, k, v, kv_len, parent = make_attn_case(19, "bf16", B, N, Hq, Hkv, 128, lens, max(lens) + N + 5)
+    desc = hb.make_attn_desc(q, k)
+    ws = torch.empty(max(hb.tree_attention_workspace(desc), 16), dtype=torch.uint8, device="cuda")
+    out = torch.empty_like(q)
+    for _ in range(3):
+        _, status = hb.tree_attention(q, k, v, kv_len, parent, out=out, workspace=ws, flags=hb.HT_ATTN_TEST_SHORT_WAITS)
+        torch.cuda.synchronize()
+        assert status.cpu().tolist() == [hb.HT_STATUS_TIMEOUT] * B
+    for _ in range(2):
+        _, status = hb.tree_attention(q, k, v, kv_len, parent, out=out, workspace=ws)
+        torch.cuda.synchronize()
+        assert status.cpu().tolist() == [0] * B
+        check_sampled_units(hb, oracle, q, k, v, kv_len.cpu().numpy(), parent, out, 6, torch.bfloat16, seed=3)
+
+
 @pytest.mark.parametrize("shape", [(3, 9, 4, 2), (3, 40, 32, 8), (40, 9, 8, 4)], ids=lambda s: "B%dN%dHq%dHkv%d" % s)
 def test_attention_tensor_core_paths_skip_bad_sequences(hb, oracle, shape):
     """Status words and untouched rows on the 16-bit kernels (clusters, tile pairs, persistent)."""
