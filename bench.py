@@ -1,6 +1,6 @@
 """Benchmark of the tree-verify step (one JSON line on stdout).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c2|c4] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c1|c2|c4] [--impl reference]
 
 A step is one pass of the whole hot path over one batch of synthetic input: per layer a
 tree-attention call, the hidden-transfer projection at the transfer layer, greedy
@@ -40,22 +40,10 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4"])
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
-    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling small cases)")
-    ap.add_argument("--kv", type=int, default=0, help="override the KV length of c3 (profiling small cases)")
-    ap.add_argument("--splits", type=int, default=0)
-    ap.add_argument("--simt", action="store_true", help="force the fp32-ALU attention kernel")
     ap.add_argument("--eager", action="store_true", help="enqueue every library call from the host instead of replaying a CUDA graph of the step")
     ap.add_argument("--no-extras", action="store_true", help="skip e2e, cpu baseline and per-kernel timing")
     ap.add_argument("--fused", choices=["auto", "on", "off"], default="auto",
                     help="verification and compaction as one launch (ht_verify_greedy_compact) or as two calls; auto: one launch for few (layer, sequence) pairs")
-    ap.add_argument("--sweep", default="", help="instead of the step benchmark, time ht_tree_attention alone on a set of "
-                    "workloads and print one JSON line per point: 'configs' (c2, c2 at KV 2048, a c3 layer, c4) or "
-                    "'c5' (the 48 grouped-query points) or 'c5-quick' (12 of them); 'transfer' times ht_transfer alone, with a "
-                    "pseudo state per sequence (B rows) and per tree node (B x T rows)")
-    ap.add_argument("--paged", type=int, default=0, help="with --sweep configs / c5: the same workloads with the cache cut into pages "
-                    "of this many rows, placed in a seeded random order in a pool (ht_tree_attention_paged)")
-    ap.add_argument("--only", default="", help="with --sweep: keep the workloads whose name contains this text")
-    ap.add_argument("--sweep-reps", type=int, default=0, help="with --sweep: calls per graph (profiling small cases)")
     return ap.parse_args()
 
 
@@ -67,12 +55,7 @@ def make_workload(args):
         return wl.config_c2()
     if args.workload == "c4":
         return wl.config_c4()
-    kw = {}
-    if args.layers:
-        kw["layers"] = args.layers
-    if args.kv:
-        kw["kv"] = args.kv
-    return wl.config_c3(**kw)
+    return wl.config_c3()
 
 
 def workload_config(w, n_gpus):
@@ -226,14 +209,25 @@ class ClockSampler:
 # profiles/attn_tc_kernel_c3_layer.md (dram__bytes_read.sum + dram__bytes_write.sum).  It is only
 # reported while the kernel source is the one that was profiled.
 NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.4e6,
-               "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh"],
-               "sha256": "d66636ddd95c59df34ad061efdbffc6603c6424f70aa605dff8ee93e7b7a18d9"}
+               "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh",
+                          "paper_2404_12022_b200/csrc/ht_common.cuh"],
+               "sha256": "to be taken with the next capture"}
+
+
+def traffic_digest():
+    """SHA-256 of the attention kernel's sources and of the compiler flags they are built with."""
+    import hashlib
+    from paper_2404_12022_b200 import build
+    h = hashlib.sha256()
+    for f in NCU_TRAFFIC["source"]:
+        h.update(open(os.path.join(ROOT, f), "rb").read())
+    h.update(" ".join(build.NVCC_FLAGS).encode())
+    return h.hexdigest()
 
 
 def ncu_traffic(w):
-    import hashlib
     try:
-        digest = hashlib.sha256(b"".join(open(os.path.join(ROOT, f), "rb").read() for f in NCU_TRAFFIC["source"])).hexdigest()
+        digest = traffic_digest()
     except OSError:
         return None
     if digest != NCU_TRAFFIC["sha256"] or w.name != NCU_TRAFFIC["workload"] or w.kv_len[0] != 4096 or w.B != 4:
@@ -282,7 +276,7 @@ def run_native(args):
 
     w = make_workload(args)
     inp = wl.make_inputs(w, "cuda")
-    step = VerifyStep(inp, num_splits=args.splits, flags=hb.HT_ATTN_FORCE_SIMT if args.simt else 0, fused={"auto": None, "on": True, "off": False}[args.fused])
+    step = VerifyStep(inp, fused={"auto": None, "on": True, "off": False}[args.fused])
     stream = torch.cuda.current_stream().cuda_stream
 
     def barrier():
@@ -300,13 +294,14 @@ def run_native(args):
         run_step()
     barrier()
     sampler = ClockSampler(local) if rank == 0 else None
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    marks[0].record()
+    for i in range(args.steps):
         run_step()
-    e1.record()
+        marks[i + 1].record()          # a mark per step (median and minimum); the figure is first mark to last
     barrier()
-    ms_total = e0.elapsed_time(e1)
+    ms_total = marks[0].elapsed_time(marks[-1])
+    per_step_us = [marks[i].elapsed_time(marks[i + 1]) * 1e3 for i in range(args.steps)]
     clocks = sampler.stop() if sampler else None
     step_bytes = step.step_bytes()
     ms_step, value = replica_aggregate(ms_total, args.steps, step_bytes, world, "cuda")
@@ -318,7 +313,8 @@ def run_native(args):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": w.dtype, "data": "synthetic", "config": workload_config(w, world),
-            "step_us": ms_step * 1e3, "step_bytes": step_bytes, "clocks": clocks,
+            "step_us": ms_step * 1e3, "step_us_median": statistics.median(per_step_us), "step_us_min": min(per_step_us),
+            "step_bytes": step_bytes, "clocks": clocks,
             "launch": "eager C-ABI calls" if args.eager else "CUDA graph of the step's C-ABI calls"}
     # launches of this library's kernels per step: the attention calls' (ht_tree_attention_launches), transfer (one
     # per batch slice of 16), verification with the compaction in the same launch
@@ -326,6 +322,7 @@ def run_native(args):
 
     if rank == 0 and not args.no_extras:
         line["roofline"], line["kernels"] = per_kernel_pass(args, step, stream, torch)
+        line["sustained"] = sustained_pass(run_step, step, local, line["kernels"]["attention"]["share"], torch)
         line["e2e"] = e2e_pass(args, step, inp, torch, world)
         sample = OracleSample(w)
         dt, done = time_oracle(sample, 1000, 0, budget_s=12.0)
@@ -337,6 +334,36 @@ def run_native(args):
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(line), flush=True)
+
+
+def sustained_pass(run_step, step, device_index, attention_share, torch, seconds=2.0):
+    """The same step replayed back to back for at least `seconds`, with the SM clock sampled meanwhile: what the
+    step costs once the power cap has settled the clocks (the timed run above is a burst).  ms x MHz tells how much
+    of a difference between two runs is clock."""
+    peak, _ = measured_peaks()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    run_step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(device_index)
+    t0 = time.perf_counter()
+    n = 0
+    e0.record()
+    while time.perf_counter() - t0 < seconds:
+        for _ in range(50):
+            run_step()
+        n += 50
+        torch.cuda.synchronize()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / n
+    attn_bytes = sum(step.attention_bytes(i) for i in range(step.layers))
+    attn_gbs = attn_bytes / (ms * 1e-3 * attention_share) / 1e9
+    return {"steps": n, "ms_per_step": ms, "value": step.step_bytes() / (ms * 1e-3) / 1e9, "unit": UNIT,
+            "sm_mhz": clocks["sm_mhz"], "reasons": clocks["reasons"],
+            "ms_x_mhz": ms * clocks["sm_mhz"] if clocks["sm_mhz"] else None,
+            "attention_gbs": attn_gbs, "attention_frac": attn_gbs / peak,
+            "note": "attention_gbs = attention bytes of a step / (the step's sustained time x the attention calls' share of the per-kernel pass)"}
 
 
 def kernels_per_attention(step, i):
@@ -525,153 +552,8 @@ def e2e_pass(args, step, inp, torch, world):
             "note": "KV cache and transfer weights resident; per-step inputs from pinned host memory, copies of layer i+1 overlap the kernels of layer i"}
 
 
-# ------------------------------------------------------------------------------------------
-# Attention-only sweep over the other workloads (not the bench line; feeds the results tables)
-# ------------------------------------------------------------------------------------------
-
-def sweep_points(which):
-    from paper_2404_12022_b200 import workloads as wl
-    import dataclasses
-    if which == "configs":
-        c2 = wl.config_c2()
-        return [c2, dataclasses.replace(c2, name="c2_at_kv2048", kv_len=[2048]), wl.config_c3(layers=1), wl.config_c4()]
-    pts = wl.c5_points()
-    if which == "c5-quick":
-        pts = [p for p in pts if p[2] == 4 and p[1] in (16, 64, 256)]
-    return [wl.config_c5(*p) for p in pts]
-
-
-def run_sweep(args):
-    """CUDA-event time of ht_tree_attention per call, replayed from a CUDA graph of `reps` calls
-    that rotate over enough copies of the cache to exceed twice the L2 (cold-L2 protocol)."""
-    import torch
-    from paper_2404_12022_b200 import binding as hb
-    from paper_2404_12022_b200 import workloads as wl
-    torch.cuda.set_device(0)
-    peak, how = measured_peaks()
-    l2 = torch.cuda.get_device_properties(0).L2_cache_size
-    for w in [x for x in sweep_points(args.sweep) if args.only in x.name]:
-        inp = wl.make_inputs(w, "cuda", with_logits=False, with_transfer=False, layers=[w.layers - 1])
-        q, kv_len, parent = inp.q[0], inp.kv_len, inp.parent
-        e = w.elem_bytes()
-        cache_bytes = 2 * inp.k_cache[0].numel() * e
-        nbuf = int(min(64, max(2, -(-2 * l2 // cache_bytes))))
-        ks = [inp.k_cache[0]] + [wl.normal_tensor(w.seed, 10 + i, tuple(inp.k_cache[0].shape), "cuda", 1.0, w.torch_dtype())
-                                 for i in range(nbuf - 1)]
-        vs = [inp.v_cache[0]] + [wl.normal_tensor(w.seed, 100 + i, tuple(inp.k_cache[0].shape), "cuda", 1.0, w.torch_dtype())
-                                 for i in range(nbuf - 1)]
-        out = torch.empty_like(q)
-        st = torch.zeros(w.B, dtype=torch.int32, device="cuda")
-        desc = hb.make_attn_desc(q, ks[0])
-        ws = torch.empty(max(hb.tree_attention_workspace(desc), 16), dtype=torch.uint8, device="cuda")
-        reps = args.sweep_reps or max(nbuf, 16)
-        call = lambda i: hb.tree_attention(q, ks[i % nbuf], vs[i % nbuf], kv_len, parent, out=out, workspace=ws, status=st)
-        if args.paged:
-            ps = args.paged
-            B, Hkv, cap, D = ks[0].shape
-            per = cap // ps
-            assert per * ps == cap, "--paged must divide the cache capacity %d" % cap
-            g = torch.Generator(device="cpu").manual_seed(w.seed)
-            table = torch.randperm(B * per, generator=g).to(torch.int32).reshape(B, per).cuda()
-
-            def to_pool(c):      # page table[b][i] of the pool holds rows [i ps, (i + 1) ps) of sequence b
-                pool = torch.empty((B * per, Hkv, ps, D), dtype=c.dtype, device="cuda")
-                pool[table.reshape(-1).long()] = c.view(B, Hkv, per, ps, D).permute(0, 2, 1, 3, 4).reshape(B * per, Hkv, ps, D)
-                return pool
-            ks = [to_pool(c) for c in ks]
-            vs = [to_pool(c) for c in vs]
-            call = lambda i: hb.tree_attention_paged(q, ks[i % nbuf], vs[i % nbuf], table, kv_len, parent, out=out,
-                                                     workspace=ws, status=st)
-        for i in range(3):
-            call(i)
-        torch.cuda.synchronize()
-        graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side), torch.cuda.graph(graph, stream=side):
-            for i in range(reps):
-                call(i)
-        torch.cuda.synchronize()
-        graph.replay()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        times = []
-        for _ in range(5):
-            e0.record(); graph.replay(); e1.record(); torch.cuda.synchronize()
-            times.append(e0.elapsed_time(e1) / reps * 1e3)
-        us = statistics.median(times)
-        rows = q.shape[1]
-        byts = sum(2 * w.Hkv * (L + rows) * w.D * e for L in w.kv_len) + 2 * w.B * rows * w.Hq * w.D * e + 4 * w.B * rows
-        flops = sum(4 * rows * w.Hq * (L + rows) * w.D for L in w.kv_len)
-        assert int(st.abs().sum()) == 0
-        print(json.dumps({"workload": w.name, "batch": w.B, "kv_len": w.kv_len[0] if len(set(w.kv_len)) == 1 else "ragged",
-                          "rows": rows, "q_heads": w.Hq, "kv_heads": w.Hkv, "dtype": w.dtype, "us": round(us, 2),
-                          "hbm_gbs": round(byts / us / 1e3, 1), "frac_of_measured_hbm": round(byts / us / 1e3 / peak, 3),
-                          "frac_of_8tbs": round(byts / us / 1e3 / 8000.0, 3), "tflops": round(flops / us / 1e6, 1),
-                          "flop_per_byte": round(flops / byts, 1), "cold_l2_copies": nbuf,
-                          "cache": ("pages of %d rows" % args.paged) if args.paged else "contiguous"}), flush=True)
-        del ks, vs, inp, ws, graph
-
-
-# (name, source rows, k, d): the configurations' projections with pseudo states hanging off one node per
-# sequence (B rows) and off every tree node (B x T rows)
-TRANSFER_POINTS = [("c2_per_sequence", 1, 3, 4096), ("c3_per_sequence", 4, 3, 4096), ("c4_per_sequence", 8, 4, 5120),
-                   ("c5_per_sequence_b16", 16, 3, 8192), ("c2_per_node", 88, 3, 4096), ("c3_per_node", 352, 3, 4096),
-                   ("c4_per_node", 512, 4, 5120), ("c5_per_node_b4_t256", 1024, 3, 8192),
-                   ("c5_per_node_b16_t256", 4096, 3, 8192)]
-
-
-def run_transfer_sweep(args):
-    """CUDA-event time of ht_transfer per call, replayed from a CUDA graph whose calls rotate over
-    enough copies of W to exceed twice the L2."""
-    import torch
-    from paper_2404_12022_b200 import binding as hb
-    from paper_2404_12022_b200 import workloads as wl
-    torch.cuda.set_device(0)
-    peak, how = measured_peaks()
-    l2 = torch.cuda.get_device_properties(0).L2_cache_size
-    tensor_peak = None
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(path):
-        tensor_peak = float(json.load(open(path)).get("bf16_tflops", 0.0)) or None
-    for name, B, k, d in [x for x in TRANSFER_POINTS if args.only in x[0]]:
-        wbytes = k * d * d * 2
-        ncopy = int(max(2, -(-2 * l2 // wbytes)))
-        h = wl.normal_tensor(31, 1, (B, d), "cuda", 1.0, torch.bfloat16)
-        Ws = [wl.normal_tensor(31, 2 + i, (k, d, d), "cuda", 0.02, torch.bfloat16) for i in range(ncopy)]
-        out = torch.empty((B, k, d), dtype=torch.bfloat16, device="cuda")
-        for i in range(3):
-            hb.transfer(h, Ws[i % ncopy], out)
-        torch.cuda.synchronize()
-        reps = args.sweep_reps or ncopy * (4 if B <= 512 else 1)
-        graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side), torch.cuda.graph(graph, stream=side):
-            for i in range(reps):
-                hb.transfer(h, Ws[i % ncopy], out)
-        torch.cuda.synchronize()
-        graph.replay()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        times = []
-        for _ in range(5):
-            e0.record(); graph.replay(); e1.record(); torch.cuda.synchronize()
-            times.append(e0.elapsed_time(e1) / reps * 1e3)
-        us = statistics.median(times)
-        byts = wbytes + B * d * 2 + B * k * d * 2
-        flops = 2.0 * B * k * d * d
-        line = {"workload": "transfer_" + name, "rows": B, "k": k, "d": d, "dtype": "bf16", "us": round(us, 2),
-                "hbm_gbs": round(byts / us / 1e3, 1), "frac_of_measured_hbm": round(byts / us / 1e3 / peak, 3),
-                "tflops": round(flops / us / 1e6, 1), "flop_per_byte": round(flops / byts, 1), "cold_l2_copies": ncopy}
-        if tensor_peak:
-            line["frac_of_measured_bf16"] = round(flops / us / 1e6 / tensor_peak, 3)
-        print(json.dumps(line), flush=True)
-        del Ws, graph
-
-
 def main():
     args = parse_args()
-    if args.sweep == "transfer":
-        return run_transfer_sweep(args)
-    if args.sweep:
-        return run_sweep(args)
     if args.impl == "reference":
         run_reference(args)
     else:

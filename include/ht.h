@@ -2,14 +2,17 @@
  * ht.h -- C ABI of the B200 tree-verify library for Hidden Transfer decoding
  * (arXiv 2404.12022).  One decoding round verifies a flattened draft tree and the
  * pseudo positions produced by the hidden-transfer projection in a single forward; this
- * library holds the four data-parallel operations of that forward that are specific to
- * the method.  Everything else of the transformer layer (norms, Q/K/V/O and MLP GEMMs,
- * rotary embedding, lm-head) is the caller's.
+ * library holds the data-parallel operations of that forward that are specific to the
+ * method (projection, tree attention, verification, compaction) and the steps around them
+ * (rotary embedding + cache append, draft tree, a paged cache).  Everything else of the
+ * transformer layer (norms, Q/K/V/O and MLP GEMMs, lm-head) is the caller's.
  *
  * Conventions for every entry point
  *   - Pointers are DEVICE pointers unless a comment says "host".  The caller owns every
- *     buffer, workspace included; the library allocates no device memory and keeps no
- *     state between calls.
+ *     buffer, workspace included; the library allocates no device memory.  What it keeps
+ *     between calls is per-device set-up only (kernel attributes, SM count, how many of a
+ *     kernel's blocks the device holds, the address of the built-in scratch array of
+ *     ht_tree_attention_static); a cudaDeviceReset makes that stale.
  *   - Work is enqueued on the caller's stream (`stream` is a cudaStream_t passed as
  *     void*; NULL = the default stream) and the call returns without synchronising.
  *   - The return value is a host-checkable status (HT_OK or HT_ERR_*).  When it is not
@@ -105,7 +108,8 @@ const char *ht_last_error_string(void);
  * hanging off one node), or one per tree node of every sequence (the reading in which
  * every token gets its pseudo states), B x T rows, for which the 16-bit types run as a
  * matrix product on the tensor cores in one pass over W.  That kernel's waits are bounded
- * (about a second); should one run out, the outputs of the affected tile are NaN.
+ * (about a second); should one run out, the outputs of the affected tile are NaN -- the call
+ * has no status argument, so a NaN tile is the only signal (NaN inputs give NaN too).
  * All pointers are device pointers, 16-byte aligned; nothing is retained after the call.
  */
 int ht_transfer(const void *h_src, const void *W, void *out, int B, int k, int d, int dtype,
@@ -165,7 +169,7 @@ int ht_tree_attention(const ht_attn_desc *desc /* host */, const void *q, const 
  *                      needed entries lies outside [0, n_pages): page 0 is read in its place (no
  *                      access outside the pool) and the sequence's rows of `out` are meaningless.
  * q, kv_len, parent, out, workspace (ht_tree_attention_workspace(desc) bytes) as in
- * ht_tree_attention.  Supported: fp16 / bf16, D = 128, Hq / Hkv a power of two, N <= 512,
+ * ht_tree_attention.  Supported: fp16 / bf16, D = 128, Hq / Hkv a power of two, N <= 1024,
  * B <= 256 (the tensor-core kernels); anything else returns HT_ERR_UNSUPPORTED.
  */
 typedef struct {

@@ -3,9 +3,17 @@
 #include <stdarg.h>
 #include <stdio.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "compact.cuh"
 
 namespace ht {
+
+// A named range around every entry point, for timelines taken with a profiler (a no-op without one attached).
+struct Range {
+    explicit Range(const char *name) { nvtxRangePushA(name); }
+    ~Range() { nvtxRangePop(); }
+};
 
 static thread_local char g_err[512] = "no error";
 
@@ -63,6 +71,7 @@ const char *ht_last_error_string(void) { return g_err; }
 
 int ht_transfer(const void *h_src, const void *W, void *out, int B, int k, int d, int dtype,
                 void *stream) {
+    Range range("ht_transfer");
     if (B < 0 || k < 0 || d < 0) return fail(HT_ERR_INVALID_ARG, "negative size");
     if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     if ((long long)B * k * d == 0) return HT_OK;
@@ -95,6 +104,7 @@ int ht_tree_attention_launches(const ht_attn_desc *desc) {
 int ht_tree_attention(const ht_attn_desc *desc, const void *q, const void *k_cache, const void *v_cache,
                       const int32_t *kv_len, const int32_t *parent, void *out, void *workspace,
                       size_t workspace_bytes, int32_t *status, void *stream) {
+    Range range("ht_tree_attention");
     int rc = check_attn_desc(desc);
     if (rc != HT_OK) return rc;
     if (desc->B == 0 || desc->N == 0) return HT_OK;
@@ -117,6 +127,7 @@ int ht_tree_attention_paged(const ht_attn_desc *desc, const ht_paged_desc *pages
                             const void *v_pages, const int32_t *block_table, const int32_t *kv_len,
                             const int32_t *parent, void *out, void *workspace, size_t workspace_bytes,
                             int32_t *status, void *stream) {
+    Range range("ht_tree_attention_paged");
     if (!desc || !pages) return fail(HT_ERR_INVALID_ARG, "NULL descriptor");
     const int ps = pages->page_size;
     if (ps < 16 || (ps & (ps - 1)) != 0) return fail(HT_ERR_INVALID_ARG, "page_size must be a power of two >= 16");
@@ -140,7 +151,7 @@ int ht_tree_attention_paged(const ht_attn_desc *desc, const ht_paged_desc *pages
     if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out) || (workspace && !aligned16(workspace)))
         return fail(HT_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
     if (!attn_tc_applicable(d))
-        return fail(HT_ERR_UNSUPPORTED, "paged cache: fp16 / bf16, D = 128, Hq / Hkv a power of two, N <= 512, B <= 256, no flags or splits");
+        return fail(HT_ERR_UNSUPPORTED, "paged cache: fp16 / bf16, D = 128, Hq / Hkv a power of two, N <= 1024, B <= 256, no kernel choice by flag, no splits");
     const size_t need = attn_tc_workspace(d);      // does not depend on the capacity
     if (need > 0 && (!workspace || workspace_bytes < need))
         return fail(HT_ERR_WORKSPACE, "workspace holds %zu bytes, %zu needed", workspace ? workspace_bytes : 0, need);
@@ -152,6 +163,7 @@ int ht_verify_greedy(const void *logits, int dtype, const int32_t *tokens, const
                      const int32_t *root_pred, int B, int N, int T, int V, int max_path, int32_t *pred,
                      int32_t *accept_len, int32_t *accept_path, int32_t *next_token, int32_t *status,
                      void *stream) {
+    Range range("ht_verify_greedy");
     if (B < 0 || N < 0 || T < 0 || T > N) return fail(HT_ERR_INVALID_ARG, "need 0 <= T <= N and B >= 0");
     if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     if (B == 0) return HT_OK;
@@ -188,6 +200,7 @@ int ht_verify_greedy_compact(const void *logits, int dtype, const int32_t *token
                              int32_t *pred, int32_t *accept_len, int32_t *accept_path, int32_t *next_token,
                              int32_t *status, void *k_cache, void *v_cache, const ht_cache_desc *desc,
                              const int32_t *kv_len, int32_t *new_kv_len, int32_t *compact_status, void *stream) {
+    Range range("ht_verify_greedy_compact");
     if (B < 0 || N < 0 || T < 0 || T > N) return fail(HT_ERR_INVALID_ARG, "need 0 <= T <= N and B >= 0");
     if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     int rc = check_cache_desc(desc, max_path);
@@ -217,6 +230,7 @@ int ht_verify_greedy_compact(const void *logits, int dtype, const int32_t *token
 int ht_kv_compact(void *k_cache, void *v_cache, const ht_cache_desc *desc, const int32_t *kv_len,
                   const int32_t *accept_len, const int32_t *accept_path, int max_path,
                   int32_t *new_kv_len, int32_t *status, void *stream) {
+    Range range("ht_kv_compact");
     if (!desc) return fail(HT_ERR_INVALID_ARG, "desc is NULL");
     if (desc->layers <= 0 || desc->B < 0 || desc->Hkv <= 0 || desc->cap <= 0 || desc->D <= 0 || desc->N < 0)
         return fail(HT_ERR_INVALID_ARG, "bad cache sizes");
@@ -245,6 +259,7 @@ int ht_draft_tree(const void *logits, int dtype, int B, int rows, int V, int fir
                   const int32_t *tmpl_parent, const int32_t *tmpl_rank, int T, const int32_t *root_token,
                   const int32_t *base_pos, int32_t *topk, int32_t *tokens, int32_t *pos, int32_t *status,
                   void *stream) {
+    Range range("ht_draft_tree");
     if (B < 0 || rows < 0 || P < 0 || first_row < 0) return fail(HT_ERR_INVALID_ARG, "negative size");
     if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     if (B == 0) return HT_OK;
@@ -262,6 +277,7 @@ int ht_draft_tree(const void *logits, int dtype, int B, int rows, int V, int fir
 int ht_rope_kv_append(const ht_attn_desc *desc, const void *q_in, const void *k_in, const void *v_in, const int32_t *pos,
                       const int32_t *kv_len, float rope_base, void *q_out, void *k_cache, void *v_cache, int32_t *status,
                       void *stream) {
+    Range range("ht_rope_kv_append");
     int rc = check_attn_desc(desc);
     if (rc != HT_OK) return rc;
     if (desc->B == 0 || desc->N == 0) return HT_OK;
@@ -293,6 +309,7 @@ static int check_paged_desc(const ht_paged_desc *pages, int Hkv, int D) {
 int ht_rope_kv_append_paged(const ht_attn_desc *desc, const ht_paged_desc *pages, const void *q_in, const void *k_in,
                             const void *v_in, const int32_t *pos, const int32_t *kv_len, const int32_t *block_table,
                             float rope_base, void *q_out, void *k_pages, void *v_pages, int32_t *status, void *stream) {
+    Range range("ht_rope_kv_append_paged");
     if (!desc) return fail(HT_ERR_INVALID_ARG, "NULL descriptor");
     int rc = check_paged_desc(pages, desc->Hkv, desc->D);
     if (rc != HT_OK) return rc;
@@ -316,6 +333,7 @@ int ht_rope_kv_append_paged(const ht_attn_desc *desc, const ht_paged_desc *pages
 int ht_kv_compact_paged(void *k_pages, void *v_pages, const ht_cache_desc *desc, const ht_paged_desc *pages,
                         const int32_t *block_table, const int32_t *kv_len, const int32_t *accept_len,
                         const int32_t *accept_path, int max_path, int32_t *new_kv_len, int32_t *status, void *stream) {
+    Range range("ht_kv_compact_paged");
     if (!desc) return fail(HT_ERR_INVALID_ARG, "desc is NULL");
     if (desc->layers <= 0 || desc->B < 0 || desc->Hkv <= 0 || desc->D <= 0 || desc->N < 0)
         return fail(HT_ERR_INVALID_ARG, "bad cache sizes");
