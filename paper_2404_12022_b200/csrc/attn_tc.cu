@@ -133,7 +133,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // up while that kernel was still finishing, and everything it may have written is read from here on.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0, kPaged);
+    plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0, kPaged, p.n_rt);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -169,7 +169,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             cur_v.init(t_begin, t_end);
             cur_p.init(t_begin, t_end);
             if (kPaged)
-                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p, lane);
+                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p, lane, p.n_rt);
             for (int e = 0; e < 2 * n; ++e) {
                 if (kPaged ? __any_sync(0xFFFFFFFFu, *abort_flag != 0) : (*abort_flag != 0)) break;
                 // entry e of the consumption order: K_0, K_1, V_0, K_2, V_1, ..., V_{n-1}
@@ -203,7 +203,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
                 if (kPaged && !is_v) {
                     // the ids of tile j were asked for kPgAhead tiles ago; ask for those of tile j + kPgAhead
-                    pages_request(p, pp, sm.pre, sm.nkt, sm.pg, j + kPgAhead, cur_p, lane);
+                    pages_request(p, pp, sm.pre, sm.nkt, sm.pg, j + kPgAhead, cur_p, lane, p.n_rt);
                     cp_async_wait<kPgAhead>();
                 }
                 if (lane == 0) mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
@@ -356,6 +356,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 cu.t0 = sm.pre[sg.b] + (sg.hk * p.n_rt + sg.rt) * sg.nkt;
                 cu.c_lo = cu.t0 / per;
                 cu.c_hi = (cu.t0 + sg.nkt - 1) / per;
+                cu.cta_mul = 1; cu.cta_add = 0;
             }
 
             float m_ref = -INFINITY, l_sum = 0.f;

@@ -461,7 +461,7 @@ __device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nk
 // Validates every sequence and fills len / nkt / pre.  Called by all threads of a block.
 template <int NT>
 __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, int32_t *s_nkt, int32_t *s_pre,
-                                               bool write_status, bool errors_only = false) {
+                                               bool write_status, bool errors_only, int units_per_head) {
     // The lengths are asked for first and used last, so that their round trip to memory overlaps
     // the scan of the parent arrays (B <= kMaxB <= NT: one sequence per thread).
     const int my_b = threadIdx.x;
@@ -490,7 +490,7 @@ __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, 
         int acc = 0;
         for (int b = 0; b < p.B; ++b) {
             s_pre[b] = acc;
-            acc += s_nkt[b] * p.Hkv * p.n_rt;
+            acc += s_nkt[b] * p.Hkv * units_per_head;
         }
         s_pre[p.B] = acc;
     }
@@ -505,8 +505,8 @@ __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, 
 // never stalls the fetches.
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ void pages_request(const Params &p, const PagedParams &pp, const int32_t *pre, const int32_t *nkt,
-                                              int32_t (*pg)[kPgSub], int jt, TileCursor &cur, int lane) {
-    if (cur.next(pre, nkt, p.B, p.n_rt)) {               // `cur` walks the range one tile per call: this is tile jt
+                                              int32_t (*pg)[kPgSub], int jt, TileCursor &cur, int lane, int n_rt_list) {
+    if (cur.next(pre, nkt, p.B, n_rt_list)) {               // `cur` walks the range one tile per call: this is tile jt
         const int sub = pp.page_size >= kTile ? 1 : kTile >> pp.page_shift;
         const int first = (cur.kt() * kTile) >> pp.page_shift;
         if (lane < sub) {                                // lane x: page x of the tile
@@ -584,7 +584,8 @@ __device__ __forceinline__ uint32_t pack2_rest(float lo, float hi, uint32_t w) {
 
 // A unit that was cut between CTAs: which one, and which CTAs hold its parts.
 struct CutUnit {
-    int valid, unit, b, hk, rt, t0, c_lo, c_hi;
+    int valid, unit, b, hk, rt, t0, c_lo, c_hi;      // c_lo .. c_hi: places in the list's partition that hold the parts
+    int cta_mul, cta_add;                            // the CTA at place c is c * cta_mul + cta_add
 };
 
 // Merge of the parts of a cut unit by the 256 softmax threads of the CTA that delivered the
@@ -604,7 +605,7 @@ __device__ __noinline__ void merge_parts(const Params &p, const CutUnit &cu, int
     for (int x = 0; x < 64; ++x) acc[x] = 0.f;
 #pragma unroll 1
     for (int c = cu.c_lo; c <= cu.c_hi; ++c) {
-        const int slot = 2 * c + ((max(cu.t0, c * per) == c * per) ? 0 : 1);
+        const int slot = 2 * (c * cu.cta_mul + cu.cta_add) + ((max(cu.t0, c * per) == c * per) ? 0 : 1);
         const float *pslot = p.part + ((size_t)slot * subs + sub) * kSlotFloats;
         const float m = __ldcg(pslot + kRows * kD + row), lp = __ldcg(pslot + kRows * kD + kRows + row);
         float4 v[16];

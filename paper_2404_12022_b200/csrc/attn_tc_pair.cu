@@ -148,17 +148,33 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // up while that kernel was still finishing, and everything it may have written is read from here on.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0, kPaged);
+    // Without clusters, where a KV head has several tile pairs (units), the list of tiles is that of the HEADS: it is
+    // cut into grid / n_rt ranges, and the n_rt CTAs of a range take one tile pair each.  They start together and walk
+    // the same K / V tiles at the same pace, so that a tile crosses DRAM once and reaches the others from L2.  (With
+    // the units laid end to end instead, the CTAs that share a head's tiles meet them dozens of tiles apart: twice the
+    // algorithmic DRAM traffic on 4 x 8192 keys x 67 rows.)
+    const bool clustered = p.cluster_k > 1;
+    const bool grouped = !clustered && p.n_rt > 1;
+    const int lrt = grouped ? 1 : p.n_rt;                                   // units per head in the list
+    const int my_rt = grouped ? (int)blockIdx.x % p.n_rt : 0;               // grouped: this CTA's tile pair
+    const int my_pos = grouped ? (int)blockIdx.x / p.n_rt : (int)blockIdx.x; // place in the list's partition
+    const int n_pos = grouped ? p.grid / p.n_rt : p.grid;
+    plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0, kPaged, lrt);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
 
     const int total = sm.pre[p.B];
-    const int per = choose_per(total, p.grid, sm.nkt, p.B, p.n_rt);
-    int t_begin = min((int)blockIdx.x * per, total);
+    const int per = choose_per(total, n_pos, sm.nkt, p.B, lrt);
+    int t_begin = my_pos < n_pos ? min(my_pos * per, total) : total;
     int t_end = min(t_begin + per, total);
-    const bool clustered = p.cluster_k > 1;
+    // the segment that holds tile t of the list; grouped: the tile pair is the CTA's own
+    auto find = [&](int t, int te, int &hint) {
+        Segment sg = locate(sm.pre, sm.nkt, p.B, lrt, t, te, hint);
+        if (grouped) sg.rt = my_rt;
+        return sg;
+    };
     uint32_t c_rank = 0;
     if (clustered) {
         // One cluster per (sequence, KV head, tile pair); its CTAs take equal shares of the unit's tiles.  (No
@@ -183,11 +199,11 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             TileCursor cur_p;                         // page-id lookahead
             cur_p.init(t_begin, t_end);
             if (kPaged)
-                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p, lane);
+                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p, lane, lrt);
             bool stop = false;
             for (int t = t_begin; t < t_end && !stop;) {
                 if (kPaged ? __any_sync(0xFFFFFFFFu, *abort_flag != 0) : (*abort_flag != 0)) break;
-                const Segment s = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
+                const Segment s = find(t, t_end, b_hint);
                 const bool two = 2 * s.rt + 1 < p.n_row_tiles;
                 {
                     bool ok = seg_i == 0 || mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag);
@@ -212,7 +228,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const CUtensorMap *tm = (i & 1) ? &tm_v : &tm_k;
                     const int jt = t - t_begin + (i >> 1);            // tile of this CTA's range
                     if (kPaged && !(i & 1)) {
-                        pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt + kPgAhead, cur_p, lane);
+                        pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt + kPgAhead, cur_p, lane, lrt);
                         cp_async_wait<kPgAhead>();
                     }
                     if (lane == 0) mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
@@ -290,7 +306,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 pend = false;
             };
             for (int t = t_begin; t < t_end;) {
-                const Segment sg = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
+                const Segment sg = find(t, t_end, b_hint);
                 const bool act = s == 0 || 2 * sg.rt + 1 < p.n_row_tiles;
                 const int L = sm.len[sg.b];
                 alive = alive && mbar_wait_quick(smem_u32(&sm.q_full), seg_i & 1, abort_flag);
@@ -356,7 +372,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         int anc_b = -1, anc_rt = -1;                   // sequence / tile pair the ancestor words were built for
         uint32_t uses_s[2] = {0, 0}, uses_o[2] = {0, 0};   // uses of s_full[s][h] / o_done[s][h] so far
         for (int t = t_begin; t < t_end;) {
-            const Segment sg = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
+            const Segment sg = find(t, t_end, b_hint);
             const int L = sm.len[sg.b];
             const int row_tile = 2 * sg.rt + s;
             const bool active = row_tile < p.n_row_tiles;
@@ -384,7 +400,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 CutUnit &cu = cut[cut_k];
                 cu.unit = (sg.b * p.Hkv + sg.hk) * p.n_rt + sg.rt;
                 cu.b = sg.b; cu.hk = sg.hk; cu.rt = sg.rt;
-                cu.t0 = sm.pre[sg.b] + (sg.hk * p.n_rt + sg.rt) * sg.nkt;
+                cu.t0 = sm.pre[sg.b] + (grouped ? sg.hk : sg.hk * p.n_rt + sg.rt) * sg.nkt;
+                cu.cta_mul = grouped ? p.n_rt : 1; cu.cta_add = my_rt;
                 cu.c_lo = cu.t0 / per;
                 cu.c_hi = (cu.t0 + sg.nkt - 1) / per;
             }
@@ -561,8 +578,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 float g0, gb = 0.f;
                 if (dir) {
                     const CutUnit &cu = cut[cut_k];
-                    const int oc = (cu.c_lo == (int)blockIdx.x) ? cu.c_hi : cu.c_lo;
-                    oslot = p.part + ((size_t)(2 * oc + ((max(cu.t0, oc * per) == oc * per) ? 0 : 1)) * 2 + s) * kSlotFloats;
+                    const int oc = (cu.c_lo == my_pos) ? cu.c_hi : cu.c_lo;
+                    oslot = p.part + ((size_t)(2 * (oc * cu.cta_mul + cu.cta_add) + ((max(cu.t0, oc * per) == oc * per) ? 0 : 1)) * 2 + s) * kSlotFloats;
                     __threadfence();
                     const float m_o = __ldcg(oslot + kRows * kD + row), l_o = __ldcg(oslot + kRows * kD + kRows + row);
                     const float Mn = fmaxf(m_ref, m_o);
