@@ -42,8 +42,7 @@ def parse_args():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--eager", action="store_true", help="enqueue every library call from the host instead of replaying a CUDA graph of the step")
     ap.add_argument("--no-extras", action="store_true", help="skip e2e, cpu baseline and per-kernel timing")
-    ap.add_argument("--fused", choices=["auto", "on", "off"], default="auto",
-                    help="verification and compaction as one launch (ht_verify_greedy_compact) or as two calls; auto: one launch for few (layer, sequence) pairs")
+    ap.add_argument("--fused", action="store_true", help="verification and compaction as one launch (ht_verify_greedy_compact) instead of two calls")
     return ap.parse_args()
 
 
@@ -208,10 +207,10 @@ class ClockSampler:
 # DRAM traffic per launch of the attention kernel on a c3 layer, from the ncu capture summarised in
 # profiles/attn_tc_kernel_c3_layer.md (dram__bytes_read.sum + dram__bytes_write.sum).  It is only
 # reported while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.4e6,
+NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 289.2e6,
                "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh",
                           "paper_2404_12022_b200/csrc/ht_common.cuh"],
-               "sha256": "to be taken with the next capture"}
+               "sha256": "40a20d579b84e51d9b99b0744500ec43a6ddff94080805e84171374a646ce596"}
 
 
 def traffic_digest():
@@ -276,7 +275,7 @@ def run_native(args):
 
     w = make_workload(args)
     inp = wl.make_inputs(w, "cuda")
-    step = VerifyStep(inp, fused={"auto": None, "on": True, "off": False}[args.fused])
+    step = VerifyStep(inp, fused=args.fused)
     stream = torch.cuda.current_stream().cuda_stream
 
     def barrier():

@@ -2,9 +2,9 @@
 
 ``VerifyStep`` owns the descriptors, outputs and workspace of a workload so that a step is
 nothing but C-ABI calls on the current stream: per layer ``ht_tree_attention`` (with the
-pseudo rows joining after the transfer layer), one ``ht_transfer``, and verification plus
-compaction over all layers as one launch (``ht_verify_greedy_compact``; ``fused=False``: one
-``ht_verify_greedy`` and one ``ht_kv_compact``).  The dense parts of the
+pseudo rows joining after the transfer layer), one ``ht_transfer``, one ``ht_verify_greedy``
+and one ``ht_kv_compact`` over all layers (``fused=True``: the last two as one launch,
+``ht_verify_greedy_compact``).  The dense parts of the
 transformer layer between those calls are outside this library; their outputs (q, the new
 K/V rows, the logits) are inputs here.
 """
@@ -20,12 +20,12 @@ from .workloads import Inputs
 
 
 class VerifyStep:
-    def __init__(self, inp: Inputs, num_splits: int = 0, flags: int = 0, fused: Optional[bool] = None):
+    def __init__(self, inp: Inputs, num_splits: int = 0, flags: int = 0, fused: bool = False):
         # Verification and compaction as one launch (ht_verify_greedy_compact) or as two calls.  The chain of
-        # dependent steps is the same either way (argmax, count, path search, rows); measured behind an attention
-        # call, one launch is ahead for one sequence and one layer (16.1 against 17.1 us on config 2) and behind
-        # once the compaction has many (layer, sequence) items (21.5 against 19.9 us on config 3's 32 layers).
-        self.fused = (inp.k_cache.shape[0] * inp.w.B <= 4) if fused is None else fused
+        # dependent steps is the same either way (argmax, count, path search, rows), and so is the time within a
+        # microsecond or two: replayed in the graph of a whole step the two calls come out ahead (config 2: 51.5
+        # against 55.7 us per step; config 3's 32 layers: 19.9 against 21.5 us for the pair), so they are the default.
+        self.fused = fused
         w = inp.w
         self.inp = inp
         self.w = w

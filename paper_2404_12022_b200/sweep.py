@@ -171,7 +171,7 @@ def run_step(args):
     torch.cuda.set_device(0)
     w = wl.config_c3(layers=args.layers, kv=args.kv)
     inp = wl.make_inputs(w, "cuda")
-    step = VerifyStep(inp, fused={"auto": None, "on": True, "off": False}[args.fused])
+    step = VerifyStep(inp, fused=args.fused)
     stream = torch.cuda.current_stream().cuda_stream
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for _ in range(3):
@@ -227,7 +227,7 @@ def main():
     s.add_argument("--layers", type=int, default=2)
     s.add_argument("--kv", type=int, default=4096)
     s.add_argument("--steps", type=int, default=1)
-    s.add_argument("--fused", choices=["auto", "on", "off"], default="auto")
+    s.add_argument("--fused", action="store_true")
     sub.add_parser("peak")
     args = ap.parse_args()
     {"attention": run_attention, "transfer": run_transfer, "step": run_step, "peak": run_peak}[args.what](args)
