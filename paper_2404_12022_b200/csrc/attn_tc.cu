@@ -184,7 +184,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int kt = is_v ? cur_v.kt() : cur_k.kt();
                 if (!is_v && cur_k.first()) {
                     // first tile of a segment: its Q tile, once the previous segment's scores are done with Q
-                    bool ok = seg_i == 0 || mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag);
+                    bool ok = seg_i == 0 || mbar_wait_quick(smem_u32(&sm.q_empty), (seg_i - 1) & 1, abort_flag);
                     if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     if (lane == 0) {
@@ -196,7 +196,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 }
                 const int slot = ring_i % kStages, use = ring_i / kStages;
                 {
-                    bool ok = use == 0 || mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag);
+                    bool ok = use == 0 || mbar_wait_quick(smem_u32(&sm.kv_empty[slot]), (use - 1) & 1, abort_flag);
                     if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                 }

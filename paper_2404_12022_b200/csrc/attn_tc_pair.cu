@@ -206,7 +206,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const Segment s = find(t, t_end, b_hint);
                 const bool two = 2 * s.rt + 1 < p.n_row_tiles;
                 {
-                    bool ok = seg_i == 0 || mbar_wait(&sm.q_empty, (seg_i - 1) & 1, abort_flag);
+                    bool ok = seg_i == 0 || mbar_wait_quick(smem_u32(&sm.q_empty), (seg_i - 1) & 1, abort_flag);
                     if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                 }
@@ -222,7 +222,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int i = 0; i < 2 * s.len; ++i) {
                     const int kt = s.kt0 + (i >> 1);
                     const int slot = ring_i % kPStages, use = ring_i / kPStages;
-                    bool ok = use == 0 || mbar_wait(&sm.kv_empty[slot], (use - 1) & 1, abort_flag);
+                    bool ok = use == 0 || mbar_wait_quick(smem_u32(&sm.kv_empty[slot]), (use - 1) & 1, abort_flag);
                     if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) { stop = true; break; }
                     const CUtensorMap *tm = (i & 1) ? &tm_v : &tm_k;

@@ -110,7 +110,7 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
             int issued = 0, slot = 0, use = 0;         // slot and round of the ring, kept by counting (no division per step)
             for (int ks = 0; ks < nk; ++ks, ++slot) {
                 if (slot == p.stages) { slot = 0; ++use; }
-                if (use > 0 && !mbar_wait(&bar.empty[slot], (use - 1) & 1, abort_flag)) break;
+                if (use > 0 && !mbar_wait_quick(smem_u32(&bar.empty[slot]), (use - 1) & 1, abort_flag)) break;
                 unsigned char *a = base + (size_t)slot * p.stage_bytes;
                 if (ks < n_main) {
                     mbar_expect_tx(&bar.full[slot], (chunk_h + chunk_w) * p.kc);
@@ -140,7 +140,7 @@ transfer_tc_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_consta
             int slot = 0, use = 0;
             for (int ks = 0; ks < nk; ++ks, ++slot) {
                 if (slot == p.stages) { slot = 0; ++use; }
-                if (!mbar_wait(&bar.full[slot], use & 1, abort_flag)) { all = false; break; }
+                if (!mbar_wait_quick(smem_u32(&bar.full[slot]), use & 1, abort_flag)) { all = false; break; }
                 tc_fence_after();
                 // The descriptors differ in their address field only (16-byte units in the low bits, never
                 // carrying out of it inside this CTA's shared memory): one template each, then additions.
