@@ -63,6 +63,13 @@ enum {
 
 /* ht_attn_desc.flags */
 #define HT_ATTN_FORCE_SIMT 1u /* use the fp32-ALU kernel even where a tensor-core kernel applies */
+/* The caller vouches that the first 64 KiB of the workspace are as a cudaMemset to zero, or any earlier
+ * ht_tree_attention / ht_tree_attention_paged call on this workspace that reported no HT_STATUS_TIMEOUT, left
+ * them: the call then leaves out the small kernel that clears the arrival counters kept there (every call
+ * leaves the counters it used at zero).  Worth about a microsecond per call in a chain of calls; with the flag
+ * set on a workspace that is not in that state, results of sequences whose work was split are undefined
+ * (nothing faults, nothing waits). */
+#define HT_ATTN_WORKSPACE_CLEAN 2u
 /* Test hook, never to be set in production: the tensor-core kernels' device-side waits give up after about a
  * microsecond instead of a second, so that their give-up path can be exercised: the call returns, the sequences'
  * status words read HT_STATUS_TIMEOUT and `out` is meaningless.  Nothing faults and nothing is left in flight:
@@ -130,8 +137,9 @@ int ht_transfer(const void *h_src, const void *W, void *out, int B, int k, int d
  *            every ancestor c of r.  fp32 (fp16 / bf16 inputs: tensor-core products with
  *            fp32 accumulation) softmax and accumulation, rounded once to `dtype`.
  *   workspace, workspace_bytes  scratch of at least ht_tree_attention_workspace(desc)
- *            bytes, 16-byte aligned; contents need no initialisation and are undefined
- *            afterwards.  Calls that run concurrently need distinct workspaces.
+ *            bytes, 16-byte aligned; contents need no initialisation (but see
+ *            HT_ATTN_WORKSPACE_CLEAN) and, beyond the first 64 KiB, are undefined afterwards.
+ *            Calls that run concurrently need distinct workspaces.
  *   status   [B] int32 out: HT_STATUS_BAD_TREE / HT_STATUS_BAD_LEN sequences are skipped
  *            (their rows of `out` are left untouched).
  * Cache rows at or beyond kv_len[b] + N are never used for a result, whatever they hold.
@@ -143,8 +151,9 @@ int ht_transfer(const void *h_src, const void *W, void *out, int B, int k, int d
  */
 size_t ht_tree_attention_workspace(const ht_attn_desc *desc /* host */);
 /* Number of this library's kernels that one ht_tree_attention call with this descriptor enqueues (1 or 2:
- * a kernel that zeroes arrival counters, or one that merges split partials, may accompany the attention
- * kernel); 0 for a descriptor the call would reject or that has nothing to do. */
+ * a kernel that zeroes arrival counters -- left out under HT_ATTN_WORKSPACE_CLEAN -- or one that merges split
+ * partials, may accompany the attention kernel); 0 for a descriptor the call would reject or that has nothing
+ * to do. */
 int ht_tree_attention_launches(const ht_attn_desc *desc /* host */);
 int ht_tree_attention(const ht_attn_desc *desc /* host */, const void *q, const void *k_cache,
                       const void *v_cache, const int32_t *kv_len, const int32_t *parent, void *out,

@@ -484,7 +484,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             sm.ml[s][row][1] = l_sum;
             // With one other part and that part already in the workspace, this CTA finishes the unit
             // from its registers; otherwise it leaves its own part there.
-            if (tid256 == 0) sm.direct = !clustered && !complete && cut[cut_k].c_hi - cut[cut_k].c_lo == 1 && delivered_old == 1u;
+            if (tid256 == 0) {
+                sm.direct = !clustered && !complete && cut[cut_k].c_hi - cut[cut_k].c_lo == 1 && delivered_old == 1u;
+                // nobody touches the unit's counter any more: it is left at zero for the next call on this workspace
+                if (sm.direct) p.tickets[cut[cut_k].unit] = 0u;
+            }
             tc_fence_before();
             softmax_groups_sync();
             tc_fence_after();
@@ -608,8 +612,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
         if (cut[0].valid || cut[1].valid) {
             if (tid256 == 0)
-                for (int k = 0; k < 2; ++k)
+                for (int k = 0; k < 2; ++k) {
                     sm.merge_here[k] = cut[k].valid && ticket[k] == (unsigned)(cut[k].c_hi - cut[k].c_lo);
+                    if (sm.merge_here[k]) p.tickets[cut[k].unit] = 0u;      // all parts have arrived: zero again for the next call
+                }
             softmax_groups_sync();
             for (int k = 0; k < 2; ++k)
                 if (sm.merge_here[k]) {
@@ -710,9 +716,21 @@ static int cluster_size(const ht_attn_desc &d) {
     return 0;
 }
 
+// The units' arrival counters sit at the start of the workspace, in an area of a fixed size whatever the
+// descriptor (so that calls with different shapes on one workspace leave it clean for one another); more units than
+// it holds get an area of their own size, which is then always cleared by the kernel.
+constexpr size_t kTicketArea = 64 * 1024;
 static size_t ticket_bytes(const ht_attn_desc &d) {
     const size_t units = (size_t)d.B * d.Hkv * units_per_head(d);
-    return (units * sizeof(unsigned int) + 255) / 256 * 256;
+    const size_t need = (units * sizeof(unsigned int) + 255) / 256 * 256;
+    return need > kTicketArea ? need : kTicketArea;
+}
+// Is the kernel that zeroes the counters (and, for a paged cache, the status words) part of the call?
+static bool needs_prepare(const ht_attn_desc &d, bool paged) {
+    if (paged) return true;                                   // the paged kernels report bad pages from any CTA
+    if (cluster_size(d) > 1) return false;                    // clusters use no counters
+    const size_t units = (size_t)d.B * d.Hkv * units_per_head(d);
+    return !(d.flags & HT_ATTN_WORKSPACE_CLEAN) || units * sizeof(unsigned int) > kTicketArea;
 }
 
 // Arrival counters of the units, then two partial-result slots per CTA (a slot holds one part
@@ -730,8 +748,8 @@ static AttnKernelFn attn_tc_fn(bool bf16, bool paged, bool clustered) {
     return fns[(bf16 ? 1 : 0) + (paged ? 2 : 0) + (clustered ? 4 : 0)];
 }
 
-// Kernels per call: the attention kernel, and ahead of it the one that zeroes the tickets unless clusters are used.
-int attn_tc_launches(const ht_attn_desc &d) { return cluster_size(d) > 1 ? 1 : 2; }
+// Kernels per call: the attention kernel, and ahead of it the one that zeroes the arrival counters where it is needed.
+int attn_tc_launches(const ht_attn_desc &d) { return needs_prepare(d, false) ? 2 : 1; }
 
 // The kernels' dynamic shared memory limit is raised once per device.
 static cudaError_t ensure_smem_attr(size_t smem) {
@@ -825,7 +843,7 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     if (units > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "too many (sequence, head, row tile) units");
     const int k = cluster_size(d);
     cudaError_t e = cudaSuccess;
-    if (k <= 1 || pages) {                        // clusters use no tickets; the paged kernels report bad pages from any CTA
+    if (needs_prepare(d, pages != nullptr)) {
         const int n_t = k <= 1 ? (int)units : 0, n_s = pages ? d.B : 0;
         const int n = n_t > n_s ? n_t : n_s;
         cudaLaunchConfig_t cfg = {};

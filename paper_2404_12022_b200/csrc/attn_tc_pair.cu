@@ -563,7 +563,11 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tc_fence_after();
             }
             // --- segment epilogue: write the result, finish a cut unit, or leave a part ---
-            if (tid256 == 0) sm.direct = !clustered && !complete && cut[cut_k].c_hi - cut[cut_k].c_lo == 1 && delivered_old == 1u;
+            if (tid256 == 0) {
+                sm.direct = !clustered && !complete && cut[cut_k].c_hi - cut[cut_k].c_lo == 1 && delivered_old == 1u;
+                // nobody touches the unit's counter any more: it is left at zero for the next call on this workspace
+                if (sm.direct) p.tickets[cut[cut_k].unit] = 0u;
+            }
             tc_fence_before();
             softmax_groups_sync();
             tc_fence_after();
@@ -682,8 +686,10 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
         if (cut[0].valid || cut[1].valid) {
             if (tid256 == 0)
-                for (int k = 0; k < 2; ++k)
+                for (int k = 0; k < 2; ++k) {
                     sm.merge_here[k] = cut[k].valid && ticket[k] == (unsigned)(cut[k].c_hi - cut[k].c_lo);
+                    if (sm.merge_here[k]) p.tickets[cut[k].unit] = 0u;      // all parts have arrived: zero again for the next call
+                }
             softmax_groups_sync();
             for (int k = 0; k < 2; ++k)
                 if (sm.merge_here[k]) {

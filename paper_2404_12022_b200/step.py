@@ -38,12 +38,13 @@ class VerifyStep:
         ws_bytes = 0
         for i in range(self.layers):
             q = inp.q[i]
-            desc = hb.make_attn_desc(q, inp.k_cache[i], 0.0, num_splits, flags)
+            # the step owns its workspace: zeroed below, and left clean by every call
+            desc = hb.make_attn_desc(q, inp.k_cache[i], 0.0, num_splits, flags | hb.HT_ATTN_WORKSPACE_CLEAN)
             self.descs.append(desc)
             self.parents.append(inp.parent if q.shape[1] == w.N else inp.parent_tree)
             self.outs.append(torch.empty_like(q))
             ws_bytes = max(ws_bytes, hb.tree_attention_workspace(desc))
-        self.workspace = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
+        self.workspace = torch.zeros(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
         self.ws_bytes = ws_bytes
         self.attn_status = torch.zeros((self.layers, w.B), dtype=torch.int32, device=dev)
         self.pseudo = torch.empty((w.B, w.k, w.d), dtype=inp.h_src.dtype, device=dev)

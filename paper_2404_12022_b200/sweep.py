@@ -61,9 +61,11 @@ def run_attention(args):
         out = torch.empty_like(q)
         st = torch.zeros(w.B, dtype=torch.int32, device="cuda")
         desc = hb.make_attn_desc(q, ks[0])
-        ws = torch.empty(max(hb.tree_attention_workspace(desc), 16), dtype=torch.uint8, device="cuda")
+        ws = torch.zeros(max(hb.tree_attention_workspace(desc), 16), dtype=torch.uint8, device="cuda")
+        clean = hb.HT_ATTN_WORKSPACE_CLEAN          # zeroed once, left clean by every call: as a decoding loop keeps it
         reps = args.reps or max(nbuf, 16)
-        call = lambda i: hb.tree_attention(q, ks[i % nbuf], vs[i % nbuf], kv_len, parent, out=out, workspace=ws, status=st)
+        call = lambda i: hb.tree_attention(q, ks[i % nbuf], vs[i % nbuf], kv_len, parent, out=out, workspace=ws, status=st,
+                                           flags=clean)
         if args.paged:
             ps = args.paged
             B, Hkv, cap, D = ks[0].shape

@@ -280,6 +280,29 @@ def test_attention_calls_in_a_row_see_each_others_results(hb, shape):
     assert bool(((a.float() - b.float()).abs() <= ulp * a.float().abs() + 1e-6).all())
 
 
+def test_attention_on_a_workspace_kept_clean_leaves_out_the_counter_kernel(hb, oracle):
+    """HT_ATTN_WORKSPACE_CLEAN: a workspace zeroed once serves calls of different shapes one after the other (units cut
+    in two and in many, finished directly or by the last arrival; one-tile and tile-pair kernel; a cluster launch in
+    between), each leaving its arrival counters at zero; every call is one kernel, and every result matches the
+    oracle on sampled units."""
+    shapes = [(4, 91, 32, 32, [1500, 1487, 1474, 1461]), (1, 19, 32, 32, [9000]), (2, 19, 64, 8, [3000, 2500]),
+              (5, 37, 32, 32, [900, 640, 33, 1200, 512]), (1, 91, 32, 32, [1024]), (1, 40, 32, 4, [20000]),
+              (4, 91, 32, 32, [1500, 1487, 1474, 1461])]
+    cases = [make_attn_case(23 + i, "bf16", B, N, Hq, Hkv, 128, lens, max(lens) + N + 5) for i, (B, N, Hq, Hkv, lens) in enumerate(shapes)]
+    need = max(hb.tree_attention_workspace(hb.make_attn_desc(c[0], c[1])) for c in cases)
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        outs = []
+        for q, k, v, kv_len, parent in cases:                     # back to back, nothing drained in between
+            assert hb.tree_attention_launches(hb.make_attn_desc(q, k, flags=hb.HT_ATTN_WORKSPACE_CLEAN)) == 1
+            outs.append(hb.tree_attention(q, k, v, kv_len, parent, workspace=ws, flags=hb.HT_ATTN_WORKSPACE_CLEAN))
+        torch.cuda.synchronize()
+        assert int(ws[:65536].view(torch.int32).abs().max()) == 0          # every counter is back at zero
+        for i, ((q, k, v, kv_len, parent), (out, status)) in enumerate(zip(cases, outs)):
+            assert status.cpu().tolist() == [0] * q.shape[0]
+            check_sampled_units(hb, oracle, q, k, v, kv_len.cpu().numpy(), parent, out, 3, torch.bfloat16, seed=i)
+
+
 @pytest.mark.parametrize("shape", [(5, 37, 32, 32, [900, 640, 33, 1200, 512]), (2, 19, 64, 8, [3000, 2500])],
                          ids=lambda s: "B%dN%dHq%dHkv%d" % s[:4])
 def test_attention_waits_that_run_out_are_reported_and_leave_the_device_usable(hb, oracle, shape):
