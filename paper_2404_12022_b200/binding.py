@@ -22,6 +22,7 @@ HT_ERR_INVALID_ARG, HT_ERR_UNSUPPORTED, HT_ERR_BAD_TREE, HT_ERR_WORKSPACE, HT_ER
 HT_STATUS_OK, HT_STATUS_BAD_TREE, HT_STATUS_BAD_LEN, HT_STATUS_BAD_PATH, HT_STATUS_PATH_TOO_LONG = range(5)
 HT_ATTN_FORCE_SIMT = 1
 HT_ATTN_WORKSPACE_CLEAN = 2
+HT_ATTN_CONTEXT_FINAL = 4
 HT_ATTN_TEST_SHORT_WAITS = 0x80000000
 HT_STATUS_BAD_PAGE, HT_STATUS_TIMEOUT = 5, 6
 

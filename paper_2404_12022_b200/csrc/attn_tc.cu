@@ -99,6 +99,13 @@ __device__ __forceinline__ void softmax_pass2(uint32_t s_addr, float *xa, float 
     }
 }
 
+// The Q tile of a segment: the N x g rows of the KV head's query heads, two 64-feature slabs.
+__device__ __forceinline__ void fetch_q_tile(Smem &sm, const CUtensorMap &tm_q, const Params &p, int hk, int rt, int b) {
+    mbar_expect_tx(&sm.q_full, kEntryBytes);
+    tma_load_4d(sm.q, &tm_q, &sm.q_full, 0, hk * p.g, rt * p.rows_per_tile_nodes, b);
+    tma_load_4d(sm.q + kSlabBytes, &tm_q, &sm.q_full, 64, hk * p.g, rt * p.rows_per_tile_nodes, b);
+}
+
 // kPaged: the cache is a pool of pages (separate instantiations, so that the contiguous kernels carry none of that code).
 // kClustered: launched as clusters (p.cluster_k > 1); a template parameter so that the persistent form carries no cluster code.
 template <bool kBf16, bool kPaged, bool kClustered>
@@ -131,9 +138,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
     // The launch is serialized programmatically behind the kernel before it in the stream: the CTA has set itself
     // up while that kernel was still finishing, and everything it may have written is read from here on.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0, kPaged, p.n_rt);
+    // `early` (the caller vouches that lengths, trees and the cache rows below the lengths were final before that
+    // kernel began): the plan is made and the first context tiles are fetched right away, and each role waits for
+    // the kernel ahead where it first touches what that kernel may have written or may still read -- the producer
+    // before the Q tile and before the first tile with tree rows, the softmax threads before their first scores
+    // (status words, workspace and `out` are written behind that), the issuer before its first product.
+    const bool early = !kPaged && p.early != 0;
+    if (!early) wait_for_kernel_ahead();
+    plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0 && !early, kPaged, p.n_rt);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -164,6 +176,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (kPaged || lane == 0) {
             int ring_i = 0, seg_i = 0;
             const int n = t_end - t_begin;
+            bool waited = !early;                  // early: the range's first Q tile is fetched by the issuing thread, behind its wait
+            auto release = [&]() {
+                if (!waited) {
+                    wait_for_kernel_ahead();
+                    waited = true;
+                }
+            };
             TileCursor cur_k, cur_v, cur_p;          // the K and V streams of the ring order, and the page-id lookahead
             cur_k.init(t_begin, t_end);
             cur_v.init(t_begin, t_end);
@@ -184,16 +203,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int kt = is_v ? cur_v.kt() : cur_k.kt();
                 if (!is_v && cur_k.first()) {
                     // first tile of a segment: its Q tile, once the previous segment's scores are done with Q
+                    if (seg_i > 0) release();
                     bool ok = seg_i == 0 || mbar_wait_quick(smem_u32(&sm.q_empty), (seg_i - 1) & 1, abort_flag);
                     if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
-                    if (lane == 0) {
-                        mbar_expect_tx(&sm.q_full, kEntryBytes);
-                        tma_load_4d(sm.q, &tm_q, &sm.q_full, 0, s.hk * p.g, s.rt * p.rows_per_tile_nodes, s.b);
-                        tma_load_4d(sm.q + kSlabBytes, &tm_q, &sm.q_full, 64, s.hk * p.g, s.rt * p.rows_per_tile_nodes, s.b);
-                    }
+                    if (lane == 0 && !(early && seg_i == 0)) fetch_q_tile(sm, tm_q, p, s.hk, s.rt, s.b);
                     ++seg_i;
                 }
+                // early: context tiles only, and no more of them than the ring holds, ahead of the wait
+                if (!waited && ((kt + 1) * kTile > sm.len[s.b] || ring_i >= kStages)) release();
                 const int slot = ring_i % kStages, use = ring_i / kStages;
                 {
                     bool ok = use == 0 || mbar_wait_quick(smem_u32(&sm.kv_empty[slot]), (use - 1) & 1, abort_flag);
@@ -220,12 +238,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 cp_async_wait<0>();
                 __syncwarp();
             }
+            release();
             if (lane == 0 && *abort_flag) {
                 // Every copy this warp issued must have landed before the CTA exits: wait, with the
                 // usual bound, for the latest armed phase of each ring slot and of the Q buffer.
                 for (int e = max(0, ring_i - kStages); e < ring_i; ++e)
                     mbar_wait(&sm.kv_full[e % kStages], (e / kStages) & 1, abort_flag, false);
-                if (seg_i > 0) mbar_wait(&sm.q_full, (seg_i - 1) & 1, abort_flag, false);
+                // (early: the first Q tile was fetched by the issuing thread, whatever else happened)
+                const int q_fetches = early && n > 0 && seg_i == 0 ? 1 : seg_i;
+                if (q_fetches > 0) mbar_wait(&sm.q_full, (q_fetches - 1) & 1, abort_flag, false);
             }
         }
         if (clustered) {                               // the two barriers of the exchange (whole warp)
@@ -239,6 +260,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // and descriptor words are formed once, each product is one instruction sequence, and the abort flag is
         // looked at only when a wait has to spin.
         if (lane == 0) {
+            if (early) {
+                // q is the kernel ahead's to write: the range's first Q tile is fetched here, behind the wait, while the
+                // producer is busy with the first context tiles
+                wait_for_kernel_ahead();
+                if (t_end > t_begin) {
+                    int hint = 0;
+                    const Segment s0 = locate(sm.pre, sm.nkt, p.B, p.n_rt, t_begin, t_end, hint);
+                    fetch_q_tile(sm, tm_q, p, s0.hk, s0.rt, s0.b);
+                }
+            }
             const uint32_t idesc_qk = instr_desc(kBf16, 0), idesc_pv = instr_desc(kBf16, 1);
             const uint32_t hi_k = desc_hi(1, 1024 >> 4), hi_v = desc_hi(kSlabBytes >> 4, 1024 >> 4);
             const uint32_t q_lo = desc_lo_with_lbo(smem_u32(sm.q), 1);
@@ -321,6 +352,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         unsigned int ticket[2] = {0u, 0u};
         cut[0].valid = cut[1].valid = 0;
         int anc_b = -1, anc_rt = -1;           // sequence / row tile the ancestor words were built for
+        bool waited = !early;
+        // early: the status words (all of them from the first CTA) go out behind the wait
+        auto release = [&]() {
+            if (!waited) {
+                wait_for_kernel_ahead();
+                waited = true;
+                if (blockIdx.x == 0 && tid256 < p.B) {
+                    const int L = sm.len[tid256];
+                    p.status[tid256] = (L < 0 || (long long)L + p.N > p.cap) ? HT_STATUS_BAD_LEN
+                                       : (sm.nkt[tid256] == 0 ? HT_STATUS_BAD_TREE : HT_STATUS_OK);
+                }
+            }
+        };
         for (int t = t_begin; t < t_end;) {
             const Segment sg = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
             const int L = sm.len[sg.b];
@@ -342,6 +386,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 anc_b = sg.b;
                 anc_rt = sg.rt;
             }
+            release();
 
             // A segment that is only part of its unit: which CTAs hold the other parts.  How many of
             // them have been delivered is asked anew at every tile and looked at in the epilogue, so
@@ -599,6 +644,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             J += sg.len;
             t += sg.len;
         }
+        release();
         if (clustered) {
             if (t_end <= t_begin) {                    // an empty share still delivers a part: nothing seen
                 cluster_sync_all();
@@ -831,6 +877,7 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     p.grid = sm_count();
     p.cluster_k = 0;
     p.wait_kcycles = (d.flags & HT_ATTN_TEST_SHORT_WAITS) ? tc::kWaitKcyclesTest : tc::kWaitKcycles;
+    p.early = (d.flags & HT_ATTN_CONTEXT_FINAL) ? 1 : 0;
     tc::PagedParams pp;
     pp.block_table = pages ? block_table : nullptr;
     pp.page_size = pages ? pages->page_size : 0;

@@ -37,7 +37,14 @@ struct Params {
     int grid;
     int cluster_k;         // > 1: launched as clusters of this many CTAs, one cluster per (sequence, KV head)
     int wait_kcycles;      // how long a wait on an mbarrier may last, in units of 1024 clock cycles
+    int early;             // HT_ATTN_CONTEXT_FINAL: lengths, trees and context rows may be read while the kernel ahead still runs
 };
+// The launch is serialized programmatically behind the kernel before it in the stream: a thread passes this point once
+// that kernel has completed and what it wrote is visible, and only then lets this kernel's own dependents be set up.
+__device__ __forceinline__ void wait_for_kernel_ahead() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 enum : int {
     kWaitKcycles = 2000000,            // about a second
     kWaitKcyclesTest = 0               // HT_ATTN_TEST_SHORT_WAITS: a wait for anything not yet there runs out at once

@@ -38,8 +38,10 @@ class VerifyStep:
         ws_bytes = 0
         for i in range(self.layers):
             q = inp.q[i]
-            # the step owns its workspace: zeroed below, and left clean by every call
-            desc = hb.make_attn_desc(q, inp.k_cache[i], 0.0, num_splits, flags | hb.HT_ATTN_WORKSPACE_CLEAN)
+            # the step owns its workspace: zeroed below, and left clean by every call; lengths, trees and context
+            # rows are final long before a layer's call (the compaction moves rows at or behind the lengths only)
+            desc = hb.make_attn_desc(q, inp.k_cache[i], 0.0, num_splits,
+                                     flags | hb.HT_ATTN_WORKSPACE_CLEAN | hb.HT_ATTN_CONTEXT_FINAL)
             self.descs.append(desc)
             self.parents.append(inp.parent if q.shape[1] == w.N else inp.parent_tree)
             self.outs.append(torch.empty_like(q))

@@ -62,7 +62,9 @@ def run_attention(args):
         st = torch.zeros(w.B, dtype=torch.int32, device="cuda")
         desc = hb.make_attn_desc(q, ks[0])
         ws = torch.zeros(max(hb.tree_attention_workspace(desc), 16), dtype=torch.uint8, device="cuda")
-        clean = hb.HT_ATTN_WORKSPACE_CLEAN          # zeroed once, left clean by every call: as a decoding loop keeps it
+        # the workspace is zeroed once and left clean by every call, lengths, trees and caches are final: what a
+        # decoding loop can promise
+        clean = hb.HT_ATTN_WORKSPACE_CLEAN | hb.HT_ATTN_CONTEXT_FINAL
         reps = args.reps or max(nbuf, 16)
         call = lambda i: hb.tree_attention(q, ks[i % nbuf], vs[i % nbuf], kv_len, parent, out=out, workspace=ws, status=st,
                                            flags=clean)

@@ -254,10 +254,13 @@ def test_attention_at_the_largest_sizes_the_tensor_core_kernels_take(hb, oracle,
 
 @pytest.mark.parametrize("shape", [(4, 91, 32, 32, 1500), (1, 91, 32, 32, 1024), (2, 40, 32, 4, 700), (3, 19, 16, 16, 3000)],
                          ids=lambda s: "B%dN%dHq%dHkv%dL%d" % s)
-def test_attention_calls_in_a_row_see_each_others_results(hb, shape):
+@pytest.mark.parametrize("final", [False, True], ids=["plain", "context_final"])
+def test_attention_calls_in_a_row_see_each_others_results(hb, shape, final):
     """The launches of consecutive calls overlap at their edges (a call's CTAs set themselves up while the call before
     it finishes).  Six calls, each taking the previous call's output as its queries and sharing one workspace, must give
-    what the same calls give with the device drained between them."""
+    what the same calls give with the device drained between them.  With HT_ATTN_CONTEXT_FINAL (lengths, trees and
+    context rows are final; q is the kernel ahead's output) a call plans and fetches its first context tiles while the
+    call before it is still finishing, and must wait for it before it reads q."""
     B, N, Hq, Hkv, L = shape
     q0, k, v, kv_len, parent = make_attn_case(91, "bf16", B, N, Hq, Hkv, 128, [L - 13 * b for b in range(B)], L + N, garbage=False)
     desc = hb.make_attn_desc(q0, k)
@@ -266,7 +269,8 @@ def test_attention_calls_in_a_row_see_each_others_results(hb, shape):
     def chain(drain):
         q = q0
         for _ in range(6):
-            out, status = hb.tree_attention(q, k, v, kv_len, parent, workspace=ws)
+            out, status = hb.tree_attention(q, k, v, kv_len, parent, workspace=ws,
+                                            flags=hb.HT_ATTN_CONTEXT_FINAL if final and not drain else 0)
             if drain:
                 torch.cuda.synchronize()
             q = out
