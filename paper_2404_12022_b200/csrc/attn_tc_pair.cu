@@ -145,9 +145,11 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     // The launch is serialized programmatically behind the kernel before it in the stream: the CTA has set itself
-    // up while that kernel was still finishing, and everything it may have written is read from here on.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // up while that kernel was still finishing, and everything it may have written is read from here on.  `early`
+    // (lengths, trees and the cache rows below the lengths were final before that kernel began): as in the one-tile
+    // kernel, plan and first context tiles do not wait, and each role waits where it first needs to.
+    const bool early = !kPaged && p.early != 0;
+    if (!early) wait_for_kernel_ahead();
     // Without clusters, where a KV head has several tile pairs (units), the list of tiles is that of the HEADS: it is
     // cut into grid / n_rt ranges, and the n_rt CTAs of a range take one tile pair each.  They start together and walk
     // the same K / V tiles at the same pace, so that a tile crosses DRAM once and reaches the others from L2.  (With
@@ -159,7 +161,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int my_rt = grouped ? (int)blockIdx.x % p.n_rt : 0;               // grouped: this CTA's tile pair
     const int my_pos = grouped ? (int)blockIdx.x / p.n_rt : (int)blockIdx.x; // place in the list's partition
     const int n_pos = grouped ? p.grid / p.n_rt : p.grid;
-    plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0, kPaged, lrt);
+    plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0 && !early, kPaged, lrt);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -187,6 +189,16 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         t_end = t0 + min(((int)c_rank + 1) * share, nk);
     }
     unsigned char *const xarea = &sm.q[0][0];          // Q buffers and ring, idle once the CTA's tiles are done
+    // The Q tiles of a segment's tile pair (one where the pair has no second tile).
+    auto fetch_q = [&](const Segment &s) {
+        const bool two = 2 * s.rt + 1 < p.n_row_tiles;
+        mbar_expect_tx(&sm.q_full, two ? 2 * kEntryBytes : kEntryBytes);
+        for (int x = 0; x < (two ? 2 : 1); ++x) {
+            const int node0 = (2 * s.rt + x) * p.rows_per_tile_nodes;
+            tma_load_4d(sm.q[x], &tm_q, &sm.q_full, 0, s.hk * p.g, node0, s.b);
+            tma_load_4d(sm.q[x] + kSlabBytes, &tm_q, &sm.q_full, 64, s.hk * p.g, node0, s.b);
+        }
+    };
     // Cluster mode: the unit's parts are exchanged between two barriers of the whole cluster (the softmax threads pass
     // them around their sends, the other warps once their work is done).
 
@@ -201,26 +213,28 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (kPaged)
                 for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p, lane, lrt);
             bool stop = false;
+            bool waited = !early;                  // early: the range's first Q tiles are fetched by stream 0's issuing thread, behind its wait
+            auto release = [&]() {
+                if (!waited) {
+                    wait_for_kernel_ahead();
+                    waited = true;
+                }
+            };
             for (int t = t_begin; t < t_end && !stop;) {
                 if (kPaged ? __any_sync(0xFFFFFFFFu, *abort_flag != 0) : (*abort_flag != 0)) break;
                 const Segment s = find(t, t_end, b_hint);
-                const bool two = 2 * s.rt + 1 < p.n_row_tiles;
+                if (seg_i > 0) release();
                 {
                     bool ok = seg_i == 0 || mbar_wait_quick(smem_u32(&sm.q_empty), (seg_i - 1) & 1, abort_flag);
                     if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                 }
-                if (lane == 0) {
-                    mbar_expect_tx(&sm.q_full, two ? 2 * kEntryBytes : kEntryBytes);
-                    for (int x = 0; x < (two ? 2 : 1); ++x) {
-                        const int node0 = (2 * s.rt + x) * p.rows_per_tile_nodes;
-                        tma_load_4d(sm.q[x], &tm_q, &sm.q_full, 0, s.hk * p.g, node0, s.b);
-                        tma_load_4d(sm.q[x] + kSlabBytes, &tm_q, &sm.q_full, 64, s.hk * p.g, node0, s.b);
-                    }
-                }
+                if (lane == 0 && !(early && seg_i == 0)) fetch_q(s);
                 ++seg_i;
                 for (int i = 0; i < 2 * s.len; ++i) {
                     const int kt = s.kt0 + (i >> 1);
+                    // early: context tiles only, and no more of them than the ring holds, ahead of the wait
+                    if (!waited && ((kt + 1) * kTile > sm.len[s.b] || ring_i >= kPStages)) release();
                     const int slot = ring_i % kPStages, use = ring_i / kPStages;
                     bool ok = use == 0 || mbar_wait_quick(smem_u32(&sm.kv_empty[slot]), (use - 1) & 1, abort_flag);
                     if (kPaged) ok = __all_sync(0xFFFFFFFFu, ok);
@@ -247,11 +261,14 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 cp_async_wait<0>();
                 __syncwarp();
             }
+            release();
             if (lane == 0 && *abort_flag) {
-                // Every copy this warp issued must have landed before the CTA exits.
+                // Every copy this warp issued must have landed before the CTA exits.  (early: the first Q tiles
+                // were fetched by stream 0's issuing thread, whatever else happened)
                 for (int e = max(0, ring_i - kPStages); e < ring_i; ++e)
                     mbar_wait(&sm.kv_full[e % kPStages], (e / kPStages) & 1, abort_flag, false);
-                if (seg_i > 0) mbar_wait(&sm.q_full, (seg_i - 1) & 1, abort_flag, false);
+                const int q_fetches = early && t_end > t_begin && seg_i == 0 ? 1 : seg_i;
+                if (q_fetches > 0) mbar_wait(&sm.q_full, (q_fetches - 1) & 1, abort_flag, false);
             }
         }
         if (clustered) { cluster_sync_all(); cluster_sync_all(); }
@@ -269,6 +286,15 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // abort flag is looked at only when a wait has to spin.
         if (lane == 0) {
             const int s = warp - 9;
+            if (early) {
+                // q is the kernel ahead's to write: the range's first Q tiles are fetched here (stream 0's thread),
+                // behind the wait, while the producer is busy with the first context tiles
+                wait_for_kernel_ahead();
+                if (s == 0 && t_end > t_begin) {
+                    int hint = 0;
+                    fetch_q(find(t_begin, t_end, hint));
+                }
+            }
             const uint32_t idesc_qk = instr_desc(kBf16, 0, kHalf), idesc_pv = instr_desc(kBf16, 1, 128);
             const uint32_t hi_k = desc_hi(1, 1024 >> 4), hi_v = desc_hi(kSlabBytes >> 4, 1024 >> 4);
             const uint32_t q_lo = desc_lo_with_lbo(smem_u32(sm.q[s]), 1);
@@ -371,6 +397,19 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         cut[0].valid = cut[1].valid = 0;
         int anc_b = -1, anc_rt = -1;                   // sequence / tile pair the ancestor words were built for
         uint32_t uses_s[2] = {0, 0}, uses_o[2] = {0, 0};   // uses of s_full[s][h] / o_done[s][h] so far
+        bool waited = !early;
+        // early: the status words (all of them from the first CTA) go out behind the wait
+        auto release = [&]() {
+            if (!waited) {
+                wait_for_kernel_ahead();
+                waited = true;
+                if (blockIdx.x == 0 && tid256 < p.B) {
+                    const int L = sm.len[tid256];
+                    p.status[tid256] = (L < 0 || (long long)L + p.N > p.cap) ? HT_STATUS_BAD_LEN
+                                       : (sm.nkt[tid256] == 0 ? HT_STATUS_BAD_TREE : HT_STATUS_OK);
+                }
+            }
+        };
         for (int t = t_begin; t < t_end;) {
             const Segment sg = find(t, t_end, b_hint);
             const int L = sm.len[sg.b];
@@ -392,6 +431,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 anc_b = sg.b;
                 anc_rt = sg.rt;
             }
+            release();
             // A segment that is only part of its unit: see the one-tile kernel.
             const bool complete = sg.kt0 == 0 && sg.len == sg.nkt;
             const int cut_k = (t == t_begin) ? 0 : 1;
@@ -670,6 +710,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             J += sg.len;
             t += sg.len;
         }
+        release();
         if (clustered && t_end <= t_begin) {
             // an empty share still takes part in the cluster's exchange, with parts that saw nothing
             const int unit = (int)blockIdx.x / p.cluster_k, b = unit / (p.Hkv * p.n_rt);
