@@ -653,44 +653,85 @@ constexpr int kXchgBytes = kXchgRecvOffset + kRows * kD * 4 + 16 * 2 * kRows * 4
 static_assert(kXchgBytes <= (1 + kStages) * kEntryBytes, "the exchange area is the Q buffer and the ring");
 
 // Second half of the reduction: behind the barrier every part has arrived everywhere, and nobody writes into a
-// peer's shared memory any more, so a CTA may leave as soon as it has merged what it holds.  Received slices
-// lie at area + kXchgRecvOffset as [sender][group in slice][row] float4, followed by [sender][m | l][row].
+// peer's shared memory any more, so a CTA may leave as soon as it has merged what it holds.
+//
+// The merge of one row's received parts.  It runs once per CTA, so what counts is the length of its chain of
+// dependent instructions, not their number: all loads are independent of one another (the k <= 8 parts unrolled
+// with predicates), the parts' weights are formed once, and the row's features leave as 16-byte stores.
+__device__ __forceinline__ float lds_f32(uint32_t a) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ float4 lds_f32x4(uint32_t a) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
+    return v;
+}
+// Weights of the k parts of `row`, 1 / (sum of the weighted row sums) folded in.  recv_ml: [sender][m | l][row] floats.
+__device__ __forceinline__ void merge_weights(uint32_t recv_ml, int k, int row, float (&f)[8]) {
+    float m[8], M = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        m[c] = c < k ? lds_f32(recv_ml + (uint32_t)(c * 2 * kRows + row) * 4u) : -INFINITY;
+        f[c] = c < k ? lds_f32(recv_ml + (uint32_t)(c * 2 * kRows + kRows + row) * 4u) : 0.f;     // the part's row sum, for now
+    }
+#pragma unroll
+    for (int c = 0; c < 8; ++c) M = fmaxf(M, m[c]);
+    float l = 0.f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const float w = m[c] == -INFINITY ? 0.f : ex2(m[c] - M);
+        l = fmaf(w, f[c], l);
+        f[c] = w;
+    }
+    const float inv = 1.f / l;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) f[c] *= inv;
+}
+// X groups of 4 features from group x0 on: recv holds [sender][group in slice (cgps of them)][row] float4; the
+// 8 X bytes of the result go to dst (16-byte aligned, X even).
+template <bool kBf16, int X>
+__device__ __forceinline__ void merge_groups(uint32_t recv, int k, int cgps, int row, int x0, const float (&f)[8], unsigned char *dst) {
+    uint32_t w[2 * X];
+#pragma unroll
+    for (int x = 0; x < X; ++x) {
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+            if (c < k && f[c] != 0.f) {            // a part that saw nothing sent no features: what lies there is not data
+                const float4 v = lds_f32x4(recv + (uint32_t)((c * cgps + x0 + x) * kRows + row) * 16u);
+                o.x = fmaf(f[c], v.x, o.x); o.y = fmaf(f[c], v.y, o.y); o.z = fmaf(f[c], v.z, o.z); o.w = fmaf(f[c], v.w, o.w);
+            }
+        w[2 * x] = pack2<kBf16>(o.x, o.y);
+        w[2 * x + 1] = pack2<kBf16>(o.z, o.w);
+    }
+#pragma unroll
+    for (int i = 0; i < X / 2; ++i)
+        *reinterpret_cast<uint4 *>(dst + i * 16) = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+}
+
+// One-tile kernel: received slices lie at area + kXchgRecvOffset as [sender][group in slice][row] float4, followed by
+// [sender][m | l][row]; thread (row, half) merges half of the CTA's slice of the row's features.
 template <bool kBf16>
 __device__ __noinline__ void cluster_merge(const Params &p, unsigned char *area, int rank, int b, int hk, int row_tile,
                                            bool valid, int tid256, volatile int *abort_flag) {
     const int k = p.cluster_k;
-    const int cg_per_slice = 32 / k;
-    const float4 *recv4 = reinterpret_cast<const float4 *>(area + kXchgRecvOffset);
-    const float *recv_ml = reinterpret_cast<const float *>(area + kXchgRecvOffset) + kRows * kD;
+    const int cgps = 32 / k;                      // groups of 4 features per slice: 16, 8 or 4
     cluster_sync_all();
     const int row = tid256 & 127, half = tid256 >> 7;
     const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
     if (!valid || node >= p.N || *abort_flag) return;
-    float M = -INFINITY;
-    for (int c = 0; c < k; ++c) M = fmaxf(M, recv_ml[c * 2 * kRows + row]);
-    float l = 0.f;
-    for (int c = 0; c < k; ++c) {
-        const float m = recv_ml[c * 2 * kRows + row];
-        if (m != -INFINITY) l = fmaf(exp2f(m - M), recv_ml[c * 2 * kRows + kRows + row], l);
-    }
-    const float inv = 1.f / l;
+    const uint32_t recv = smem_u32(area) + kXchgRecvOffset, recv_ml = recv + kRows * kD * 4;
+    float f[8];
+    merge_weights(recv_ml, k, row, f);
     const int head = hk * p.g + row % p.g;
-    const int x_per_half = cg_per_slice / 2 > 0 ? cg_per_slice / 2 : 1;
-    for (int xi = 0; xi < x_per_half; ++xi) {
-        const int x = half * x_per_half + xi;
-        if (x >= cg_per_slice) break;
-        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int c = 0; c < k; ++c) {
-            const float m = recv_ml[c * 2 * kRows + row];
-            if (m == -INFINITY) continue;
-            const float f = exp2f(m - M);
-            const float4 v = recv4[(c * cg_per_slice + x) * kRows + row];
-            o.x = fmaf(f, v.x, o.x); o.y = fmaf(f, v.y, o.y); o.z = fmaf(f, v.z, o.z); o.w = fmaf(f, v.w, o.w);
-        }
-        unsigned char *dst = static_cast<unsigned char *>(p.out) +
-                             ((((size_t)b * p.N + node) * p.Hq + head) * kD + (rank * cg_per_slice + x) * 4) * 2;
-        *reinterpret_cast<uint2 *>(dst) = make_uint2(pack2<kBf16>(o.x * inv, o.y * inv), pack2<kBf16>(o.z * inv, o.w * inv));
-    }
+    const int x0 = half * (cgps / 2);
+    unsigned char *dst = static_cast<unsigned char *>(p.out) +
+                         ((((size_t)b * p.N + node) * p.Hq + head) * kD + (rank * cgps + x0) * 4) * 2;
+    if (k == 2) merge_groups<kBf16, 8>(recv, k, cgps, row, x0, f, dst);
+    else if (k == 4) merge_groups<kBf16, 4>(recv, k, cgps, row, x0, f, dst);
+    else merge_groups<kBf16, 2>(recv, k, cgps, row, x0, f, dst);
 }
 
 }  // namespace tc

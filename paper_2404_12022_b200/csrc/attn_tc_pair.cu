@@ -63,6 +63,8 @@ constexpr int kPXchgMl = kRows * kD * 4;                         // bytes from a
 constexpr int kPXchgStream = kPXchgMl + 8 * 2 * kRows * 4;       // up to 8 senders
 static_assert(2 * kPXchgStream <= (2 + kPStages) * kEntryBytes, "the exchange area is the Q buffers and the ring");
 
+// A stream's received parts lie at `area` as [sender][group in slice][row] float4, followed (at kPXchgMl) by
+// [sender][m | l][row]; thread `row` of the stream merges the CTA's whole slice of the row's features.
 template <bool kBf16>
 __device__ __noinline__ void cluster_merge_pair(const Params &p, const unsigned char *area, int rank, int b, int hk, int row_tile,
                                                 bool valid, int row, volatile int *abort_flag) {
@@ -70,28 +72,18 @@ __device__ __noinline__ void cluster_merge_pair(const Params &p, const unsigned 
     const int k = p.cluster_k, cgps = 32 / k;
     const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
     if (!valid || row_tile >= p.n_row_tiles || node >= p.N || *abort_flag) return;
-    const float4 *recv4 = reinterpret_cast<const float4 *>(area);
-    const float *recv_ml = reinterpret_cast<const float *>(area + kPXchgMl);
-    float M = -INFINITY;
-    for (int c = 0; c < k; ++c) M = fmaxf(M, recv_ml[c * 2 * kRows + row]);
-    float l = 0.f;
-    for (int c = 0; c < k; ++c) {
-        const float m = recv_ml[c * 2 * kRows + row];
-        if (m != -INFINITY) l = fmaf(exp2f(m - M), recv_ml[c * 2 * kRows + kRows + row], l);
-    }
-    const float inv = 1.f / l;
+    const uint32_t recv = smem_u32(area), recv_ml = recv + kPXchgMl;
+    float f[8];
+    merge_weights(recv_ml, k, row, f);
     const int head = hk * p.g + row % p.g;
     unsigned char *dst = static_cast<unsigned char *>(p.out) + ((((size_t)b * p.N + node) * p.Hq + head) * kD + rank * cgps * 4) * 2;
-    for (int x = 0; x < cgps; ++x) {
-        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int c = 0; c < k; ++c) {
-            const float m = recv_ml[c * 2 * kRows + row];
-            if (m == -INFINITY) continue;
-            const float f = exp2f(m - M);
-            const float4 v = recv4[(c * cgps + x) * kRows + row];
-            o.x = fmaf(f, v.x, o.x); o.y = fmaf(f, v.y, o.y); o.z = fmaf(f, v.z, o.z); o.w = fmaf(f, v.w, o.w);
-        }
-        *reinterpret_cast<uint2 *>(dst + x * 8) = make_uint2(pack2<kBf16>(o.x * inv, o.y * inv), pack2<kBf16>(o.z * inv, o.w * inv));
+    if (k == 2) {
+        merge_groups<kBf16, 8>(recv, k, cgps, row, 0, f, dst);
+        merge_groups<kBf16, 8>(recv, k, cgps, row, 8, f, dst + 64);
+    } else if (k == 4) {
+        merge_groups<kBf16, 8>(recv, k, cgps, row, 0, f, dst);
+    } else {
+        merge_groups<kBf16, 4>(recv, k, cgps, row, 0, f, dst);
     }
 }
 
