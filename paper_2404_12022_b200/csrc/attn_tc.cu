@@ -162,10 +162,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // barrier here: the first remote access comes after the one all threads pass ahead of the exchange.)
         c_rank = cluster_ctarank();
         const int unit = (int)blockIdx.x / p.cluster_k, b = unit / p.Hkv, hk = unit - b * p.Hkv;
-        const int nk = sm.nkt[b], share = (nk + p.cluster_k - 1) / p.cluster_k;
+        const int nk = sm.nkt[b];
         const int t0 = sm.pre[b] + hk * nk;
-        t_begin = t0 + min((int)c_rank * share, nk);
-        t_end = t0 + min(((int)c_rank + 1) * share, nk);
+        int lo, hi;
+        cluster_share(nk, sm.len[b], p.cluster_k, (int)c_rank, lo, hi);
+        t_begin = t0 + lo;
+        t_end = t0 + hi;
     }
 
     if (warp == 8) {
@@ -405,7 +407,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
 
             float m_ref = -INFINITY, l_sum = 0.f;
-            int n_mine = 0, last_jj = 0;
 #pragma unroll 1
             for (int i = 0; i < sg.len; ++i) {
                 const int jj = J + i;
@@ -517,14 +518,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 }
                 tc_fence_before();
                 mbar_arrive(&sm.p_ready[s]);
-                ++n_mine;
-                last_jj = jj;
             }
-            // --- segment epilogue: merge the two streams, write the result or a partial ---
-            if (n_mine > 0) {
-                mbar_wait(&sm.o_done[s], (last_jj >> 1) & 1, abort_flag);
-                tc_fence_after();
-            }
+            // --- segment epilogue: merge the two streams, write the result or a partial.  The streams' maxima and sums
+            // are exchanged and the weights formed while the last products are still running; the accumulators are read
+            // behind the wait for both streams' last product (every thread reads both). ---
             sm.ml[s][row][0] = m_ref;
             sm.ml[s][row][1] = l_sum;
             // With one other part and that part already in the workspace, this CTA finishes the unit
@@ -534,14 +531,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 // nobody touches the unit's counter any more: it is left at zero for the next call on this workspace
                 if (sm.direct) p.tickets[cut[cut_k].unit] = 0u;
             }
-            tc_fence_before();
             softmax_groups_sync();
-            tc_fence_after();
-            // In a cluster the part goes straight from the accumulators into the peers' shared memory (each
-            // peer owns a slice of the features), so the barrier that says "every CTA of the cluster is done with
-            // its Q buffer and ring" comes first: every thread of every CTA takes part in it, the producer and
-            // issuer warps once their work is done.
-            if (clustered) cluster_sync_all();
             const float m0 = sm.ml[0][row][0], l0 = sm.ml[0][row][1];
             const float m1 = sm.ml[1][row][0], l1 = sm.ml[1][row][1];
             const bool direct = sm.direct;
@@ -577,6 +567,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 g0 = f0 * inv;
                 g1 = f1 * inv;
             }
+            {
+                const int last_any = J + sg.len - 1;                       // the segment's last tile; x's last: same parity
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
+                    const int lx = ((last_any & 1) == x) ? last_any : last_any - 1;
+                    if (lx >= J) mbar_wait(&sm.o_done[x], (lx >> 1) & 1, abort_flag);
+                }
+                tc_fence_after();
+            }
+            // In a cluster the part goes straight from the accumulators into the peers' shared memory (each
+            // peer owns a slice of the features), so the barrier that says "every CTA of the cluster is done with
+            // its Q buffer and ring" comes first: every thread of every CTA takes part in it, the producer and
+            // issuer warps once their work is done.
+            if (clustered) cluster_sync_all();
             const bool final = (complete && !clustered) || direct;
 #pragma unroll 1
             for (int c2 = 0; c2 < (warp_real ? 2 : 0); ++c2) {

@@ -436,6 +436,17 @@ struct TileCursor {
 
 __device__ __forceinline__ int tiles_per_cta(int total, int grid) { return (total + grid - 1) / grid; }
 
+// Shares of a unit's nkt tiles among the k CTAs of a cluster.  A tile with tree keys costs about two context tiles
+// (mask, P as a hi + lo pair, twice the P V products), so the shares are equal in cost rather than in tiles: with
+// 8 context tiles and the tree tile over 4 CTAs, 3 + 3 + 2 + 1 instead of 3 + 3 + 3 + 0.
+__device__ __forceinline__ void cluster_share(int nkt, int L, int k, int rank, int &lo, int &hi) {
+    const int n_ctx = min(L / kTile, nkt);                 // tiles of context keys only
+    const int cost = n_ctx + 2 * (nkt - n_ctx), share = (cost + k - 1) / k;
+    auto tile_at = [&](int c) { return min(c <= n_ctx ? c : n_ctx + (c - n_ctx) / 2, nkt); };
+    lo = tile_at(rank * share);
+    hi = rank == k - 1 ? nkt : tile_at((rank + 1) * share);
+}
+
 // Tiles per CTA.  An even share cuts nearly every unit in two, and every cut costs a partial
 // result in the workspace and a merge at the end: about as much as half a dozen tiles, whatever the
 // unit's length.  So when all sequences are equally long and some whole multiple or whole fraction of a

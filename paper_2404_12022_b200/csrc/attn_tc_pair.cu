@@ -175,10 +175,12 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // cluster barrier here: the first remote access comes after the one all threads pass ahead of the exchange.)
         c_rank = cluster_ctarank();
         const int unit = (int)blockIdx.x / p.cluster_k, b = unit / (p.Hkv * p.n_rt);
-        const int nk = sm.nkt[b], share = (nk + p.cluster_k - 1) / p.cluster_k;
+        const int nk = sm.nkt[b];
         const int t0 = sm.pre[b] + (unit - b * p.Hkv * p.n_rt) * nk;
-        t_begin = t0 + min((int)c_rank * share, nk);
-        t_end = t0 + min(((int)c_rank + 1) * share, nk);
+        int lo, hi;
+        cluster_share(nk, sm.len[b], p.cluster_k, (int)c_rank, lo, hi);
+        t_begin = t0 + lo;
+        t_end = t0 + hi;
     }
     unsigned char *const xarea = &sm.q[0][0];          // Q buffers and ring, idle once the CTA's tiles are done
     // The Q tiles of a segment's tile pair (one where the pair has no second tile).
