@@ -31,9 +31,9 @@ struct CompactSmem {
     int bad_page;
 };
 
-// Called by all kCompactThreads threads of a block; `a` = accept_len[b] and `L` = kv_len[b] as the caller read them
+// Called by all kThreads threads of a block; `a` = accept_len[b] and `L` = kv_len[b] as the caller read them
 // (the fused kernel reads the former with acquire semantics, and the latter while it waits for the former).  Ends with a barrier, so that the shared arrays may be reused at once.
-template <int kPerThread>               // 16-byte vectors a thread holds between gather and scatter
+template <int kPerThread, int kThreads = kCompactThreads>   // 16-byte vectors a thread holds between gather and scatter; threads of the block
 __device__ __forceinline__ void compact_item(const CompactArgs &c, CompactSmem &sm, int layer, int b, int grp, int a, int L) {
     if ((int)threadIdx.x < c.max_path) sm.path[threadIdx.x] = c.accept_path[(size_t)b * c.max_path + threadIdx.x];
     if (threadIdx.x == 0) sm.bad_page = 0;
@@ -84,7 +84,7 @@ __device__ __forceinline__ void compact_item(const CompactArgs &c, CompactSmem &
     const int pair_lo = (int)((long long)pairs * grp / c.groups), pair_hi = (int)((long long)pairs * (grp + 1) / c.groups);
     const int vec_per_row = c.row_bytes / 16;
     const int per_pair = a * vec_per_row;                        // <= 4096 (checked by the caller)
-    const int pairs_per_pass = max(1, kPerThread * kCompactThreads / per_pair);
+    const int pairs_per_pass = max(1, kPerThread * kThreads / per_pair);
     unsigned char *const base_k = c.k_cache + (long long)layer * c.stride_layer_b;
     unsigned char *const base_v = c.v_cache + (long long)layer * c.stride_layer_b;
     const long long seq_off = (long long)b * c.stride_b_b;
@@ -94,7 +94,7 @@ __device__ __forceinline__ void compact_item(const CompactArgs &c, CompactSmem &
         uint4 regs[kPerThread];
 #pragma unroll
         for (int i = 0; i < kPerThread; ++i) {
-            const int t = threadIdx.x + i * kCompactThreads;
+            const int t = threadIdx.x + i * kThreads;
             if (t < total) {
                 const int pr = t / per_pair, rem = t - pr * per_pair;
                 const int j = rem / vec_per_row, v = rem - j * vec_per_row;
@@ -108,7 +108,7 @@ __device__ __forceinline__ void compact_item(const CompactArgs &c, CompactSmem &
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < kPerThread; ++i) {
-            const int t = threadIdx.x + i * kCompactThreads;
+            const int t = threadIdx.x + i * kThreads;
             if (t < total) {
                 const int pr = t / per_pair, rem = t - pr * per_pair;
                 const int j = rem / vec_per_row, v = rem - j * vec_per_row;

@@ -4,8 +4,9 @@
 // accepted path's K/V rows (Fig. 1 caption) in the same launch.
 //
 // One launch, a grid no larger than the GPU holds at once.  A block streams logits rows
-// (16-byte loads, all of a row in flight at once, shuffle reductions) and stores each row's
-// argmax; the block that finishes a sequence's last row runs the path search for that
+// (asynchronous 16-byte copies into shared memory, 64 KB of a row in flight at once whatever the
+// compiler makes of the registers; every thread reads back what it copied, shuffle reductions)
+// and stores each row's argmax; the block that finishes a sequence's last row runs the path search for that
 // sequence -- a few hundred integer operations.  Arrivals are counted in the upper bits of the
 // sequence's accept_len word: the caller hands it over holding a small value (zero, or the
 // length an earlier call left there), the last block overwrites it with the new length, so
@@ -43,10 +44,41 @@ __device__ __forceinline__ int ld_acquire(const int32_t *p) {
     return v;
 }
 
-// Path search of one sequence by one block.  Every thread walks the root path of its nodes (parent[c] < c
-// makes the walk finite), checks the match rule on the way and proposes (depth, node);
+// The tree of one sequence in shared memory: parents and draft tokens are inputs (staged while the logits stream, by
+// every block, for the sequence of the row it works on), the rows' argmax is what the other blocks of the launch wrote
+// (staged by the block that searches, once all rows have arrived).
+constexpr int kStage = 1024;                 // trees of up to this many rows are staged
+struct TreeSmem {
+    int32_t par[kStage], tok[kStage], prd[kStage];
+    int bad, root, staged_b;
+    unsigned long long key[32];
+};
+
+__device__ __forceinline__ void stage_tree(TreeSmem &ts, int b, const int32_t *__restrict__ tokens, const int32_t *__restrict__ parent,
+                                           const int32_t *__restrict__ root_pred, int N, int T) {
+    if (ts.staged_b == b) return;                      // (uniform over the block: written behind a barrier below)
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        ts.bad = 0;
+        ts.root = root_pred ? root_pred[b] : -1;
+        ts.staged_b = b;
+    }
+    __syncthreads();
+    const int32_t *par = parent + (size_t)b * N;
+    for (int c = threadIdx.x; c < N; c += blockDim.x) {
+        const int pc = par[c];
+        if (N <= kStage) {
+            ts.par[c] = pc;
+            if (c < T) ts.tok[c] = tokens[(size_t)b * T + c];
+        }
+        if (pc < -1 || pc >= c) ts.bad = 1;
+    }
+}
+
+// Path search of one sequence by one block (its tree staged by stage_tree).  Every thread walks the root path of its
+// nodes (parent[c] < c makes the walk finite), checks the match rule on the way and proposes (depth, node);
 // the block keeps the deepest valid node, lowest index on ties.
-__device__ __forceinline__ void accept_sequence(const int b, const int32_t *__restrict__ tokens, const int32_t *__restrict__ parent,
+__device__ __forceinline__ void accept_sequence(TreeSmem &ts, const int b, const int32_t *__restrict__ tokens, const int32_t *__restrict__ parent,
               const int32_t *__restrict__ root_pred, const int32_t *pred, int N, int T,
               int max_path, int32_t *accept_len, int32_t *__restrict__ accept_path,
               int32_t *__restrict__ next_token, int32_t *__restrict__ status, const int done_mark) {
@@ -54,39 +86,29 @@ __device__ __forceinline__ void accept_sequence(const int b, const int32_t *__re
     const int32_t *tok = tokens + (size_t)b * T;
     const int32_t *prd = pred + (size_t)b * N;
     int32_t *path = accept_path + (size_t)b * max_path;
-    __shared__ int s_bad;
-    __shared__ unsigned long long s_key[8];
     // The walks below are chains of dependent reads: with the tree's three arrays in shared memory they
     // cost one round trip to L2 in all instead of one per level (trees of up to kStage rows).
-    constexpr int kStage = 1024;
-    __shared__ int32_t s_par[kStage], s_tok[kStage], s_prd[kStage];
-    if (threadIdx.x == 0) s_bad = 0;
-    __syncthreads();
     if (N <= kStage) {
-        for (int c = threadIdx.x; c < N; c += blockDim.x) {
-            const int pc = par[c];
-            s_par[c] = pc;
-            s_prd[c] = __ldcg(prd + c);
-            if (c < T) s_tok[c] = tok[c];
-            if (pc < -1 || pc >= c) s_bad = 1;
-        }
-        par = s_par; tok = s_tok; prd = s_prd;
-    } else {
-        for (int c = threadIdx.x; c < N; c += blockDim.x)
-            if (par[c] < -1 || par[c] >= c) s_bad = 1;
+        for (int c = threadIdx.x; c < N; c += blockDim.x) ts.prd[c] = __ldcg(prd + c);
+        par = ts.par; tok = ts.tok; prd = ts.prd;
     }
     for (int j = threadIdx.x; j < max_path; j += blockDim.x) path[j] = -1;
     __syncthreads();
-    if (s_bad) {
+    // the word other blocks wait on (fused form) is stored with release semantics, behind everything else
+    auto finish = [&](int word) {
+        if (done_mark) st_release(accept_len + b, done_mark | word);
+        else accept_len[b] = word;
+    };
+    if (ts.bad) {
         if (threadIdx.x == 0) {
             status[b] = HT_STATUS_BAD_TREE;
             next_token[b] = -1;
-            st_release(accept_len + b, done_mark);
+            finish(0);
         }
         return;
     }
     const bool has_root = root_pred != nullptr;
-    const int rp = has_root ? root_pred[b] : -1;
+    const int rp = ts.root;
     // key = depth << 32 | (0xFFFFFFFF - node): max picks the deepest, then the lowest node
     unsigned long long key = 0;
     for (int n = threadIdx.x; n < T; n += blockDim.x) {
@@ -108,18 +130,16 @@ __device__ __forceinline__ void accept_sequence(const int b, const int32_t *__re
         const unsigned long long o = __shfl_xor_sync(0xffffffffu, key, off);
         key = o > key ? o : key;
     }
-    if ((threadIdx.x & 31) == 0) s_key[threadIdx.x >> 5] = key;
+    if ((threadIdx.x & 31) == 0) ts.key[threadIdx.x >> 5] = key;
     __syncthreads();
     if (threadIdx.x == 0) {
-        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) key = s_key[w] > key ? s_key[w] : key;
+        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) key = ts.key[w] > key ? ts.key[w] : key;
         const int len = (int)(key >> 32);
         const int node = (int)(0xFFFFFFFFu - (unsigned)(key & 0xFFFFFFFFu));
-        // the length goes last, with release semantics: it is also the word other blocks wait on (fused form: marked
-        // "done", since a small value is also what the word held before the sequence's first row arrived)
         if (len > max_path) {
             status[b] = HT_STATUS_PATH_TOO_LONG;
             next_token[b] = -1;
-            st_release(accept_len + b, done_mark);
+            finish(0);
         } else {
             status[b] = HT_STATUS_OK;
             if (len == 0) {
@@ -129,12 +149,14 @@ __device__ __forceinline__ void accept_sequence(const int b, const int32_t *__re
                 for (int c = node; c >= 0; c = par[c]) path[j--] = c;
                 next_token[b] = ld_pred(prd + node);
             }
-            st_release(accept_len + b, done_mark | len);
+            finish(len);
         }
     }
 }
 
-constexpr int kVerifyThreads = 256;
+constexpr int kVerifyThreads = 512;
+constexpr int kVerifyInFlight = 8;           // 16-byte copies per thread in flight: 64 KB per block
+constexpr int kVerifySmem = kVerifyThreads * kVerifyInFlight * 16;
 constexpr unsigned kTicket = 256u;           // arrivals are counted in units of this on the accept_len word: lengths stay below it
 constexpr int kDoneMark = 1 << 30;           // fused form: the length is in the word's low bits, the compaction may begin
 
@@ -147,25 +169,31 @@ __device__ __forceinline__ int row_argmax(const T *__restrict__ row, int V) {
     const bool vec_ok = ((size_t)V * sizeof(T)) % 16 == 0;
     if (vec_ok) {
         const int nvec = V / VE;
-        constexpr int U = 16;                      // independent 16-byte loads in flight per thread: 64 KB per block and pass
+        constexpr int U = kVerifyInFlight;
+        extern __shared__ uint4 s_stage[];             // [U][kVerifyThreads]: a thread reads back its own copies only
         for (int j0 = threadIdx.x; j0 < nvec; j0 += U * kVerifyThreads) {
-            uint4 raw[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int j = j0 + u * kVerifyThreads;
-                raw[u] = __ldcs(reinterpret_cast<const uint4 *>(row + (size_t)min(j, nvec - 1) * VE));   // past the end: the last vector again
+                if (j < nvec)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(&s_stage[u * kVerifyThreads + threadIdx.x])),
+                                 "l"(row + (size_t)j * VE) : "memory");
             }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const int j = min(j0 + u * kVerifyThreads, nvec - 1);
-                float f[VE];
-                unpack16<T>(raw[u], f);
+                const int j = j0 + u * kVerifyThreads;
+                if (j < nvec) {
+                    float f[VE];
+                    unpack16<T>(s_stage[u * kVerifyThreads + threadIdx.x], f);
 #pragma unroll
-                for (int e = 0; e < VE; ++e) {
-                    // A thread meets its elements in increasing index order, so "larger value, lower index
-                    // on ties" is "strictly larger than the best so far".  NaN compares false and is
-                    // skipped; so is -inf, which a row without anything larger settles below.
-                    if (f[e] > best.v) best = Best{f[e], j * VE + e};
+                    for (int e = 0; e < VE; ++e) {
+                        // A thread meets its elements in increasing index order, so "larger value, lower index
+                        // on ties" is "strictly larger than the best so far".  NaN compares false and is
+                        // skipped; so is -inf, which a row without anything larger settles below.
+                        if (f[e] > best.v) best = Best{f[e], j * VE + e};
+                    }
                 }
             }
         }
@@ -215,30 +243,35 @@ struct VerifyArgs {
 
 // kFused: the blocks go on to the compaction once their rows are done.
 template <typename T, bool kFused>
-__global__ void __launch_bounds__(kVerifyThreads, 4)
+__global__ void __launch_bounds__(kVerifyThreads, 2)
 verify_kernel(const VerifyArgs v, const CompactArgs c) {
     // The launch is serialized programmatically behind the kernel ahead of it in the stream: from here on everything
     // that kernel wrote may be read.  A kernel serialized behind this one may set itself up meanwhile.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __shared__ int s_last;
+    __shared__ TreeSmem ts;
+    if (threadIdx.x == 0) ts.staged_b = -1;
+    __syncthreads();
     const int n_rows = v.B * v.rows;
     for (int idx = blockIdx.x; idx < n_rows; idx += gridDim.x) {
         const int b = idx / v.rows, r = idx - b * v.rows;
+        // the sequence's tree (inputs) is on its way into shared memory while the row streams
+        stage_tree(ts, b, v.tokens, v.parent, v.root_pred, v.N, v.T);
         const int best = row_argmax<T>(static_cast<const T *>(v.logits) + ((size_t)b * v.N + r) * v.V, v.V);
         if (threadIdx.x == 0) {
             v.pred[(size_t)b * v.N + r] = best;
-            // The block that stores a sequence's last argmax searches its tree.
-            __threadfence();
-            const unsigned before = atomicAdd(reinterpret_cast<unsigned int *>(v.accept_len + b), kTicket);
+            // The block that stores a sequence's last argmax searches its tree: the count is added with release
+            // semantics (the store above comes first) and read with acquire semantics (the other rows' stores are
+            // visible behind it, to the whole block behind the barrier below).
+            unsigned before;
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(before) : "l"(v.accept_len + b), "r"(kTicket) : "memory");
             s_last = before / kTicket == (unsigned)(v.rows - 1);
         }
         __syncthreads();
-        if (s_last) {
-            __threadfence();
-            accept_sequence(b, v.tokens, v.parent, v.root_pred, v.pred, v.N, v.T, v.max_path, v.accept_len, v.accept_path,
+        if (s_last)
+            accept_sequence(ts, b, v.tokens, v.parent, v.root_pred, v.pred, v.N, v.T, v.max_path, v.accept_len, v.accept_path,
                             v.next_token, v.status, kFused ? kDoneMark : 0);
-        }
         __syncthreads();
     }
     if (!kFused) return;
@@ -275,7 +308,7 @@ verify_kernel(const VerifyArgs v, const CompactArgs c) {
             __syncthreads();
             continue;
         }
-        compact_item<8>(c, csm, layer, b, grp, a, L);
+        compact_item<4, kVerifyThreads>(c, csm, layer, b, grp, a, L);
         if (threadIdx.x == 0) {
             const unsigned before = atomicAdd(reinterpret_cast<unsigned int *>(v.accept_len + b), kTicket);
             if ((before & ~(unsigned)kDoneMark) / kTicket == (unsigned)(c.layers * c.groups - 1)) v.accept_len[b] = a;
@@ -284,10 +317,11 @@ verify_kernel(const VerifyArgs v, const CompactArgs c) {
 }
 
 template <typename... KArgs, typename... Args>
-static cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t s, Args... args) {
+static cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t s, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -302,7 +336,8 @@ template <typename Kernel>
 static int resident_blocks(Kernel kernel) {
     int dev = 0, sms = 0, per_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kVerifyThreads, 0) != cudaSuccess || sms <= 0 || per_sm <= 0) {
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kVerifySmem) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kVerifyThreads, kVerifySmem) != cudaSuccess || sms <= 0 || per_sm <= 0) {
         cudaGetLastError();
         return 148;
     }
@@ -322,8 +357,8 @@ static cudaError_t launch_verify_t(const VerifyArgs &v, const CompactArgs *compa
     }
     const long long want = (long long)v.B * v.rows;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
-    if (compact) return launch_chained(verify_kernel<T, true>, grid, (unsigned)kVerifyThreads, s, v, *compact);
-    return launch_chained(verify_kernel<T, false>, grid, (unsigned)kVerifyThreads, s, v, CompactArgs{});
+    if (compact) return launch_chained(verify_kernel<T, true>, grid, (unsigned)kVerifyThreads, (size_t)kVerifySmem, s, v, *compact);
+    return launch_chained(verify_kernel<T, false>, grid, (unsigned)kVerifyThreads, (size_t)kVerifySmem, s, v, CompactArgs{});
 }
 
 int launch_verify(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
