@@ -162,24 +162,34 @@ constexpr int kDoneMark = 1 << 30;           // fused form: the length is in the
 
 // Argmax of one logits row by the block: lowest index on ties, NaN never wins, a row of NaNs gives 0.  All threads
 // return the same index.
+// This thread's copies of one pass over a row (vectors j0, j0 + kVerifyThreads, ...) into its slots of the staging area.
+template <typename T>
+__device__ __forceinline__ void row_issue(const T *__restrict__ row, int nvec, int j0) {
+    extern __shared__ uint4 s_stage[];                 // [kVerifyInFlight][kVerifyThreads]: a thread reads back its own copies only
+#pragma unroll
+    for (int u = 0; u < kVerifyInFlight; ++u) {
+        const int j = j0 + u * kVerifyThreads;
+        if (j < nvec)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(&s_stage[u * kVerifyThreads + threadIdx.x])),
+                         "l"(row + (size_t)j * Vec16<T>::n) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+template <typename T>
+__device__ __forceinline__ bool row_vectorized(int V) { return ((size_t)V * sizeof(T)) % 16 == 0; }
+
+// The caller has issued the row's first pass (row_issue with j0 = threadIdx.x) where the row is vectorized.
 template <typename T>
 __device__ __forceinline__ int row_argmax(const T *__restrict__ row, int V) {
     constexpr int VE = Vec16<T>::n;
     Best best{-INFINITY, INT_MAX};
-    const bool vec_ok = ((size_t)V * sizeof(T)) % 16 == 0;
+    const bool vec_ok = row_vectorized<T>(V);
     if (vec_ok) {
         const int nvec = V / VE;
         constexpr int U = kVerifyInFlight;
-        extern __shared__ uint4 s_stage[];             // [U][kVerifyThreads]: a thread reads back its own copies only
+        extern __shared__ uint4 s_stage[];
         for (int j0 = threadIdx.x; j0 < nvec; j0 += U * kVerifyThreads) {
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int j = j0 + u * kVerifyThreads;
-                if (j < nvec)
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(&s_stage[u * kVerifyThreads + threadIdx.x])),
-                                 "l"(row + (size_t)j * VE) : "memory");
-            }
-            asm volatile("cp.async.commit_group;" ::: "memory");
+            if (j0 != (int)threadIdx.x) row_issue<T>(row, nvec, j0);
             asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
             for (int u = 0; u < U; ++u) {
@@ -256,9 +266,11 @@ verify_kernel(const VerifyArgs v, const CompactArgs c) {
     const int n_rows = v.B * v.rows;
     for (int idx = blockIdx.x; idx < n_rows; idx += gridDim.x) {
         const int b = idx / v.rows, r = idx - b * v.rows;
-        // the sequence's tree (inputs) is on its way into shared memory while the row streams
+        // the row's first 64 KB are asked for, then the sequence's tree (inputs) goes into shared memory while they stream
+        const T *row = static_cast<const T *>(v.logits) + ((size_t)b * v.N + r) * v.V;
+        if (row_vectorized<T>(v.V)) row_issue<T>(row, v.V / Vec16<T>::n, threadIdx.x);
         stage_tree(ts, b, v.tokens, v.parent, v.root_pred, v.N, v.T);
-        const int best = row_argmax<T>(static_cast<const T *>(v.logits) + ((size_t)b * v.N + r) * v.V, v.V);
+        const int best = row_argmax<T>(row, v.V);
         if (threadIdx.x == 0) {
             v.pred[(size_t)b * v.N + r] = best;
             // The block that stores a sequence's last argmax searches its tree: the count is added with release
