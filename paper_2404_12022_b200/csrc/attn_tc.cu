@@ -145,30 +145,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // (status words, workspace and `out` are written behind that), the issuer before its first product.
     const bool early = !kPaged && p.early != 0;
     if (!early) wait_for_kernel_ahead();
-    plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0 && !early, kPaged, p.n_rt);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = sm.tmem_base;
-
-    const int total = sm.pre[p.B];
-    const int per = choose_per(total, p.grid, sm.nkt, p.B, p.n_rt);
-    int t_begin = min((int)blockIdx.x * per, total);
-    int t_end = min(t_begin + per, total);
+    // Persistent form: CTA i takes the i-th range of the tile list.  Cluster form: one cluster per (sequence, KV head);
+    // its CTAs take cost-equal shares of the unit's tiles.  (No cluster barrier here: the first remote access comes
+    // after the one all threads pass ahead of the exchange.)  One thread works the range and its first segment out.
     constexpr bool clustered = kClustered;
     uint32_t c_rank = 0;
+    RangeAsk ask;
+    ask.n_pos = p.grid; ask.my_pos = (int)blockIdx.x;
+    ask.cluster_k = 0; ask.cl_rank = 0; ask.cl_b = 0; ask.cl_unit = 0;
     if (clustered) {
-        // One cluster per (sequence, KV head); the cluster's CTAs take equal shares of its tiles.  (No cluster
-        // barrier here: the first remote access comes after the one all threads pass ahead of the exchange.)
         c_rank = cluster_ctarank();
-        const int unit = (int)blockIdx.x / p.cluster_k, b = unit / p.Hkv, hk = unit - b * p.Hkv;
-        const int nk = sm.nkt[b];
-        const int t0 = sm.pre[b] + hk * nk;
-        int lo, hi;
-        cluster_share(nk, sm.len[b], p.cluster_k, (int)c_rank, lo, hi);
-        t_begin = t0 + lo;
-        t_end = t0 + hi;
+        const int unit = (int)blockIdx.x / p.cluster_k;
+        ask.cluster_k = p.cluster_k; ask.cl_rank = (int)c_rank;
+        ask.cl_b = unit / p.Hkv;
+        ask.cl_unit = unit - ask.cl_b * p.Hkv;
     }
+    tc_fence_before();                              // (the tensor memory's base address crosses the plan's last barrier)
+    plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0 && !early, kPaged, 1, ask, sm.plan);   // one unit per KV head in this kernel
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+    const Range range = read_range(sm.plan);
+    const int per = range.per, t_begin = range.t_begin, t_end = range.t_end;
+    const Segment first = range.first;
 
     if (warp == 8) {
         // ------------------------------- TMA producer -------------------------------
@@ -186,18 +184,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 }
             };
             TileCursor cur_k, cur_v, cur_p;          // the K and V streams of the ring order, and the page-id lookahead
-            cur_k.init(t_begin, t_end);
-            cur_v.init(t_begin, t_end);
-            cur_p.init(t_begin, t_end);
+            cur_k.init(t_begin, t_end, first);
+            cur_v.init(t_begin, t_end, first);
+            cur_p.init(t_begin, t_end, first);
             if (kPaged)
-                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p, lane, p.n_rt);
+                for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p, lane, 1);
             for (int e = 0; e < 2 * n; ++e) {
                 if (kPaged ? __any_sync(0xFFFFFFFFu, *abort_flag != 0) : (*abort_flag != 0)) break;
                 // entry e of the consumption order: K_0, K_1, V_0, K_2, V_1, ..., V_{n-1}
                 const bool is_v = e == 2 * n - 1 || (e != 0 && (e & 1) == 0);
                 const int j = e == 0 ? 0 : (e == 2 * n - 1 ? n - 1 : (is_v ? (e - 2) / 2 : (e + 1) / 2));
-                if (is_v) cur_v.next(sm.pre, sm.nkt, p.B, p.n_rt);   // tile j of its stream
-                else cur_k.next(sm.pre, sm.nkt, p.B, p.n_rt);
+                if (is_v) cur_v.next(sm.pre, sm.nkt, p.B, 1);   // tile j of its stream
+                else cur_k.next(sm.pre, sm.nkt, p.B, 1);
                 struct { int b, hk, rt; } s;
                 s.b = is_v ? cur_v.s.b : cur_k.s.b;
                 s.hk = is_v ? cur_v.s.hk : cur_k.s.hk;
@@ -223,7 +221,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
                 if (kPaged && !is_v) {
                     // the ids of tile j were asked for kPgAhead tiles ago; ask for those of tile j + kPgAhead
-                    pages_request(p, pp, sm.pre, sm.nkt, sm.pg, j + kPgAhead, cur_p, lane, p.n_rt);
+                    pages_request(p, pp, sm.pre, sm.nkt, sm.pg, j + kPgAhead, cur_p, lane, 1);
                     cp_async_wait<kPgAhead>();
                 }
                 if (lane == 0) mbar_expect_tx(&sm.kv_full[slot], kEntryBytes);
@@ -266,11 +264,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 // q is the kernel ahead's to write: the range's first Q tile is fetched here, behind the wait, while the
                 // producer is busy with the first context tiles
                 wait_for_kernel_ahead();
-                if (t_end > t_begin) {
-                    int hint = 0;
-                    const Segment s0 = locate(sm.pre, sm.nkt, p.B, p.n_rt, t_begin, t_end, hint);
-                    fetch_q_tile(sm, tm_q, p, s0.hk, s0.rt, s0.b);
-                }
+                if (t_end > t_begin) fetch_q_tile(sm, tm_q, p, first.hk, first.rt, first.b);
             }
             const uint32_t idesc_qk = instr_desc(kBf16, 0), idesc_pv = instr_desc(kBf16, 1);
             const uint32_t hi_k = desc_hi(1, 1024 >> 4), hi_v = desc_hi(kSlabBytes >> 4, 1024 >> 4);
@@ -309,7 +303,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             };
             if (n == 1) v_slot = 1;                                          // a single tile: K_0, V_0
             for (int t = t_begin; t < t_end;) {
-                const Segment sg = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
+                const Segment sg = t == t_begin ? first : locate(sm.pre, sm.nkt, p.B, 1, t, t_end, b_hint);
                 const int L = sm.len[sg.b];
                 alive = alive && mbar_wait_quick(smem_u32(&sm.q_full), seg_i & 1, abort_flag);
                 for (int i = 0; i < sg.len; ++i) {
@@ -368,7 +362,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
         };
         for (int t = t_begin; t < t_end;) {
-            const Segment sg = locate(sm.pre, sm.nkt, p.B, p.n_rt, t, t_end, b_hint);
+            const Segment sg = t == t_begin ? first : locate(sm.pre, sm.nkt, p.B, 1, t, t_end, b_hint);
             const int L = sm.len[sg.b];
             // --- ancestor masks of this tile's rows (kept while sequence and row tile stay the same) ---
             const int node = sg.rt * p.rows_per_tile_nodes + row / p.g;

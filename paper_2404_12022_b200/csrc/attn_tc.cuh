@@ -16,6 +16,7 @@ constexpr int kEntryBytes = kTile * kD * 2;
 constexpr int kSlabBytes = kEntryBytes / 2;   // [128 rows][64 elements] = 16 KiB
 constexpr int kThreads = 320;
 constexpr int kMaxB = 256;
+constexpr int kPlanWords = 12;         // per, t_begin, t_end, first segment (b, hk, rt, kt0, len, nkt)
 constexpr int kMaxWords = 32;              // ancestor words per row -> N <= 1024
 constexpr int kSlotFloats = kRows * kD + 2 * kRows;   // one partial result: O as [32 feature groups][128 rows][4], m[128], l[128]
 constexpr uint32_t kTmemCols = 512;
@@ -66,6 +67,7 @@ struct __align__(1024) Smem {
     int32_t len[kMaxB];
     int32_t nkt[kMaxB];
     int32_t pre[kMaxB + 1];
+    int32_t plan[kPlanWords];          // the CTA's share of the tiles and its first segment (plan_sequences)
     unsigned long long kv_full[kStages], kv_empty[kStages], q_full, q_empty, s_full[2], p_ready[2], o_done[2], mma_drain;
     int abort, wait_kcycles;           // the abort flag, and right behind it the limit of a wait (the waits read both as one 8-byte word)
     uint32_t tmem_base;
@@ -394,6 +396,18 @@ struct Segment {
     int b, hk, rt, kt0, len, nkt;
 };
 
+// a / b for 0 <= a, 0 < b.  The plan is a chain of dependent instructions that every launch runs through before its
+// first fetch, and the compiler's 32-bit division is some 35 of them: below 2^22 the quotient comes from the
+// reciprocal in single precision (within one of the truth: both operands are exact, the product is off by a few
+// units in its last place) and is put right by the remainder.
+__device__ __forceinline__ int fast_div(int a, int b) {
+    if ((a | b) >> 22) return a / b;
+    int q = __float2int_rz(__fdividef((float)a, (float)b));
+    const int r = a - q * b;
+    q += r >= b ? 1 : (r < 0 ? -1 : 0);
+    return q;
+}
+
 __device__ __forceinline__ Segment locate(const int32_t *pre, const int32_t *nkt, int B, int n_rt, int t, int t_end, int &b_hint) {
     int b = b_hint;
     while (b < B - 1 && t >= pre[b + 1]) ++b;
@@ -402,9 +416,9 @@ __device__ __forceinline__ Segment locate(const int32_t *pre, const int32_t *nkt
     s.b = b;
     s.nkt = nkt[b];
     const int local = t - pre[b];
-    const int unit = local / s.nkt;
+    const int unit = fast_div(local, s.nkt);
     s.kt0 = local - unit * s.nkt;
-    s.hk = unit / n_rt;
+    s.hk = n_rt == 1 ? unit : fast_div(unit, n_rt);
     s.rt = unit - s.hk * n_rt;
     s.len = min(s.nkt - s.kt0, t_end - t);
     return s;
@@ -417,6 +431,11 @@ struct TileCursor {
     int t, t_end, b_hint;
     __device__ __forceinline__ void init(int t_begin, int t_end_) {
         t = t_begin; t_end = t_end_; b_hint = 0; i = 0; s.len = 0; s.kt0 = 0;
+    }
+    // ... with the range's first segment already known (an empty range: first.len == 0)
+    __device__ __forceinline__ void init(int t_begin, int t_end_, const Segment &first) {
+        t = t_begin; t_end = t_end_; b_hint = first.b; i = 0; s = first;
+        if (s.len == 0) s.kt0 = 0;
     }
     // Moves to the next tile; false past the end of the range.  Afterwards s.b / s.hk / s.rt are the tile's
     // unit, kt() its index within the unit's tiles and first() tells whether it opens a segment.
@@ -434,14 +453,14 @@ struct TileCursor {
     __device__ __forceinline__ bool first() const { return i == 1; }
 };
 
-__device__ __forceinline__ int tiles_per_cta(int total, int grid) { return (total + grid - 1) / grid; }
+__device__ __forceinline__ int tiles_per_cta(int total, int grid) { return fast_div(total + grid - 1, grid); }
 
 // Shares of a unit's nkt tiles among the k CTAs of a cluster.  A tile with tree keys costs about two context tiles
 // (mask, P as a hi + lo pair, twice the P V products), so the shares are equal in cost rather than in tiles: with
 // 8 context tiles and the tree tile over 4 CTAs, 3 + 3 + 2 + 1 instead of 3 + 3 + 3 + 0.
 __device__ __forceinline__ void cluster_share(int nkt, int L, int k, int rank, int &lo, int &hi) {
-    const int n_ctx = min(L / kTile, nkt);                 // tiles of context keys only
-    const int cost = n_ctx + 2 * (nkt - n_ctx), share = (cost + k - 1) / k;
+    const int n_ctx = max(0, min(L / kTile, nkt));         // tiles of context keys only (a refused length: none)
+    const int cost = n_ctx + 2 * (nkt - n_ctx), share = (cost + k - 1) >> (__ffs(k) - 1);     // k is a power of two
     auto tile_at = [&](int c) { return min(c <= n_ctx ? c : n_ctx + (c - n_ctx) / 2, nkt); };
     lo = tile_at(rank * share);
     hi = rank == k - 1 ? nkt : tile_at((rank + 1) * share);
@@ -468,49 +487,145 @@ __device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nk
     if (n == 0 || even == 0) return even;
     int cand;
     if (n >= even) {
-        const int k = n / even;                       // largest count of parts whose length is >= even
-        cand = (n + k - 1) / k;
+        const int k = fast_div(n, even);              // largest count of parts whose length is >= even
+        cand = fast_div(n + k - 1, k);
     } else {
-        cand = (even + n - 1) / n * n;                // whole units
+        cand = fast_div(even + n - 1, n) * n;         // whole units
     }
     return (cand - even <= 8 || (n_rt > 1 && cand * 20 <= even * 21)) ? cand : even;
 }
 
-// Validates every sequence and fills len / nkt / pre.  Called by all threads of a block.
+// Which share of the tile list a CTA takes.  Persistent form: place `my_pos` of `n_pos` ranges of `per` tiles
+// (choose_per).  Cluster form (cluster_k > 1): the CTA's cost-equal share of the one unit its cluster works on,
+// sequence cl_b, unit cl_unit of that sequence's units.
+struct RangeAsk {
+    int n_pos, my_pos;
+    int cluster_k, cl_rank, cl_b, cl_unit;
+};
+struct Range {
+    int per, t_begin, t_end;
+    Segment first;                 // the segment that holds tile t_begin (len == 0: the range is empty)
+};
+__device__ __forceinline__ Range read_range(const int32_t *w) {
+    Range r;
+    r.per = w[0]; r.t_begin = w[1]; r.t_end = w[2];
+    r.first.b = w[3]; r.first.hk = w[4]; r.first.rt = w[5]; r.first.kt0 = w[6]; r.first.len = w[7]; r.first.nkt = w[8];
+    return r;
+}
+
+// The CTA's range and first segment from the finished len / nkt / pre arrays: one thread's work (a chain of
+// dependent integer instructions with half a dozen divisions; run by every thread it would also queue up at the
+// conversion units), left in shared memory for everybody.
+__device__ __forceinline__ void plan_range(const int32_t *s_len, const int32_t *s_nkt, const int32_t *s_pre, int B, int Hkv,
+                                           int units_per_head, const RangeAsk &ask, int32_t *w) {
+    const int total = s_pre[B];
+    Range r;
+    r.first.b = 0; r.first.hk = 0; r.first.rt = 0; r.first.kt0 = 0; r.first.len = 0; r.first.nkt = 0;
+    if (ask.cluster_k > 1) {
+        r.per = 0;
+        const int nk = s_nkt[ask.cl_b];
+        int lo, hi;
+        cluster_share(nk, s_len[ask.cl_b], ask.cluster_k, ask.cl_rank, lo, hi);
+        const int t0 = s_pre[ask.cl_b] + ask.cl_unit * nk;
+        r.t_begin = t0 + lo;
+        r.t_end = t0 + hi;
+        r.first.b = ask.cl_b;
+        r.first.hk = units_per_head == 1 ? ask.cl_unit : fast_div(ask.cl_unit, units_per_head);
+        r.first.rt = ask.cl_unit - r.first.hk * units_per_head;
+        r.first.kt0 = lo; r.first.len = hi - lo; r.first.nkt = nk;
+    } else {
+        r.per = choose_per(total, ask.n_pos, s_nkt, B, units_per_head);
+        r.t_begin = ask.my_pos < ask.n_pos ? min(ask.my_pos * r.per, total) : total;
+        r.t_end = min(r.t_begin + r.per, total);
+        if (r.t_end > r.t_begin) {
+            int hint = 0;
+            r.first = locate(s_pre, s_nkt, B, units_per_head, r.t_begin, r.t_end, hint);
+        }
+    }
+    w[0] = r.per; w[1] = r.t_begin; w[2] = r.t_end;
+    w[3] = r.first.b; w[4] = r.first.hk; w[5] = r.first.rt; w[6] = r.first.kt0; w[7] = r.first.len; w[8] = r.first.nkt;
+}
+
+// Validates every sequence and fills len / nkt / pre.  Called by all threads of a block; ends with a barrier.  Every
+// launch runs through this before its first fetch, so the common case (no malformed tree) takes two barriers: one
+// that also tells whether any thread met a bad parent entry, and the one at the end.
 template <int NT>
 __device__ __forceinline__ void plan_sequences(const Params &p, int32_t *s_len, int32_t *s_nkt, int32_t *s_pre,
-                                               bool write_status, bool errors_only, int units_per_head) {
+                                               bool write_status, bool errors_only, int units_per_head,
+                                               const RangeAsk &ask, int32_t *s_plan) {
     // The lengths are asked for first and used last, so that their round trip to memory overlaps
     // the scan of the parent arrays (B <= kMaxB <= NT: one sequence per thread).
     const int my_b = threadIdx.x;
     const int my_L = my_b < p.B ? p.kv_len[my_b] : 0;
-    for (int b = threadIdx.x; b < p.B; b += NT) s_nkt[b] = 0;       // 0 = legal so far
-    __syncthreads();
-    for (int i = threadIdx.x; i < p.B * p.N; i += NT) {
-        const int b = i / p.N, c = i - b * p.N;
-        const int par = p.parent[i];
-        if (par < -1 || par >= c) s_nkt[b] = -1;                     // benign race: all writers store -1
+    const int entries = p.B * p.N;
+    bool saw_bad = false;
+    {
+        // entry i = (sequence b, row c); a step of NT entries moves (b, c) by (db, dc) with one carry at most
+        const int par0 = (int)threadIdx.x < entries ? p.parent[threadIdx.x] : -1;   // on its way while (b, c) are formed
+        int b = fast_div((int)threadIdx.x, p.N), c = (int)threadIdx.x - b * p.N;
+        const int db = fast_div(NT, p.N), dc = NT - db * p.N;
+        for (int i = threadIdx.x; i < entries; i += NT) {
+            const int par = i == (int)threadIdx.x ? par0 : p.parent[i];
+            saw_bad = saw_bad || par < -1 || par >= c;
+            b += db;
+            c += dc;
+            if (c >= p.N) { c -= p.N; ++b; }
+        }
     }
-    __syncthreads();
+    if (__syncthreads_or(saw_bad)) {
+        // some tree is malformed: which sequences, through shared memory (0 = legal so far)
+        for (int b = threadIdx.x; b < p.B; b += NT) s_nkt[b] = 0;
+        __syncthreads();
+        for (int i = threadIdx.x; i < entries; i += NT) {
+            const int b = i / p.N, c = i - b * p.N;
+            const int par = p.parent[i];
+            if (par < -1 || par >= c) s_nkt[b] = -1;                 // benign race: all writers store -1
+        }
+        __syncthreads();
+        saw_bad = my_b < p.B && s_nkt[my_b] < 0;                     // now: is this thread's own sequence malformed
+        __syncthreads();
+    } else {
+        saw_bad = false;
+    }
+    int my_n = 0;                                                    // this thread's sequence: its tiles per unit
     if (my_b < p.B) {
         const int b = my_b, L = my_L;
         int code = HT_STATUS_OK;
-        if (s_nkt[b] < 0) code = HT_STATUS_BAD_TREE;
+        if (saw_bad) code = HT_STATUS_BAD_TREE;
         if (L < 0 || (long long)L + p.N > p.cap) code = HT_STATUS_BAD_LEN;
         s_len[b] = L;
-        s_nkt[b] = code == HT_STATUS_OK ? (L + p.N + kTile - 1) / kTile : 0;
+        my_n = code == HT_STATUS_OK ? (L + p.N + kTile - 1) / kTile : 0;
+        s_nkt[b] = my_n;
         // paged cache: the status words were zeroed ahead of the launch, and a fetch may already have
         // reported a bad page for this sequence, so only errors are written
         if (write_status && (code != HT_STATUS_OK || !errors_only)) p.status[b] = code;
     }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int acc = 0;
-        for (int b = 0; b < p.B; ++b) {
-            s_pre[b] = acc;
-            acc += s_nkt[b] * p.Hkv * units_per_head;
+    if (p.B <= 32) {
+        // prefix sums of the units' tiles by shuffles in the first warp
+        if (threadIdx.x < 32) {
+            const int mine = my_n * p.Hkv * units_per_head;
+            int inc = mine;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(0xFFFFFFFFu, inc, off);
+                if ((int)threadIdx.x >= off) inc += o;
+            }
+            if (my_b < p.B) s_pre[my_b] = inc - mine;
+            if (my_b == p.B - 1) s_pre[p.B] = inc;
+            __syncwarp();
+            if (threadIdx.x == 0) plan_range(s_len, s_nkt, s_pre, p.B, p.Hkv, units_per_head, ask, s_plan);
         }
-        s_pre[p.B] = acc;
+    } else {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int acc = 0;
+            for (int b = 0; b < p.B; ++b) {
+                s_pre[b] = acc;
+                acc += s_nkt[b] * p.Hkv * units_per_head;
+            }
+            s_pre[p.B] = acc;
+            plan_range(s_len, s_nkt, s_pre, p.B, p.Hkv, units_per_head, ask, s_plan);
+        }
     }
     __syncthreads();
 }

@@ -94,6 +94,7 @@ struct __align__(1024) PSmem {
     int32_t len[kMaxB];
     int32_t nkt[kMaxB];
     int32_t pre[kMaxB + 1];
+    int32_t plan[kPlanWords];          // the CTA's share of the tiles and its first segment (plan_sequences)
     unsigned long long kv_full[kPStages], kv_empty[kPStages], q_full, q_empty, s_full[2][2], p_ready[2][2], o_done[2][2], mma_drain;
     int abort, wait_kcycles;           // the abort flag, and right behind it the limit of a wait (the waits read both as one 8-byte word)
     uint32_t tmem_base;
@@ -153,35 +154,38 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int my_rt = grouped ? (int)blockIdx.x % p.n_rt : 0;               // grouped: this CTA's tile pair
     const int my_pos = grouped ? (int)blockIdx.x / p.n_rt : (int)blockIdx.x; // place in the list's partition
     const int n_pos = grouped ? p.grid / p.n_rt : p.grid;
-    plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0 && !early, kPaged, lrt);
-    tc_fence_before();
-    __syncthreads();
+    // Cluster form: one cluster per (sequence, KV head, tile pair); its CTAs take cost-equal shares of the unit's tiles.
+    // (No cluster barrier here: the first remote access comes after the one all threads pass ahead of the exchange.)
+    // One thread works the CTA's range and its first segment out.
+    uint32_t c_rank = 0;
+    RangeAsk ask;
+    ask.n_pos = n_pos; ask.my_pos = my_pos;
+    ask.cluster_k = 0; ask.cl_rank = 0; ask.cl_b = 0; ask.cl_unit = 0;
+    if (clustered) {
+        c_rank = cluster_ctarank();
+        const int unit = (int)blockIdx.x / p.cluster_k;
+        ask.cluster_k = p.cluster_k; ask.cl_rank = (int)c_rank;
+        ask.cl_b = unit / (p.Hkv * p.n_rt);
+        ask.cl_unit = unit - ask.cl_b * p.Hkv * p.n_rt;
+    }
+    tc_fence_before();                              // (the tensor memory's base address crosses the plan's last barrier)
+    plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0 && !early, kPaged, lrt, ask, sm.plan);
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
-
-    const int total = sm.pre[p.B];
-    const int per = choose_per(total, n_pos, sm.nkt, p.B, lrt);
-    int t_begin = my_pos < n_pos ? min(my_pos * per, total) : total;
-    int t_end = min(t_begin + per, total);
+    const Range range = read_range(sm.plan);
+    const int per = range.per, t_begin = range.t_begin, t_end = range.t_end;
+    Segment first = range.first;
+    if (grouped) first.rt = my_rt;
     // the segment that holds tile t of the list; grouped: the tile pair is the CTA's own
     auto find = [&](int t, int te, int &hint) {
+        if (t == t_begin) {
+            hint = first.b;
+            return first;
+        }
         Segment sg = locate(sm.pre, sm.nkt, p.B, lrt, t, te, hint);
         if (grouped) sg.rt = my_rt;
         return sg;
     };
-    uint32_t c_rank = 0;
-    if (clustered) {
-        // One cluster per (sequence, KV head, tile pair); its CTAs take equal shares of the unit's tiles.  (No
-        // cluster barrier here: the first remote access comes after the one all threads pass ahead of the exchange.)
-        c_rank = cluster_ctarank();
-        const int unit = (int)blockIdx.x / p.cluster_k, b = unit / (p.Hkv * p.n_rt);
-        const int nk = sm.nkt[b];
-        const int t0 = sm.pre[b] + (unit - b * p.Hkv * p.n_rt) * nk;
-        int lo, hi;
-        cluster_share(nk, sm.len[b], p.cluster_k, (int)c_rank, lo, hi);
-        t_begin = t0 + lo;
-        t_end = t0 + hi;
-    }
     unsigned char *const xarea = &sm.q[0][0];          // Q buffers and ring, idle once the CTA's tiles are done
     // The Q tiles of a segment's tile pair (one where the pair has no second tile).
     auto fetch_q = [&](const Segment &s) {
@@ -203,7 +207,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (kPaged || lane == 0) {
             int b_hint = 0, ring_i = 0, seg_i = 0;
             TileCursor cur_p;                         // page-id lookahead
-            cur_p.init(t_begin, t_end);
+            cur_p.init(t_begin, t_end, first);
             if (kPaged)
                 for (int jt = 0; jt < kPgAhead; ++jt) pages_request(p, pp, sm.pre, sm.nkt, sm.pg, jt, cur_p, lane, lrt);
             bool stop = false;
