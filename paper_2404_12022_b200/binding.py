@@ -197,7 +197,7 @@ def tree_attention(q, k_cache, v_cache, kv_len, parent, out=None, workspace=None
 
 
 def tree_attention_paged(q, k_pages, v_pages, block_table, kv_len, parent, out=None, workspace=None, status=None,
-                         scale: float = 0.0):
+                         scale: float = 0.0, flags: int = 0):
     """q [B, N, Hq, D]; page pools [n_pages, Hkv, page_size, D] (may be strided over page / head);
     block_table [B, max_pages] int32; kv_len [B] int32; parent [B, N] int32.  Returns (out, status)."""
     _need(q, name="q")
@@ -215,7 +215,7 @@ def tree_attention_paged(q, k_pages, v_pages, block_table, kv_len, parent, out=N
     if block_table.dim() != 2 or block_table.shape[0] != B or tuple(parent.shape) != (B, N) or tuple(kv_len.shape) != (B,):
         raise ValueError("block_table must be [B, max_pages], parent [B, N], kv_len [B]")
     max_pages = block_table.shape[1]
-    desc = AttnDesc(B, N, Hq, Hkv, D, max_pages * page_size, _DTYPES[q.dtype], scale, 0, 0, 0, 0)
+    desc = AttnDesc(B, N, Hq, Hkv, D, max_pages * page_size, _DTYPES[q.dtype], scale, 0, 0, 0, flags)
     pages = PagedDesc(page_size, max_pages, n_pages, k_pages.stride(0), k_pages.stride(1))
     if out is None:
         out = torch.empty_like(q)

@@ -143,7 +143,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // the kernel ahead where it first touches what that kernel may have written or may still read -- the producer
     // before the Q tile and before the first tile with tree rows, the softmax threads before their first scores
     // (status words, workspace and `out` are written behind that), the issuer before its first product.
-    const bool early = !kPaged && p.early != 0;
+    const bool early = p.early != 0;
+    if (kPaged && early)
+        for (int b = threadIdx.x; b < p.B; b += blockDim.x) sm.bad_page[b] = 0;     // (the plan's barriers come before any fetch)
     if (!early) wait_for_kernel_ahead();
     // Persistent form: CTA i takes the i-th range of the tile list.  Cluster form: one cluster per (sequence, KV head);
     // its CTAs take cost-equal shares of the unit's tiles.  (No cluster barrier here: the first remote access comes
@@ -181,6 +183,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (!waited) {
                     wait_for_kernel_ahead();
                     waited = true;
+                    if (kPaged) {                       // bad page entries met so far (the whole warp is here)
+                        __syncwarp();
+                        for (int b = lane; b < p.B; b += 32)
+                            if (sm.bad_page[b]) p.status[b] = HT_STATUS_BAD_PAGE;
+                    }
                 }
             };
             TileCursor cur_k, cur_v, cur_p;          // the K and V streams of the ring order, and the page-id lookahead
@@ -228,7 +235,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (kPaged) {
                     __syncwarp();                                     // the barrier is armed before any lane's copy can complete
                     fetch_kv_tile_paged(p, pp, sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt, sm.len[s.b] + p.N,
-                                        sm.pg[j % kPgTiles], lane);
+                                        sm.pg[j % kPgTiles], lane, waited ? nullptr : sm.bad_page);
                 } else {
                     fetch_kv_tile(sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt);
                 }
@@ -356,8 +363,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 waited = true;
                 if (blockIdx.x == 0 && tid256 < p.B) {
                     const int L = sm.len[tid256];
-                    p.status[tid256] = (L < 0 || (long long)L + p.N > p.cap) ? HT_STATUS_BAD_LEN
-                                       : (sm.nkt[tid256] == 0 ? HT_STATUS_BAD_TREE : HT_STATUS_OK);
+                    const int code = (L < 0 || (long long)L + p.N > p.cap) ? HT_STATUS_BAD_LEN
+                                     : (sm.nkt[tid256] == 0 ? HT_STATUS_BAD_TREE : HT_STATUS_OK);
+                    // (paged cache: the words were cleared ahead of the launch and a fetch may have reported a bad page)
+                    if (!kPaged || code != HT_STATUS_OK) p.status[tid256] = code;
                 }
             }
         };

@@ -68,6 +68,7 @@ struct __align__(1024) Smem {
     int32_t nkt[kMaxB];
     int32_t pre[kMaxB + 1];
     int32_t plan[kPlanWords];          // the CTA's share of the tiles and its first segment (plan_sequences)
+    unsigned char bad_page[kMaxB];     // paged cache, early start: sequences whose bad page entry is reported behind the wait
     unsigned long long kv_full[kStages], kv_empty[kStages], q_full, q_empty, s_full[2], p_ready[2], o_done[2], mma_drain;
     int abort, wait_kcycles;           // the abort flag, and right behind it the limit of a wait (the waits read both as one 8-byte word)
     uint32_t tmem_base;
@@ -662,15 +663,21 @@ __device__ __forceinline__ void fetch_kv_tile(unsigned char *dst, const CUtensor
 // it asked for itself.  An id outside the pool is replaced by page 0 (no access outside the pool), and
 // reported in the sequence's status word if any of the page's rows is a key of the sequence (rows past
 // kv_len + N are masked and zeroed anyway).
+// `later`: not null while the kernel ahead in the stream may still be running (it is the one that clears the status
+// words): the report is left there and written out behind the wait.
 __device__ __forceinline__ void fetch_kv_tile_paged(const Params &p, const PagedParams &pp, unsigned char *dst, const CUtensorMap *tm,
-                                                    void *bar, int b, int hk, int kt, int keys, const int32_t *pg, int lane) {
+                                                    void *bar, int b, int hk, int kt, int keys, const int32_t *pg, int lane,
+                                                    unsigned char *later) {
     const int ps = pp.page_size;
     const int sub = ps >= kTile ? 1 : kTile >> pp.page_shift;
     if (lane < sub) {
         const int row0 = ps >= kTile ? (kt * kTile) & (ps - 1) : 0;
         int page = pg[lane];
         if ((unsigned)page >= (unsigned)pp.n_pages) {
-            if (kt * kTile + (lane << pp.page_shift) < keys) p.status[b] = HT_STATUS_BAD_PAGE;
+            if (kt * kTile + (lane << pp.page_shift) < keys) {
+                if (later) later[b] = 1;
+                else p.status[b] = HT_STATUS_BAD_PAGE;
+            }
             page = 0;
         }
         const int off = (lane << pp.page_shift) * 128;      // rows of a slab are 128 bytes apart

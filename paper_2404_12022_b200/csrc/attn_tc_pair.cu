@@ -95,6 +95,7 @@ struct __align__(1024) PSmem {
     int32_t nkt[kMaxB];
     int32_t pre[kMaxB + 1];
     int32_t plan[kPlanWords];          // the CTA's share of the tiles and its first segment (plan_sequences)
+    unsigned char bad_page[kMaxB];     // paged cache, early start: sequences whose bad page entry is reported behind the wait
     unsigned long long kv_full[kPStages], kv_empty[kPStages], q_full, q_empty, s_full[2][2], p_ready[2][2], o_done[2][2], mma_drain;
     int abort, wait_kcycles;           // the abort flag, and right behind it the limit of a wait (the waits read both as one 8-byte word)
     uint32_t tmem_base;
@@ -141,7 +142,9 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // up while that kernel was still finishing, and everything it may have written is read from here on.  `early`
     // (lengths, trees and the cache rows below the lengths were final before that kernel began): as in the one-tile
     // kernel, plan and first context tiles do not wait, and each role waits where it first needs to.
-    const bool early = !kPaged && p.early != 0;
+    const bool early = p.early != 0;
+    if (kPaged && early)
+        for (int b = threadIdx.x; b < p.B; b += blockDim.x) sm.bad_page[b] = 0;     // (the plan's barriers come before any fetch)
     if (!early) wait_for_kernel_ahead();
     // Without clusters, where a KV head has several tile pairs (units), the list of tiles is that of the HEADS: it is
     // cut into grid / n_rt ranges, and the n_rt CTAs of a range take one tile pair each.  They start together and walk
@@ -216,6 +219,11 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (!waited) {
                     wait_for_kernel_ahead();
                     waited = true;
+                    if (kPaged) {                       // bad page entries met so far (the whole warp is here)
+                        __syncwarp();
+                        for (int b = lane; b < p.B; b += 32)
+                            if (sm.bad_page[b]) p.status[b] = HT_STATUS_BAD_PAGE;
+                    }
                 }
             };
             for (int t = t_begin; t < t_end && !stop;) {
@@ -247,7 +255,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (kPaged) {
                         __syncwarp();                                 // the barrier is armed before any lane's copy can complete
                         fetch_kv_tile_paged(p, pp, sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt, sm.len[s.b] + p.N,
-                                            sm.pg[jt % kPgTiles], lane);
+                                            sm.pg[jt % kPgTiles], lane, waited ? nullptr : sm.bad_page);
                     } else {
                         fetch_kv_tile(sm.ring[slot], tm, &sm.kv_full[slot], s.b, s.hk, kt);
                     }
@@ -403,8 +411,10 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 waited = true;
                 if (blockIdx.x == 0 && tid256 < p.B) {
                     const int L = sm.len[tid256];
-                    p.status[tid256] = (L < 0 || (long long)L + p.N > p.cap) ? HT_STATUS_BAD_LEN
-                                       : (sm.nkt[tid256] == 0 ? HT_STATUS_BAD_TREE : HT_STATUS_OK);
+                    const int code = (L < 0 || (long long)L + p.N > p.cap) ? HT_STATUS_BAD_LEN
+                                     : (sm.nkt[tid256] == 0 ? HT_STATUS_BAD_TREE : HT_STATUS_OK);
+                    // (paged cache: the words were cleared ahead of the launch and a fetch may have reported a bad page)
+                    if (!kPaged || code != HT_STATUS_OK) p.status[tid256] = code;
                 }
             }
         };

@@ -83,7 +83,7 @@ def run_attention(args):
             ks = [to_pool(c) for c in ks]
             vs = [to_pool(c) for c in vs]
             call = lambda i: hb.tree_attention_paged(q, ks[i % nbuf], vs[i % nbuf], table, kv_len, parent, out=out,
-                                                     workspace=ws, status=st)
+                                                     workspace=ws, status=st, flags=hb.HT_ATTN_CONTEXT_FINAL)
         for i in range(3):
             call(i)
         torch.cuda.synchronize()

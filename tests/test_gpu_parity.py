@@ -711,7 +711,9 @@ def test_paged_attention_random_shapes_against_the_contiguous_entry_point(hb):
         tree = str(rng.choice(["random", "chain", "roots"]))
         q, pk, pv, table, kv_len, parent, k, v = make_paged_case(500 + trial, dtype, B, N, Hkv * g, Hkv, lens, ps, tree,
                                                                 extra_pages=int(rng.integers(0, 3)))
-        out, status = hb.tree_attention_paged(q, pk, pv, table, kv_len, parent)
+        # every third trial with the early start (lengths, tree, block table and context rows are final here)
+        out, status = hb.tree_attention_paged(q, pk, pv, table, kv_len, parent,
+                                              flags=hb.HT_ATTN_CONTEXT_FINAL if trial % 3 == 0 else 0)
         ref, _ = hb.tree_attention(q, k, v, kv_len, parent)
         torch.cuda.synchronize()
         what = "trial %d: B=%d N=%d Hq=%d Hkv=%d lens=%s %s %s pages of %d" % (trial, B, N, Hkv * g, Hkv, lens, tree, dtype, ps)
@@ -722,21 +724,25 @@ def test_paged_attention_random_shapes_against_the_contiguous_entry_point(hb):
         assert bool(((a - r).abs() <= 1e-3 + 2 * eps * r.abs()).all()), what + ": max diff %.3e" % float((a - r).abs().max())
 
 
-def test_paged_attention_reports_bad_pages_and_lengths(hb):
+@pytest.mark.parametrize("final", [False, True], ids=["plain", "context_final"])
+def test_paged_attention_reports_bad_pages_and_lengths(hb, final):
+    """(With the early start a bad entry among the context pages is met before the status words have been cleared
+    for this call: the report must still arrive.)"""
     from oracle import paged_oracle
+    flags = hb.HT_ATTN_CONTEXT_FINAL if final else 0
     B, N, Hq, Hkv, lens, ps = 3, 19, 8, 8, [100, 200, 300], 32
     q, pk, pv, table, kv_len, parent, k, v = make_paged_case(77, "bf16", B, N, Hq, Hkv, lens, ps)
-    good, status = hb.tree_attention_paged(q, pk, pv, table, kv_len, parent)
+    good, status = hb.tree_attention_paged(q, pk, pv, table, kv_len, parent, flags=flags)
     assert status.cpu().tolist() == [0, 0, 0]
     t2 = table.clone()
     t2[1, 2] = pk.shape[0] + 5                     # a page sequence 1 needs, outside the pool
-    out, status = hb.tree_attention_paged(q, pk, pv, t2, kv_len, parent)
+    out, status = hb.tree_attention_paged(q, pk, pv, t2, kv_len, parent, flags=flags)
     assert status.cpu().tolist() == [0, 5, 0]
     assert torch.equal(out[0], good[0]) and torch.equal(out[2], good[2])
     long = kv_len.clone()
     long[2] = table.shape[1] * ps - N + 1          # one row more than the table can address
     out = torch.full_like(good, 7.0)
-    out, status = hb.tree_attention_paged(q, pk, pv, table, long, parent, out=out)
+    out, status = hb.tree_attention_paged(q, pk, pv, table, long, parent, out=out, flags=flags)
     assert status.cpu().tolist() == [0, 0, 2]
     assert torch.equal(out[0], good[0]) and bool((out[2] == 7.0).all())
 
