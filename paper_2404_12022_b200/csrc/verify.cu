@@ -154,16 +154,18 @@ __device__ __forceinline__ void accept_sequence(TreeSmem &ts, const int b, const
     }
 }
 
-constexpr int kVerifyThreads = 512;
-constexpr int kVerifyInFlight = 8;           // 16-byte copies per thread in flight: 64 KB per block
-constexpr int kVerifySmem = kVerifyThreads * kVerifyInFlight * 16;
+// Two shapes of block, 128 KB of logits in flight per SM either way: 512 threads (64 KB of a row at once, two blocks
+// per SM) while the rows are few, so that a row is there in one round trip; 256 threads (32 KB at once, four blocks
+// per SM) when there are more rows than twice the SMs, so that all of them are under way at once.
+constexpr int kVerifyInFlight = 8;           // 16-byte copies per thread in flight
+constexpr int verify_smem(int threads) { return threads * kVerifyInFlight * 16; }
 constexpr unsigned kTicket = 256u;           // arrivals are counted in units of this on the accept_len word: lengths stay below it
 constexpr int kDoneMark = 1 << 30;           // fused form: the length is in the word's low bits, the compaction may begin
 
 // Argmax of one logits row by the block: lowest index on ties, NaN never wins, a row of NaNs gives 0.  All threads
 // return the same index.
 // This thread's copies of one pass over a row (vectors j0, j0 + kVerifyThreads, ...) into its slots of the staging area.
-template <typename T>
+template <typename T, int kVerifyThreads>
 __device__ __forceinline__ void row_issue(const T *__restrict__ row, int nvec, int j0) {
     extern __shared__ uint4 s_stage[];                 // [kVerifyInFlight][kVerifyThreads]: a thread reads back its own copies only
 #pragma unroll
@@ -179,7 +181,7 @@ template <typename T>
 __device__ __forceinline__ bool row_vectorized(int V) { return ((size_t)V * sizeof(T)) % 16 == 0; }
 
 // The caller has issued the row's first pass (row_issue with j0 = threadIdx.x) where the row is vectorized.
-template <typename T>
+template <typename T, int kVerifyThreads>
 __device__ __forceinline__ int row_argmax(const T *__restrict__ row, int V) {
     constexpr int VE = Vec16<T>::n;
     Best best{-INFINITY, INT_MAX};
@@ -189,7 +191,7 @@ __device__ __forceinline__ int row_argmax(const T *__restrict__ row, int V) {
         constexpr int U = kVerifyInFlight;
         extern __shared__ uint4 s_stage[];
         for (int j0 = threadIdx.x; j0 < nvec; j0 += U * kVerifyThreads) {
-            if (j0 != (int)threadIdx.x) row_issue<T>(row, nvec, j0);
+            if (j0 != (int)threadIdx.x) row_issue<T, kVerifyThreads>(row, nvec, j0);
             asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
             for (int u = 0; u < U; ++u) {
@@ -252,8 +254,8 @@ struct VerifyArgs {
 };
 
 // kFused: the blocks go on to the compaction once their rows are done.
-template <typename T, bool kFused>
-__global__ void __launch_bounds__(kVerifyThreads, 2)
+template <typename T, bool kFused, int kVerifyThreads>
+__global__ void __launch_bounds__(kVerifyThreads, 1024 / kVerifyThreads)
 verify_kernel(const VerifyArgs v, const CompactArgs c) {
     // The launch is serialized programmatically behind the kernel ahead of it in the stream: from here on everything
     // that kernel wrote may be read.  A kernel serialized behind this one may set itself up meanwhile.
@@ -268,9 +270,9 @@ verify_kernel(const VerifyArgs v, const CompactArgs c) {
         const int b = idx / v.rows, r = idx - b * v.rows;
         // the row's first 64 KB are asked for, then the sequence's tree (inputs) goes into shared memory while they stream
         const T *row = static_cast<const T *>(v.logits) + ((size_t)b * v.N + r) * v.V;
-        if (row_vectorized<T>(v.V)) row_issue<T>(row, v.V / Vec16<T>::n, threadIdx.x);
+        if (row_vectorized<T>(v.V)) row_issue<T, kVerifyThreads>(row, v.V / Vec16<T>::n, threadIdx.x);
         stage_tree(ts, b, v.tokens, v.parent, v.root_pred, v.N, v.T);
-        const int best = row_argmax<T>(row, v.V);
+        const int best = row_argmax<T, kVerifyThreads>(row, v.V);
         if (threadIdx.x == 0) {
             v.pred[(size_t)b * v.N + r] = best;
             // The block that stores a sequence's last argmax searches its tree: the count is added with release
@@ -320,7 +322,7 @@ verify_kernel(const VerifyArgs v, const CompactArgs c) {
             __syncthreads();
             continue;
         }
-        compact_item<4, kVerifyThreads>(c, csm, layer, b, grp, a, L);
+        compact_item<2048 / kVerifyThreads, kVerifyThreads>(c, csm, layer, b, grp, a, L);
         if (threadIdx.x == 0) {
             const unsigned before = atomicAdd(reinterpret_cast<unsigned int *>(v.accept_len + b), kTicket);
             if ((before & ~(unsigned)kDoneMark) / kTicket == (unsigned)(c.layers * c.groups - 1)) v.accept_len[b] = a;
@@ -343,34 +345,47 @@ static cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsig
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// Blocks of a verification kernel the GPU holds at once.
+// Blocks of a verification kernel the GPU holds at once (and its shared memory limit raised, once).
 template <typename Kernel>
-static int resident_blocks(Kernel kernel) {
+static int resident_blocks(Kernel kernel, int threads) {
     int dev = 0, sms = 0, per_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kVerifySmem) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kVerifyThreads, kVerifySmem) != cudaSuccess || sms <= 0 || per_sm <= 0) {
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, verify_smem(threads)) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, verify_smem(threads)) != cudaSuccess || sms <= 0 || per_sm <= 0) {
         cudaGetLastError();
         return 148;
     }
     return sms * per_sm;
 }
 
-template <typename T>
-static cudaError_t launch_verify_t(const VerifyArgs &v, const CompactArgs *compact, cudaStream_t s) {
-    static int cap_plain[64], cap_fused[64];          // per device
+template <typename T, bool kFused, int kThreads>
+static cudaError_t launch_verify_shape(const VerifyArgs &v, const CompactArgs &c, cudaStream_t s, int *blocks_out) {
+    static int caps[64];                              // per device
     int dev = 0;
     cudaGetDevice(&dev);
-    int *slot = (dev >= 0 && dev < 64) ? (compact ? &cap_fused[dev] : &cap_plain[dev]) : nullptr;
+    int *slot = (dev >= 0 && dev < 64) ? &caps[dev] : nullptr;
     int cap = slot ? *slot : 0;
     if (cap == 0) {
-        cap = compact ? resident_blocks(verify_kernel<T, true>) : resident_blocks(verify_kernel<T, false>);
+        cap = resident_blocks(verify_kernel<T, kFused, kThreads>, kThreads);
         if (slot) *slot = cap;
+    }
+    if (blocks_out) {
+        *blocks_out = cap;
+        return cudaSuccess;
     }
     const long long want = (long long)v.B * v.rows;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
-    if (compact) return launch_chained(verify_kernel<T, true>, grid, (unsigned)kVerifyThreads, (size_t)kVerifySmem, s, v, *compact);
-    return launch_chained(verify_kernel<T, false>, grid, (unsigned)kVerifyThreads, (size_t)kVerifySmem, s, v, CompactArgs{});
+    return launch_chained(verify_kernel<T, kFused, kThreads>, grid, (unsigned)kThreads, (size_t)verify_smem(kThreads), s, v, c);
+}
+
+template <typename T>
+static cudaError_t launch_verify_t(const VerifyArgs &v, const CompactArgs *compact, cudaStream_t s) {
+    int wide = 0;                                     // blocks of the 512-thread shape the GPU holds
+    cudaError_t e = compact ? launch_verify_shape<T, true, 512>(v, *compact, s, &wide) : launch_verify_shape<T, false, 512>(v, CompactArgs{}, s, &wide);
+    if (e != cudaSuccess) return e;
+    const bool few = (long long)v.B * v.rows <= wide;
+    if (compact) return few ? launch_verify_shape<T, true, 512>(v, *compact, s, nullptr) : launch_verify_shape<T, true, 256>(v, *compact, s, nullptr);
+    return few ? launch_verify_shape<T, false, 512>(v, CompactArgs{}, s, nullptr) : launch_verify_shape<T, false, 256>(v, CompactArgs{}, s, nullptr);
 }
 
 int launch_verify(const void *logits, int dtype, const int32_t *tokens, const int32_t *parent,
