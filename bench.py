@@ -207,7 +207,7 @@ class ClockSampler:
 # DRAM traffic per launch of the attention kernel on a c3 layer, from the ncu capture of the committed build summarised
 # at the end of profiles/attn_tc_kernel_c3_layer.md (dram__bytes_read.sum + dram__bytes_write.sum, mean of two launches).  It is only
 # reported while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 287.5e6,
+NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 287.7e6,
                "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh",
                           "paper_2404_12022_b200/csrc/ht_common.cuh"],
                "sha256": "993c72d0b1ffbf1ec2f4e4feb818e5504ccbbfcfe7aace9b6e2936a554e4a60f"}
