@@ -31,7 +31,15 @@
 //                        a list of 128-key tiles; CTA i takes tiles [i*per, (i+1)*per).  A
 //                        unit that is cut writes (m, l, O) partials to the workspace and
 //                        takes a ticket; the CTA that delivers the last part of a unit
-//                        merges all parts -- nobody waits on another CTA.
+//                        merges all parts -- nobody waits on another CTA.  The ticket words
+//                        reset themselves (a caller that keeps its workspace needs no kernel
+//                        to clear them: HT_ATTN_WORKSPACE_CLEAN).  Few units: clusters, with
+//                        the parts reduced through distributed shared memory.
+//   launch             : serialized programmatically behind the kernel ahead in the stream.
+//                        With the caller's word that lengths, trees and context rows were
+//                        final before that kernel began (HT_ATTN_CONTEXT_FINAL) the plan and
+//                        the first context tiles do not wait for it; each role waits where it
+//                        first touches what that kernel may still write or read.
 //
 // Every wait on an mbarrier is bounded; when one runs out the CTA raises an abort flag,
 // reports HT_STATUS_TIMEOUT, runs to the end of its control flow without further waiting,
