@@ -254,14 +254,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 __syncwarp();
             }
             release();
-            if (lane == 0 && *abort_flag) {
-                // Every copy this warp issued must have landed before the CTA exits: wait, with the
-                // usual bound, for the latest armed phase of each ring slot and of the Q buffer.
-                for (int e = max(0, ring_i - kStages); e < ring_i; ++e)
-                    mbar_wait(&sm.kv_full[e % kStages], (e / kStages) & 1, abort_flag, false);
-                // (early: the first Q tile was fetched by the issuing thread, whatever else happened)
-                const int q_fetches = early && n > 0 && seg_i == 0 ? 1 : seg_i;
-                if (q_fetches > 0) mbar_wait(&sm.q_full, (q_fetches - 1) & 1, abort_flag, false);
+            if (lane == 0) {
+                // how many ring entries and Q tiles were asked for: should the CTA give up, the teardown waits for the
+                // last of them (early: the first Q tile was fetched by the issuing thread, whatever else happened)
+                sm.plan[9] = ring_i;
+                sm.plan[10] = early && n > 0 && seg_i == 0 ? 1 : seg_i;
             }
         }
         if (clustered) {                               // the two barriers of the exchange (whole warp)
@@ -693,6 +690,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (sm.abort && threadIdx.x == 0) {
         for (int b = 0; b < p.B; ++b)
             if (sm.nkt[b] > 0) p.status[b] = HT_STATUS_TIMEOUT;
+    }
+    if (sm.abort && threadIdx.x == 8 * 32) {
+        // Some wait of this CTA ran out, wherever: every copy it asked for must have landed before it exits (this
+        // warp leaves last: it frees the tensor memory below).  Wait, with the full bound, for the latest armed
+        // phase of each ring slot and of the Q buffer.
+        const int ring_i = sm.plan[9], q_fetches = sm.plan[10];
+        for (int e = max(0, ring_i - kStages); e < ring_i; ++e)
+            mbar_wait(&sm.kv_full[e % kStages], (e / kStages) & 1, abort_flag, false);
+        if (q_fetches > 0) mbar_wait(&sm.q_full, (q_fetches - 1) & 1, abort_flag, false);
     }
     if (warp == 8) {
         tc_fence_after();

@@ -545,6 +545,7 @@ __device__ __forceinline__ void plan_range(const int32_t *s_len, const int32_t *
     }
     w[0] = r.per; w[1] = r.t_begin; w[2] = r.t_end;
     w[3] = r.first.b; w[4] = r.first.hk; w[5] = r.first.rt; w[6] = r.first.kt0; w[7] = r.first.len; w[8] = r.first.nkt;
+    w[9] = 0; w[10] = 0;           // (the producer's tally of what it asked for, read by the teardown of a CTA that gave up)
 }
 
 // Validates every sequence and fills len / nkt / pre.  Called by all threads of a block; ends with a barrier.  Every

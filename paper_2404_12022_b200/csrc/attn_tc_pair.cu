@@ -268,13 +268,11 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 __syncwarp();
             }
             release();
-            if (lane == 0 && *abort_flag) {
-                // Every copy this warp issued must have landed before the CTA exits.  (early: the first Q tiles
-                // were fetched by stream 0's issuing thread, whatever else happened)
-                for (int e = max(0, ring_i - kPStages); e < ring_i; ++e)
-                    mbar_wait(&sm.kv_full[e % kPStages], (e / kPStages) & 1, abort_flag, false);
-                const int q_fetches = early && t_end > t_begin && seg_i == 0 ? 1 : seg_i;
-                if (q_fetches > 0) mbar_wait(&sm.q_full, (q_fetches - 1) & 1, abort_flag, false);
+            if (lane == 0) {
+                // how many ring entries and Q fetches were asked for: should the CTA give up, the teardown waits for the
+                // last of them (early: the first Q tiles were fetched by stream 0's issuing thread, whatever else happened)
+                sm.plan[9] = ring_i;
+                sm.plan[10] = early && t_end > t_begin && seg_i == 0 ? 1 : seg_i;
             }
         }
         if (clustered) { cluster_sync_all(); cluster_sync_all(); }
@@ -756,6 +754,14 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (sm.abort && threadIdx.x == 0) {
         for (int b = 0; b < p.B; ++b)
             if (sm.nkt[b] > 0) p.status[b] = HT_STATUS_TIMEOUT;
+    }
+    if (sm.abort && threadIdx.x == 8 * 32) {
+        // Some wait of this CTA ran out, wherever: every copy it asked for must have landed before it exits (this
+        // warp leaves last: it frees the tensor memory below).
+        const int ring_i = sm.plan[9], q_fetches = sm.plan[10];
+        for (int e = max(0, ring_i - kPStages); e < ring_i; ++e)
+            mbar_wait(&sm.kv_full[e % kPStages], (e / kPStages) & 1, abort_flag, false);
+        if (q_fetches > 0) mbar_wait(&sm.q_full, (q_fetches - 1) & 1, abort_flag, false);
     }
     if (warp == 8) {
         tc_fence_after();

@@ -319,8 +319,9 @@ def test_attention_waits_that_run_out_are_reported_and_leave_the_device_usable(h
     desc = hb.make_attn_desc(q, k)
     ws = torch.empty(max(hb.tree_attention_workspace(desc), 16), dtype=torch.uint8, device="cuda")
     out = torch.empty_like(q)
-    for _ in range(3):
-        _, status = hb.tree_attention(q, k, v, kv_len, parent, out=out, workspace=ws, flags=hb.HT_ATTN_TEST_SHORT_WAITS)
+    for i in range(4):                     # the last two with the early start (plan and first fetches ahead of the wait)
+        _, status = hb.tree_attention(q, k, v, kv_len, parent, out=out, workspace=ws,
+                                      flags=hb.HT_ATTN_TEST_SHORT_WAITS | (hb.HT_ATTN_CONTEXT_FINAL if i >= 2 else 0))
         torch.cuda.synchronize()
         assert status.cpu().tolist() == [hb.HT_STATUS_TIMEOUT] * B
     for _ in range(2):
@@ -328,6 +329,15 @@ def test_attention_waits_that_run_out_are_reported_and_leave_the_device_usable(h
         torch.cuda.synchronize()
         assert status.cpu().tolist() == [0] * B
         check_sampled_units(hb, oracle, q, k, v, kv_len.cpu().numpy(), parent, out, 6, torch.bfloat16, seed=3)
+    # a call that gave up may leave arrival counters behind: the workspace is zeroed again before it is called clean
+    _, status = hb.tree_attention(q, k, v, kv_len, parent, out=out, workspace=ws, flags=hb.HT_ATTN_TEST_SHORT_WAITS)
+    ws.zero_()
+    for _ in range(2):
+        _, status = hb.tree_attention(q, k, v, kv_len, parent, out=out, workspace=ws,
+                                      flags=hb.HT_ATTN_WORKSPACE_CLEAN | hb.HT_ATTN_CONTEXT_FINAL)
+        torch.cuda.synchronize()
+        assert status.cpu().tolist() == [0] * B
+        check_sampled_units(hb, oracle, q, k, v, kv_len.cpu().numpy(), parent, out, 6, torch.bfloat16, seed=4)
 
 
 @pytest.mark.parametrize("shape", [(3, 9, 4, 2), (3, 40, 32, 8), (40, 9, 8, 4)], ids=lambda s: "B%dN%dHq%dHkv%d" % s)
