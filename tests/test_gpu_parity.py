@@ -201,12 +201,17 @@ def test_attention_every_work_split(hb, oracle, dtype, case):
     assert bool(((a - b2).abs() <= ulp * a.abs() + 1e-6).all())
 
 
-def test_attention_random_shapes_tensor_core_kernels_against_the_alu_kernel(hb, oracle):
+@pytest.mark.parametrize("promises", [False, True], ids=["plain", "clean_workspace_context_final"])
+def test_attention_random_shapes_tensor_core_kernels_against_the_alu_kernel(hb, oracle, promises):
     """Forty seeded random shapes (batch, rows, head grouping, ragged lengths, tree kinds) through
     whichever tensor-core kernel and work split they select, compared with the fp32-ALU kernel of
     the same library on the GPU (itself checked against the oracle above); the first sequence and
-    KV head of every shape also against the oracle."""
+    KV head of every shape also against the oracle.  Second round: all forty on ONE workspace, zeroed once, with
+    HT_ATTN_WORKSPACE_CLEAN and HT_ATTN_CONTEXT_FINAL, the calls enqueued back to back -- every kind of split must leave
+    its arrival counters at zero for whatever shape comes next, and the early start must change no result."""
     rng = np.random.default_rng(2024)
+    flags = (hb.HT_ATTN_WORKSPACE_CLEAN | hb.HT_ATTN_CONTEXT_FINAL) if promises else 0
+    ws = torch.zeros(64 << 20, dtype=torch.uint8, device="cuda") if promises else None
     for trial in range(40):
         g = int(rng.choice([1, 1, 2, 4, 8, 16]))
         Hkv = int(rng.choice([1, 2, 4, 8, 32]))
@@ -219,9 +224,14 @@ def test_attention_random_shapes_tensor_core_kernels_against_the_alu_kernel(hb, 
         dtype = "bf16" if trial % 2 else "f16"
         tree = str(rng.choice(["random", "chain", "roots"]))
         q, k, v, kv_len, parent = make_attn_case(100 + trial, dtype, B, N, Hkv * g, Hkv, 128, lens, cap, tree)
-        out, status = hb.tree_attention(q, k, v, kv_len, parent)
+        if promises:
+            assert hb.tree_attention_workspace(hb.make_attn_desc(q, k)) <= ws.numel()
+            hb.tree_attention(q, k, v, kv_len, parent, workspace=ws, flags=flags)          # twice in a row, undrained
+        out, status = hb.tree_attention(q, k, v, kv_len, parent, workspace=ws, flags=flags)
         ref, _ = hb.tree_attention(q, k, v, kv_len, parent, flags=hb.HT_ATTN_FORCE_SIMT)
         torch.cuda.synchronize()
+        if promises:
+            assert int(ws[:65536].view(torch.int32).abs().max()) == 0
         what = "trial %d: B=%d N=%d Hq=%d Hkv=%d lens=%s %s %s" % (trial, B, N, Hkv * g, Hkv, lens, tree, dtype)
         assert status.cpu().tolist() == [0] * B, what
         a, r = out.float(), ref.float()
@@ -508,6 +518,58 @@ def test_config_c4_ragged_full_size_sampled(hb, oracle):
     assert_close(f32np(pseudo), oracle.transfer(f32np(inp.h_src), f32np(inp.W)), torch.bfloat16, "c4 transfer")
     _verify_and_compact(hb, oracle, inp)
     assert sorted(set(inp.want_len)) == sorted(set(inp.want_len) & {0, 1, 2, 3, 4})
+
+
+@pytest.mark.parametrize("which", ["c2", "c3_two_layers", "c4"])
+def test_step_from_its_graph_as_the_benchmark_replays_it(hb, oracle, which):
+    """The launch configuration the step benchmark times: the step's C-ABI calls captured in a CUDA graph, the
+    attention calls with HT_ATTN_WORKSPACE_CLEAN and HT_ATTN_CONTEXT_FINAL on the step's own workspace, programmatic
+    serialization between the kernels.  One replay on fresh caches: attention of every materialised layer against the
+    oracle (sampled units, both gates), projection, verification and compaction against the oracle (integers and
+    moved rows bit for bit).  A second replay on restored caches must give the same integers and rows."""
+    from paper_2404_12022_b200.step import VerifyStep
+    w = {"c2": wl.config_c2, "c3_two_layers": wl.config_c3, "c4": wl.config_c4}[which]()
+    inp = wl.make_inputs(w, "cuda", layers=[3, 20]) if which == "c3_two_layers" else wl.make_inputs(w, "cuda")
+    k0, v0 = inp.k_cache.clone(), inp.v_cache.clone()
+    step = VerifyStep(inp)
+    step.run()                                           # (once per device set-up; it also compacts: caches restored below)
+    torch.cuda.synchronize()
+    step.capture()
+    view = torch.int32 if inp.k_cache.dtype == torch.float32 else torch.int16
+    results = []
+    for _ in range(2):
+        inp.k_cache.copy_(k0)
+        inp.v_cache.copy_(v0)
+        step.accept_len.zero_()
+        torch.cuda.synchronize()
+        step.replay()
+        torch.cuda.synchronize()
+        results.append((step.pred.clone(), step.accept_len.clone(), step.accept_path.clone(), step.next_token.clone(),
+                        step.new_kv_len.clone(), inp.k_cache.view(view).clone(), [o.clone() for o in step.outs]))
+    pred, alen, apath, nxt, new_len, k_after, outs = results[0]
+    assert int(step.attn_status.abs().sum()) == 0 and int(step.verify_status.abs().sum()) == 0 and int(step.compact_status.abs().sum()) == 0
+    # attention (the caches' context and tree rows as they were before the compaction)
+    kv = inp.kv_len.cpu().numpy()
+    for i in range(step.layers):
+        check_sampled_units(hb, oracle, inp.q[i], k0[i], v0[i], kv, step.parents[i], outs[i], 6, inp.q[i].dtype, seed=i, gates=True)
+    assert_close(f32np(step.pseudo), oracle.transfer(f32np(inp.h_src), f32np(inp.W)), inp.h_src.dtype, which + " transfer")
+    o_pred, o_alen, o_apath, o_nxt, o_status = oracle.verify_greedy(
+        f32np(inp.logits), inp.tokens.cpu().numpy(), inp.parent.cpu().numpy(),
+        None if inp.root_pred is None else inp.root_pred.cpu().numpy(), w.max_path)
+    assert np.array_equal(pred.cpu().numpy(), o_pred) and np.array_equal(alen.cpu().numpy(), o_alen)
+    assert np.array_equal(apath.cpu().numpy(), o_apath) and np.array_equal(nxt.cpu().numpy(), o_nxt)
+    assert o_alen.tolist() == inp.want_len
+    k_ref, v_ref, len_ref, st_ref = oracle.kv_compact(k0.view(view).cpu().numpy(), v0.view(view).cpu().numpy(), w.N, kv, o_alen, o_apath)
+    assert np.array_equal(new_len.cpu().numpy(), len_ref)
+    ka = k_after.cpu().numpy()
+    for b in range(w.B):
+        assert np.array_equal(ka[:, b, :, :int(len_ref[b])], k_ref[:, b, :, :int(len_ref[b])])
+    # the second replay: same integers, same rows; attention to the last place or the one next to it
+    for x, y in zip(results[0][:6], results[1][:6]):
+        assert torch.equal(x, y)
+    ulp = 2.0 ** -10 if inp.q[0].dtype == torch.float16 else 2.0 ** -7
+    for x, y in zip(results[0][6], results[1][6]):
+        assert bool(((x.float() - y.float()).abs() <= ulp * x.float().abs() + 1e-6).all())
 
 
 def check_sampled_rows(oracle, q, k, v, kv_len, parent, out, n_rows, seed, what):
