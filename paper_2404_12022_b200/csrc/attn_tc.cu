@@ -898,11 +898,11 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     p.grid = sm_count();
     p.cluster_k = 0;
     p.wait_kcycles = (d.flags & HT_ATTN_TEST_SHORT_WAITS) ? tc::kWaitKcyclesTest : tc::kWaitKcycles;
-    // An early start pays at the edges of a launch (about 3 us); CTAs that start when their SM happens to come free
-    // no longer walk a shared head's tiles in step, which costs long launches a little (0.5-1 % from about a hundred
-    // tiles per CTA on): there the kernel waits at its start as usual.
+    // An early start pays at the edges of a launch (about 3 us).  In the tile-pair kernel, CTAs that start when their
+    // SM happens to come free no longer walk a shared head's tiles in step, which costs long launches a little (0.5-1 %
+    // from about a hundred tiles per CTA on): there the kernel waits at its start as usual.
     const long long tiles_bound = (long long)d.B * d.Hkv * units_per_head(d) * ((d.cap + tc::kTile - 1) / tc::kTile);
-    p.early = ((d.flags & HT_ATTN_CONTEXT_FINAL) && tiles_bound <= 96ll * sm_count()) ? 1 : 0;
+    p.early = ((d.flags & HT_ATTN_CONTEXT_FINAL) && (!pair_mode(d) || tiles_bound <= 96ll * sm_count())) ? 1 : 0;
     tc::PagedParams pp;
     pp.block_table = pages ? block_table : nullptr;
     pp.page_size = pages ? pages->page_size : 0;
