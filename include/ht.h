@@ -70,12 +70,14 @@ enum {
  * set on a workspace that is not in that state, results of sequences whose work was split are undefined
  * (nothing faults, nothing waits). */
 #define HT_ATTN_WORKSPACE_CLEAN 2u
-/* The caller vouches that kv_len, parent, the cache rows below kv_len[b] of every sequence (and, for a paged cache,
- * the block-table entries of those rows) were final before the two kernels ahead of this call in `stream` began (in a decoding step they are: the lengths change at the
- * compaction, the rows below them are earlier steps', and the tree is drafted before the first layer).  The
- * tensor-core kernels then make their plan and fetch their first context tiles while the kernel ahead is still
- * finishing, and wait for it only before they read q or rows at or beyond kv_len[b] and before they write
- * anything (about 3 us per call in a chain of calls).  The fp32-ALU kernel ignores the flag. */
+/* The caller vouches that kv_len, parent, the cache rows below kv_len[b] of every sequence (and, for a paged
+ * cache, the block-table entries of those rows) were final before the two kernels ahead of this call in `stream`
+ * began.  (In a decoding step they are: the lengths change at the compaction, the rows below them are earlier
+ * steps', and the tree is drafted before the first layer.)  The tensor-core kernels then make their plan and
+ * fetch their first context tiles while the kernel ahead is still finishing, and wait for it only before they
+ * read q or rows at or beyond kv_len[b] and before they write anything: about 3 us per call in a chain of calls.
+ * A broken promise gives wrong results for the call, never a fault or a wait.  The fp32-ALU kernel ignores the
+ * flag. */
 #define HT_ATTN_CONTEXT_FINAL 4u
 /* Test hook, never to be set in production: the tensor-core kernels' device-side waits give up after about a
  * microsecond instead of a second, so that their give-up path can be exercised: the call returns, the sequences'
