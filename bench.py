@@ -210,7 +210,7 @@ class ClockSampler:
 NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 287.7e6,
                "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh",
                           "paper_2404_12022_b200/csrc/ht_common.cuh"],
-               "sha256": "993c72d0b1ffbf1ec2f4e4feb818e5504ccbbfcfe7aace9b6e2936a554e4a60f"}
+               "sha256": "4857c30647b030ea865f093c4d8acd5878e0d535de7b4174ff6c11bb381c67f2"}
 
 
 def traffic_digest():
