@@ -105,6 +105,14 @@ typedef struct {
     int64_t stride_h;     /* elements; 0 = cap*D */
 } ht_cache_desc;
 
+/* Knobs read once per process from the environment, for cross-checks and bug reports (results never need them):
+ *   HT_LOG=1                        every entry point prints its arguments and the kernel it chose to stderr
+ *   HT_FORCE_PATH=simt|mma|tcgen05  attention on the fp32-ALU kernel (simt); ht_transfer of 16-bit inputs on the
+ *                                   warp-level kernel (mma) or, where the shape allows, on the tcgen05 kernel
+ *   HT_SPLITS=n                     attention with n KV splits where the descriptor leaves the choice
+ *                                   (num_splits == 0): the split-KV ALU kernel, as an explicit num_splits selects it
+ * ht_tree_attention_workspace() and ht_tree_attention_launches() answer for the kernel the knobs select. */
+
 /* Library version (major*10000 + minor*100 + patch). */
 int ht_version(void);
 

@@ -2,6 +2,8 @@
 // meaning of every argument are in include/ht.h.
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include <nvtx3/nvToolsExt.h>
 
@@ -16,6 +18,41 @@ struct Range {
 };
 
 static thread_local char g_err[512] = "no error";
+
+const Knobs &knobs() {
+    static const Knobs k = [] {
+        Knobs x{false, 0, 0};
+        const char *e = getenv("HT_LOG");
+        x.log = e && *e && strcmp(e, "0") != 0;
+        e = getenv("HT_SPLITS");
+        if (e) {
+            const long v = strtol(e, nullptr, 10);
+            x.splits = v > 0 && v <= 1024 ? (int)v : 0;
+        }
+        e = getenv("HT_FORCE_PATH");
+        if (e) x.path = !strcmp(e, "simt") ? 1 : (!strcmp(e, "mma") ? 2 : (!strcmp(e, "tcgen05") ? 3 : 0));
+        return x;
+    }();
+    return k;
+}
+
+void trace(const char *fmt, ...) {
+    if (!knobs().log) return;
+    va_list ap;
+    va_start(ap, fmt);
+    fputs("[ht] ", stderr);
+    vfprintf(stderr, fmt, ap);
+    fputc('\n', stderr);
+    va_end(ap);
+}
+
+// The descriptor as the knobs of the environment leave it.
+static ht_attn_desc with_knobs(const ht_attn_desc &d) {
+    ht_attn_desc x = d;
+    if (knobs().path == 1) x.flags |= HT_ATTN_FORCE_SIMT;
+    if (knobs().splits > 0 && x.num_splits == 0) x.num_splits = knobs().splits;
+    return x;
+}
 
 // Do the int32 arrays [a, a + n) and [b, b + n) share an element?
 static bool overlap_i32(const int32_t *a, const int32_t *b, long long n) {
@@ -72,6 +109,7 @@ const char *ht_last_error_string(void) { return g_err; }
 int ht_transfer(const void *h_src, const void *W, void *out, int B, int k, int d, int dtype,
                 void *stream) {
     Range range("ht_transfer");
+    trace("ht_transfer B=%d k=%d d=%d dtype=%d", B, k, d, dtype);
     if (B < 0 || k < 0 || d < 0) return fail(HT_ERR_INVALID_ARG, "negative size");
     if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     if ((long long)B * k * d == 0) return HT_OK;
@@ -87,13 +125,18 @@ int ht_transfer(const void *h_src, const void *W, void *out, int B, int k, int d
 size_t ht_tree_attention_workspace(const ht_attn_desc *desc) {
     if (check_attn_desc(desc) != HT_OK) return 0;
     if (desc->B == 0 || desc->N == 0) return 0;
+    // (the maximum over the kernels the descriptor may get, whatever the environment's knobs say)
     size_t need = attn_simt_workspace(*desc, nullptr);
+    const ht_attn_desc k = with_knobs(*desc);
+    const size_t need_k = attn_simt_workspace(k, nullptr);
+    need = need_k > need ? need_k : need;
     if (attn_tc_applicable(*desc)) need = attn_tc_workspace(*desc) > need ? attn_tc_workspace(*desc) : need;
     return (need + 255) / 256 * 256;
 }
 
-int ht_tree_attention_launches(const ht_attn_desc *desc) {
-    if (check_attn_desc(desc) != HT_OK) return 0;
+int ht_tree_attention_launches(const ht_attn_desc *user_desc) {
+    if (check_attn_desc(user_desc) != HT_OK) return 0;
+    const ht_attn_desc d = with_knobs(*user_desc), *desc = &d;
     if (desc->B == 0 || desc->N == 0) return 0;
     if (attn_tc_applicable(*desc)) return attn_tc_launches(*desc);
     int splits = 1;
@@ -101,12 +144,16 @@ int ht_tree_attention_launches(const ht_attn_desc *desc) {
     return splits > 1 ? 2 : 1;
 }
 
-int ht_tree_attention(const ht_attn_desc *desc, const void *q, const void *k_cache, const void *v_cache,
+int ht_tree_attention(const ht_attn_desc *user_desc, const void *q, const void *k_cache, const void *v_cache,
                       const int32_t *kv_len, const int32_t *parent, void *out, void *workspace,
                       size_t workspace_bytes, int32_t *status, void *stream) {
     Range range("ht_tree_attention");
-    int rc = check_attn_desc(desc);
+    int rc = check_attn_desc(user_desc);
     if (rc != HT_OK) return rc;
+    const ht_attn_desc d = with_knobs(*user_desc), *desc = &d;
+    trace("ht_tree_attention B=%d N=%d Hq=%d Hkv=%d D=%d cap=%d dtype=%d splits=%d flags=0x%x -> %s", desc->B, desc->N, desc->Hq,
+          desc->Hkv, desc->D, desc->cap, desc->dtype, desc->num_splits, desc->flags,
+          attn_tc_applicable(*desc) ? "tcgen05" : "simt");
     if (desc->B == 0 || desc->N == 0) return HT_OK;
     if (!q || !k_cache || !v_cache || !kv_len || !parent || !out || !status)
         return fail(HT_ERR_INVALID_ARG, "NULL pointer");
@@ -128,6 +175,7 @@ int ht_tree_attention_paged(const ht_attn_desc *desc, const ht_paged_desc *pages
                             const int32_t *parent, void *out, void *workspace, size_t workspace_bytes,
                             int32_t *status, void *stream) {
     Range range("ht_tree_attention_paged");
+    if (desc && pages) trace("ht_tree_attention_paged B=%d N=%d Hq=%d Hkv=%d D=%d page_size=%d max_pages=%d n_pages=%d dtype=%d flags=0x%x", desc->B, desc->N, desc->Hq, desc->Hkv, desc->D, pages->page_size, pages->max_pages, pages->n_pages, desc->dtype, desc->flags);
     if (!desc || !pages) return fail(HT_ERR_INVALID_ARG, "NULL descriptor");
     const int ps = pages->page_size;
     if (ps < 16 || (ps & (ps - 1)) != 0) return fail(HT_ERR_INVALID_ARG, "page_size must be a power of two >= 16");
@@ -164,6 +212,7 @@ int ht_verify_greedy(const void *logits, int dtype, const int32_t *tokens, const
                      int32_t *accept_len, int32_t *accept_path, int32_t *next_token, int32_t *status,
                      void *stream) {
     Range range("ht_verify_greedy");
+    trace("ht_verify_greedy B=%d N=%d T=%d V=%d max_path=%d dtype=%d root_pred=%s", B, N, T, V, max_path, dtype, root_pred ? "given" : "none");
     if (B < 0 || N < 0 || T < 0 || T > N) return fail(HT_ERR_INVALID_ARG, "need 0 <= T <= N and B >= 0");
     if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     if (B == 0) return HT_OK;
@@ -201,6 +250,7 @@ int ht_verify_greedy_compact(const void *logits, int dtype, const int32_t *token
                              int32_t *status, void *k_cache, void *v_cache, const ht_cache_desc *desc,
                              const int32_t *kv_len, int32_t *new_kv_len, int32_t *compact_status, void *stream) {
     Range range("ht_verify_greedy_compact");
+    trace("ht_verify_greedy_compact B=%d N=%d T=%d V=%d max_path=%d dtype=%d layers=%d", B, N, T, V, max_path, dtype, desc ? desc->layers : -1);
     if (B < 0 || N < 0 || T < 0 || T > N) return fail(HT_ERR_INVALID_ARG, "need 0 <= T <= N and B >= 0");
     if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     int rc = check_cache_desc(desc, max_path);
@@ -231,6 +281,7 @@ int ht_kv_compact(void *k_cache, void *v_cache, const ht_cache_desc *desc, const
                   const int32_t *accept_len, const int32_t *accept_path, int max_path,
                   int32_t *new_kv_len, int32_t *status, void *stream) {
     Range range("ht_kv_compact");
+    if (desc) trace("ht_kv_compact layers=%d B=%d Hkv=%d cap=%d D=%d N=%d max_path=%d", desc->layers, desc->B, desc->Hkv, desc->cap, desc->D, desc->N, max_path);
     if (!desc) return fail(HT_ERR_INVALID_ARG, "desc is NULL");
     if (desc->layers <= 0 || desc->B < 0 || desc->Hkv <= 0 || desc->cap <= 0 || desc->D <= 0 || desc->N < 0)
         return fail(HT_ERR_INVALID_ARG, "bad cache sizes");
@@ -260,6 +311,7 @@ int ht_draft_tree(const void *logits, int dtype, int B, int rows, int V, int fir
                   const int32_t *base_pos, int32_t *topk, int32_t *tokens, int32_t *pos, int32_t *status,
                   void *stream) {
     Range range("ht_draft_tree");
+    trace("ht_draft_tree B=%d rows=%d V=%d first_row=%d P=%d K=%d dtype=%d", B, rows, V, first_row, P, K, dtype);
     if (B < 0 || rows < 0 || P < 0 || first_row < 0) return fail(HT_ERR_INVALID_ARG, "negative size");
     if (!valid_dtype(dtype)) return fail(HT_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     if (B == 0) return HT_OK;
@@ -278,6 +330,7 @@ int ht_rope_kv_append(const ht_attn_desc *desc, const void *q_in, const void *k_
                       const int32_t *kv_len, float rope_base, void *q_out, void *k_cache, void *v_cache, int32_t *status,
                       void *stream) {
     Range range("ht_rope_kv_append");
+    if (desc) trace("ht_rope_kv_append B=%d N=%d Hq=%d Hkv=%d D=%d dtype=%d", desc->B, desc->N, desc->Hq, desc->Hkv, desc->D, desc->dtype);
     int rc = check_attn_desc(desc);
     if (rc != HT_OK) return rc;
     if (desc->B == 0 || desc->N == 0) return HT_OK;
@@ -310,6 +363,7 @@ int ht_rope_kv_append_paged(const ht_attn_desc *desc, const ht_paged_desc *pages
                             const void *v_in, const int32_t *pos, const int32_t *kv_len, const int32_t *block_table,
                             float rope_base, void *q_out, void *k_pages, void *v_pages, int32_t *status, void *stream) {
     Range range("ht_rope_kv_append_paged");
+    if (desc && pages) trace("ht_rope_kv_append_paged B=%d N=%d Hq=%d Hkv=%d D=%d page_size=%d dtype=%d", desc->B, desc->N, desc->Hq, desc->Hkv, desc->D, pages->page_size, desc->dtype);
     if (!desc) return fail(HT_ERR_INVALID_ARG, "NULL descriptor");
     int rc = check_paged_desc(pages, desc->Hkv, desc->D);
     if (rc != HT_OK) return rc;
@@ -334,6 +388,7 @@ int ht_kv_compact_paged(void *k_pages, void *v_pages, const ht_cache_desc *desc,
                         const int32_t *block_table, const int32_t *kv_len, const int32_t *accept_len,
                         const int32_t *accept_path, int max_path, int32_t *new_kv_len, int32_t *status, void *stream) {
     Range range("ht_kv_compact_paged");
+    if (desc && pages) trace("ht_kv_compact_paged layers=%d B=%d Hkv=%d D=%d N=%d page_size=%d max_path=%d", desc->layers, desc->B, desc->Hkv, desc->D, desc->N, pages->page_size, max_path);
     if (!desc) return fail(HT_ERR_INVALID_ARG, "desc is NULL");
     if (desc->layers <= 0 || desc->B < 0 || desc->Hkv <= 0 || desc->D <= 0 || desc->N < 0)
         return fail(HT_ERR_INVALID_ARG, "bad cache sizes");

@@ -18,6 +18,20 @@ int check_attn_desc(const ht_attn_desc *d);
 // Checks the launch status of the kernel just enqueued.
 int check_launch(const char *what);
 
+// Knobs read once from the environment, for cross-checks and bug reports (never needed for results):
+//   HT_LOG=1                       every entry point prints its arguments and the kernel it chose to stderr
+//   HT_FORCE_PATH=simt|mma|tcgen05 attention on the fp32-ALU kernel (simt); the projection of 16-bit inputs on the
+//                                  warp-level kernel (mma) or, where its shape allows, on the tcgen05 kernel
+//   HT_SPLITS=n                    attention: n KV splits where the descriptor leaves the choice (num_splits == 0),
+//                                  which selects the split-KV ALU kernel, as an explicit num_splits does
+struct Knobs {
+    bool log;
+    int splits;           // 0: not set
+    int path;             // 0: not set, 1: simt, 2: mma, 3: tcgen05
+};
+const Knobs &knobs();
+void trace(const char *fmt, ...);      // a line on stderr when HT_LOG is set
+
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline int elem_bytes(int dtype) { return dtype == HT_F32 ? 4 : 2; }

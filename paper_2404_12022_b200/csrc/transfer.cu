@@ -280,8 +280,8 @@ static int launch_typed16(const void *h, const void *W, void *out, int B, int k,
 static bool use_tc(int B, int k, int d, int dtype) {
     if (!transfer_tc_applicable(B, k, d, dtype)) return false;
     const char *e = getenv("HT_TRANSFER_KERNEL");
-    if (e && !strcmp(e, "tc")) return true;
-    if (e && !strcmp(e, "mma")) return false;
+    if ((e && !strcmp(e, "tc")) || knobs().path == 3) return true;
+    if ((e && !strcmp(e, "mma")) || knobs().path == 2) return false;
     // 9 to 16 rows take the warp-level kernel's two-tile form (24.5 us on config 3's W against 19.3 with up to 8
     // rows); the tcgen05 kernel is ahead of that once W is large enough to amortise its set-up (21.6 us there).
     return B > 16 || (B > 8 && (long long)k * d * d * 2 >= (64ll << 20));
@@ -289,7 +289,11 @@ static bool use_tc(int B, int k, int d, int dtype) {
 
 int launch_transfer(const void *h, const void *W, void *out, int B, int k, int d, int dtype,
                     cudaStream_t s) {
-    if (use_tc(B, k, d, dtype)) return launch_transfer_tc(h, W, out, B, k, d, dtype, s);
+    if (use_tc(B, k, d, dtype)) {
+        trace("ht_transfer -> tcgen05 kernel");
+        return launch_transfer_tc(h, W, out, B, k, d, dtype, s);
+    }
+    trace("ht_transfer -> %s kernel", dtype == HT_F32 ? "fp32-ALU" : "m16n8k16");
     switch (dtype) {
         case HT_F32: return launch_typed<float>(h, W, out, B, k, d, s);
         case HT_F16: return launch_typed16<__half>(h, W, out, B, k, d, s);

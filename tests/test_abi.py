@@ -105,3 +105,40 @@ def test_binding_refuses_cpu_tensors_and_has_no_fallback():
         hb.transfer(torch.zeros(1, 8), torch.zeros(1, 8, 8))
     src = open(os.path.join(ROOT, "paper_2404_12022_b200", "binding.py")).read()
     assert "oracle" not in src.replace("no fallback", "")
+
+
+def _in_child(env, code):
+    import subprocess
+    import sys
+    e = dict(os.environ)
+    e.update(env)
+    r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, env=e, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr
+    return r.stdout, r.stderr
+
+
+_KNOB_PROBE = """
+import ctypes
+from paper_2404_12022_b200 import binding as hb
+lib = hb.load()
+d = hb.AttnDesc(4, 91, 32, 32, 128, 4224, hb.HT_BF16, 0.0, 0, 0, 0, 0)
+clean = hb.AttnDesc(4, 91, 32, 32, 128, 4224, hb.HT_BF16, 0.0, 0, 0, 0, hb.HT_ATTN_WORKSPACE_CLEAN)
+print(lib.ht_tree_attention_launches(ctypes.byref(d)), lib.ht_tree_attention_launches(ctypes.byref(clean)),
+      lib.ht_tree_attention_workspace(ctypes.byref(d)))
+print(lib.ht_transfer(None, None, None, 0, 3, 8, hb.HT_F32, None))
+"""
+
+
+def test_knobs_of_the_environment(lib):
+    """HT_FORCE_PATH, HT_SPLITS and HT_LOG are read by the library itself (once per process, so each setting gets a
+    child process); the calls made here are answered on the host."""
+    plain, err = _in_child({}, _KNOB_PROBE)
+    assert plain.split()[:2] == ["2", "1"] and err.strip() == ""         # tensor-core kernel: with / without the counter kernel
+    ws_plain = int(plain.split()[2])
+    forced, _ = _in_child({"HT_FORCE_PATH": "simt"}, _KNOB_PROBE)
+    assert forced.split()[0] == forced.split()[1] and forced.split()[0] in ("1", "2")   # the ALU kernel, whatever the flags
+    assert int(forced.split()[2]) >= ws_plain                             # the workspace is the maximum over the kernels
+    split, _ = _in_child({"HT_SPLITS": "4"}, _KNOB_PROBE)
+    assert split.split()[:2] == ["2", "2"]                                 # split-KV ALU kernel + its merge
+    out, err = _in_child({"HT_LOG": "1"}, _KNOB_PROBE)
+    assert out.split()[3] == "0" and "[ht] ht_transfer B=0 k=3 d=8" in err
