@@ -769,10 +769,17 @@ static bool pair_mode(const ht_attn_desc &d) { return row_tiles(d) >= 2; }
 static int units_per_head(const ht_attn_desc &d) { return pair_mode(d) ? (row_tiles(d) + 1) / 2 : 1; }
 
 // Cluster size when the (sequence, KV head[, tile pair]) units are so few that a CTA per unit would
-// leave most SMs idle: the largest of 8, 4, 2 whose clusters fit the GPU at once.
+// leave most SMs idle: the largest of 16 (see below), 8, 4, 2 whose clusters fit the GPU at once.
+static int clusters16_fit();
+
 static int cluster_size(const ht_attn_desc &d) {
     const long long units = (long long)d.B * d.Hkv * units_per_head(d);
     const int sms = sm_count();
+    // A handful of units with long caches: clusters of 16, beyond the portable size, where the device can hold one per
+    // unit at once (a B200 holds seven: one sequence on four KV heads gets them, one on eight does not).  Measured
+    // against clusters of eight: 4 x 32768 keys x 152 rows 77.2 -> 49.5 us, x 8000 keys 25.8 -> 20.5 us, x 4096 keys
+    // 19.1 -> 17.4 us (tile pairs); one tile of 91 rows: 47.9 -> 32.9 us at 32768 keys, level at 8000, behind at 4096.
+    if (units * 16 <= sms && d.cap > (pair_mode(d) ? 4096 : 8192) && clusters16_fit() >= units) return 16;
     for (int k = 8; k >= 2; k /= 2)
         if (units * k <= sms) {
             // Clusters leave SMs idle when units * k falls well short of the GPU; that only pays while the
@@ -828,9 +835,46 @@ static cudaError_t ensure_smem_attr(size_t smem) {
     for (int i = 0; i < 8; ++i) {
         e = cudaFuncSetAttribute(attn_tc_fn(i & 1, (i >> 1) & 1, i >> 2), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
+        if (i >> 2) {                        // the cluster form may be launched in clusters of 16
+            e = cudaFuncSetAttribute(attn_tc_fn(i & 1, (i >> 1) & 1, 1), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            if (e != cudaSuccess) return e;
+        }
     }
     if (dev >= 0 && dev < 64) done[dev] = true;
     return cudaSuccess;
+}
+
+// Clusters of 16 CTAs of these kernels (one CTA per SM: all of its shared and tensor memory) that the device holds at
+// once; 0 where it cannot be asked (no device) or cannot hold any.  The tile-pair kernel has the same footprint.
+static int clusters16_fit() {
+    static int cached[64];                   // 0: not asked yet, -1: none
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return 0;
+    }
+    if (cached[dev] == 0) {
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(16 * 8);
+        cfg.blockDim = dim3(tc::kThreads);
+        cfg.dynamicSmemBytes = sizeof(tc::Smem) + 1024;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 16;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (ensure_smem_attr(sizeof(tc::Smem) + 1024) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&n, attn_tc_fn(true, false, true), &cfg) != cudaSuccess) {
+            cudaGetLastError();
+            n = 0;
+        }
+        trace("clusters of 16 CTAs the device holds at once: %d", n);
+        cached[dev] = n > 0 ? n : -1;
+    }
+    return cached[dev] > 0 ? cached[dev] : 0;
 }
 
 static int make_map(CUtensorMap *map, const void *base, int dtype, const cuuint64_t dims[4], const cuuint64_t strides_b[3],
@@ -937,10 +981,13 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
         p.cluster_k = k;
         p.grid = (int)units * k;
     }
+    trace("ht_tree_attention -> %s kernel, %s, %d CTAs%s%s", pair_mode(d) ? "tile-pair" : "one-tile",
+          k > 1 ? (k == 16 ? "clusters of 16" : (k == 8 ? "clusters of 8" : (k == 4 ? "clusters of 4" : "clusters of 2"))) : "persistent",
+          p.grid, p.early ? ", early start" : "", needs_prepare(d, pages != nullptr) ? ", counters cleared by a kernel" : "");
     if (pair_mode(d)) return launch_attn_tc_pair_kernel(tm_q, tm_k, tm_v, p, pp, d.dtype == HT_BF16, pages != nullptr, s);
     e = ensure_smem_attr(sizeof(tc::Smem) + 1024);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-    // Few (sequence, KV head) units: one cluster of 8, 4 or 2 CTAs per unit, parts reduced through
+    // Few (sequence, KV head) units: one cluster of 16, 8, 4 or 2 CTAs per unit, parts reduced through
     // distributed shared memory; otherwise one persistent CTA per SM.  Either way the launch is serialized
     // programmatically behind the kernel before it.
     cudaLaunchConfig_t cfg = {};

@@ -790,7 +790,7 @@ static_assert(kXchgBytes <= (1 + kStages) * kEntryBytes, "the exchange area is t
 // peer's shared memory any more, so a CTA may leave as soon as it has merged what it holds.
 //
 // The merge of one row's received parts.  It runs once per CTA, so what counts is the length of its chain of
-// dependent instructions, not their number: all loads are independent of one another (the k <= 8 parts unrolled
+// dependent instructions, not their number: all loads are independent of one another (the k <= 16 parts unrolled
 // with predicates), the parts' weights are formed once, and the row's features leave as 16-byte stores.
 __device__ __forceinline__ float lds_f32(uint32_t a) {
     float v;
@@ -803,42 +803,47 @@ __device__ __forceinline__ float4 lds_f32x4(uint32_t a) {
     return v;
 }
 // Weights of the k parts of `row`, 1 / (sum of the weighted row sums) folded in.  recv_ml: [sender][m | l][row] floats.
-__device__ __forceinline__ void merge_weights(uint32_t recv_ml, int k, int row, float (&f)[8]) {
-    float m[8], M = -INFINITY;
+constexpr int kMaxCluster = 16;        // CTAs per cluster at most (16 is beyond the portable size: asked for per kernel)
+__device__ __forceinline__ void merge_weights(uint32_t recv_ml, int k, int row, float (&f)[kMaxCluster]) {
+    float m[kMaxCluster], M = -INFINITY;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
+    for (int c = 0; c < kMaxCluster; ++c) {
         m[c] = c < k ? lds_f32(recv_ml + (uint32_t)(c * 2 * kRows + row) * 4u) : -INFINITY;
         f[c] = c < k ? lds_f32(recv_ml + (uint32_t)(c * 2 * kRows + kRows + row) * 4u) : 0.f;     // the part's row sum, for now
     }
 #pragma unroll
-    for (int c = 0; c < 8; ++c) M = fmaxf(M, m[c]);
+    for (int c = 0; c < kMaxCluster; ++c) M = fmaxf(M, m[c]);
     float l = 0.f;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
+    for (int c = 0; c < kMaxCluster; ++c) {
         const float w = m[c] == -INFINITY ? 0.f : ex2(m[c] - M);
         l = fmaf(w, f[c], l);
         f[c] = w;
     }
     const float inv = 1.f / l;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) f[c] *= inv;
+    for (int c = 0; c < kMaxCluster; ++c) f[c] *= inv;
 }
 // X groups of 4 features from group x0 on: recv holds [sender][group in slice (cgps of them)][row] float4; the
-// 8 X bytes of the result go to dst (16-byte aligned, X even).
+// 8 X bytes of the result go to dst (16-byte aligned for even X, 8-byte aligned for X = 1).
 template <bool kBf16, int X>
-__device__ __forceinline__ void merge_groups(uint32_t recv, int k, int cgps, int row, int x0, const float (&f)[8], unsigned char *dst) {
+__device__ __forceinline__ void merge_groups(uint32_t recv, int k, int cgps, int row, int x0, const float (&f)[kMaxCluster], unsigned char *dst) {
     uint32_t w[2 * X];
 #pragma unroll
     for (int x = 0; x < X; ++x) {
         float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
+        for (int c = 0; c < kMaxCluster; ++c)
             if (c < k && f[c] != 0.f) {            // a part that saw nothing sent no features: what lies there is not data
                 const float4 v = lds_f32x4(recv + (uint32_t)((c * cgps + x0 + x) * kRows + row) * 16u);
                 o.x = fmaf(f[c], v.x, o.x); o.y = fmaf(f[c], v.y, o.y); o.z = fmaf(f[c], v.z, o.z); o.w = fmaf(f[c], v.w, o.w);
             }
         w[2 * x] = pack2<kBf16>(o.x, o.y);
         w[2 * x + 1] = pack2<kBf16>(o.z, o.w);
+    }
+    if (X == 1) {
+        *reinterpret_cast<uint2 *>(dst) = make_uint2(w[0], w[1]);
+        return;
     }
 #pragma unroll
     for (int i = 0; i < X / 2; ++i)
@@ -851,13 +856,13 @@ template <bool kBf16>
 __device__ __noinline__ void cluster_merge(const Params &p, unsigned char *area, int rank, int b, int hk, int row_tile,
                                            bool valid, int tid256, volatile int *abort_flag) {
     const int k = p.cluster_k;
-    const int cgps = 32 / k;                      // groups of 4 features per slice: 16, 8 or 4
+    const int cgps = 32 / k;                      // groups of 4 features per slice: 16, 8, 4 or 2
     cluster_sync_all();
     const int row = tid256 & 127, half = tid256 >> 7;
     const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
     if (!valid || node >= p.N || *abort_flag) return;
     const uint32_t recv = smem_u32(area) + kXchgRecvOffset, recv_ml = recv + kRows * kD * 4;
-    float f[8];
+    float f[kMaxCluster];
     merge_weights(recv_ml, k, row, f);
     const int head = hk * p.g + row % p.g;
     const int x0 = half * (cgps / 2);
@@ -865,7 +870,8 @@ __device__ __noinline__ void cluster_merge(const Params &p, unsigned char *area,
                          ((((size_t)b * p.N + node) * p.Hq + head) * kD + (rank * cgps + x0) * 4) * 2;
     if (k == 2) merge_groups<kBf16, 8>(recv, k, cgps, row, x0, f, dst);
     else if (k == 4) merge_groups<kBf16, 4>(recv, k, cgps, row, x0, f, dst);
-    else merge_groups<kBf16, 2>(recv, k, cgps, row, x0, f, dst);
+    else if (k == 8) merge_groups<kBf16, 2>(recv, k, cgps, row, x0, f, dst);
+    else merge_groups<kBf16, 1>(recv, k, cgps, row, x0, f, dst);
 }
 
 }  // namespace tc

@@ -60,7 +60,7 @@ __device__ __forceinline__ void ex2_poly_x2(unsigned long long x2, float &p0, fl
 // followed by [sender][m | l][row]; behind the second barrier of the cluster the same thread merges the k slices of
 // its row and writes the CTA's features of the result.
 constexpr int kPXchgMl = kRows * kD * 4;                         // bytes from a stream's area to its m, l
-constexpr int kPXchgStream = kPXchgMl + 8 * 2 * kRows * 4;       // up to 8 senders
+constexpr int kPXchgStream = kPXchgMl + kMaxCluster * 2 * kRows * 4;   // up to 16 senders
 static_assert(2 * kPXchgStream <= (2 + kPStages) * kEntryBytes, "the exchange area is the Q buffers and the ring");
 
 // A stream's received parts lie at `area` as [sender][group in slice][row] float4, followed (at kPXchgMl) by
@@ -73,7 +73,7 @@ __device__ __noinline__ void cluster_merge_pair(const Params &p, const unsigned 
     const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
     if (!valid || row_tile >= p.n_row_tiles || node >= p.N || *abort_flag) return;
     const uint32_t recv = smem_u32(area), recv_ml = recv + kPXchgMl;
-    float f[8];
+    float f[kMaxCluster];
     merge_weights(recv_ml, k, row, f);
     const int head = hk * p.g + row % p.g;
     unsigned char *dst = static_cast<unsigned char *>(p.out) + ((((size_t)b * p.N + node) * p.Hq + head) * kD + rank * cgps * 4) * 2;
@@ -82,8 +82,10 @@ __device__ __noinline__ void cluster_merge_pair(const Params &p, const unsigned 
         merge_groups<kBf16, 8>(recv, k, cgps, row, 8, f, dst + 64);
     } else if (k == 4) {
         merge_groups<kBf16, 8>(recv, k, cgps, row, 0, f, dst);
-    } else {
+    } else if (k == 8) {
         merge_groups<kBf16, 4>(recv, k, cgps, row, 0, f, dst);
+    } else {
+        merge_groups<kBf16, 2>(recv, k, cgps, row, 0, f, dst);
     }
 }
 
@@ -785,8 +787,10 @@ int launch_attn_tc_pair_kernel(const CUtensorMap &tm_q, const CUtensorMap &tm_k,
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
     if (!(dev >= 0 && dev < 64 && done[dev])) {
-        for (int i = 0; i < 4 && e == cudaSuccess; ++i)
+        for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
             e = cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(fns[i], cudaFuncAttributeNonPortableClusterSizeAllowed, 1);   // clusters of 16
+        }
         if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         if (dev >= 0 && dev < 64) done[dev] = true;
     }

@@ -262,6 +262,27 @@ def test_attention_at_the_largest_sizes_the_tensor_core_kernels_take(hb, oracle,
     check_sampled_units(hb, oracle, q, k, v, kv_len.cpu().numpy(), parent, out, 2, torch.bfloat16, seed=N)
 
 
+@pytest.mark.parametrize("shape", [(1, 19, 8, 8, 12000), (1, 91, 4, 4, 30001), (1, 19, 64, 8, 9000), (1, 67, 64, 8, 20000), (2, 33, 4, 4, 8300)],
+                         ids=lambda s: "B%dN%dHq%dHkv%dL%d" % s)
+@pytest.mark.parametrize("final", [False, True], ids=["plain", "context_final"])
+def test_attention_few_units_with_long_caches(hb, oracle, shape, final):
+    """A handful of (sequence, KV head) units with caches beyond 8192 rows: clusters of sixteen CTAs per unit where the
+    device holds them (one-tile and tile-pair kernel; shares with and without tiles, the tree rows in one tile or
+    two), against the oracle on sampled units and against the ALU kernel everywhere."""
+    B, N, Hq, Hkv, L = shape
+    lens = [L - 777 * b for b in range(B)]
+    q, k, v, kv_len, parent = make_attn_case(57, "bf16", B, N, Hq, Hkv, 128, lens, L + N + 3)
+    out, status = hb.tree_attention(q, k, v, kv_len, parent, flags=hb.HT_ATTN_CONTEXT_FINAL if final else 0)
+    ref, _ = hb.tree_attention(q, k, v, kv_len, parent, flags=hb.HT_ATTN_FORCE_SIMT)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0] * B
+    a, r = out.float(), ref.float()
+    eps = 2.0 ** -7
+    assert torch.isfinite(a).all()
+    assert bool(((a - r).abs() <= 2e-3 + 2 * eps * r.abs() + 3 * eps).all()), "max diff %.3e" % float((a - r).abs().max())
+    check_sampled_units(hb, oracle, q, k, v, kv_len.cpu().numpy(), parent, out, 2, torch.bfloat16, seed=N, gates=True)
+
+
 @pytest.mark.parametrize("shape", [(4, 91, 32, 32, 1500), (1, 91, 32, 32, 1024), (2, 40, 32, 4, 700), (3, 19, 16, 16, 3000)],
                          ids=lambda s: "B%dN%dHq%dHkv%dL%d" % s)
 @pytest.mark.parametrize("final", [False, True], ids=["plain", "context_final"])
