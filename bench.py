@@ -210,7 +210,7 @@ class ClockSampler:
 NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 287.7e6,
                "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh",
                           "paper_2404_12022_b200/csrc/ht_common.cuh"],
-               "sha256": "4857c30647b030ea865f093c4d8acd5878e0d535de7b4174ff6c11bb381c67f2"}
+               "sha256": "5d0ba9b2a6b316fa6a222158943b17410744748bf9b2d7a2236da0bc133c52ac"}
 
 
 def traffic_digest():
