@@ -162,13 +162,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     uint32_t c_rank = 0;
     RangeAsk ask;
     ask.n_pos = p.grid; ask.my_pos = (int)blockIdx.x;
-    ask.cluster_k = 0; ask.cl_rank = 0; ask.cl_b = 0; ask.cl_unit = 0;
+    ask.cluster_k = 0; ask.cl_rank = 0; ask.cl_units_per_seq = 1;
     if (clustered) {
+        // (two clusters on a unit, p.cluster_split == 2: their CTAs share the unit's tiles like one cluster of twice the size)
         c_rank = cluster_ctarank();
-        const int unit = (int)blockIdx.x / p.cluster_k;
-        ask.cluster_k = p.cluster_k; ask.cl_rank = (int)c_rank;
-        ask.cl_b = unit / p.Hkv;
-        ask.cl_unit = unit - ask.cl_b * p.Hkv;
+        ask.cluster_k = p.cluster_k * p.cluster_split;
+        ask.cl_rank = (int)blockIdx.x % ask.cluster_k;
+        ask.cl_units_per_seq = p.Hkv;
     }
     tc_fence_before();                              // (the tensor memory's base address crosses the plan's last barrier)
     plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0 && !early, kPaged, 1, ask, sm.plan);   // one unit per KV head in this kernel
@@ -664,7 +664,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 for (int c = 0; c < p.cluster_k; ++c)
                     st_peer_f1(map_to_peer(xrecv + (uint32_t)(kRows * kD + ((int)c_rank * 2 + s) * kRows + row) * 4u, (uint32_t)c), s == 0 ? -INFINITY : 0.f);
             }
-            const int unit = (int)blockIdx.x / p.cluster_k, b = unit / p.Hkv;
+            const int unit = (int)blockIdx.x / (p.cluster_k * p.cluster_split), b = unit / p.Hkv;
             cluster_merge<kBf16>(p, &sm.q[0], (int)c_rank, b, unit - b * p.Hkv, 0, sm.nkt[b] > 0, tid256, abort_flag);
         }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
@@ -771,6 +771,7 @@ static int units_per_head(const ht_attn_desc &d) { return pair_mode(d) ? (row_ti
 // Cluster size when the (sequence, KV head[, tile pair]) units are so few that a CTA per unit would
 // leave most SMs idle: the largest of 16 (see below), 8, 4, 2 whose clusters fit the GPU at once.
 static int clusters16_fit();
+static int clusters_fit(int k);
 
 static int cluster_size(const ht_attn_desc &d) {
     const long long units = (long long)d.B * d.Hkv * units_per_head(d);
@@ -779,7 +780,12 @@ static int cluster_size(const ht_attn_desc &d) {
     // unit at once (a B200 holds seven: one sequence on four KV heads gets them, one on eight does not).  Measured
     // against clusters of eight: 4 x 32768 keys x 152 rows 77.2 -> 49.5 us, x 8000 keys 25.8 -> 20.5 us, x 4096 keys
     // 19.1 -> 17.4 us (tile pairs); one tile of 91 rows: 47.9 -> 32.9 us at 32768 keys, level at 8000, behind at 4096.
-    if (units * 16 <= sms && d.cap > (pair_mode(d) ? 4096 : 8192) && clusters16_fit() >= units) return 16;
+    // Where it does not, two clusters of eight or four of four share a unit (cluster_split below), if the device holds those.
+    if (units * 16 <= sms && d.cap > (pair_mode(d) ? 4096 : 8192)) {
+        if (clusters_fit(16) >= units) return 16;
+        if (clusters_fit(8) >= 2 * units) return 8;
+        if (clusters_fit(4) >= 4 * units) return 4;
+    }
     for (int k = 8; k >= 2; k /= 2)
         if (units * k <= sms) {
             // Clusters leave SMs idle when units * k falls well short of the GPU; that only pays while the
@@ -799,10 +805,23 @@ static size_t ticket_bytes(const ht_attn_desc &d) {
     const size_t need = (units * sizeof(unsigned int) + 255) / 256 * 256;
     return need > kTicketArea ? need : kTicketArea;
 }
+// Several clusters on a unit, where clusters of sixteen would be taken but the device does not hold one per unit (a
+// B200 holds 7 of sixteen, 15 of eight, 33 of four: one sequence on eight KV heads gets four clusters of four per
+// unit): each reduces its share of the keys through distributed shared memory, and the results meet in the workspace
+// (an arrival counter per set of CTAs of one rank; the last finishes).
+static int cluster_split(const ht_attn_desc &d) {
+    const long long units = (long long)d.B * d.Hkv * units_per_head(d);
+    if (!(units * 16 <= sm_count() && d.cap > (pair_mode(d) ? 4096 : 8192))) return 1;
+    if (clusters_fit(16) >= units) return 1;
+    if (clusters_fit(8) >= 2 * units) return 2;
+    if (clusters_fit(4) >= 4 * units) return 4;
+    return 1;
+}
+
 // Is the kernel that zeroes the counters (and, for a paged cache, the status words) part of the call?
 static bool needs_prepare(const ht_attn_desc &d, bool paged) {
     if (paged) return true;                                   // the paged kernels report bad pages from any CTA
-    if (cluster_size(d) > 1) return false;                    // clusters use no counters
+    if (cluster_size(d) > 1 && cluster_split(d) == 1) return false;   // one cluster per unit: no counters
     const size_t units = (size_t)d.B * d.Hkv * units_per_head(d);
     return !(d.flags & HT_ATTN_WORKSPACE_CLEAN) || units * sizeof(unsigned int) > kTicketArea;
 }
@@ -846,22 +865,23 @@ static cudaError_t ensure_smem_attr(size_t smem) {
 
 // Clusters of 16 CTAs of these kernels (one CTA per SM: all of its shared and tensor memory) that the device holds at
 // once; 0 where it cannot be asked (no device) or cannot hold any.  The tile-pair kernel has the same footprint.
-static int clusters16_fit() {
-    static int cached[64];                   // 0: not asked yet, -1: none
+static int clusters_fit(int k) {
+    static int cached[64][3];                // per device and size 4 / 8 / 16; 0: not asked yet, -1: none
+    const int slot = k == 16 ? 2 : (k == 8 ? 1 : 0);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
         cudaGetLastError();
         return 0;
     }
-    if (cached[dev] == 0) {
+    if (cached[dev][slot] == 0) {
         int n = 0;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(16 * 8);
+        cfg.gridDim = dim3((unsigned)(k * 64));
         cfg.blockDim = dim3(tc::kThreads);
         cfg.dynamicSmemBytes = sizeof(tc::Smem) + 1024;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 16;
+        attr[0].val.clusterDim.x = (unsigned)k;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
@@ -871,11 +891,12 @@ static int clusters16_fit() {
             cudaGetLastError();
             n = 0;
         }
-        trace("clusters of 16 CTAs the device holds at once: %d", n);
-        cached[dev] = n > 0 ? n : -1;
+        trace("clusters of %d CTAs the device holds at once: %d", k, n);
+        cached[dev][slot] = n > 0 ? n : -1;
     }
-    return cached[dev] > 0 ? cached[dev] : 0;
+    return cached[dev][slot] > 0 ? cached[dev][slot] : 0;
 }
+static int clusters16_fit() { return clusters_fit(16); }
 
 static int make_map(CUtensorMap *map, const void *base, int dtype, const cuuint64_t dims[4], const cuuint64_t strides_b[3],
                     const cuuint32_t box[4]) {
@@ -941,6 +962,7 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     p.is_bf16 = d.dtype == HT_BF16;
     p.grid = sm_count();
     p.cluster_k = 0;
+    p.cluster_split = 1;
     p.wait_kcycles = (d.flags & HT_ATTN_TEST_SHORT_WAITS) ? tc::kWaitKcyclesTest : tc::kWaitKcycles;
     // An early start pays at the edges of a launch (about 3 us).  In the tile-pair kernel, CTAs that start when their
     // SM happens to come free no longer walk a shared head's tiles in step, which costs long launches a little (0.5-1 %
@@ -957,10 +979,10 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     const size_t smem = offsetof(tc::Smem, anc) + (size_t)((d.N + 31) / 32) * tc::kRows * sizeof(uint32_t) + 1024;
     const long long units = (long long)d.B * d.Hkv * p.n_rt;
     if (units > 0x7fffffffLL) return fail(HT_ERR_UNSUPPORTED, "too many (sequence, head, row tile) units");
-    const int k = cluster_size(d);
+    const int k = cluster_size(d), split = k > 1 ? cluster_split(d) : 1;
     cudaError_t e = cudaSuccess;
     if (needs_prepare(d, pages != nullptr)) {
-        const int n_t = k <= 1 ? (int)units : 0, n_s = pages ? d.B : 0;
+        const int n_t = k <= 1 ? (int)units : (split > 1 ? (int)units * k : 0), n_s = pages ? d.B : 0;
         const int n = n_t > n_s ? n_t : n_s;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)((n + 255) / 256 < 64 ? (n + 255) / 256 : 64));
@@ -979,10 +1001,12 @@ int launch_attn_tc(const ht_attn_desc &d, const void *q, const void *kc, const v
     }
     if (k > 1) {
         p.cluster_k = k;
-        p.grid = (int)units * k;
+        p.cluster_split = split;
+        p.grid = (int)units * k * split;
     }
+    if (knobs().log) trace("clusters the device holds: %d of 4, %d of 8, %d of 16", clusters_fit(4), clusters_fit(8), clusters_fit(16));
     trace("ht_tree_attention -> %s kernel, %s, %d CTAs%s%s", pair_mode(d) ? "tile-pair" : "one-tile",
-          k > 1 ? (k == 16 ? "clusters of 16" : (k == 8 ? "clusters of 8" : (k == 4 ? "clusters of 4" : "clusters of 2"))) : "persistent",
+          k > 1 ? (k == 16 ? "clusters of 16" : (k == 8 ? (split == 2 ? "two clusters of 8 per unit" : "clusters of 8") : (k == 4 ? (split == 4 ? "four clusters of 4 per unit" : "clusters of 4") : "clusters of 2"))) : "persistent",
           p.grid, p.early ? ", early start" : "", needs_prepare(d, pages != nullptr) ? ", counters cleared by a kernel" : "");
     if (pair_mode(d)) return launch_attn_tc_pair_kernel(tm_q, tm_k, tm_v, p, pp, d.dtype == HT_BF16, pages != nullptr, s);
     e = ensure_smem_attr(sizeof(tc::Smem) + 1024);

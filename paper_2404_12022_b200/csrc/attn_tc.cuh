@@ -37,6 +37,7 @@ struct Params {
     int is_bf16;
     int grid;
     int cluster_k;         // > 1: launched as clusters of this many CTAs, one cluster per (sequence, KV head)
+    int cluster_split;     // clusters per unit: 1, or 2 (each reduces its half of the keys; the two results meet in the workspace)
     int wait_kcycles;      // how long a wait on an mbarrier may last, in units of 1024 clock cycles
     int early;             // HT_ATTN_CONTEXT_FINAL: lengths, trees and context rows may be read while the kernel ahead still runs
 };
@@ -497,11 +498,12 @@ __device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nk
 }
 
 // Which share of the tile list a CTA takes.  Persistent form: place `my_pos` of `n_pos` ranges of `per` tiles
-// (choose_per).  Cluster form (cluster_k > 1): the CTA's cost-equal share of the one unit its cluster works on,
-// sequence cl_b, unit cl_unit of that sequence's units.
+// (choose_per).  Cluster form (cluster_k > 1): the CTA's cost-equal share of the one unit its cluster (or set of
+// clusters) works on.
 struct RangeAsk {
     int n_pos, my_pos;
-    int cluster_k, cl_rank, cl_b, cl_unit;
+    int cluster_k, cl_rank;                     // cluster form: CTAs that share a unit (side by side in the grid), this CTA's place among them
+    int cl_units_per_seq;                       // ... and units per sequence: Hkv, or Hkv x tile pairs per head
 };
 struct Range {
     int per, t_begin, t_end;
@@ -524,15 +526,19 @@ __device__ __forceinline__ void plan_range(const int32_t *s_len, const int32_t *
     r.first.b = 0; r.first.hk = 0; r.first.rt = 0; r.first.kt0 = 0; r.first.len = 0; r.first.nkt = 0;
     if (ask.cluster_k > 1) {
         r.per = 0;
-        const int nk = s_nkt[ask.cl_b];
+        // ask.cluster_k CTAs share the unit (one cluster, or several clusters side by side in the grid); ask.cl_rank
+        // is this CTA's place among them
+        const int unit = (int)blockIdx.x / ask.cluster_k;
+        const int cl_b = unit / ask.cl_units_per_seq, cl_unit = unit - cl_b * ask.cl_units_per_seq;
+        const int nk = s_nkt[cl_b];
         int lo, hi;
-        cluster_share(nk, s_len[ask.cl_b], ask.cluster_k, ask.cl_rank, lo, hi);
-        const int t0 = s_pre[ask.cl_b] + ask.cl_unit * nk;
+        cluster_share(nk, s_len[cl_b], ask.cluster_k, ask.cl_rank, lo, hi);
+        const int t0 = s_pre[cl_b] + cl_unit * nk;
         r.t_begin = t0 + lo;
         r.t_end = t0 + hi;
-        r.first.b = ask.cl_b;
-        r.first.hk = units_per_head == 1 ? ask.cl_unit : fast_div(ask.cl_unit, units_per_head);
-        r.first.rt = ask.cl_unit - r.first.hk * units_per_head;
+        r.first.b = cl_b;
+        r.first.hk = units_per_head == 1 ? cl_unit : fast_div(cl_unit, units_per_head);
+        r.first.rt = cl_unit - r.first.hk * units_per_head;
         r.first.kt0 = lo; r.first.len = hi - lo; r.first.nkt = nk;
     } else {
         r.per = choose_per(total, ask.n_pos, s_nkt, B, units_per_head);
@@ -804,7 +810,9 @@ __device__ __forceinline__ float4 lds_f32x4(uint32_t a) {
 }
 // Weights of the k parts of `row`, 1 / (sum of the weighted row sums) folded in.  recv_ml: [sender][m | l][row] floats.
 constexpr int kMaxCluster = 16;        // CTAs per cluster at most (16 is beyond the portable size: asked for per kernel)
-__device__ __forceinline__ void merge_weights(uint32_t recv_ml, int k, int row, float (&f)[kMaxCluster]) {
+// raw != nullptr: the weights stay relative to the maximum, which is returned with the weighted sum (raw[0] = M,
+// raw[1] = l): the cluster's result is then a part itself (two clusters share the unit).
+__device__ __forceinline__ void merge_weights(uint32_t recv_ml, int k, int row, float (&f)[kMaxCluster], float *raw = nullptr) {
     float m[kMaxCluster], M = -INFINITY;
 #pragma unroll
     for (int c = 0; c < kMaxCluster; ++c) {
@@ -820,26 +828,38 @@ __device__ __forceinline__ void merge_weights(uint32_t recv_ml, int k, int row, 
         l = fmaf(w, f[c], l);
         f[c] = w;
     }
+    if (raw) {
+        raw[0] = M;
+        raw[1] = l;
+        return;
+    }
     const float inv = 1.f / l;
 #pragma unroll
     for (int c = 0; c < kMaxCluster; ++c) f[c] *= inv;
 }
-// X groups of 4 features from group x0 on: recv holds [sender][group in slice (cgps of them)][row] float4; the
-// 8 X bytes of the result go to dst (16-byte aligned for even X, 8-byte aligned for X = 1).
-template <bool kBf16, int X>
-__device__ __forceinline__ void merge_groups(uint32_t recv, int k, int cgps, int row, int x0, const float (&f)[kMaxCluster], unsigned char *dst) {
-    uint32_t w[2 * X];
+// X groups of 4 features from group x0 on, summed over the parts with their weights: recv holds
+// [sender][group in slice (cgps of them)][row] float4.
+template <int X>
+__device__ __forceinline__ void merge_sums(uint32_t recv, int k, int cgps, int row, int x0, const float (&f)[kMaxCluster], float4 (&o)[X]) {
 #pragma unroll
     for (int x = 0; x < X; ++x) {
-        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        o[x] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int c = 0; c < kMaxCluster; ++c)
             if (c < k && f[c] != 0.f) {            // a part that saw nothing sent no features: what lies there is not data
                 const float4 v = lds_f32x4(recv + (uint32_t)((c * cgps + x0 + x) * kRows + row) * 16u);
-                o.x = fmaf(f[c], v.x, o.x); o.y = fmaf(f[c], v.y, o.y); o.z = fmaf(f[c], v.z, o.z); o.w = fmaf(f[c], v.w, o.w);
+                o[x].x = fmaf(f[c], v.x, o[x].x); o[x].y = fmaf(f[c], v.y, o[x].y); o[x].z = fmaf(f[c], v.z, o[x].z); o[x].w = fmaf(f[c], v.w, o[x].w);
             }
-        w[2 * x] = pack2<kBf16>(o.x, o.y);
-        w[2 * x + 1] = pack2<kBf16>(o.z, o.w);
+    }
+}
+// ... rounded and stored: 8 X bytes at dst (16-byte aligned for even X, 8-byte aligned for X = 1).
+template <bool kBf16, int X>
+__device__ __forceinline__ void store_groups(const float4 (&o)[X], float scale, unsigned char *dst) {
+    uint32_t w[2 * X];
+#pragma unroll
+    for (int x = 0; x < X; ++x) {
+        w[2 * x] = pack2<kBf16>(o[x].x * scale, o[x].y * scale);
+        w[2 * x + 1] = pack2<kBf16>(o[x].z * scale, o[x].w * scale);
     }
     if (X == 1) {
         *reinterpret_cast<uint2 *>(dst) = make_uint2(w[0], w[1]);
@@ -849,19 +869,142 @@ __device__ __forceinline__ void merge_groups(uint32_t recv, int k, int cgps, int
     for (int i = 0; i < X / 2; ++i)
         *reinterpret_cast<uint4 *>(dst + i * 16) = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
 }
+template <bool kBf16, int X>
+__device__ __forceinline__ void merge_groups(uint32_t recv, int k, int cgps, int row, int x0, const float (&f)[kMaxCluster], unsigned char *dst) {
+    float4 o[X];
+    merge_sums<X>(recv, k, cgps, row, x0, f, o);
+    store_groups<kBf16, X>(o, 1.f, dst);
+}
+
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int *ptr) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
+
+// Several clusters share a unit (p.cluster_split = 2 or 4): behind its own exchange each CTA holds, for its slice of
+// the features, a part of the unit over its cluster's share of the keys -- o (unnormalised sums), M, l per row.  The
+// CTAs of the same rank in the sibling clusters hold the other parts.  Whichever comes last finishes the rows: from
+// its registers if all the others' parts are in the workspace already, else after leaving its own there and finding,
+// by the arrival counter, that it was last after all.  Nobody waits.  Called by all 256 softmax threads (three
+// barriers at most); `flag` is a word of shared memory.  mine / theirs[]: [group in slice][row] float4, M and l behind
+// kRows * kD floats, as a part of a cut unit.
+template <bool kBf16, int X>
+__device__ __forceinline__ void finish_with_siblings(float *mine, const float *const (&theirs)[3], int n_others, unsigned int *ticket,
+                                                     int *flag, float4 (&o)[X], float M, float l, bool has_row, bool writes_ml,
+                                                     int row, int xg0, unsigned char *dst, int tid256, volatile int *abort_flag) {
+    if (tid256 == 0) *flag = *abort_flag ? 2 : (ld_acquire_gpu(ticket) == (unsigned)n_others ? 1 : 0);
+    softmax_groups_sync();
+    int state = *flag;
+    if (state == 2) return;                                 // some wait of this CTA ran out: its part is not to be trusted
+    if (state == 0) {
+        if (has_row) {
+#pragma unroll
+            for (int x = 0; x < X; ++x) reinterpret_cast<float4 *>(mine)[(xg0 + x) * kRows + row] = o[x];
+            if (writes_ml) {
+                mine[kRows * kD + row] = M;
+                mine[kRows * kD + kRows + row] = l;
+            }
+        }
+        softmax_groups_sync();                              // the CTA's part is written, and everybody has read the flag
+        if (tid256 == 0) {
+            __threadfence();
+            *flag = atomicAdd(ticket, 1u) == (unsigned)n_others ? 1 : 0;
+        }
+        softmax_groups_sync();
+        state = *flag;
+        if (state == 0) return;                             // not the last: a sibling finishes
+    }
+    __threadfence();
+    if (has_row) {
+        float m_o[3], l_o[3], Mn = M;
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+            m_o[j] = j < n_others ? __ldcg(theirs[j] + kRows * kD + row) : -INFINITY;
+            l_o[j] = j < n_others ? __ldcg(theirs[j] + kRows * kD + kRows + row) : 0.f;
+            Mn = fmaxf(Mn, m_o[j]);
+        }
+        const float fa = M == -INFINITY ? 0.f : ex2(M - Mn);
+        float fb[3], sum = l * fa;
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+            fb[j] = m_o[j] == -INFINITY ? 0.f : ex2(m_o[j] - Mn);
+            sum = fmaf(l_o[j], fb[j], sum);
+        }
+        const float inv = 1.f / sum;
+#pragma unroll
+        for (int x = 0; x < X; ++x) {
+            o[x].x *= fa; o[x].y *= fa; o[x].z *= fa; o[x].w *= fa;
+#pragma unroll
+            for (int j = 0; j < 3; ++j)
+                if (j < n_others && fb[j] != 0.f) {
+                    const float4 v = __ldcg(reinterpret_cast<const float4 *>(theirs[j]) + (xg0 + x) * kRows + row);
+                    o[x].x = fmaf(fb[j], v.x, o[x].x); o[x].y = fmaf(fb[j], v.y, o[x].y);
+                    o[x].z = fmaf(fb[j], v.z, o[x].z); o[x].w = fmaf(fb[j], v.w, o[x].w);
+                }
+        }
+        store_groups<kBf16, X>(o, inv, dst);
+    }
+    if (tid256 == 0) *ticket = 0u;                          // zero again for the next call on this workspace
+}
+// The workspace slots of the CTAs of this CTA's rank in the sibling clusters (sub: the stream's slot of a tile pair).
+__device__ __forceinline__ void sibling_slots(const Params &p, int slots_per_cta, int sub, const float *(&theirs)[3]) {
+    const int k = p.cluster_k, S = p.cluster_split;
+    const int cluster = (int)blockIdx.x / k, rank = (int)blockIdx.x - cluster * k, first = cluster / S * S;
+    int n = 0;
+    for (int j = 0; j < S; ++j)
+        if (first + j != cluster) theirs[n++] = p.part + ((size_t)(2 * ((first + j) * k + rank)) * slots_per_cta + sub) * kSlotFloats;
+    for (; n < 3; ++n) theirs[n] = nullptr;
+}
 
 // One-tile kernel: received slices lie at area + kXchgRecvOffset as [sender][group in slice][row] float4, followed by
 // [sender][m | l][row]; thread (row, half) merges half of the CTA's slice of the row's features.
 template <bool kBf16>
 __device__ __noinline__ void cluster_merge(const Params &p, unsigned char *area, int rank, int b, int hk, int row_tile,
                                            bool valid, int tid256, volatile int *abort_flag) {
+    int *const flag = &reinterpret_cast<Smem *>(area)->direct;      // (the area is the start of the CTA's shared memory)
     const int k = p.cluster_k;
     const int cgps = 32 / k;                      // groups of 4 features per slice: 16, 8, 4 or 2
     cluster_sync_all();
     const int row = tid256 & 127, half = tid256 >> 7;
     const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
-    if (!valid || node >= p.N || *abort_flag) return;
     const uint32_t recv = smem_u32(area) + kXchgRecvOffset, recv_ml = recv + kRows * kD * 4;
+    if (p.cluster_split > 1) {
+        // several clusters (of eight, or of four) share the unit: this one's result is a part
+        const bool has_row = valid && node < p.N;
+        float f[kMaxCluster], raw[2] = {-INFINITY, 0.f};
+        float4 o[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) o[x] = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int x0 = half * (cgps / 2);
+        if (has_row) {
+            merge_weights(recv_ml, k, row, f, raw);
+            if (k == 8) {
+                float4 o2[2];
+                merge_sums<2>(recv, k, cgps, row, x0, f, o2);
+                o[0] = o2[0]; o[1] = o2[1];
+            } else {
+                merge_sums<4>(recv, k, cgps, row, x0, f, o);
+            }
+        }
+        const int unit = ((int)blockIdx.x / k) / p.cluster_split;
+        const int head = hk * p.g + row % p.g;
+        unsigned char *dst = static_cast<unsigned char *>(p.out) +
+                             ((((size_t)b * p.N + node) * p.Hq + head) * kD + (rank * cgps + x0) * 4) * 2;
+        const float *theirs[3];
+        sibling_slots(p, 1, 0, theirs);
+        float *mine = p.part + (size_t)(2 * (int)blockIdx.x) * kSlotFloats;
+        if (k == 8) {
+            float4 o2[2] = {o[0], o[1]};
+            finish_with_siblings<kBf16, 2>(mine, theirs, p.cluster_split - 1, p.tickets + unit * k + rank, flag, o2, raw[0], raw[1],
+                                           has_row, half == 0, row, x0, dst, tid256, abort_flag);
+        } else {
+            finish_with_siblings<kBf16, 4>(mine, theirs, p.cluster_split - 1, p.tickets + unit * k + rank, flag, o, raw[0], raw[1],
+                                           has_row, half == 0, row, x0, dst, tid256, abort_flag);
+        }
+        return;
+    }
+    if (!valid || node >= p.N || *abort_flag) return;
     float f[kMaxCluster];
     merge_weights(recv_ml, k, row, f);
     const int head = hk * p.g + row % p.g;

@@ -63,32 +63,6 @@ constexpr int kPXchgMl = kRows * kD * 4;                         // bytes from a
 constexpr int kPXchgStream = kPXchgMl + kMaxCluster * 2 * kRows * 4;   // up to 16 senders
 static_assert(2 * kPXchgStream <= (2 + kPStages) * kEntryBytes, "the exchange area is the Q buffers and the ring");
 
-// A stream's received parts lie at `area` as [sender][group in slice][row] float4, followed (at kPXchgMl) by
-// [sender][m | l][row]; thread `row` of the stream merges the CTA's whole slice of the row's features.
-template <bool kBf16>
-__device__ __noinline__ void cluster_merge_pair(const Params &p, const unsigned char *area, int rank, int b, int hk, int row_tile,
-                                                bool valid, int row, volatile int *abort_flag) {
-    cluster_sync_all();                                 // every part has arrived everywhere; nobody writes to a peer any more
-    const int k = p.cluster_k, cgps = 32 / k;
-    const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
-    if (!valid || row_tile >= p.n_row_tiles || node >= p.N || *abort_flag) return;
-    const uint32_t recv = smem_u32(area), recv_ml = recv + kPXchgMl;
-    float f[kMaxCluster];
-    merge_weights(recv_ml, k, row, f);
-    const int head = hk * p.g + row % p.g;
-    unsigned char *dst = static_cast<unsigned char *>(p.out) + ((((size_t)b * p.N + node) * p.Hq + head) * kD + rank * cgps * 4) * 2;
-    if (k == 2) {
-        merge_groups<kBf16, 8>(recv, k, cgps, row, 0, f, dst);
-        merge_groups<kBf16, 8>(recv, k, cgps, row, 8, f, dst + 64);
-    } else if (k == 4) {
-        merge_groups<kBf16, 8>(recv, k, cgps, row, 0, f, dst);
-    } else if (k == 8) {
-        merge_groups<kBf16, 4>(recv, k, cgps, row, 0, f, dst);
-    } else {
-        merge_groups<kBf16, 2>(recv, k, cgps, row, 0, f, dst);
-    }
-}
-
 struct __align__(1024) PSmem {
     unsigned char q[2][kEntryBytes];
     unsigned char ring[kPStages][kEntryBytes];
@@ -106,6 +80,70 @@ struct __align__(1024) PSmem {
     int32_t pg[kPgTiles][kPgSub];      // paged cache: page ids of the tiles about to be fetched
     uint32_t anc[2 * kMaxWords * kRows];   // ancestor words [stream][word][row]; last member: only 2 * ceil(N / 32) words are allocated
 };
+
+// A stream's received parts lie at `area` as [sender][group in slice][row] float4, followed (at kPXchgMl) by
+// [sender][m | l][row]; thread `row` of the stream merges the CTA's whole slice of the row's features.
+// (Called by all 256 softmax threads, the threads of stream s with that stream's area.)
+template <bool kBf16>
+__device__ __noinline__ void cluster_merge_pair(const Params &p, const unsigned char *area, int rank, int b, int hk, int row_tile,
+                                                bool valid, int row, volatile int *abort_flag) {
+    cluster_sync_all();                                 // every part has arrived everywhere; nobody writes to a peer any more
+    const int s = (int)threadIdx.x >> 7;                // the stream whose area this is
+    const int k = p.cluster_k, cgps = 32 / k;
+    const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
+    const uint32_t recv = smem_u32(area), recv_ml = recv + kPXchgMl;
+    if (p.cluster_split > 1) {
+        // several clusters (of eight, or of four) share the unit: this one's result is a part
+        const bool has_row = valid && row_tile < p.n_row_tiles && node < p.N;
+        float f[kMaxCluster], raw[2] = {-INFINITY, 0.f};
+        float4 o[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) o[x] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (has_row) {
+            merge_weights(recv_ml, k, row, f, raw);
+            if (k == 8) {
+                float4 o4[4];
+                merge_sums<4>(recv, k, cgps, row, 0, f, o4);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) o[x] = o4[x];
+            } else {
+                merge_sums<8>(recv, k, cgps, row, 0, f, o);
+            }
+        }
+        const int unit = ((int)blockIdx.x / k) / p.cluster_split;
+        const int head = hk * p.g + row % p.g;
+        unsigned char *dst = static_cast<unsigned char *>(p.out) + ((((size_t)b * p.N + node) * p.Hq + head) * kD + rank * cgps * 4) * 2;
+        int *const flag = &reinterpret_cast<PSmem *>(const_cast<unsigned char *>(area) - s * kPXchgStream)->direct;   // (the areas start the CTA's shared memory)
+        const float *theirs[3];
+        sibling_slots(p, 2, s, theirs);
+        float *mine = p.part + ((size_t)(2 * (int)blockIdx.x) * 2 + s) * kSlotFloats;
+        if (k == 8) {
+            float4 o4[4] = {o[0], o[1], o[2], o[3]};
+            finish_with_siblings<kBf16, 4>(mine, theirs, p.cluster_split - 1, p.tickets + unit * k + rank, flag, o4, raw[0], raw[1],
+                                           has_row, true, row, 0, dst, (int)threadIdx.x, abort_flag);
+        } else {
+            finish_with_siblings<kBf16, 8>(mine, theirs, p.cluster_split - 1, p.tickets + unit * k + rank, flag, o, raw[0], raw[1],
+                                           has_row, true, row, 0, dst, (int)threadIdx.x, abort_flag);
+        }
+        return;
+    }
+    if (!valid || row_tile >= p.n_row_tiles || node >= p.N || *abort_flag) return;
+    float f[kMaxCluster];
+    merge_weights(recv_ml, k, row, f);
+    const int head = hk * p.g + row % p.g;
+    unsigned char *dst = static_cast<unsigned char *>(p.out) + ((((size_t)b * p.N + node) * p.Hq + head) * kD + rank * cgps * 4) * 2;
+    if (k == 2) {
+        merge_groups<kBf16, 8>(recv, k, cgps, row, 0, f, dst);
+        merge_groups<kBf16, 8>(recv, k, cgps, row, 8, f, dst + 64);
+    } else if (k == 4) {
+        merge_groups<kBf16, 8>(recv, k, cgps, row, 0, f, dst);
+    } else if (k == 8) {
+        merge_groups<kBf16, 4>(recv, k, cgps, row, 0, f, dst);
+    } else {
+        merge_groups<kBf16, 2>(recv, k, cgps, row, 0, f, dst);
+    }
+}
+
 
 template <bool kBf16, bool kPaged>
 __global__ void __launch_bounds__(kPThreads, 1)
@@ -165,13 +203,13 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     uint32_t c_rank = 0;
     RangeAsk ask;
     ask.n_pos = n_pos; ask.my_pos = my_pos;
-    ask.cluster_k = 0; ask.cl_rank = 0; ask.cl_b = 0; ask.cl_unit = 0;
+    ask.cluster_k = 0; ask.cl_rank = 0; ask.cl_units_per_seq = 1;
     if (clustered) {
         c_rank = cluster_ctarank();
-        const int unit = (int)blockIdx.x / p.cluster_k;
-        ask.cluster_k = p.cluster_k; ask.cl_rank = (int)c_rank;
-        ask.cl_b = unit / (p.Hkv * p.n_rt);
-        ask.cl_unit = unit - ask.cl_b * p.Hkv * p.n_rt;
+        // (two clusters on a unit, p.cluster_split == 2: their CTAs share the unit's tiles like one cluster of twice the size)
+        ask.cluster_k = p.cluster_k * p.cluster_split;
+        ask.cl_rank = (int)blockIdx.x % ask.cluster_k;
+        ask.cl_units_per_seq = p.Hkv * p.n_rt;
     }
     tc_fence_before();                              // (the tensor memory's base address crosses the plan's last barrier)
     plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0 && !early, kPaged, lrt, ask, sm.plan);
@@ -721,7 +759,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         release();
         if (clustered && t_end <= t_begin) {
             // an empty share still takes part in the cluster's exchange, with parts that saw nothing
-            const int unit = (int)blockIdx.x / p.cluster_k, b = unit / (p.Hkv * p.n_rt);
+            const int unit = (int)blockIdx.x / (p.cluster_k * p.cluster_split), b = unit / (p.Hkv * p.n_rt);
             const int rem = unit - b * p.Hkv * p.n_rt, hk = rem / p.n_rt, rt = rem - hk * p.n_rt;
             cluster_sync_all();
             if (2 * rt + s < p.n_row_tiles)
