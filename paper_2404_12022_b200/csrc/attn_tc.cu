@@ -162,13 +162,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     uint32_t c_rank = 0;
     RangeAsk ask;
     ask.n_pos = p.grid; ask.my_pos = (int)blockIdx.x;
-    ask.cluster_k = 0; ask.cl_rank = 0; ask.cl_units_per_seq = 1;
+    ask.cluster_k = 0; ask.cl_rank = 0; ask.cl_b = 0; ask.cl_unit = 0;
     if (clustered) {
         // (two clusters on a unit, p.cluster_split == 2: their CTAs share the unit's tiles like one cluster of twice the size)
         c_rank = cluster_ctarank();
-        ask.cluster_k = p.cluster_k * p.cluster_split;
-        ask.cl_rank = (int)blockIdx.x % ask.cluster_k;
-        ask.cl_units_per_seq = p.Hkv;
+        ask.cluster_k = p.cluster_k * p.cluster_split;                 // a power of two
+        ask.cl_rank = (int)blockIdx.x & (ask.cluster_k - 1);
+        const int unit = (int)blockIdx.x >> (__ffs(ask.cluster_k) - 1);
+        ask.cl_b = unit / p.Hkv;
+        ask.cl_unit = unit - ask.cl_b * p.Hkv;
     }
     tc_fence_before();                              // (the tensor memory's base address crosses the plan's last barrier)
     plan_sequences<kThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0 && !early, kPaged, 1, ask, sm.plan);   // one unit per KV head in this kernel

@@ -503,7 +503,7 @@ __device__ __forceinline__ int choose_per(int total, int grid, const int32_t *nk
 struct RangeAsk {
     int n_pos, my_pos;
     int cluster_k, cl_rank;                     // cluster form: CTAs that share a unit (side by side in the grid), this CTA's place among them
-    int cl_units_per_seq;                       // ... and units per sequence: Hkv, or Hkv x tile pairs per head
+    int cl_b, cl_unit;                          // ... their sequence, and which of its units
 };
 struct Range {
     int per, t_begin, t_end;
@@ -528,8 +528,7 @@ __device__ __forceinline__ void plan_range(const int32_t *s_len, const int32_t *
         r.per = 0;
         // ask.cluster_k CTAs share the unit (one cluster, or several clusters side by side in the grid); ask.cl_rank
         // is this CTA's place among them
-        const int unit = (int)blockIdx.x / ask.cluster_k;
-        const int cl_b = unit / ask.cl_units_per_seq, cl_unit = unit - cl_b * ask.cl_units_per_seq;
+        const int cl_b = ask.cl_b, cl_unit = ask.cl_unit;
         const int nk = s_nkt[cl_b];
         int lo, hi;
         cluster_share(nk, s_len[cl_b], ask.cluster_k, ask.cl_rank, lo, hi);
@@ -812,18 +811,19 @@ __device__ __forceinline__ float4 lds_f32x4(uint32_t a) {
 constexpr int kMaxCluster = 16;        // CTAs per cluster at most (16 is beyond the portable size: asked for per kernel)
 // raw != nullptr: the weights stay relative to the maximum, which is returned with the weighted sum (raw[0] = M,
 // raw[1] = l): the cluster's result is then a part itself (two clusters share the unit).
+template <int KP>                       // KP >= k: how far the loops over the parts are unrolled
 __device__ __forceinline__ void merge_weights(uint32_t recv_ml, int k, int row, float (&f)[kMaxCluster], float *raw = nullptr) {
     float m[kMaxCluster], M = -INFINITY;
 #pragma unroll
-    for (int c = 0; c < kMaxCluster; ++c) {
+    for (int c = 0; c < KP; ++c) {
         m[c] = c < k ? lds_f32(recv_ml + (uint32_t)(c * 2 * kRows + row) * 4u) : -INFINITY;
         f[c] = c < k ? lds_f32(recv_ml + (uint32_t)(c * 2 * kRows + kRows + row) * 4u) : 0.f;     // the part's row sum, for now
     }
 #pragma unroll
-    for (int c = 0; c < kMaxCluster; ++c) M = fmaxf(M, m[c]);
+    for (int c = 0; c < KP; ++c) M = fmaxf(M, m[c]);
     float l = 0.f;
 #pragma unroll
-    for (int c = 0; c < kMaxCluster; ++c) {
+    for (int c = 0; c < KP; ++c) {
         const float w = m[c] == -INFINITY ? 0.f : ex2(m[c] - M);
         l = fmaf(w, f[c], l);
         f[c] = w;
@@ -835,17 +835,17 @@ __device__ __forceinline__ void merge_weights(uint32_t recv_ml, int k, int row, 
     }
     const float inv = 1.f / l;
 #pragma unroll
-    for (int c = 0; c < kMaxCluster; ++c) f[c] *= inv;
+    for (int c = 0; c < KP; ++c) f[c] *= inv;
 }
 // X groups of 4 features from group x0 on, summed over the parts with their weights: recv holds
 // [sender][group in slice (cgps of them)][row] float4.
-template <int X>
+template <int X, int KP>
 __device__ __forceinline__ void merge_sums(uint32_t recv, int k, int cgps, int row, int x0, const float (&f)[kMaxCluster], float4 (&o)[X]) {
 #pragma unroll
     for (int x = 0; x < X; ++x) {
         o[x] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int c = 0; c < kMaxCluster; ++c)
+        for (int c = 0; c < KP; ++c)
             if (c < k && f[c] != 0.f) {            // a part that saw nothing sent no features: what lies there is not data
                 const float4 v = lds_f32x4(recv + (uint32_t)((c * cgps + x0 + x) * kRows + row) * 16u);
                 o[x].x = fmaf(f[c], v.x, o[x].x); o[x].y = fmaf(f[c], v.y, o[x].y); o[x].z = fmaf(f[c], v.z, o[x].z); o[x].w = fmaf(f[c], v.w, o[x].w);
@@ -869,10 +869,10 @@ __device__ __forceinline__ void store_groups(const float4 (&o)[X], float scale, 
     for (int i = 0; i < X / 2; ++i)
         *reinterpret_cast<uint4 *>(dst + i * 16) = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
 }
-template <bool kBf16, int X>
+template <bool kBf16, int X, int KP>
 __device__ __forceinline__ void merge_groups(uint32_t recv, int k, int cgps, int row, int x0, const float (&f)[kMaxCluster], unsigned char *dst) {
     float4 o[X];
-    merge_sums<X>(recv, k, cgps, row, x0, f, o);
+    merge_sums<X, KP>(recv, k, cgps, row, x0, f, o);
     store_groups<kBf16, X>(o, 1.f, dst);
 }
 
@@ -889,18 +889,24 @@ __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int *ptr) 
 // by the arrival counter, that it was last after all.  Nobody waits.  Called by all 256 softmax threads (three
 // barriers at most); `flag` is a word of shared memory.  mine / theirs[]: [group in slice][row] float4, M and l behind
 // kRows * kD floats, as a part of a cut unit.
-template <bool kBf16, int X>
+// The thread's groups of 4 features are worked through in n_chunks chunks of XC groups, formed anew by `sums(chunk, o)`
+// from what the CTA received wherever they are needed (few registers: this code runs once, behind a call).
+template <bool kBf16, int XC, typename Sums>
 __device__ __forceinline__ void finish_with_siblings(float *mine, const float *const (&theirs)[3], int n_others, unsigned int *ticket,
-                                                     int *flag, float4 (&o)[X], float M, float l, bool has_row, bool writes_ml,
+                                                     int *flag, Sums sums, int n_chunks, float M, float l, bool has_row, bool writes_ml,
                                                      int row, int xg0, unsigned char *dst, int tid256, volatile int *abort_flag) {
     if (tid256 == 0) *flag = *abort_flag ? 2 : (ld_acquire_gpu(ticket) == (unsigned)n_others ? 1 : 0);
     softmax_groups_sync();
     int state = *flag;
     if (state == 2) return;                                 // some wait of this CTA ran out: its part is not to be trusted
+    float4 o[XC];
     if (state == 0) {
         if (has_row) {
+            for (int ch = 0; ch < n_chunks; ++ch) {
+                sums(ch, o);
 #pragma unroll
-            for (int x = 0; x < X; ++x) reinterpret_cast<float4 *>(mine)[(xg0 + x) * kRows + row] = o[x];
+                for (int x = 0; x < XC; ++x) reinterpret_cast<float4 *>(mine)[(xg0 + ch * XC + x) * kRows + row] = o[x];
+            }
             if (writes_ml) {
                 mine[kRows * kD + row] = M;
                 mine[kRows * kD + kRows + row] = l;
@@ -932,18 +938,21 @@ __device__ __forceinline__ void finish_with_siblings(float *mine, const float *c
             sum = fmaf(l_o[j], fb[j], sum);
         }
         const float inv = 1.f / sum;
+        for (int ch = 0; ch < n_chunks; ++ch) {
+            sums(ch, o);
 #pragma unroll
-        for (int x = 0; x < X; ++x) {
-            o[x].x *= fa; o[x].y *= fa; o[x].z *= fa; o[x].w *= fa;
+            for (int x = 0; x < XC; ++x) {
+                o[x].x *= fa; o[x].y *= fa; o[x].z *= fa; o[x].w *= fa;
 #pragma unroll
-            for (int j = 0; j < 3; ++j)
-                if (j < n_others && fb[j] != 0.f) {
-                    const float4 v = __ldcg(reinterpret_cast<const float4 *>(theirs[j]) + (xg0 + x) * kRows + row);
-                    o[x].x = fmaf(fb[j], v.x, o[x].x); o[x].y = fmaf(fb[j], v.y, o[x].y);
-                    o[x].z = fmaf(fb[j], v.z, o[x].z); o[x].w = fmaf(fb[j], v.w, o[x].w);
-                }
+                for (int j = 0; j < 3; ++j)
+                    if (j < n_others && fb[j] != 0.f) {
+                        const float4 v = __ldcg(reinterpret_cast<const float4 *>(theirs[j]) + (xg0 + ch * XC + x) * kRows + row);
+                        o[x].x = fmaf(fb[j], v.x, o[x].x); o[x].y = fmaf(fb[j], v.y, o[x].y);
+                        o[x].z = fmaf(fb[j], v.z, o[x].z); o[x].w = fmaf(fb[j], v.w, o[x].w);
+                    }
+            }
+            store_groups<kBf16, XC>(o, inv, dst + ch * XC * 8);
         }
-        store_groups<kBf16, X>(o, inv, dst);
     }
     if (tid256 == 0) *ticket = 0u;                          // zero again for the next call on this workspace
 }
@@ -973,19 +982,10 @@ __device__ __noinline__ void cluster_merge(const Params &p, unsigned char *area,
         // several clusters (of eight, or of four) share the unit: this one's result is a part
         const bool has_row = valid && node < p.N;
         float f[kMaxCluster], raw[2] = {-INFINITY, 0.f};
-        float4 o[4];
-#pragma unroll
-        for (int x = 0; x < 4; ++x) o[x] = make_float4(0.f, 0.f, 0.f, 0.f);
         const int x0 = half * (cgps / 2);
         if (has_row) {
-            merge_weights(recv_ml, k, row, f, raw);
-            if (k == 8) {
-                float4 o2[2];
-                merge_sums<2>(recv, k, cgps, row, x0, f, o2);
-                o[0] = o2[0]; o[1] = o2[1];
-            } else {
-                merge_sums<4>(recv, k, cgps, row, x0, f, o);
-            }
+            if (k == 8) merge_weights<8>(recv_ml, k, row, f, raw);
+            else merge_weights<4>(recv_ml, k, row, f, raw);
         }
         const int unit = ((int)blockIdx.x / k) / p.cluster_split;
         const int head = hk * p.g + row % p.g;
@@ -994,27 +994,27 @@ __device__ __noinline__ void cluster_merge(const Params &p, unsigned char *area,
         const float *theirs[3];
         sibling_slots(p, 1, 0, theirs);
         float *mine = p.part + (size_t)(2 * (int)blockIdx.x) * kSlotFloats;
-        if (k == 8) {
-            float4 o2[2] = {o[0], o[1]};
-            finish_with_siblings<kBf16, 2>(mine, theirs, p.cluster_split - 1, p.tickets + unit * k + rank, flag, o2, raw[0], raw[1],
-                                           has_row, half == 0, row, x0, dst, tid256, abort_flag);
-        } else {
-            finish_with_siblings<kBf16, 4>(mine, theirs, p.cluster_split - 1, p.tickets + unit * k + rank, flag, o, raw[0], raw[1],
-                                           has_row, half == 0, row, x0, dst, tid256, abort_flag);
-        }
+        auto sums = [&](int ch, float4 (&o)[2]) {                // two groups at a time: clusters of eight have two per thread, of four four
+            if (k == 8) merge_sums<2, 8>(recv, k, cgps, row, x0 + 2 * ch, f, o);
+            else merge_sums<2, 4>(recv, k, cgps, row, x0 + 2 * ch, f, o);
+        };
+        finish_with_siblings<kBf16, 2>(mine, theirs, p.cluster_split - 1, p.tickets + unit * k + rank, flag, sums, k == 8 ? 1 : 2,
+                                       raw[0], raw[1], has_row, half == 0, row, x0, dst, tid256, abort_flag);
         return;
     }
     if (!valid || node >= p.N || *abort_flag) return;
     float f[kMaxCluster];
-    merge_weights(recv_ml, k, row, f);
+    if (k <= 4) merge_weights<4>(recv_ml, k, row, f);
+    else if (k == 8) merge_weights<8>(recv_ml, k, row, f);
+    else merge_weights<16>(recv_ml, k, row, f);
     const int head = hk * p.g + row % p.g;
     const int x0 = half * (cgps / 2);
     unsigned char *dst = static_cast<unsigned char *>(p.out) +
                          ((((size_t)b * p.N + node) * p.Hq + head) * kD + (rank * cgps + x0) * 4) * 2;
-    if (k == 2) merge_groups<kBf16, 8>(recv, k, cgps, row, x0, f, dst);
-    else if (k == 4) merge_groups<kBf16, 4>(recv, k, cgps, row, x0, f, dst);
-    else if (k == 8) merge_groups<kBf16, 2>(recv, k, cgps, row, x0, f, dst);
-    else merge_groups<kBf16, 1>(recv, k, cgps, row, x0, f, dst);
+    if (k == 2) merge_groups<kBf16, 8, 2>(recv, k, cgps, row, x0, f, dst);
+    else if (k == 4) merge_groups<kBf16, 4, 4>(recv, k, cgps, row, x0, f, dst);
+    else if (k == 8) merge_groups<kBf16, 2, 8>(recv, k, cgps, row, x0, f, dst);
+    else merge_groups<kBf16, 1, 16>(recv, k, cgps, row, x0, f, dst);
 }
 
 }  // namespace tc

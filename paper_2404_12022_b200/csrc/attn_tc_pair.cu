@@ -84,7 +84,9 @@ struct __align__(1024) PSmem {
 // A stream's received parts lie at `area` as [sender][group in slice][row] float4, followed (at kPXchgMl) by
 // [sender][m | l][row]; thread `row` of the stream merges the CTA's whole slice of the row's features.
 // (Called by all 256 softmax threads, the threads of stream s with that stream's area.)
-template <bool kBf16>
+// kSplit: the instantiation that knows of several clusters per unit (p.cluster_split > 1); the others carry none of that
+// code, whose register needs would otherwise reach into the callers'.
+template <bool kBf16, bool kSplit>
 __device__ __noinline__ void cluster_merge_pair(const Params &p, const unsigned char *area, int rank, int b, int hk, int row_tile,
                                                 bool valid, int row, volatile int *abort_flag) {
     cluster_sync_all();                                 // every part has arrived everywhere; nobody writes to a peer any more
@@ -92,23 +94,13 @@ __device__ __noinline__ void cluster_merge_pair(const Params &p, const unsigned 
     const int k = p.cluster_k, cgps = 32 / k;
     const int node = row_tile * p.rows_per_tile_nodes + row / p.g;
     const uint32_t recv = smem_u32(area), recv_ml = recv + kPXchgMl;
-    if (p.cluster_split > 1) {
+    if (kSplit && p.cluster_split > 1) {
         // several clusters (of eight, or of four) share the unit: this one's result is a part
         const bool has_row = valid && row_tile < p.n_row_tiles && node < p.N;
         float f[kMaxCluster], raw[2] = {-INFINITY, 0.f};
-        float4 o[8];
-#pragma unroll
-        for (int x = 0; x < 8; ++x) o[x] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (has_row) {
-            merge_weights(recv_ml, k, row, f, raw);
-            if (k == 8) {
-                float4 o4[4];
-                merge_sums<4>(recv, k, cgps, row, 0, f, o4);
-#pragma unroll
-                for (int x = 0; x < 4; ++x) o[x] = o4[x];
-            } else {
-                merge_sums<8>(recv, k, cgps, row, 0, f, o);
-            }
+            if (k == 8) merge_weights<8>(recv_ml, k, row, f, raw);
+            else merge_weights<4>(recv_ml, k, row, f, raw);
         }
         const int unit = ((int)blockIdx.x / k) / p.cluster_split;
         const int head = hk * p.g + row % p.g;
@@ -117,35 +109,35 @@ __device__ __noinline__ void cluster_merge_pair(const Params &p, const unsigned 
         const float *theirs[3];
         sibling_slots(p, 2, s, theirs);
         float *mine = p.part + ((size_t)(2 * (int)blockIdx.x) * 2 + s) * kSlotFloats;
-        if (k == 8) {
-            float4 o4[4] = {o[0], o[1], o[2], o[3]};
-            finish_with_siblings<kBf16, 4>(mine, theirs, p.cluster_split - 1, p.tickets + unit * k + rank, flag, o4, raw[0], raw[1],
-                                           has_row, true, row, 0, dst, (int)threadIdx.x, abort_flag);
-        } else {
-            finish_with_siblings<kBf16, 8>(mine, theirs, p.cluster_split - 1, p.tickets + unit * k + rank, flag, o, raw[0], raw[1],
-                                           has_row, true, row, 0, dst, (int)threadIdx.x, abort_flag);
-        }
+        auto sums = [&](int ch, float4 (&o)[4]) {                // four groups at a time: clusters of eight have four per thread, of four eight
+            if (k == 8) merge_sums<4, 8>(recv, k, cgps, row, 4 * ch, f, o);
+            else merge_sums<4, 4>(recv, k, cgps, row, 4 * ch, f, o);
+        };
+        finish_with_siblings<kBf16, 4>(mine, theirs, p.cluster_split - 1, p.tickets + unit * k + rank, flag, sums, k == 8 ? 1 : 2,
+                                       raw[0], raw[1], has_row, true, row, 0, dst, (int)threadIdx.x, abort_flag);
         return;
     }
     if (!valid || row_tile >= p.n_row_tiles || node >= p.N || *abort_flag) return;
     float f[kMaxCluster];
-    merge_weights(recv_ml, k, row, f);
+    if (k <= 4) merge_weights<4>(recv_ml, k, row, f);
+    else if (k == 8) merge_weights<8>(recv_ml, k, row, f);
+    else merge_weights<16>(recv_ml, k, row, f);
     const int head = hk * p.g + row % p.g;
     unsigned char *dst = static_cast<unsigned char *>(p.out) + ((((size_t)b * p.N + node) * p.Hq + head) * kD + rank * cgps * 4) * 2;
     if (k == 2) {
-        merge_groups<kBf16, 8>(recv, k, cgps, row, 0, f, dst);
-        merge_groups<kBf16, 8>(recv, k, cgps, row, 8, f, dst + 64);
+        merge_groups<kBf16, 8, 2>(recv, k, cgps, row, 0, f, dst);
+        merge_groups<kBf16, 8, 2>(recv, k, cgps, row, 8, f, dst + 64);
     } else if (k == 4) {
-        merge_groups<kBf16, 8>(recv, k, cgps, row, 0, f, dst);
+        merge_groups<kBf16, 8, 4>(recv, k, cgps, row, 0, f, dst);
     } else if (k == 8) {
-        merge_groups<kBf16, 4>(recv, k, cgps, row, 0, f, dst);
+        merge_groups<kBf16, 4, 8>(recv, k, cgps, row, 0, f, dst);
     } else {
-        merge_groups<kBf16, 2>(recv, k, cgps, row, 0, f, dst);
+        merge_groups<kBf16, 2, 16>(recv, k, cgps, row, 0, f, dst);
     }
 }
 
 
-template <bool kBf16, bool kPaged>
+template <bool kBf16, bool kPaged, bool kSplit>
 __global__ void __launch_bounds__(kPThreads, 1)
 attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const Params p, const PagedParams pp) {
@@ -203,13 +195,15 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     uint32_t c_rank = 0;
     RangeAsk ask;
     ask.n_pos = n_pos; ask.my_pos = my_pos;
-    ask.cluster_k = 0; ask.cl_rank = 0; ask.cl_units_per_seq = 1;
+    ask.cluster_k = 0; ask.cl_rank = 0; ask.cl_b = 0; ask.cl_unit = 0;
     if (clustered) {
         c_rank = cluster_ctarank();
         // (two clusters on a unit, p.cluster_split == 2: their CTAs share the unit's tiles like one cluster of twice the size)
-        ask.cluster_k = p.cluster_k * p.cluster_split;
-        ask.cl_rank = (int)blockIdx.x % ask.cluster_k;
-        ask.cl_units_per_seq = p.Hkv * p.n_rt;
+        ask.cluster_k = p.cluster_k * p.cluster_split;                 // a power of two
+        ask.cl_rank = (int)blockIdx.x & (ask.cluster_k - 1);
+        const int unit = (int)blockIdx.x >> (__ffs(ask.cluster_k) - 1);
+        ask.cl_b = unit / (p.Hkv * p.n_rt);
+        ask.cl_unit = unit - ask.cl_b * p.Hkv * p.n_rt;
     }
     tc_fence_before();                              // (the tensor memory's base address crosses the plan's last barrier)
     plan_sequences<kPThreads>(p, sm.len, sm.nkt, sm.pre, blockIdx.x == 0 && !early, kPaged, lrt, ask, sm.plan);
@@ -740,7 +734,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 cluster_sync_all();
                 if (active) emit(nullptr, false, false, true);
                 tc_fence_before();
-                cluster_merge_pair<kBf16>(p, xarea + s * kPXchgStream, (int)c_rank, sg.b, sg.hk, row_tile, true, row, abort_flag);
+                cluster_merge_pair<kBf16, kSplit>(p, xarea + s * kPXchgStream, (int)c_rank, sg.b, sg.hk, row_tile, true, row, abort_flag);
             } else if (active) {
                 emit(p.part + ((size_t)(2 * (int)blockIdx.x + cut_k) * 2 + s) * kSlotFloats, final || direct, direct, false);
             }
@@ -768,7 +762,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     st_peer_f1(ml, -INFINITY);
                     st_peer_f1(ml + kRows * 4, 0.f);
                 }
-            cluster_merge_pair<kBf16>(p, xarea + s * kPXchgStream, (int)c_rank, b, hk, 2 * rt + s, sm.nkt[b] > 0, row, abort_flag);
+            cluster_merge_pair<kBf16, kSplit>(p, xarea + s * kPXchgStream, (int)c_rank, b, hk, 2 * rt + s, sm.nkt[b] > 0, row, abort_flag);
         }
         // --- cut units: the CTA that delivers the last part of a unit merges all parts; nobody waits ---
         if (cut[0].valid || cut[1].valid) {
@@ -815,9 +809,11 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 int launch_attn_tc_pair_kernel(const CUtensorMap &tm_q, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const tc::Params &p,
                                const tc::PagedParams &pp, bool bf16, bool paged, cudaStream_t s) {
     typedef void (*Fn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const tc::Params, const tc::PagedParams);
-    const Fn fns[4] = {tc::attn_tc_pair_kernel<false, false>, tc::attn_tc_pair_kernel<true, false>,
-                       tc::attn_tc_pair_kernel<false, true>, tc::attn_tc_pair_kernel<true, true>};
-    const Fn fn = fns[(bf16 ? 1 : 0) + (paged ? 2 : 0)];
+    const Fn fns[8] = {tc::attn_tc_pair_kernel<false, false, false>, tc::attn_tc_pair_kernel<true, false, false>,
+                       tc::attn_tc_pair_kernel<false, true, false>,  tc::attn_tc_pair_kernel<true, true, false>,
+                       tc::attn_tc_pair_kernel<false, false, true>,  tc::attn_tc_pair_kernel<true, false, true>,
+                       tc::attn_tc_pair_kernel<false, true, true>,   tc::attn_tc_pair_kernel<true, true, true>};
+    const Fn fn = fns[(bf16 ? 1 : 0) + (paged ? 2 : 0) + (p.cluster_split > 1 ? 4 : 0)];
     static bool done[64];
     const size_t smem_max = sizeof(tc::PSmem) + 1024;
     const size_t smem = offsetof(tc::PSmem, anc) + (size_t)2 * ((p.N + 31) / 32) * tc::kRows * sizeof(uint32_t) + 1024;
@@ -825,7 +821,7 @@ int launch_attn_tc_pair_kernel(const CUtensorMap &tm_q, const CUtensorMap &tm_k,
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(HT_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
     if (!(dev >= 0 && dev < 64 && done[dev])) {
-        for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+        for (int i = 0; i < 8 && e == cudaSuccess; ++i) {
             e = cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
             if (e == cudaSuccess) e = cudaFuncSetAttribute(fns[i], cudaFuncAttributeNonPortableClusterSizeAllowed, 1);   // clusters of 16
         }
