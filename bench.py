@@ -207,10 +207,10 @@ class ClockSampler:
 # DRAM traffic per launch of the attention kernel on a c3 layer, from the ncu capture of the committed build summarised
 # at the end of profiles/attn_tc_kernel_c3_layer.md (dram__bytes_read.sum + dram__bytes_write.sum, mean of two launches).  It is only
 # reported while the kernel source is the one that was profiled.
-NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 287.7e6,
+NCU_TRAFFIC = {"workload": "c3_llama7b_step_bf16", "bytes_per_launch": 287.6e6,
                "source": ["paper_2404_12022_b200/csrc/attn_tc.cu", "paper_2404_12022_b200/csrc/attn_tc.cuh",
                           "paper_2404_12022_b200/csrc/ht_common.cuh"],
-               "sha256": "5d0ba9b2a6b316fa6a222158943b17410744748bf9b2d7a2236da0bc133c52ac"}
+               "sha256": "eaae2896afb6cfc62190630292e100236acc25093f3c70e33ac50d261a13661e"}
 
 
 def traffic_digest():
