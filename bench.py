@@ -62,7 +62,9 @@ def workload_config(w, n_gpus):
             "head_dim": w.D, "kv_len": (w.kv_len[0] if len(set(w.kv_len)) == 1 else "ragged %d..%d" % (min(w.kv_len), max(w.kv_len))),
             "tree_nodes": w.T, "pseudo_rows": w.P, "hidden": w.d, "transfer_steps": w.k, "vocab": w.V,
             "parallelism": "replicas x%d" % n_gpus if n_gpus > 1 else "single GPU",
-            "l2_policy": "inputs larger than L2 (KV cache of a step >> 126 MB)"}
+            "l2_policy": "inputs larger than L2 (KV cache of a step >> 126 MB)",
+            "attention_flags": "HT_ATTN_WORKSPACE_CLEAN | HT_ATTN_CONTEXT_FINAL (the step keeps its workspace; lengths, trees "
+                               "and context rows are final before a layer's call)"}
 
 
 # ------------------------------------------------------------------------------------------
